@@ -1,0 +1,324 @@
+"""fp64 CPU oracle for the multi-agent PPO hot path.  TEST INFRASTRUCTURE ONLY.
+
+This file is the reference the CUDA library is judged against.  It is plain numpy in float64,
+slow and direct: every quantity is its definition written out, one block of rows at a time,
+with the full logit vector of each row materialised.  It shares no code with the CUDA path and
+imports nothing from it.  Only tests, the smoke check and the benchmark's CPU-baseline leg may
+call it; the product never does.
+
+What each function follows:
+
+* ``role_advantage``  - the additive role reward r_v = lam_node r_node + lam_turn r_turn +
+  lam_traj r_traj (Section "Agent-Specific Reward Interface", the lambda-weighted equation) with
+  rewards committed per role invocation (Section "Optimization Objective and System Interface");
+  role identity is kept even when parameters are shared (Section "Parameter Sharing in the
+  System"), so statistics are per (rollout group, role), never per model.  The normalisation
+  itself (mean / std per segment, epsilon added to std) is not printed in the paper; it is the
+  reading fixed for this path.
+* ``logprob_fwd``     - "old log probabilities, reference-policy log probabilities" of the
+  paragraph "Advantage computation and policy evaluation": log-softmax of the LM-head logits
+  of the model that phi assigns to the token's role, gathered at the target token, and the
+  Shannon entropy of that softmax.
+* ``ppo_loss_fwd_bwd``- the "PPO-style" update of Section "PPO-Style Training Loop" with the
+  standard clipped surrogate, a KL-to-reference penalty (k1/k2/k3 estimators) and an entropy
+  bonus, averaged over valid tokens per model (paragraph "Model-specific updates and
+  synchronization": each worker group updates its own actor), and its exact gradient with
+  respect to the hidden states and each LM-head matrix.
+* ``gae``             - the generalized-advantage equation printed in the same section
+  (A_t = sum_l (gamma lambda)^l delta_{t+l}), evaluated as the literal double sum.
+
+Pins: tests/test_oracle_pins.py (closed forms, invariants, library special cases, finite
+differences, autograd third opinion, brute force).  No function here is unpinned.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+F64 = np.float64
+
+
+def to_f64(x) -> np.ndarray:
+    """Exact widening.  uint16 arrays are bf16 bit patterns; anything else is cast."""
+    x = np.asarray(x)
+    if x.dtype == np.uint16:
+        return (x.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(F64)
+    return x.astype(F64)
+
+
+# ----------------------------------------------------------------------------------------------
+# stage 1: role-level advantage
+# ----------------------------------------------------------------------------------------------
+
+def role_advantage(inv_role, inv_group, inv_traj, r_node, r_turn, r_traj, lam,
+                   n_roles, n_groups, cu_seqlens, tok_mask=None, eps=1e-6, ddof=0):
+    """Combine rewards per invocation, normalise per (group, role), broadcast to tokens.
+
+    Returns dict(r, adv_inv, adv_tok, seg_n, seg_mean, seg_std); segment index = g*n_roles+v.
+    """
+    inv_role = np.asarray(inv_role, dtype=np.int64)
+    inv_group = np.asarray(inv_group, dtype=np.int64)
+    inv_traj = np.asarray(inv_traj, dtype=np.int64)
+    S = inv_role.shape[0]
+    lam = np.ones((n_roles, 3), F64) if lam is None else to_f64(lam).reshape(n_roles, 3)
+    rn = np.zeros(S, F64) if r_node is None else to_f64(r_node)
+    rt = np.zeros(S, F64) if r_turn is None else to_f64(r_turn)
+    rj = np.zeros(S, F64) if r_traj is None else to_f64(r_traj)[inv_traj]
+    r = lam[inv_role, 0] * rn + lam[inv_role, 1] * rt + lam[inv_role, 2] * rj
+
+    n_seg = n_groups * n_roles
+    seg = inv_group * n_roles + inv_role
+    seg_n = np.zeros(n_seg, np.int64)
+    seg_mean = np.zeros(n_seg, F64)
+    seg_std = np.zeros(n_seg, F64)
+    adv_inv = np.zeros(S, F64)
+    for q in range(n_seg):
+        members = np.nonzero(seg == q)[0]
+        n = members.size
+        seg_n[q] = n
+        if n == 0:
+            continue
+        mu = r[members].sum() / n
+        seg_mean[q] = mu
+        if n - ddof <= 0:
+            continue                                    # A = 0, std reported as 0
+        sigma = np.sqrt(((r[members] - mu) ** 2).sum() / (n - ddof))
+        seg_std[q] = sigma
+        if sigma + eps == 0.0:
+            continue                                    # all rewards equal and eps = 0: A = 0
+        adv_inv[members] = (r[members] - mu) / (sigma + eps)
+
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    n_tok = int(cu[-1])
+    mask = np.ones(n_tok, F64) if tok_mask is None else (np.asarray(tok_mask) != 0).astype(F64)
+    adv_tok = np.zeros(n_tok, F64)
+    for s in range(S):
+        adv_tok[cu[s]:cu[s + 1]] = adv_inv[s]
+    adv_tok *= mask
+    return dict(r=r, adv_inv=adv_inv, adv_tok=adv_tok, seg_n=seg_n, seg_mean=seg_mean, seg_std=seg_std)
+
+
+# ----------------------------------------------------------------------------------------------
+# token routing through phi
+# ----------------------------------------------------------------------------------------------
+
+def token_invocation(cu_seqlens) -> np.ndarray:
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    return np.repeat(np.arange(cu.size - 1, dtype=np.int64), np.diff(cu))
+
+
+def token_role_model(cu_seqlens, inv_role, role_model):
+    tok_inv = token_invocation(cu_seqlens)
+    tok_role = np.asarray(inv_role, dtype=np.int64)[tok_inv]
+    tok_model = np.asarray(role_model, dtype=np.int64)[tok_role]
+    return tok_role, tok_model
+
+
+# ----------------------------------------------------------------------------------------------
+# stage 2: log-prob, entropy, log-sum-exp
+# ----------------------------------------------------------------------------------------------
+
+def _row_stats(Z):
+    """lse, entropy and probabilities of each row of a logit block Z [n, V] (float64)."""
+    m = Z.max(axis=1, keepdims=True)
+    E = np.exp(Z - m)
+    s = E.sum(axis=1, keepdims=True)
+    lse = (m + np.log(s))[:, 0]
+    P = E / s
+    logP = Z - lse[:, None]
+    ent = -(P * logP).sum(axis=1)
+    return lse, ent, P
+
+
+def logprob_fwd(hidden, W, cu_seqlens, inv_role, role_model, target, tok_mask=None,
+                inv_temperature=1.0, rows=None, block=256):
+    """logp, entropy, lse per token (zeros where mask == 0).
+
+    ``rows`` restricts the computation to the given token indices (sampled parity at full size);
+    other rows are returned as zero.
+    """
+    n_tok = int(np.asarray(cu_seqlens)[-1])
+    _, tok_model = token_role_model(cu_seqlens, inv_role, role_model)
+    mask = np.ones(n_tok, bool) if tok_mask is None else (np.asarray(tok_mask) != 0)
+    target = np.asarray(target, dtype=np.int64)
+    want = mask.copy()
+    if rows is not None:
+        sel = np.zeros(n_tok, bool)
+        sel[np.asarray(rows, dtype=np.int64)] = True
+        want &= sel
+    logp = np.zeros(n_tok, F64)
+    ent = np.zeros(n_tok, F64)
+    lse = np.zeros(n_tok, F64)
+    for k in range(len(W)):
+        idx = np.nonzero(want & (tok_model == k))[0]
+        if idx.size == 0:
+            continue
+        Wk = to_f64(W[k])
+        for b0 in range(0, idx.size, block):
+            ib = idx[b0:b0 + block]
+            Z = inv_temperature * (to_f64(hidden[ib]) @ Wk.T)
+            l, e, _ = _row_stats(Z)
+            lse[ib] = l
+            ent[ib] = e
+            logp[ib] = Z[np.arange(ib.size), target[ib]] - l
+    return dict(logp=logp, entropy=ent, lse=lse)
+
+
+# ----------------------------------------------------------------------------------------------
+# stage 3: PPO-clip + KL-to-reference (+ entropy bonus): forward and backward
+# ----------------------------------------------------------------------------------------------
+
+def kl_term(d, mode):
+    """KL-to-reference estimators as functions of d = ref_logp - logp, and d(kl)/d(logp)."""
+    if mode == 1:
+        return -d, np.ones_like(d)
+    if mode == 2:
+        return 0.5 * d * d, -d
+    if mode == 3:
+        return np.exp(d) - d - 1.0, 1.0 - np.exp(d)
+    raise ValueError("kl_mode must be 1, 2 or 3")
+
+
+def ppo_token_terms(logp, entropy, old_logp, ref_logp, adv, clip_lo, clip_hi, kl_coef, kl_mode, ent_coef):
+    """Per-token loss pieces and the derivative of the token loss w.r.t. its log-prob."""
+    rho = np.exp(logp - old_logp)
+    rho_c = np.clip(rho, 1.0 - clip_lo, 1.0 + clip_hi)
+    unclipped = -rho * adv
+    clipped = -rho_c * adv
+    u = (unclipped >= clipped)                      # ties -> unclipped branch
+    pg = np.where(u, unclipped, clipped)
+    d = ref_logp - logp
+    kl, dkl = kl_term(d, kl_mode)
+    tok_loss = pg + kl_coef * kl - ent_coef * entropy
+    dl_dlogp = np.where(u, -adv * rho, 0.0) + kl_coef * dkl
+    return dict(rho=rho, pg=pg, kl=kl, u=u, tok_loss=tok_loss, dl_dlogp=dl_dlogp)
+
+
+def ppo_loss_fwd_bwd(hidden, W, cu_seqlens, inv_role, role_model, target, tok_mask,
+                     old_logp, ref_logp, adv_tok, clip_lo=0.2, clip_hi=0.2, kl_coef=0.0, kl_mode=3,
+                     ent_coef=0.0, norm=None, inv_temperature=1.0, n_roles=None,
+                     want_dW=True, dW_models=None, rows=None, block=256):
+    """Loss per model, metrics, per-token outputs, dHidden [N,H] and dW_k [V,H] (float64).
+
+    ``norm``      : optional per-model denominator M_k (gradient accumulation across calls).
+    ``dW_models`` : models whose dW is materialised (default: all); others are returned as None.
+    ``rows``      : if given, only these token rows are evaluated (sampled parity at full size).
+                    M_k still counts every valid row of the batch, so the per-token outputs and
+                    dHidden rows of the selected rows are exact (a row's gradient needs only that
+                    row, W_k and M_k); ``loss`` and ``dW`` are then the contribution of the
+                    selected rows alone.
+    """
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    n_tok = int(cu[-1])
+    K = len(W)
+    H = np.asarray(hidden).shape[1]
+    tok_role, tok_model = token_role_model(cu, inv_role, role_model)
+    R = int(n_roles if n_roles is not None else np.asarray(role_model).size)
+    mask = np.ones(n_tok, bool) if tok_mask is None else (np.asarray(tok_mask) != 0)
+    target = np.asarray(target, dtype=np.int64)
+    old_logp = to_f64(old_logp)
+    ref_logp = to_f64(ref_logp)
+    adv = to_f64(adv_tok)
+    tau = float(inv_temperature)
+
+    logp = np.zeros(n_tok, F64)
+    ent = np.zeros(n_tok, F64)
+    lse = np.zeros(n_tok, F64)
+    tok_loss = np.zeros(n_tok, F64)
+    pg = np.zeros(n_tok, F64)
+    kl = np.zeros(n_tok, F64)
+    rho = np.zeros(n_tok, F64)
+    clipped_flag = np.zeros(n_tok, F64)
+    a = np.zeros(n_tok, F64)
+    b = np.zeros(n_tok, F64)
+    M = np.zeros(K, F64)
+    loss = np.zeros(K, F64)
+    dW = [None] * K
+    dW_models = range(K) if dW_models is None else dW_models
+
+    # the counts M_k come first: every token's coefficient is scaled by 1/M_k
+    for k in range(K):
+        cnt = float((mask & (tok_model == k)).sum())
+        M[k] = float(norm[k]) if norm is not None else max(cnt, 1.0)
+
+    want = mask.copy()
+    if rows is not None:
+        sel_rows = np.zeros(n_tok, bool)
+        sel_rows[np.asarray(rows, dtype=np.int64)] = True
+        want &= sel_rows
+    # dHidden: all N rows (zeros where masked), or, with ``rows``, one line per evaluated row
+    dh_index = np.arange(n_tok) if rows is None else np.nonzero(want)[0]
+    dh_pos = np.full(n_tok, -1, np.int64)
+    dh_pos[dh_index] = np.arange(dh_index.size)
+    dHidden = np.zeros((dh_index.size, H), F64)
+
+    for k in range(K):
+        idx = np.nonzero(want & (tok_model == k))[0]
+        Wk = to_f64(W[k]) if idx.size or (want_dW and k in dW_models) else None
+        if want_dW and k in dW_models:
+            dW[k] = np.zeros((Wk.shape[0], H), F64)
+        for b0 in range(0, idx.size, block):
+            ib = idx[b0:b0 + block]
+            hb = to_f64(hidden[ib])
+            Z = tau * (hb @ Wk.T)
+            l, e, P = _row_stats(Z)
+            lp = Z[np.arange(ib.size), target[ib]] - l
+            t = ppo_token_terms(lp, e, old_logp[ib], ref_logp[ib], adv[ib],
+                                clip_lo, clip_hi, kl_coef, kl_mode, ent_coef)
+            logp[ib], ent[ib], lse[ib] = lp, e, l
+            tok_loss[ib], pg[ib], kl[ib], rho[ib] = t["tok_loss"], t["pg"], t["kl"], t["rho"]
+            clipped_flag[ib] = (~t["u"]).astype(F64)
+            a[ib] = t["dl_dlogp"] / M[k]
+            b[ib] = -ent_coef / M[k]
+            # dL/dz for every vocabulary entry of every selected row
+            Gm = -a[ib][:, None] * P - b[ib][:, None] * P * (Z - l[:, None] + e[:, None])
+            Gm[np.arange(ib.size), target[ib]] += a[ib]
+            dHidden[dh_pos[ib]] = tau * (Gm @ Wk)
+            if dW[k] is not None:
+                dW[k] += tau * (Gm.T @ hb)
+        loss[k] = tok_loss[idx].sum() / M[k]
+
+    def _metrics(sel):
+        n = float(sel.sum())
+        dn = max(n, 1.0)
+        return np.array([n, pg[sel].sum() / dn, kl[sel].sum() / dn, ent[sel].sum() / dn,
+                         clipped_flag[sel].sum() / dn, rho[sel].sum() / dn,
+                         logp[sel].sum() / dn, adv[sel].sum() / dn], F64)
+
+    metrics_model = np.stack([_metrics(want & (tok_model == k)) for k in range(K)])
+    metrics_role = np.stack([_metrics(want & (tok_role == v)) for v in range(R)])
+    return dict(loss=loss, M=M, logp=logp, entropy=ent, lse=lse, tok_loss=tok_loss, a=a, b=b,
+                dHidden=dHidden, dh_index=dh_index, dW=dW, metrics_model=metrics_model, metrics_role=metrics_role)
+
+
+def ppo_loss_value(hidden, W, cu_seqlens, inv_role, role_model, target, tok_mask,
+                   old_logp, ref_logp, adv_tok, **kw):
+    """Loss per model only (used by the finite-difference pin)."""
+    out = ppo_loss_fwd_bwd(hidden, W, cu_seqlens, inv_role, role_model, target, tok_mask,
+                           old_logp, ref_logp, adv_tok, want_dW=False, **kw)
+    return out["loss"]
+
+
+# ----------------------------------------------------------------------------------------------
+# token-level generalized advantage estimation (the advantage formula the paper prints)
+# ----------------------------------------------------------------------------------------------
+
+def gae(rewards, values, cu_seqlens, gamma, lam):
+    """A_t = sum_{l=0}^{T-t} (gamma*lam)^l delta_{t+l},  delta_t = r_t + gamma V(s_{t+1}) - V(s_t),
+    per sequence, with V past the last token taken as 0.  Returns (advantages, returns=A+V)."""
+    r = to_f64(rewards)
+    v = to_f64(values)
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    A = np.zeros_like(r)
+    for s in range(cu.size - 1):
+        lo, hi = int(cu[s]), int(cu[s + 1])
+        T = hi - lo
+        if T == 0:
+            continue
+        vs = np.concatenate([v[lo:hi], [0.0]])
+        delta = r[lo:hi] + gamma * vs[1:] - vs[:-1]
+        for t in range(T):
+            acc = 0.0
+            for l in range(T - t):
+                acc += (gamma * lam) ** l * delta[t + l]
+            A[lo + t] = acc
+    return A, A + v
