@@ -1,0 +1,167 @@
+/*
+ * unity.h - C ABI of libunity: the per-token policy computation of a multi-agent PPO update
+ * (role-level advantages; grouped LM-head log-prob / entropy; PPO-clip + KL loss with backward)
+ * for one NVIDIA B200 (sm_100a).
+ *
+ * Conventions
+ * -----------
+ * - Every function returns an int status: 0 (UNITY_OK) or a negative UNITY_ERR_* code.  Nothing
+ *   throws, aborts or traps.  unity_last_error() gives a text for the last failure of a context.
+ * - Unless marked (host), data pointers are DEVICE pointers owned by the caller; the library never
+ *   frees or keeps them beyond the call.  Arrays marked (host) are read during the call.
+ * - Work is enqueued on the stream given to unity_create.  unity_logprob_fwd and
+ *   unity_ppo_loss_fwd_bwd synchronise that stream once, early, to read the K per-model row counts
+ *   (a few bytes) that size the grouped launches; everything else is asynchronous.  Device-side
+ *   errors (bad indices in the data, a bounded wait that expired) are sticky in a status word
+ *   read by unity_check_status.
+ * - The library allocates no device memory per call: all scratch lives in the caller's workspace.
+ * - Rows with tok_mask == 0 receive 0 in every per-token output and cost no tensor work.
+ * - Limits: 1 <= K <= UNITY_MAX_MODELS, 1 <= n_roles <= UNITY_MAX_ROLES, H % 64 == 0, V % 8 == 0,
+ *   hidden / W / dHidden / dW base addresses 16-byte aligned and densely packed (row pitch = H).
+ * - One context per stream; a context is not re-entrant.
+ */
+#ifndef UNITY_H_
+#define UNITY_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define UNITY_OK 0
+#define UNITY_ERR_INVALID_ARG (-1)   /* null pointer, negative size, parameter out of range      */
+#define UNITY_ERR_SHAPE (-2)         /* H, V, K, n_roles outside the limits above                */
+#define UNITY_ERR_ALIGNMENT (-3)     /* a matrix pointer is not 16-byte aligned                  */
+#define UNITY_ERR_WORKSPACE (-4)     /* workspace smaller than unity_workspace_bytes(...)        */
+#define UNITY_ERR_CUDA (-5)          /* a CUDA runtime / driver call failed                      */
+#define UNITY_ERR_UNSUPPORTED_ARCH (-6) /* device is not compute capability 10.x                 */
+#define UNITY_ERR_BAD_INDEX (-7)     /* device status: target / role / group / model id out of range;
+                                        the offending row or invocation was treated as masked    */
+#define UNITY_ERR_TIMEOUT (-8)       /* device status: a bounded in-kernel wait expired          */
+
+#define UNITY_MAX_MODELS 16
+#define UNITY_MAX_ROLES 64
+#define UNITY_N_METRICS 8            /* per class: n_valid, mean pg loss, mean KL, mean entropy,
+                                        clip fraction, mean ratio, mean logp, mean advantage     */
+
+typedef struct unity_ctx unity_ctx;
+
+/* Create a context bound to `device` and `cuda_stream` (a cudaStream_t; NULL = default stream).
+ * `workspace` is caller-owned device memory of `workspace_bytes` bytes (256-byte aligned) that the
+ * context uses as scratch until unity_destroy.  Fails with UNITY_ERR_UNSUPPORTED_ARCH off sm_100. */
+int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace, size_t workspace_bytes);
+int unity_destroy(unity_ctx* ctx);
+
+/* Scratch bytes that make every call with these sizes run with full-size chunks.  A smaller
+ * workspace still works down to unity_workspace_min_bytes (smaller gradient chunks). */
+size_t unity_workspace_bytes(int64_t n_tok, int32_t H, int32_t V, int32_t K, int32_t n_inv);
+size_t unity_workspace_min_bytes(int64_t n_tok, int32_t H, int32_t V, int32_t K, int32_t n_inv);
+
+/* Synchronise the stream, return the sticky device status (UNITY_OK, UNITY_ERR_BAD_INDEX,
+ * UNITY_ERR_TIMEOUT or UNITY_ERR_CUDA) and clear it. */
+int unity_check_status(unity_ctx* ctx);
+const char* unity_last_error(const unity_ctx* ctx);
+
+/* Number of kernels this context has launched since creation (for benchmark bookkeeping). */
+int64_t unity_launch_count(const unity_ctx* ctx);
+
+/* ------------------------------------------------------------------------------------------------
+ * Stage 1: role-level advantage.
+ *
+ * Per role invocation s with role v: r_s = lam[v][0]*r_node[s] + lam[v][1]*r_turn[s] +
+ * lam[v][2]*r_traj[inv_traj[s]]  - the additive node / turn / trajectory combination of Section
+ * "Agent-Specific Reward Interface" (the lambda-weighted equation), rewards being attributed to role
+ * invocations (Section "Optimization Objective and System Interface").  Then, per segment
+ * (rollout group g, role v) - role identity is kept even when roles share one model (Section
+ * "Parameter Sharing in the System") - with n members, mean mu and sigma = sqrt(sum (r-mu)^2 /
+ * (n-ddof)):  A_s = (r_s - mu) / (sigma + eps), and A_s = 0 when n-ddof <= 0 or sigma+eps == 0.
+ * Finally adv_tok[i] = A_{inv(i)} * tok_mask[i] for every response token of the invocation
+ * (paragraph "Batch construction": delayed rewards are aligned with token sequences).
+ *
+ *   inv_role, inv_group, inv_traj : int32 [n_inv]; an id out of range flags UNITY_ERR_BAD_INDEX and
+ *                                   the invocation is left out of the statistics with A = 0
+ *   r_node, r_turn : f32 [n_inv] or NULL (= 0);  r_traj : f32 [n_traj] or NULL (= 0)
+ *   lam            : (host) f32 [n_roles*3] (node, turn, traj) or NULL (= all 1)
+ *   cu_seqlens     : int64 [n_inv+1], non-decreasing, cu_seqlens[0] = 0, cu_seqlens[n_inv] = n_tok
+ *   tok_mask       : u8 [n_tok] or NULL (= all 1)
+ *   adv_inv        : out f32 [n_inv];  adv_tok : out f32 [n_tok] (NULL allowed when n_tok == 0)
+ *   seg_mean, seg_std : out f32 [n_groups*n_roles] or NULL; index g*n_roles+v; 0 for empty segments
+ * Deterministic: fixed-order reductions, no floating-point atomics.
+ */
+typedef struct {
+    float eps; /* default 1e-6 */
+    int ddof;  /* 0 (population) or 1 (sample) */
+} unity_adv_params;
+
+int unity_role_advantage(unity_ctx* ctx, int32_t n_inv, int32_t n_traj, int32_t n_roles, int32_t n_groups,
+                         const int32_t* inv_role, const int32_t* inv_group, const int32_t* inv_traj,
+                         const float* r_node, const float* r_turn, const float* r_traj, const float* lam,
+                         const unity_adv_params* params, int64_t n_tok, const int64_t* cu_seqlens,
+                         const uint8_t* tok_mask, float* adv_inv, float* adv_tok, float* seg_mean, float* seg_std);
+
+/* ------------------------------------------------------------------------------------------------
+ * Shared description of the response-token rows for stages 2 and 3.  Token i belongs to the
+ * invocation s with cu_seqlens[s] <= i < cu_seqlens[s+1]; its role is inv_role[s]; the model that
+ * serves it is role_model[role] - the agent-to-model mapping phi of Section "Agent--LLM Mapping"
+ * (full sharing, partial sharing, full separation are just different tables).
+ */
+typedef struct {
+    int64_t n_tok;
+    int32_t H, V, K, n_inv, n_roles;
+    const void* hidden;          /* bf16 [n_tok, H] row-major                                   */
+    const void* const* W;        /* (host) K device pointers, each bf16 [V, H] row-major        */
+    const int64_t* cu_seqlens;   /* int64 [n_inv+1]                                             */
+    const int32_t* inv_role;     /* int32 [n_inv]                                               */
+    const int32_t* role_model;   /* (host) int32 [n_roles], values in [0, K)                    */
+    const int32_t* target;       /* int32 [n_tok], 0 <= target < V (else BAD_INDEX, row masked) */
+    const uint8_t* tok_mask;     /* u8 [n_tok] or NULL (= all 1)                                */
+    float inv_temperature;       /* logits are multiplied by this; must be > 0; default 1       */
+} unity_rows;
+
+/* Stage 2: the log-probabilities every worker group evaluates for the old, reference and current
+ * policy (paragraph "Advantage computation and policy evaluation").  For each valid row, with
+ * z = inv_temperature * W_{model(i)} h_i over the whole vocabulary:
+ *   lse = log sum_v exp z_v ;  logp[i] = z_target - lse ;  entropy[i] = - sum_v p_v log p_v.
+ * The logits exist only in tensor memory; nothing of size n_tok x V is written.
+ *   logp : out f32 [n_tok];  entropy, lse : out f32 [n_tok] or NULL.
+ */
+int unity_logprob_fwd(unity_ctx* ctx, const unity_rows* rows, float* logp, float* entropy, float* lse);
+
+/* Stage 3: the PPO-style policy update of one batch (Section "PPO-Style Training Loop"; paragraph
+ * "Model-specific updates and synchronization": each model has its own loss and gradients).
+ * Per valid row, with logp and entropy H as in stage 2 and rho = exp(logp - old_logp):
+ *   pg  = max(-rho*A, -clip(rho, 1-clip_lo, 1+clip_hi)*A)            (ties take the unclipped branch)
+ *   d   = ref_logp - logp ;  kl = -d (mode 1) | d*d/2 (mode 2) | exp(d)-d-1 (mode 3)
+ *   l_i = pg + kl_coef*kl - ent_coef*H
+ *   loss[k] = (1/M_k) sum_{valid i of model k} l_i ,  M_k = norm[k] if given else max(#valid rows, 1)
+ * Backward: dHidden[i,:] = dL/dh_i (bf16, zeros on masked rows) and dW[k] = dL/dW_k (f32), where the
+ * logits are recomputed per vocabulary chunk; only a bounded chunk of logit gradients is ever stored.
+ *   old_logp, ref_logp, adv_tok : f32 [n_tok]
+ *   loss     : out f32 [K]
+ *   metrics  : out f32 [(K + n_roles) * UNITY_N_METRICS] or NULL: K per-model records then n_roles
+ *              per-role records (role metrics stay separate under parameter sharing)
+ *   logp, entropy, tok_loss : out f32 [n_tok] or NULL
+ *   dHidden  : out bf16 [n_tok, H];  dW : (host) K device pointers, each f32 [V, H]
+ * norm + accumulate_dW make gradient accumulation over micro-batches exact.
+ * Deterministic: no floating-point atomics anywhere.
+ */
+typedef struct {
+    float clip_lo, clip_hi; /* 0.2, 0.2 */
+    float kl_coef;
+    int kl_mode;            /* 1, 2 or 3 (default 3) */
+    float ent_coef;
+    const float* norm;      /* (host) f32 [K] or NULL */
+    int accumulate_dW;      /* 0: overwrite dW, 1: add to it */
+} unity_ppo_params;
+
+int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_ppo_params* params,
+                           const float* old_logp, const float* ref_logp, const float* adv_tok, float* loss,
+                           float* metrics, float* logp, float* entropy, float* tok_loss, void* dHidden,
+                           void* const* dW);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* UNITY_H_ */

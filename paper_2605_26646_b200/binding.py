@@ -1,0 +1,249 @@
+"""ctypes binding of libunity.so: argument marshalling only.
+
+Every function mirrors the C entry point of the same name in ``include/unity.h``; tensors are
+torch CUDA tensors whose ``data_ptr()`` is passed through, small host tables are python
+sequences.  No arithmetic of the path happens here, and there is no fallback: if the shared
+library cannot be loaded the import of a symbol raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import torch
+
+from . import build as _build
+
+UNITY_OK = 0
+ERR_NAMES = {0: "UNITY_OK", -1: "UNITY_ERR_INVALID_ARG", -2: "UNITY_ERR_SHAPE", -3: "UNITY_ERR_ALIGNMENT",
+             -4: "UNITY_ERR_WORKSPACE", -5: "UNITY_ERR_CUDA", -6: "UNITY_ERR_UNSUPPORTED_ARCH",
+             -7: "UNITY_ERR_BAD_INDEX", -8: "UNITY_ERR_TIMEOUT"}
+UNITY_MAX_MODELS = 16
+UNITY_MAX_ROLES = 64
+UNITY_N_METRICS = 8
+
+EXPORTS = ["unity_create", "unity_destroy", "unity_workspace_bytes", "unity_workspace_min_bytes",
+           "unity_check_status", "unity_last_error", "unity_launch_count", "unity_role_advantage",
+           "unity_logprob_fwd", "unity_ppo_loss_fwd_bwd"]
+
+
+class UnityError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"{ERR_NAMES.get(code, code)}: {msg}")
+        self.code = code
+
+
+class unity_adv_params(C.Structure):
+    _fields_ = [("eps", C.c_float), ("ddof", C.c_int)]
+
+
+class unity_rows(C.Structure):
+    _fields_ = [("n_tok", C.c_int64), ("H", C.c_int32), ("V", C.c_int32), ("K", C.c_int32),
+                ("n_inv", C.c_int32), ("n_roles", C.c_int32),
+                ("hidden", C.c_void_p), ("W", C.POINTER(C.c_void_p)), ("cu_seqlens", C.c_void_p),
+                ("inv_role", C.c_void_p), ("role_model", C.POINTER(C.c_int32)), ("target", C.c_void_p),
+                ("tok_mask", C.c_void_p), ("inv_temperature", C.c_float)]
+
+
+class unity_ppo_params(C.Structure):
+    _fields_ = [("clip_lo", C.c_float), ("clip_hi", C.c_float), ("kl_coef", C.c_float), ("kl_mode", C.c_int),
+                ("ent_coef", C.c_float), ("norm", C.POINTER(C.c_float)), ("accumulate_dW", C.c_int)]
+
+
+_LIB = None
+
+
+def load_library(path: Optional[str] = None) -> C.CDLL:
+    """Load (building first if the sources are newer) libunity.so.  Raises if that is impossible."""
+    global _LIB
+    if _LIB is not None and path is None:
+        return _LIB
+    if path is None:
+        path = _build.LIB_PATH
+        if _build.needs_build():
+            _build.build()
+    if not os.path.exists(path):
+        raise RuntimeError(f"libunity.so not found at {path}: build it with python -m paper_2605_26646_b200.build")
+    lib = C.CDLL(path)
+    vp, i32, i64, f32p = C.c_void_p, C.c_int32, C.c_int64, C.POINTER(C.c_float)
+    lib.unity_create.argtypes = [C.POINTER(vp), C.c_int, vp, vp, C.c_size_t]
+    lib.unity_create.restype = C.c_int
+    lib.unity_destroy.argtypes = [vp]
+    lib.unity_destroy.restype = C.c_int
+    for fn in (lib.unity_workspace_bytes, lib.unity_workspace_min_bytes):
+        fn.argtypes = [i64, i32, i32, i32, i32]
+        fn.restype = C.c_size_t
+    lib.unity_check_status.argtypes = [vp]
+    lib.unity_check_status.restype = C.c_int
+    lib.unity_last_error.argtypes = [vp]
+    lib.unity_last_error.restype = C.c_char_p
+    lib.unity_launch_count.argtypes = [vp]
+    lib.unity_launch_count.restype = i64
+    lib.unity_role_advantage.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, f32p,
+                                         C.POINTER(unity_adv_params), i64, vp, vp, vp, vp, vp, vp]
+    lib.unity_role_advantage.restype = C.c_int
+    lib.unity_logprob_fwd.argtypes = [vp, C.POINTER(unity_rows), vp, vp, vp]
+    lib.unity_logprob_fwd.restype = C.c_int
+    lib.unity_ppo_loss_fwd_bwd.argtypes = [vp, C.POINTER(unity_rows), C.POINTER(unity_ppo_params), vp, vp, vp,
+                                           vp, vp, vp, vp, vp, vp, C.POINTER(vp)]
+    lib.unity_ppo_loss_fwd_bwd.restype = C.c_int
+    if path == _build.LIB_PATH:
+        _LIB = lib
+    return lib
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None, name="tensor", host=False) -> Optional[int]:
+    if t is None:
+        return None
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name}: expected {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if not host and not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    return t.data_ptr()
+
+
+def _raise(ctx, code: int):
+    if code != UNITY_OK:
+        raise UnityError(code, load_library().unity_last_error(ctx).decode())
+
+
+# ------------------------------------------------------------------------------------------------
+# functions with the names of the C entry points
+# ------------------------------------------------------------------------------------------------
+def unity_workspace_bytes(n_tok: int, H: int, V: int, K: int, n_inv: int) -> int:
+    return int(load_library().unity_workspace_bytes(n_tok, H, V, K, n_inv))
+
+
+def unity_workspace_min_bytes(n_tok: int, H: int, V: int, K: int, n_inv: int) -> int:
+    return int(load_library().unity_workspace_min_bytes(n_tok, H, V, K, n_inv))
+
+
+def unity_create(device: int, stream_ptr: int, workspace: torch.Tensor) -> C.c_void_p:
+    ctx = C.c_void_p()
+    code = load_library().unity_create(C.byref(ctx), device, stream_ptr, workspace.data_ptr(),
+                                       workspace.numel() * workspace.element_size())
+    if code != UNITY_OK:
+        raise UnityError(code, "unity_create failed")
+    return ctx
+
+
+def unity_destroy(ctx) -> None:
+    load_library().unity_destroy(ctx)
+
+
+def unity_check_status(ctx) -> None:
+    _raise(ctx, load_library().unity_check_status(ctx))
+
+
+def unity_launch_count(ctx) -> int:
+    return int(load_library().unity_launch_count(ctx))
+
+
+def unity_role_advantage(ctx, n_traj: int, n_roles: int, n_groups: int, inv_role, inv_group, inv_traj,
+                         r_node, r_turn, r_traj, lam: Optional[Sequence[float]], eps: float, ddof: int,
+                         cu_seqlens, tok_mask, adv_inv, adv_tok, seg_mean=None, seg_std=None) -> None:
+    n_inv = int(inv_role.numel())
+    n_tok = int(adv_tok.numel()) if adv_tok is not None else 0
+    lam_arr = None
+    if lam is not None:
+        flat = [float(x) for row in lam for x in (row if hasattr(row, "__iter__") else [row])]
+        lam_arr = (C.c_float * len(flat))(*flat)
+    p = unity_adv_params(eps, ddof)
+    i32, f32 = torch.int32, torch.float32
+    code = load_library().unity_role_advantage(
+        ctx, n_inv, n_traj, n_roles, n_groups, _ptr(inv_role, i32, "inv_role"), _ptr(inv_group, i32, "inv_group"),
+        _ptr(inv_traj, i32, "inv_traj"), _ptr(r_node, f32, "r_node"), _ptr(r_turn, f32, "r_turn"),
+        _ptr(r_traj, f32, "r_traj"), lam_arr, C.byref(p), n_tok, _ptr(cu_seqlens, torch.int64, "cu_seqlens"),
+        _ptr(tok_mask, torch.uint8, "tok_mask"), _ptr(adv_inv, f32, "adv_inv"), _ptr(adv_tok, f32, "adv_tok"),
+        _ptr(seg_mean, f32, "seg_mean"), _ptr(seg_std, f32, "seg_std"))
+    _raise(ctx, code)
+
+
+def _make_rows(hidden, W, cu_seqlens, inv_role, role_model, target, tok_mask, inv_temperature, keep):
+    K = len(W)
+    n_tok, H = int(hidden.shape[0]), int(hidden.shape[1])
+    V = int(W[0].shape[0])
+    for k, w in enumerate(W):
+        if tuple(w.shape) != (V, H):
+            raise ValueError(f"W[{k}] has shape {tuple(w.shape)}, expected {(V, H)}")
+    Wp = (C.c_void_p * K)(*[_ptr(w, torch.bfloat16, "W") for w in W])
+    rm = (C.c_int32 * len(role_model))(*[int(x) for x in role_model])
+    keep.extend([Wp, rm])
+    rows = unity_rows(n_tok, H, V, K, int(inv_role.numel()), len(role_model),
+                      _ptr(hidden, torch.bfloat16, "hidden"), Wp, _ptr(cu_seqlens, torch.int64, "cu_seqlens"),
+                      _ptr(inv_role, torch.int32, "inv_role"), rm, _ptr(target, torch.int32, "target"),
+                      _ptr(tok_mask, torch.uint8, "tok_mask"), float(inv_temperature))
+    return rows
+
+
+def unity_logprob_fwd(ctx, hidden, W, cu_seqlens, inv_role, role_model, target, tok_mask, inv_temperature,
+                      logp, entropy=None, lse=None) -> None:
+    keep = []
+    rows = _make_rows(hidden, W, cu_seqlens, inv_role, role_model, target, tok_mask, inv_temperature, keep)
+    f32 = torch.float32
+    code = load_library().unity_logprob_fwd(ctx, C.byref(rows), _ptr(logp, f32, "logp"),
+                                            _ptr(entropy, f32, "entropy"), _ptr(lse, f32, "lse"))
+    _raise(ctx, code)
+
+
+def unity_ppo_loss_fwd_bwd(ctx, hidden, W, cu_seqlens, inv_role, role_model, target, tok_mask, inv_temperature,
+                           clip_lo, clip_hi, kl_coef, kl_mode, ent_coef, norm: Optional[Sequence[float]],
+                           accumulate_dW: bool, old_logp, ref_logp, adv_tok, loss, metrics, logp, entropy,
+                           tok_loss, dHidden, dW) -> None:
+    keep = []
+    rows = _make_rows(hidden, W, cu_seqlens, inv_role, role_model, target, tok_mask, inv_temperature, keep)
+    norm_arr = None
+    if norm is not None:
+        norm_arr = (C.c_float * len(norm))(*[float(x) for x in norm])
+    p = unity_ppo_params(clip_lo, clip_hi, kl_coef, kl_mode, ent_coef, norm_arr, 1 if accumulate_dW else 0)
+    dWp = (C.c_void_p * len(dW))(*[_ptr(g, torch.float32, "dW") for g in dW])
+    f32 = torch.float32
+    code = load_library().unity_ppo_loss_fwd_bwd(
+        ctx, C.byref(rows), C.byref(p), _ptr(old_logp, f32, "old_logp"), _ptr(ref_logp, f32, "ref_logp"),
+        _ptr(adv_tok, f32, "adv_tok"), _ptr(loss, f32, "loss"), _ptr(metrics, f32, "metrics"),
+        _ptr(logp, f32, "logp"), _ptr(entropy, f32, "entropy"), _ptr(tok_loss, f32, "tok_loss"),
+        _ptr(dHidden, torch.bfloat16, "dHidden"), dWp)
+    _raise(ctx, code)
+
+
+# ------------------------------------------------------------------------------------------------
+class Context:
+    """Owns a workspace tensor and a unity_ctx bound to a torch stream."""
+
+    def __init__(self, device: int = 0, workspace_bytes: int = 1 << 28, stream: Optional[torch.cuda.Stream] = None):
+        self.device = int(device)
+        with torch.cuda.device(self.device):
+            self.stream = stream or torch.cuda.current_stream()
+            self.workspace = torch.empty(int(workspace_bytes), dtype=torch.uint8, device=f"cuda:{self.device}")
+        self.ctx = unity_create(self.device, self.stream.cuda_stream, self.workspace)
+
+    def close(self):
+        if self.ctx is not None:
+            unity_destroy(self.ctx)
+            self.ctx = None
+            self.workspace = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def check_status(self):
+        unity_check_status(self.ctx)
+
+    @property
+    def launch_count(self) -> int:
+        return unity_launch_count(self.ctx)
+
+    def role_advantage(self, *a, **kw):
+        return unity_role_advantage(self.ctx, *a, **kw)
+
+    def logprob_fwd(self, *a, **kw):
+        return unity_logprob_fwd(self.ctx, *a, **kw)
+
+    def ppo_loss_fwd_bwd(self, *a, **kw):
+        return unity_ppo_loss_fwd_bwd(self.ctx, *a, **kw)

@@ -1,0 +1,147 @@
+// Internal declarations shared by the translation units of libunity (not part of the C ABI).
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "../../include/unity.h"
+
+namespace unity {
+
+constexpr int kTileM = 128;   // rows of the A operand per CTA tile (TMEM lanes)
+constexpr int kTileN = 256;   // rows of the B operand per CTA tile (TMEM columns per accumulator stage)
+constexpr int kTileK = 64;    // bf16 elements per shared-memory K slab (one 128-byte swizzle row)
+constexpr int kRouteBlock = 256;          // threads (= tokens) per block in the routing kernels
+constexpr long long kWaitBudgetCycles = 4000000000LL;   // ~2 s: bound of every in-kernel wait
+
+// Device status bits (sticky, ORed into the context's status word).
+constexpr int kStatusBadIndex = 1;
+constexpr int kStatusTimeout = 2;
+
+// ----------------------------------------------------------------------------------------------
+// GEMM  C[m, n] = sum_k A[m, k] * B[n, k]   (both operands K-major bf16, fp32 accumulation in TMEM)
+// ----------------------------------------------------------------------------------------------
+enum GemmEpilogue : int {
+    kEpiSoftmaxStats = 0,   // online (max, sum exp, sum exp*z, target logit) per row; nothing of size M x N stored
+    kEpiLogitGrad = 1,      // dL/dz in bf16 for a bounded (rows x vocab) chunk
+    kEpiAccumF32 = 2        // C (+)= acc, fp32, row-major
+};
+
+struct GemmArgs {
+    // tile grid and coordinates into the tensor maps
+    int m_tiles, n_tiles, k_iters;
+    int group_m;              // row tiles per raster group (consecutive units share these A tiles)
+    int a_row0, b_row0;       // first row of A / B (tensor-map coordinates) of tile (0, 0)
+    int a_k0, b_k0;           // first K element of A / B
+    int m_rows, n_cols;       // valid extent of C from (a_row0, b_row0): epilogue writes nothing beyond it
+    // kEpiSoftmaxStats: a unit is (row tile, vocabulary split); a CTA keeps a unit's running statistics
+    int n_splits, tiles_per_split;
+    float4* stats;            // [n_splits][stats_pitch], row relative to a_row0: (max acc, sum e, sum e*acc, target acc)
+    long long stats_pitch;
+    const int* target_p;      // [rows] packed targets (global vocabulary index), indexed from a_row0 + row
+    int vocab0;               // global vocabulary index of B row b_row0
+    float scale;              // inv_temperature (softmax) / unused otherwise
+    // kEpiLogitGrad
+    const float* coef_a;      // [rows] dL/dlogp * scale, packed order
+    const float* coef_b;      // [rows] dL/dentropy * scale
+    const float* row_lse;     // [rows]
+    const float* row_ent;     // [rows]
+    __nv_bfloat16* G;         // [m_rows, ldg] chunk-local
+    long long ldg;
+    // kEpiAccumF32
+    float* C;
+    long long ldc;
+    int beta;                 // 0: overwrite, 1: add to C
+    int* status;
+};
+
+cudaError_t launch_gemm(GemmEpilogue epi, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args,
+                        int sm_count, cudaStream_t stream);
+cudaError_t gemm_set_attributes();
+
+// ----------------------------------------------------------------------------------------------
+// streaming kernels (advantage, routing, token terms, transposes); each returns the launch error
+// ----------------------------------------------------------------------------------------------
+struct AdvArgs {
+    int n_inv, n_traj, n_roles, n_groups;
+    const int32_t *inv_role, *inv_group, *inv_traj;
+    const float *r_node, *r_turn, *r_traj;
+    int has_lam;
+    float lam[UNITY_MAX_ROLES * 3];
+    float eps;
+    int ddof;
+    long long n_tok;
+    const int64_t* cu_seqlens;
+    const uint8_t* tok_mask;
+    float *adv_inv, *adv_tok, *seg_mean, *seg_std;
+    float* r_scratch;   // [n_inv]
+    int* seg_scratch;   // [n_inv]
+    int* status;
+};
+cudaError_t launch_advantage(const AdvArgs& a, cudaStream_t stream, int* n_launches);
+
+struct RouteArgs {
+    long long n_tok;
+    int n_inv, n_roles, K, V;
+    const int64_t* cu_seqlens;
+    const int32_t* inv_role;
+    int32_t role_model[UNITY_MAX_ROLES];
+    const int32_t* target;
+    const uint8_t* tok_mask;
+    int n_blocks;                // ceil(n_tok / kRouteBlock)
+    int* blk_cnt;                // [n_blocks * K] -> exclusive prefix per model after the scan
+    int* counts;                 // [K] valid rows per model
+    int* offsets;                // [K+1] first slot of each model (multiples of kTileM), offsets[K] = total slots
+    int* tok_slot;               // [n_tok] slot of a token or -1
+    int* slot_tok;               // [max_slots] token of a slot or -1 (pre-filled with -1)
+    int8_t* tok_model;           // [n_tok] model id or -1
+    int* status;
+};
+cudaError_t launch_route(const RouteArgs& a, cudaStream_t stream, int* n_launches);
+
+cudaError_t launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* target, const int* slot_tok, int n_slots,
+                               int H, __nv_bfloat16* hp, int* target_p, cudaStream_t stream);
+
+// out[c, r] = in[r, c] for a bf16 matrix [rows, cols] with row pitch ld_in; out pitch ld_out.
+cudaError_t launch_transpose_bf16(const __nv_bfloat16* in, long long ld_in, __nv_bfloat16* out, long long ld_out,
+                                  int rows, int cols, cudaStream_t stream);
+
+struct TokenArgs {
+    int n_slots, n_splits, K, n_roles, n_inv;
+    long long n_tok;
+    const float4* stats;       // per model: base stats_base[k], pitch = padded rows of the model
+    long long stats_base[UNITY_MAX_MODELS];
+    int model_splits[UNITY_MAX_MODELS];
+    const int* slot_tok;
+    const int* tok_slot;
+    const int8_t* tok_model;
+    int offsets[UNITY_MAX_MODELS + 1];
+    float scale;               // inv_temperature
+    // forward outputs (packed and caller order)
+    float *row_lse, *row_ent, *row_logp;      // packed [n_slots]
+    float *logp, *entropy, *lse;              // caller order [n_tok], nullable
+    // loss part (null for logprob_fwd)
+    const float *old_logp, *ref_logp, *adv_tok;
+    float clip_lo, clip_hi, kl_coef, ent_coef;
+    int kl_mode;
+    float norm[UNITY_MAX_MODELS];   // M_k
+    float *coef_a, *coef_b;    // packed [n_slots], already multiplied by scale
+    float* tok_loss;           // caller order, nullable
+    const int64_t* cu_seqlens;
+    const int32_t* inv_role;
+    int32_t role_model[UNITY_MAX_ROLES];
+    float* inv_sums;           // [n_inv * 9]
+    float* loss;               // [K]
+    float* metrics;            // [(K + n_roles) * 8] nullable
+};
+cudaError_t launch_finish_forward(const TokenArgs& a, bool with_loss, cudaStream_t stream, int* n_launches);
+
+cudaError_t launch_zero_masked_rows(const int* tok_slot, long long n_tok, int H, __nv_bfloat16* dHidden,
+                                    cudaStream_t stream);
+// dHidden[slot_tok[slot0 + r], :] = bf16(dHc[r, :]) for r < n_rows with a token
+cudaError_t launch_store_dhidden(const float* dHc, const int* slot_tok, int slot0, int n_rows, int H,
+                                 __nv_bfloat16* dHidden, cudaStream_t stream);
+
+}  // namespace unity

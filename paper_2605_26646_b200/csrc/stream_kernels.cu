@@ -1,0 +1,500 @@
+// Streaming (HBM / latency bound) kernels of libunity: role-level advantage, routing of response
+// tokens to their model through the agent-to-model table, row packing, bf16 transposes, per-token PPO
+// terms with fixed-order reductions, and the dHidden write-back.  No floating-point atomics anywhere:
+// every reduction has a fixed order, so results are bitwise reproducible.
+#include "internal.h"
+
+namespace unity {
+
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+    return v;
+}
+__device__ __forceinline__ int warp_sum_int(int v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+    return v;
+}
+
+// Invocation that owns token `tok`: the s with cu[s] <= tok < cu[s+1] (zero-length invocations are skipped).
+__device__ __forceinline__ int find_invocation(const int64_t* __restrict__ cu, int n_inv, long long tok) {
+    int lo = 0, hi = n_inv;   // number of entries cu[1..n_inv] that are <= tok
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (cu[mid + 1] <= tok) lo = mid + 1; else hi = mid;
+    }
+    return min(lo, n_inv - 1);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Stage 1: advantage
+// ------------------------------------------------------------------------------------------------
+__global__ void k_adv_combine(AdvArgs a) {
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= a.n_inv) return;
+    const int v = a.inv_role[s], g = a.inv_group[s];
+    bool ok = (v >= 0 && v < a.n_roles && g >= 0 && g < a.n_groups);
+    float rj = 0.f;
+    if (a.r_traj != nullptr) {
+        const int t = a.inv_traj[s];
+        if (t >= 0 && t < a.n_traj) rj = a.r_traj[t]; else ok = false;
+    }
+    float r = 0.f;
+    int seg = -1;
+    if (ok) {
+        const float ln = a.has_lam ? a.lam[v * 3 + 0] : 1.f;
+        const float lt = a.has_lam ? a.lam[v * 3 + 1] : 1.f;
+        const float lj = a.has_lam ? a.lam[v * 3 + 2] : 1.f;
+        const float rn = a.r_node ? a.r_node[s] : 0.f;
+        const float rt = a.r_turn ? a.r_turn[s] : 0.f;
+        r = __fadd_rn(__fadd_rn(__fmul_rn(ln, rn), __fmul_rn(lt, rt)), __fmul_rn(lj, rj));
+        seg = g * a.n_roles + v;
+    } else {
+        atomicOr(a.status, kStatusBadIndex);
+    }
+    a.r_scratch[s] = r;
+    a.seg_scratch[s] = seg;
+    a.adv_inv[s] = 0.f;
+}
+
+// One warp per (group, role) segment.  Three sweeps over the invocation list with 128-bit loads:
+// count + sum -> mean; sum of squared deviations -> sigma; write the members' advantages.
+__global__ void k_adv_segment(AdvArgs a) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    const int n_seg = a.n_groups * a.n_roles;
+    if (warp >= n_seg) return;
+    const int q = warp;
+    const int n4 = a.n_inv >> 2;
+    const int4* seg4 = reinterpret_cast<const int4*>(a.seg_scratch);
+    const float4* r4 = reinterpret_cast<const float4*>(a.r_scratch);
+
+    int cnt = 0;
+    float sum = 0.f;
+    for (int i = lane; i < n4; i += 32) {
+        const int4 sg = seg4[i];
+        if (sg.x == q || sg.y == q || sg.z == q || sg.w == q) {
+            const float4 r = r4[i];
+            if (sg.x == q) { cnt++; sum += r.x; }
+            if (sg.y == q) { cnt++; sum += r.y; }
+            if (sg.z == q) { cnt++; sum += r.z; }
+            if (sg.w == q) { cnt++; sum += r.w; }
+        }
+    }
+    for (int s = (n4 << 2) + lane; s < a.n_inv; s += 32)
+        if (a.seg_scratch[s] == q) { cnt++; sum += a.r_scratch[s]; }
+    cnt = warp_sum_int(cnt);
+    sum = warp_sum(sum);
+    const float mu = cnt > 0 ? sum / static_cast<float>(cnt) : 0.f;
+
+    float m2 = 0.f;
+    for (int i = lane; i < n4; i += 32) {
+        const int4 sg = seg4[i];
+        if (sg.x == q || sg.y == q || sg.z == q || sg.w == q) {
+            const float4 r = r4[i];
+            if (sg.x == q) { const float d = r.x - mu; m2 += d * d; }
+            if (sg.y == q) { const float d = r.y - mu; m2 += d * d; }
+            if (sg.z == q) { const float d = r.z - mu; m2 += d * d; }
+            if (sg.w == q) { const float d = r.w - mu; m2 += d * d; }
+        }
+    }
+    for (int s = (n4 << 2) + lane; s < a.n_inv; s += 32)
+        if (a.seg_scratch[s] == q) { const float d = a.r_scratch[s] - mu; m2 += d * d; }
+    m2 = warp_sum(m2);
+
+    const int dof = cnt - a.ddof;
+    const float sigma = dof > 0 ? sqrtf(m2 / static_cast<float>(dof)) : 0.f;
+    const float denom = sigma + a.eps;
+    if (lane == 0) {
+        if (a.seg_mean) a.seg_mean[q] = mu;
+        if (a.seg_std) a.seg_std[q] = sigma;
+    }
+    if (cnt == 0) return;
+    for (int s = lane; s < a.n_inv; s += 32)
+        if (a.seg_scratch[s] == q) a.adv_inv[s] = (dof > 0 && denom != 0.f) ? (a.r_scratch[s] - mu) / denom : 0.f;
+}
+
+// Four tokens per thread: one 32-bit mask load, one 128-bit store.
+__global__ void k_adv_broadcast(AdvArgs a) {
+    const long long i0 = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) * 4;
+    if (i0 >= a.n_tok) return;
+    int s = find_invocation(a.cu_seqlens, a.n_inv, i0);
+    long long end = a.cu_seqlens[s + 1];
+    float adv = a.adv_inv[s];
+    float out[4];
+    const int n = static_cast<int>(min(4LL, a.n_tok - i0));
+    unsigned m4 = 0x01010101u;
+    const bool mask_al = (reinterpret_cast<uintptr_t>(a.tok_mask) & 3) == 0;
+    const bool out_al = (reinterpret_cast<uintptr_t>(a.adv_tok) & 15) == 0;
+    if (a.tok_mask) {
+        if (n == 4 && mask_al) m4 = *reinterpret_cast<const unsigned*>(a.tok_mask + i0);
+        else { m4 = 0; for (int j = 0; j < n; ++j) m4 |= static_cast<unsigned>(a.tok_mask[i0 + j]) << (8 * j); }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const long long i = i0 + j;
+        if (j < n) {
+            while (i >= end && s + 1 < a.n_inv) { ++s; end = a.cu_seqlens[s + 1]; adv = a.adv_inv[s]; }
+            out[j] = ((m4 >> (8 * j)) & 0xffu) ? adv : 0.f;
+        } else out[j] = 0.f;
+    }
+    if (n == 4 && out_al) *reinterpret_cast<float4*>(a.adv_tok + i0) = make_float4(out[0], out[1], out[2], out[3]);
+    else for (int j = 0; j < n; ++j) a.adv_tok[i0 + j] = out[j];
+}
+
+// ------------------------------------------------------------------------------------------------
+// Routing: stable partition of the valid tokens by model id (count, scan, assign)
+// ------------------------------------------------------------------------------------------------
+__global__ void k_route_count(RouteArgs a) {
+    __shared__ int cnt[UNITY_MAX_MODELS];
+    if (threadIdx.x < UNITY_MAX_MODELS) cnt[threadIdx.x] = 0;
+    __syncthreads();
+    const long long i = static_cast<long long>(blockIdx.x) * kRouteBlock + threadIdx.x;
+    if (i < a.n_tok) {
+        int model = -1;
+        const bool on = a.tok_mask ? (a.tok_mask[i] != 0) : true;
+        if (on) {
+            const int s = find_invocation(a.cu_seqlens, a.n_inv, i);
+            const int role = a.inv_role[s];
+            const int tgt = a.target[i];
+            if (role >= 0 && role < a.n_roles && tgt >= 0 && tgt < a.V) {
+                model = a.role_model[role];
+                if (model < 0 || model >= a.K) model = -1;
+            }
+            if (model < 0) atomicOr(a.status, kStatusBadIndex);
+            else atomicAdd(&cnt[model], 1);
+        }
+        a.tok_model[i] = static_cast<int8_t>(model);
+    }
+    __syncthreads();
+    if (threadIdx.x < a.K) a.blk_cnt[blockIdx.x * a.K + threadIdx.x] = cnt[threadIdx.x];
+}
+
+// One block: exclusive scan of the per-block counts of each model; then slot offsets padded to the row tile.
+__global__ void k_route_scan(RouteArgs a) {
+    __shared__ int part[1024];
+    __shared__ int total[UNITY_MAX_MODELS];
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int per = (a.n_blocks + nt - 1) / nt;
+    const int b0 = tid * per, b1 = min(b0 + per, a.n_blocks);
+    for (int k = 0; k < a.K; ++k) {
+        int s = 0;
+        for (int b = b0; b < b1; ++b) s += a.blk_cnt[b * a.K + k];
+        part[tid] = s;
+        __syncthreads();
+        for (int off = 1; off < nt; off <<= 1) {     // inclusive Hillis-Steele scan of the thread sums
+            const int v = (tid >= off) ? part[tid - off] : 0;
+            __syncthreads();
+            part[tid] += v;
+            __syncthreads();
+        }
+        int run = part[tid] - s;
+        if (tid == nt - 1) total[k] = part[tid];
+        for (int b = b0; b < b1; ++b) { const int c = a.blk_cnt[b * a.K + k]; a.blk_cnt[b * a.K + k] = run; run += c; }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        int off = 0;
+        for (int k = 0; k < a.K; ++k) {
+            a.counts[k] = total[k];
+            a.offsets[k] = off;
+            off += (total[k] + kTileM - 1) / kTileM * kTileM;
+        }
+        a.offsets[a.K] = off;
+    }
+}
+
+__global__ void k_route_assign(RouteArgs a) {
+    __shared__ int warp_cnt[kRouteBlock / 32][UNITY_MAX_MODELS];
+    const long long i = static_cast<long long>(blockIdx.x) * kRouteBlock + threadIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int model = (i < a.n_tok) ? a.tok_model[i] : -1;
+    int rank = 0;
+    for (int k = 0; k < a.K; ++k) {
+        const unsigned bal = __ballot_sync(kFull, model == k);
+        if (model == k) rank = __popc(bal & ((1u << lane) - 1u));
+        if (lane == 0) warp_cnt[warp][k] = __popc(bal);
+    }
+    __syncthreads();
+    if (i >= a.n_tok) return;
+    if (model < 0) { a.tok_slot[i] = -1; return; }
+    int before = 0;
+    for (int w = 0; w < warp; ++w) before += warp_cnt[w][model];
+    const int slot = a.offsets[model] + a.blk_cnt[blockIdx.x * a.K + model] + before + rank;
+    a.tok_slot[i] = slot;
+    a.slot_tok[slot] = static_cast<int>(i);
+}
+
+// One warp per packed row: 128-bit copies of the hidden row (zeros for padding slots).
+__global__ void k_gather_rows(const __nv_bfloat16* __restrict__ hidden, const int32_t* __restrict__ target,
+                              const int* __restrict__ slot_tok, int n_slots, int H, __nv_bfloat16* __restrict__ hp,
+                              int* __restrict__ target_p) {
+    const int slot = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (slot >= n_slots) return;
+    const int tok = slot_tok[slot];
+    const int n16 = H >> 3;
+    uint4* dst = reinterpret_cast<uint4*>(hp + static_cast<long long>(slot) * H);
+    if (tok >= 0) {
+        const uint4* src = reinterpret_cast<const uint4*>(hidden + static_cast<long long>(tok) * H);
+        for (int j = lane; j < n16; j += 32) dst[j] = src[j];
+    } else {
+        for (int j = lane; j < n16; j += 32) dst[j] = make_uint4(0, 0, 0, 0);
+    }
+    if (lane == 0) target_p[slot] = tok >= 0 ? target[tok] : 0;
+}
+
+// 64 x 64 bf16 tile transpose through shared memory; 32-bit accesses on both sides.
+__global__ void k_transpose_bf16(const __nv_bfloat16* __restrict__ in, long long ld_in, __nv_bfloat16* __restrict__ out,
+                                 long long ld_out, int rows, int cols) {
+    __shared__ __nv_bfloat16 tile[64][66];
+    const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;     // 32 x 8 threads
+    for (int rr = ty; rr < 64; rr += 8) {
+        const int r = r0 + rr, c = c0 + tx * 2;
+        __nv_bfloat162 v = __floats2bfloat162_rn(0.f, 0.f);
+        if (r < rows) {
+            if (c + 1 < cols) v = *reinterpret_cast<const __nv_bfloat162*>(in + static_cast<long long>(r) * ld_in + c);
+            else if (c < cols) v.x = in[static_cast<long long>(r) * ld_in + c];
+        }
+        tile[rr][tx * 2] = v.x;
+        tile[rr][tx * 2 + 1] = v.y;
+    }
+    __syncthreads();
+    for (int cc = ty; cc < 64; cc += 8) {
+        const int c = c0 + cc, r = r0 + tx * 2;
+        if (c >= cols) continue;
+        __nv_bfloat162 v;
+        v.x = tile[tx * 2][cc];
+        v.y = tile[tx * 2 + 1][cc];
+        if (r + 1 < rows) *reinterpret_cast<__nv_bfloat162*>(out + static_cast<long long>(c) * ld_out + r) = v;
+        else if (r < rows) out[static_cast<long long>(c) * ld_out + r] = v.x;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Per-token PPO terms
+// ------------------------------------------------------------------------------------------------
+struct PpoTerms {
+    float rho, pg, kl, tok_loss, dl_dlogp, clipped;
+};
+__device__ __forceinline__ PpoTerms ppo_terms(float logp, float ent, float old_lp, float ref_lp, float adv,
+                                              float clip_lo, float clip_hi, float kl_coef, int kl_mode,
+                                              float ent_coef) {
+    PpoTerms t;
+    t.rho = expf(logp - old_lp);
+    const float rho_c = fminf(fmaxf(t.rho, 1.f - clip_lo), 1.f + clip_hi);
+    const float unclipped = -t.rho * adv, clipped = -rho_c * adv;
+    const bool u = unclipped >= clipped;     // ties take the unclipped branch
+    t.pg = u ? unclipped : clipped;
+    t.clipped = u ? 0.f : 1.f;
+    const float d = ref_lp - logp;
+    float dkl;
+    if (kl_mode == 1) { t.kl = -d; dkl = 1.f; }
+    else if (kl_mode == 2) { t.kl = 0.5f * d * d; dkl = -d; }
+    else { const float e = expm1f(d); t.kl = e - d; dkl = -e; }
+    t.tok_loss = t.pg + kl_coef * t.kl - ent_coef * ent;
+    t.dl_dlogp = (u ? -adv * t.rho : 0.f) + kl_coef * dkl;
+    return t;
+}
+
+// One thread per packed row: merge the vocabulary splits, form lse / entropy / logp, then the loss terms.
+__global__ void k_finish_rows(TokenArgs a, int with_loss) {
+    const int slot = blockIdx.x * blockDim.x + threadIdx.x;
+    if (slot >= a.n_slots) return;
+    const int tok = a.slot_tok[slot];
+    if (tok < 0) {
+        a.row_lse[slot] = 0.f; a.row_ent[slot] = 0.f; a.row_logp[slot] = 0.f;
+        if (with_loss) { a.coef_a[slot] = 0.f; a.coef_b[slot] = 0.f; }
+        return;
+    }
+    const int k = a.tok_model[tok];
+    const long long pitch = a.offsets[k + 1] - a.offsets[k];
+    const float4* st = a.stats + a.stats_base[k] + (slot - a.offsets[k]);
+    const int n_splits = a.model_splits[k];
+    const float c = a.scale * 1.4426950408889634f;    // exp(scale*x) = exp2(c*x)
+    float m = -3.0e38f;
+    for (int j = 0; j < n_splits; ++j) m = fmaxf(m, st[j * pitch].x);
+    float s = 0.f, t = 0.f, zy = -3.0e38f;
+    for (int j = 0; j < n_splits; ++j) {
+        const float4 p = st[j * pitch];
+        const float w = exp2f((p.x - m) * c);
+        s += p.y * w;
+        t += p.z * w;
+        zy = fmaxf(zy, p.w);
+    }
+    const float lse = a.scale * m + logf(s);
+    const float ent = lse - a.scale * (t / s);
+    const float logp = a.scale * zy - lse;
+    a.row_lse[slot] = lse; a.row_ent[slot] = ent; a.row_logp[slot] = logp;
+    if (a.logp) a.logp[tok] = logp;
+    if (a.entropy) a.entropy[tok] = ent;
+    if (a.lse) a.lse[tok] = lse;
+    if (!with_loss) return;
+    const float Mk = a.norm[k];
+    const PpoTerms p = ppo_terms(logp, ent, a.old_logp[tok], a.ref_logp[tok], a.adv_tok[tok], a.clip_lo, a.clip_hi,
+                                 a.kl_coef, a.kl_mode, a.ent_coef);
+    a.coef_a[slot] = a.scale * (p.dl_dlogp / Mk);
+    a.coef_b[slot] = a.scale * (-a.ent_coef / Mk);
+    if (a.tok_loss) a.tok_loss[tok] = p.tok_loss;
+}
+
+// One warp per invocation: nine sums over its valid tokens in a fixed order.
+__global__ void k_inv_reduce(TokenArgs a) {
+    const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (s >= a.n_inv) return;
+    float acc[9];
+#pragma unroll
+    for (int j = 0; j < 9; ++j) acc[j] = 0.f;
+    const long long lo = a.cu_seqlens[s], hi = a.cu_seqlens[s + 1];
+    for (long long i = lo + lane; i < hi; i += 32) {
+        const int slot = a.tok_slot[i];
+        if (slot < 0) continue;
+        const float logp = a.row_logp[slot], ent = a.row_ent[slot], adv = a.adv_tok[i];
+        const PpoTerms p = ppo_terms(logp, ent, a.old_logp[i], a.ref_logp[i], adv, a.clip_lo, a.clip_hi, a.kl_coef,
+                                     a.kl_mode, a.ent_coef);
+        acc[0] += 1.f; acc[1] += p.pg; acc[2] += p.kl; acc[3] += ent; acc[4] += p.clipped; acc[5] += p.rho;
+        acc[6] += logp; acc[7] += adv; acc[8] += p.tok_loss;
+    }
+#pragma unroll
+    for (int j = 0; j < 9; ++j) acc[j] = warp_sum(acc[j]);
+    if (lane == 0)
+        for (int j = 0; j < 9; ++j) a.inv_sums[s * 9 + j] = acc[j];
+}
+
+// One warp per class (K models, then n_roles roles): fixed-order sum over the invocations of the class.
+__global__ void k_class_reduce(TokenArgs a) {
+    const int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (c >= a.K + a.n_roles) return;
+    float acc[9];
+#pragma unroll
+    for (int j = 0; j < 9; ++j) acc[j] = 0.f;
+    for (int s = lane; s < a.n_inv; s += 32) {
+        const int role = a.inv_role[s];
+        if (role < 0 || role >= a.n_roles) continue;
+        const bool mine = (c < a.K) ? (a.role_model[role] == c) : (role == c - a.K);
+        if (!mine) continue;
+#pragma unroll
+        for (int j = 0; j < 9; ++j) acc[j] += a.inv_sums[s * 9 + j];
+    }
+#pragma unroll
+    for (int j = 0; j < 9; ++j) acc[j] = warp_sum(acc[j]);
+    if (lane != 0) return;
+    const float dn = fmaxf(acc[0], 1.f);
+    if (a.metrics) {
+        float* m = a.metrics + c * UNITY_N_METRICS;
+        m[0] = acc[0];
+        for (int j = 1; j < 8; ++j) m[j] = acc[j] / dn;
+    }
+    if (c < a.K) a.loss[c] = acc[8] / a.norm[c];
+}
+
+__global__ void k_zero_masked_rows(const int* __restrict__ tok_slot, long long n_tok, int H,
+                                   __nv_bfloat16* __restrict__ dHidden) {
+    const long long tok = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (tok >= n_tok || tok_slot[tok] >= 0) return;
+    uint4* dst = reinterpret_cast<uint4*>(dHidden + tok * H);
+    for (int j = lane; j < (H >> 3); j += 32) dst[j] = make_uint4(0, 0, 0, 0);
+}
+
+__global__ void k_store_dhidden(const float* __restrict__ dHc, const int* __restrict__ slot_tok, int slot0, int n_rows,
+                                int H, __nv_bfloat16* __restrict__ dHidden) {
+    const int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (r >= n_rows) return;
+    const int tok = slot_tok[slot0 + r];
+    if (tok < 0) return;
+    const float4* src = reinterpret_cast<const float4*>(dHc + static_cast<long long>(r) * H);
+    uint2* dst = reinterpret_cast<uint2*>(dHidden + static_cast<long long>(tok) * H);
+    for (int j = lane; j < (H >> 2); j += 32) {
+        const float4 v = src[j];
+        __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+        uint2 o;
+        o.x = *reinterpret_cast<unsigned*>(&lo);
+        o.y = *reinterpret_cast<unsigned*>(&hi);
+        dst[j] = o;
+    }
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------
+// launchers
+// ------------------------------------------------------------------------------------------------
+cudaError_t launch_advantage(const AdvArgs& a, cudaStream_t stream, int* n_launches) {
+    if (a.n_inv > 0) {
+        k_adv_combine<<<(a.n_inv + 255) / 256, 256, 0, stream>>>(a);
+        const int n_seg = a.n_groups * a.n_roles;
+        k_adv_segment<<<(n_seg + 7) / 8, 256, 0, stream>>>(a);
+        *n_launches += 2;
+    }
+    if (a.n_tok > 0) {
+        const long long quads = (a.n_tok + 3) / 4;
+        k_adv_broadcast<<<static_cast<unsigned>((quads + 255) / 256), 256, 0, stream>>>(a);
+        *n_launches += 1;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_route(const RouteArgs& a, cudaStream_t stream, int* n_launches) {
+    k_route_count<<<a.n_blocks, kRouteBlock, 0, stream>>>(a);
+    k_route_scan<<<1, 1024, 0, stream>>>(a);
+    k_route_assign<<<a.n_blocks, kRouteBlock, 0, stream>>>(a);
+    *n_launches += 3;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* target, const int* slot_tok, int n_slots,
+                               int H, __nv_bfloat16* hp, int* target_p, cudaStream_t stream) {
+    if (n_slots == 0) return cudaSuccess;
+    k_gather_rows<<<(n_slots + 7) / 8, 256, 0, stream>>>(hidden, target, slot_tok, n_slots, H, hp, target_p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_transpose_bf16(const __nv_bfloat16* in, long long ld_in, __nv_bfloat16* out, long long ld_out,
+                                  int rows, int cols, cudaStream_t stream) {
+    if (rows == 0 || cols == 0) return cudaSuccess;
+    dim3 grid((cols + 63) / 64, (rows + 63) / 64);
+    k_transpose_bf16<<<grid, 256, 0, stream>>>(in, ld_in, out, ld_out, rows, cols);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_finish_forward(const TokenArgs& a, bool with_loss, cudaStream_t stream, int* n_launches) {
+    if (a.n_slots > 0) {
+        k_finish_rows<<<(a.n_slots + 255) / 256, 256, 0, stream>>>(a, with_loss ? 1 : 0);
+        *n_launches += 1;
+    }
+    if (with_loss) {
+        if (a.n_inv > 0) {
+            k_inv_reduce<<<(a.n_inv + 7) / 8, 256, 0, stream>>>(a);
+            *n_launches += 1;
+        }
+        k_class_reduce<<<(a.K + a.n_roles + 7) / 8, 256, 0, stream>>>(a);
+        *n_launches += 1;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_zero_masked_rows(const int* tok_slot, long long n_tok, int H, __nv_bfloat16* dHidden,
+                                    cudaStream_t stream) {
+    if (n_tok == 0) return cudaSuccess;
+    k_zero_masked_rows<<<static_cast<unsigned>((n_tok + 7) / 8), 256, 0, stream>>>(tok_slot, n_tok, H, dHidden);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_store_dhidden(const float* dHc, const int* slot_tok, int slot0, int n_rows, int H,
+                                 __nv_bfloat16* dHidden, cudaStream_t stream) {
+    if (n_rows == 0) return cudaSuccess;
+    k_store_dhidden<<<(n_rows + 7) / 8, 256, 0, stream>>>(dHc, slot_tok, slot0, n_rows, H, dHidden);
+    return cudaGetLastError();
+}
+
+}  // namespace unity

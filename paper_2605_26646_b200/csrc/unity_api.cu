@@ -1,0 +1,545 @@
+// C ABI of libunity: argument validation, workspace carving and the launch sequence of each call.
+// All arithmetic of the path runs in the kernels of stream_kernels.cu and gemm_tcgen05.cu.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "internal.h"
+
+using namespace unity;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct unity_ctx {
+    int device;
+    cudaStream_t stream;
+    char* ws;
+    size_t ws_bytes;
+    int* d_status;        // device status word
+    int* h_pinned;        // pinned host staging for the per-model counts and the status word
+    int sm_count;
+    EncodeTiledFn encode;
+    long long launches;
+    char err[512];
+};
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kChunkRows = 16384;    // token rows per gradient chunk (multiple of kTileM)
+constexpr int kChunkVocab = 8192;    // vocabulary entries per gradient chunk (multiple of kTileN)
+constexpr int kMinChunkRows = 1024;
+constexpr int kMinChunkVocab = 1024;
+
+inline size_t up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int fail(unity_ctx* ctx, int code, const char* fmt, ...) {
+    if (ctx) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(ctx->err, sizeof(ctx->err), fmt, ap);
+        va_end(ap);
+    }
+    return code;
+}
+#define CUDA_TRY(ctx, expr)                                                                              \
+    do {                                                                                                 \
+        cudaError_t e_ = (expr);                                                                         \
+        if (e_ != cudaSuccess) return fail(ctx, UNITY_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e_)); \
+    } while (0)
+
+struct Bump {
+    char* base;
+    size_t off, cap;
+    bool ok;
+    template <typename T> T* take(size_t n) {
+        off = up(off, kAlign);
+        T* p = reinterpret_cast<T*>(base + off);
+        off += n * sizeof(T);
+        if (off > cap) ok = false;
+        return p;
+    }
+};
+
+struct Layout {
+    // routing + forward
+    int* tok_slot; int* slot_tok; int8_t* tok_model; int* blk_cnt; int* counts; int* offsets;
+    __nv_bfloat16* hp; int* target_p; float4* stats; float *row_lse, *row_ent, *row_logp;
+    // loss + backward
+    float *coef_a, *coef_b, *inv_sums;
+    __nv_bfloat16 *hT, *WT, *G, *GT; float* dHc;
+    long long max_slots, stats_cap;
+    int n_blocks, chunk_rows, chunk_vocab;
+    size_t bytes;
+};
+
+long long max_slots_of(long long n_tok, int K) { return static_cast<long long>(up(n_tok, kTileM)) + static_cast<long long>(kTileM) * K; }
+
+// Carve the workspace.  chunk_rows / chunk_vocab are the wanted gradient chunk sizes (0 = forward only).
+Layout carve(char* base, size_t cap, long long n_tok, int H, int V, int K, int n_inv, int chunk_rows, int chunk_vocab,
+             bool* fits) {
+    Layout L;
+    memset(&L, 0, sizeof(L));
+    Bump b{base, 0, cap, true};
+    L.max_slots = max_slots_of(n_tok, K);
+    L.n_blocks = static_cast<int>((n_tok + kRouteBlock - 1) / kRouteBlock);
+    L.stats_cap = 4 * L.max_slots + 94720LL * K;
+    L.tok_slot = b.take<int>(n_tok);
+    L.slot_tok = b.take<int>(L.max_slots);
+    L.tok_model = b.take<int8_t>(n_tok);
+    L.blk_cnt = b.take<int>(static_cast<size_t>(L.n_blocks) * K + 1);
+    L.counts = b.take<int>(UNITY_MAX_MODELS);
+    L.offsets = b.take<int>(UNITY_MAX_MODELS + 1);
+    L.hp = b.take<__nv_bfloat16>(static_cast<size_t>(L.max_slots) * H);
+    L.target_p = b.take<int>(L.max_slots);
+    L.stats = b.take<float4>(L.stats_cap);
+    L.row_lse = b.take<float>(L.max_slots);
+    L.row_ent = b.take<float>(L.max_slots);
+    L.row_logp = b.take<float>(L.max_slots);
+    L.chunk_rows = chunk_rows;
+    L.chunk_vocab = chunk_vocab;
+    if (chunk_rows > 0) {
+        L.coef_a = b.take<float>(L.max_slots);
+        L.coef_b = b.take<float>(L.max_slots);
+        L.inv_sums = b.take<float>(static_cast<size_t>(n_inv) * 9 + 1);
+        L.hT = b.take<__nv_bfloat16>(static_cast<size_t>(H) * L.max_slots);
+        L.WT = b.take<__nv_bfloat16>(static_cast<size_t>(H) * V);
+        L.G = b.take<__nv_bfloat16>(static_cast<size_t>(chunk_rows) * chunk_vocab);
+        L.GT = b.take<__nv_bfloat16>(static_cast<size_t>(chunk_rows) * chunk_vocab);
+        L.dHc = b.take<float>(static_cast<size_t>(chunk_rows) * H);
+    }
+    L.bytes = up(b.off, kAlign);
+    if (fits) *fits = b.ok;
+    return L;
+}
+
+int wanted_chunk_rows(long long n_tok, int K) {
+    const long long ms = max_slots_of(n_tok, K);
+    return static_cast<int>(ms < kChunkRows ? ms : kChunkRows);
+}
+int wanted_chunk_vocab(int V) {
+    const long long vp = static_cast<long long>(up(V, kTileN));
+    return static_cast<int>(vp < kChunkVocab ? vp : kChunkVocab);
+}
+
+int make_tmap(unity_ctx* ctx, CUtensorMap* tm, const void* ptr, uint64_t inner, uint64_t rows, uint64_t pitch_bytes,
+              uint32_t box_rows) {
+    cuuint64_t dims[2] = {inner, rows};
+    cuuint64_t strides[1] = {pitch_bytes};
+    cuuint32_t box[2] = {static_cast<cuuint32_t>(kTileK), box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = ctx->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+        return fail(ctx, UNITY_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d): inner=%llu rows=%llu pitch=%llu", (int)r,
+                    (unsigned long long)inner, (unsigned long long)rows, (unsigned long long)pitch_bytes);
+    return UNITY_OK;
+}
+
+int validate_rows(unity_ctx* ctx, const unity_rows* r) {
+    if (!ctx) return UNITY_ERR_INVALID_ARG;
+    if (!r) return fail(ctx, UNITY_ERR_INVALID_ARG, "rows is NULL");
+    if (r->n_tok < 0 || r->n_inv < 0) return fail(ctx, UNITY_ERR_INVALID_ARG, "negative size");
+    if (r->n_tok > 0x7fffff00LL) return fail(ctx, UNITY_ERR_SHAPE, "n_tok too large");
+    if (r->K < 1 || r->K > UNITY_MAX_MODELS) return fail(ctx, UNITY_ERR_SHAPE, "K=%d outside [1,%d]", r->K, UNITY_MAX_MODELS);
+    if (r->n_roles < 1 || r->n_roles > UNITY_MAX_ROLES)
+        return fail(ctx, UNITY_ERR_SHAPE, "n_roles=%d outside [1,%d]", r->n_roles, UNITY_MAX_ROLES);
+    if (r->H < 64 || r->H % 64 != 0) return fail(ctx, UNITY_ERR_SHAPE, "H=%d must be a positive multiple of 64", r->H);
+    if (r->V < 8 || r->V % 8 != 0) return fail(ctx, UNITY_ERR_SHAPE, "V=%d must be a positive multiple of 8", r->V);
+    if (!(r->inv_temperature > 0.f)) return fail(ctx, UNITY_ERR_INVALID_ARG, "inv_temperature must be > 0");
+    if (!r->W || !r->role_model) return fail(ctx, UNITY_ERR_INVALID_ARG, "W / role_model is NULL");
+    if (r->n_tok > 0 && (!r->hidden || !r->cu_seqlens || !r->inv_role || !r->target || r->n_inv < 1))
+        return fail(ctx, UNITY_ERR_INVALID_ARG, "hidden / cu_seqlens / inv_role / target is NULL or n_inv < 1");
+    if (reinterpret_cast<uintptr_t>(r->hidden) & 15) return fail(ctx, UNITY_ERR_ALIGNMENT, "hidden not 16-byte aligned");
+    for (int k = 0; k < r->K; ++k) {
+        if (!r->W[k]) return fail(ctx, UNITY_ERR_INVALID_ARG, "W[%d] is NULL", k);
+        if (reinterpret_cast<uintptr_t>(r->W[k]) & 15) return fail(ctx, UNITY_ERR_ALIGNMENT, "W[%d] not 16-byte aligned", k);
+    }
+    for (int v = 0; v < r->n_roles; ++v)
+        if (r->role_model[v] < 0 || r->role_model[v] >= r->K)
+            return fail(ctx, UNITY_ERR_INVALID_ARG, "role_model[%d]=%d outside [0,%d)", v, r->role_model[v], r->K);
+    return UNITY_OK;
+}
+
+struct RowPlan {
+    Layout L;
+    int counts[UNITY_MAX_MODELS];
+    int offsets[UNITY_MAX_MODELS + 1];
+    int splits[UNITY_MAX_MODELS];
+    long long stats_base[UNITY_MAX_MODELS];
+    int n_slots;
+};
+
+// Routing, packing and the forward sweep: fills per-split softmax statistics for every packed row.
+int forward_sweep(unity_ctx* ctx, const unity_rows* r, RowPlan& P) {
+    const Layout& L = P.L;
+    cudaStream_t st = ctx->stream;
+    int nl = 0;
+    CUDA_TRY(ctx, cudaMemsetAsync(L.slot_tok, 0xff, sizeof(int) * L.max_slots, st));
+    RouteArgs ra;
+    memset(&ra, 0, sizeof(ra));
+    ra.n_tok = r->n_tok; ra.n_inv = r->n_inv; ra.n_roles = r->n_roles; ra.K = r->K; ra.V = r->V;
+    ra.cu_seqlens = r->cu_seqlens; ra.inv_role = r->inv_role; ra.target = r->target; ra.tok_mask = r->tok_mask;
+    for (int v = 0; v < r->n_roles; ++v) ra.role_model[v] = r->role_model[v];
+    ra.n_blocks = L.n_blocks; ra.blk_cnt = L.blk_cnt; ra.counts = L.counts; ra.offsets = L.offsets;
+    ra.tok_slot = L.tok_slot; ra.slot_tok = L.slot_tok; ra.tok_model = L.tok_model; ra.status = ctx->d_status;
+    CUDA_TRY(ctx, launch_route(ra, st, &nl));
+    CUDA_TRY(ctx, cudaMemcpyAsync(ctx->h_pinned, L.counts, sizeof(int) * UNITY_MAX_MODELS, cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(ctx, cudaStreamSynchronize(st));
+    int off = 0;
+    for (int k = 0; k < r->K; ++k) {
+        P.counts[k] = ctx->h_pinned[k];
+        P.offsets[k] = off;
+        off += static_cast<int>(up(P.counts[k], kTileM));
+    }
+    P.offsets[r->K] = off;
+    P.n_slots = off;
+
+    CUDA_TRY(ctx, launch_gather_rows(static_cast<const __nv_bfloat16*>(r->hidden), r->target, L.slot_tok, P.n_slots,
+                                     r->H, L.hp, L.target_p, st));
+    nl += P.n_slots > 0;
+
+    CUtensorMap tmA;
+    if (P.n_slots > 0) {
+        int rc = make_tmap(ctx, &tmA, L.hp, r->H, P.n_slots, static_cast<uint64_t>(r->H) * 2, kTileM);
+        if (rc) return rc;
+    }
+    const int n_tiles = (r->V + kTileN - 1) / kTileN;
+    long long sbase = 0;
+    for (int k = 0; k < r->K; ++k) {
+        P.splits[k] = 1;
+        P.stats_base[k] = sbase;
+        const int rows_k = P.offsets[k + 1] - P.offsets[k];
+        if (rows_k == 0) continue;
+        const int m_tiles = rows_k / kTileM;
+        int splits = (4 * ctx->sm_count + m_tiles - 1) / m_tiles;
+        if (splits < 4) splits = 4;
+        if (splits > 32) splits = 32;
+        if (splits > n_tiles) splits = n_tiles;
+        const int tps = (n_tiles + splits - 1) / splits;
+        splits = (n_tiles + tps - 1) / tps;
+        P.splits[k] = splits;
+        sbase += static_cast<long long>(splits) * rows_k;
+        if (sbase > L.stats_cap) return fail(ctx, UNITY_ERR_WORKSPACE, "internal: statistics scratch too small");
+
+        CUtensorMap tmB;
+        int rc = make_tmap(ctx, &tmB, r->W[k], r->H, r->V, static_cast<uint64_t>(r->H) * 2, kTileN);
+        if (rc) return rc;
+        GemmArgs g;
+        memset(&g, 0, sizeof(g));
+        g.m_tiles = m_tiles; g.n_tiles = n_tiles; g.k_iters = r->H / kTileK;
+        g.group_m = ctx->sm_count / splits > 0 ? ctx->sm_count / splits : 1;
+        g.a_row0 = P.offsets[k]; g.b_row0 = 0; g.a_k0 = 0; g.b_k0 = 0;
+        g.m_rows = rows_k; g.n_cols = r->V;
+        g.n_splits = splits; g.tiles_per_split = tps;
+        g.stats = L.stats + P.stats_base[k]; g.stats_pitch = rows_k;
+        g.target_p = L.target_p; g.vocab0 = 0; g.scale = r->inv_temperature;
+        g.status = ctx->d_status;
+        CUDA_TRY(ctx, launch_gemm(kEpiSoftmaxStats, tmA, tmB, g, ctx->sm_count, st));
+        nl += 1;
+    }
+    ctx->launches += nl;
+    return UNITY_OK;
+}
+
+void fill_token_args(TokenArgs& t, const unity_rows* r, const RowPlan& P) {
+    memset(&t, 0, sizeof(t));
+    const Layout& L = P.L;
+    t.n_slots = P.n_slots; t.K = r->K; t.n_roles = r->n_roles; t.n_inv = r->n_inv; t.n_tok = r->n_tok;
+    t.stats = L.stats;
+    for (int k = 0; k < r->K; ++k) { t.stats_base[k] = P.stats_base[k]; t.model_splits[k] = P.splits[k]; }
+    for (int k = 0; k <= r->K; ++k) t.offsets[k] = P.offsets[k];
+    t.slot_tok = L.slot_tok; t.tok_slot = L.tok_slot; t.tok_model = L.tok_model;
+    t.scale = r->inv_temperature;
+    t.row_lse = L.row_lse; t.row_ent = L.row_ent; t.row_logp = L.row_logp;
+    t.cu_seqlens = r->cu_seqlens; t.inv_role = r->inv_role;
+    for (int v = 0; v < r->n_roles; ++v) t.role_model[v] = r->role_model[v];
+}
+
+}  // namespace
+
+// ================================================================================================
+extern "C" {
+
+int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace, size_t workspace_bytes) {
+    if (!out) return UNITY_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (workspace_bytes > 0 && !workspace) return UNITY_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return UNITY_ERR_ALIGNMENT;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { cudaGetLastError(); return UNITY_ERR_CUDA; }
+    if (prop.major != 10) return UNITY_ERR_UNSUPPORTED_ARCH;
+    if (cudaSetDevice(device) != cudaSuccess) return UNITY_ERR_CUDA;
+    unity_ctx* c = new (std::nothrow) unity_ctx();
+    if (!c) return UNITY_ERR_CUDA;
+    memset(c, 0, sizeof(*c));
+    c->device = device;
+    c->stream = static_cast<cudaStream_t>(cuda_stream);
+    c->ws = static_cast<char*>(workspace);
+    c->ws_bytes = workspace_bytes;
+    c->sm_count = prop.multiProcessorCount;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess) {
+        delete c;
+        return UNITY_ERR_CUDA;
+    }
+    c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    if (cudaMalloc(&c->d_status, 256) != cudaSuccess || cudaMallocHost(&c->h_pinned, 4096) != cudaSuccess ||
+        cudaMemset(c->d_status, 0, 256) != cudaSuccess || gemm_set_attributes() != cudaSuccess) {
+        if (c->d_status) cudaFree(c->d_status);
+        if (c->h_pinned) cudaFreeHost(c->h_pinned);
+        delete c;
+        cudaGetLastError();
+        return UNITY_ERR_CUDA;
+    }
+    *out = c;
+    return UNITY_OK;
+}
+
+int unity_destroy(unity_ctx* ctx) {
+    if (!ctx) return UNITY_ERR_INVALID_ARG;
+    cudaSetDevice(ctx->device);
+    cudaStreamSynchronize(ctx->stream);
+    cudaFree(ctx->d_status);
+    cudaFreeHost(ctx->h_pinned);
+    delete ctx;
+    return UNITY_OK;
+}
+
+size_t unity_workspace_bytes(int64_t n_tok, int32_t H, int32_t V, int32_t K, int32_t n_inv) {
+    if (n_tok < 0 || H <= 0 || V <= 0 || K <= 0 || n_inv < 0) return 0;
+    return carve(nullptr, ~size_t(0), n_tok, H, V, K, n_inv, wanted_chunk_rows(n_tok, K), wanted_chunk_vocab(V), nullptr).bytes;
+}
+
+size_t unity_workspace_min_bytes(int64_t n_tok, int32_t H, int32_t V, int32_t K, int32_t n_inv) {
+    if (n_tok < 0 || H <= 0 || V <= 0 || K <= 0 || n_inv < 0) return 0;
+    int cr = wanted_chunk_rows(n_tok, K), cv = wanted_chunk_vocab(V);
+    if (cr > kMinChunkRows) cr = kMinChunkRows;
+    if (cv > kMinChunkVocab) cv = kMinChunkVocab;
+    return carve(nullptr, ~size_t(0), n_tok, H, V, K, n_inv, cr, cv, nullptr).bytes;
+}
+
+int unity_check_status(unity_ctx* ctx) {
+    if (!ctx) return UNITY_ERR_INVALID_ARG;
+    CUDA_TRY(ctx, cudaSetDevice(ctx->device));
+    CUDA_TRY(ctx, cudaMemcpyAsync(ctx->h_pinned + 512, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+    CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof(int), ctx->stream));
+    CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream));
+    const int bits = ctx->h_pinned[512];
+    if (bits & kStatusTimeout) return fail(ctx, UNITY_ERR_TIMEOUT, "a bounded in-kernel wait expired");
+    if (bits & kStatusBadIndex) return fail(ctx, UNITY_ERR_BAD_INDEX, "an index in the data was out of range (row / invocation masked)");
+    return UNITY_OK;
+}
+
+const char* unity_last_error(const unity_ctx* ctx) { return ctx ? ctx->err : "null context"; }
+
+int64_t unity_launch_count(const unity_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+// ------------------------------------------------------------------------------------------------
+int unity_role_advantage(unity_ctx* ctx, int32_t n_inv, int32_t n_traj, int32_t n_roles, int32_t n_groups,
+                         const int32_t* inv_role, const int32_t* inv_group, const int32_t* inv_traj,
+                         const float* r_node, const float* r_turn, const float* r_traj, const float* lam,
+                         const unity_adv_params* params, int64_t n_tok, const int64_t* cu_seqlens,
+                         const uint8_t* tok_mask, float* adv_inv, float* adv_tok, float* seg_mean, float* seg_std) {
+    if (!ctx) return UNITY_ERR_INVALID_ARG;
+    if (n_inv < 0 || n_traj < 0 || n_tok < 0) return fail(ctx, UNITY_ERR_INVALID_ARG, "negative size");
+    if (n_roles < 1 || n_roles > UNITY_MAX_ROLES) return fail(ctx, UNITY_ERR_SHAPE, "n_roles=%d outside [1,%d]", n_roles, UNITY_MAX_ROLES);
+    if (n_groups < 1 || static_cast<long long>(n_groups) * n_roles > (1 << 24))
+        return fail(ctx, UNITY_ERR_SHAPE, "n_groups*n_roles outside [1, 2^24]");
+    if (n_inv > 0 && (!inv_role || !inv_group || !adv_inv)) return fail(ctx, UNITY_ERR_INVALID_ARG, "inv_role / inv_group / adv_inv is NULL");
+    if (r_traj && n_inv > 0 && !inv_traj) return fail(ctx, UNITY_ERR_INVALID_ARG, "r_traj given without inv_traj");
+    if (n_tok > 0 && (!cu_seqlens || !adv_tok || n_inv < 1)) return fail(ctx, UNITY_ERR_INVALID_ARG, "cu_seqlens / adv_tok is NULL or n_inv < 1");
+    const float eps = params ? params->eps : 1e-6f;
+    const int ddof = params ? params->ddof : 0;
+    if (!(eps >= 0.f) || (ddof != 0 && ddof != 1)) return fail(ctx, UNITY_ERR_INVALID_ARG, "eps must be >= 0 and ddof 0 or 1");
+    CUDA_TRY(ctx, cudaSetDevice(ctx->device));
+    Bump b{ctx->ws, 0, ctx->ws_bytes, true};
+    AdvArgs a;
+    memset(&a, 0, sizeof(a));
+    a.r_scratch = b.take<float>(n_inv + 4);
+    a.seg_scratch = b.take<int>(n_inv + 4);
+    if (!b.ok) return fail(ctx, UNITY_ERR_WORKSPACE, "workspace too small: need %zu bytes", b.off);
+    a.n_inv = n_inv; a.n_traj = n_traj; a.n_roles = n_roles; a.n_groups = n_groups;
+    a.inv_role = inv_role; a.inv_group = inv_group; a.inv_traj = inv_traj;
+    a.r_node = r_node; a.r_turn = r_turn; a.r_traj = r_traj;
+    a.has_lam = lam != nullptr;
+    if (lam) memcpy(a.lam, lam, sizeof(float) * 3 * n_roles);
+    a.eps = eps; a.ddof = ddof; a.n_tok = n_tok; a.cu_seqlens = cu_seqlens; a.tok_mask = tok_mask;
+    a.adv_inv = adv_inv; a.adv_tok = adv_tok; a.seg_mean = seg_mean; a.seg_std = seg_std;
+    a.status = ctx->d_status;
+    int nl = 0;
+    CUDA_TRY(ctx, launch_advantage(a, ctx->stream, &nl));
+    ctx->launches += nl;
+    return UNITY_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+int unity_logprob_fwd(unity_ctx* ctx, const unity_rows* rows, float* logp, float* entropy, float* lse) {
+    int rc = validate_rows(ctx, rows);
+    if (rc) return rc;
+    if (rows->n_tok > 0 && !logp) return fail(ctx, UNITY_ERR_INVALID_ARG, "logp is NULL");
+    if (rows->n_tok == 0) return UNITY_OK;
+    CUDA_TRY(ctx, cudaSetDevice(ctx->device));
+    RowPlan P;
+    bool fits = false;
+    P.L = carve(ctx->ws, ctx->ws_bytes, rows->n_tok, rows->H, rows->V, rows->K, rows->n_inv, 0, 0, &fits);
+    if (!fits) return fail(ctx, UNITY_ERR_WORKSPACE, "workspace too small: need %zu bytes, have %zu", P.L.bytes, ctx->ws_bytes);
+    cudaStream_t st = ctx->stream;
+    CUDA_TRY(ctx, cudaMemsetAsync(logp, 0, sizeof(float) * rows->n_tok, st));
+    if (entropy) CUDA_TRY(ctx, cudaMemsetAsync(entropy, 0, sizeof(float) * rows->n_tok, st));
+    if (lse) CUDA_TRY(ctx, cudaMemsetAsync(lse, 0, sizeof(float) * rows->n_tok, st));
+    rc = forward_sweep(ctx, rows, P);
+    if (rc) return rc;
+    TokenArgs t;
+    fill_token_args(t, rows, P);
+    t.logp = logp; t.entropy = entropy; t.lse = lse;
+    int nl = 0;
+    CUDA_TRY(ctx, launch_finish_forward(t, false, st, &nl));
+    ctx->launches += nl;
+    return UNITY_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_ppo_params* params,
+                           const float* old_logp, const float* ref_logp, const float* adv_tok, float* loss,
+                           float* metrics, float* logp, float* entropy, float* tok_loss, void* dHidden,
+                           void* const* dW) {
+    int rc = validate_rows(ctx, rows);
+    if (rc) return rc;
+    if (!params || !loss || !dW) return fail(ctx, UNITY_ERR_INVALID_ARG, "params / loss / dW is NULL");
+    if (params->kl_mode < 1 || params->kl_mode > 3) return fail(ctx, UNITY_ERR_INVALID_ARG, "kl_mode must be 1, 2 or 3");
+    if (!(params->clip_lo >= 0.f) || !(params->clip_hi >= 0.f)) return fail(ctx, UNITY_ERR_INVALID_ARG, "clip ranges must be >= 0");
+    if (rows->n_tok > 0 && (!old_logp || !ref_logp || !adv_tok || !dHidden))
+        return fail(ctx, UNITY_ERR_INVALID_ARG, "old_logp / ref_logp / adv_tok / dHidden is NULL");
+    if (reinterpret_cast<uintptr_t>(dHidden) & 15) return fail(ctx, UNITY_ERR_ALIGNMENT, "dHidden not 16-byte aligned");
+    const int K = rows->K, H = rows->H, V = rows->V;
+    for (int k = 0; k < K; ++k) {
+        if (!dW[k]) return fail(ctx, UNITY_ERR_INVALID_ARG, "dW[%d] is NULL", k);
+        if (reinterpret_cast<uintptr_t>(dW[k]) & 15) return fail(ctx, UNITY_ERR_ALIGNMENT, "dW[%d] not 16-byte aligned", k);
+        if (params->norm && !(params->norm[k] > 0.f)) return fail(ctx, UNITY_ERR_INVALID_ARG, "norm[%d] must be > 0", k);
+    }
+    CUDA_TRY(ctx, cudaSetDevice(ctx->device));
+    cudaStream_t st = ctx->stream;
+
+    // choose gradient chunk sizes that fit the workspace
+    int cr = wanted_chunk_rows(rows->n_tok, K), cv = wanted_chunk_vocab(V);
+    RowPlan P;
+    bool fits = false;
+    while (true) {
+        P.L = carve(ctx->ws, ctx->ws_bytes, rows->n_tok, H, V, K, rows->n_inv, cr, cv, &fits);
+        if (fits) break;
+        if (cr > kMinChunkRows && cr >= cv) cr = static_cast<int>(up(cr / 2, kTileM));
+        else if (cv > kMinChunkVocab) cv = static_cast<int>(up(cv / 2, kTileN));
+        else if (cr > kMinChunkRows) cr = static_cast<int>(up(cr / 2, kTileM));
+        else return fail(ctx, UNITY_ERR_WORKSPACE, "workspace too small: need at least %zu bytes, have %zu", P.L.bytes, ctx->ws_bytes);
+    }
+    const Layout& L = P.L;
+
+    CUDA_TRY(ctx, cudaMemsetAsync(loss, 0, sizeof(float) * K, st));
+    if (rows->n_tok == 0) {
+        if (metrics) CUDA_TRY(ctx, cudaMemsetAsync(metrics, 0, sizeof(float) * (K + rows->n_roles) * UNITY_N_METRICS, st));
+        if (!params->accumulate_dW)
+            for (int k = 0; k < K; ++k) CUDA_TRY(ctx, cudaMemsetAsync(dW[k], 0, sizeof(float) * V * H, st));
+        return UNITY_OK;
+    }
+    if (logp) CUDA_TRY(ctx, cudaMemsetAsync(logp, 0, sizeof(float) * rows->n_tok, st));
+    if (entropy) CUDA_TRY(ctx, cudaMemsetAsync(entropy, 0, sizeof(float) * rows->n_tok, st));
+    if (tok_loss) CUDA_TRY(ctx, cudaMemsetAsync(tok_loss, 0, sizeof(float) * rows->n_tok, st));
+
+    rc = forward_sweep(ctx, rows, P);
+    if (rc) return rc;
+    int nl = 0;
+
+    TokenArgs t;
+    fill_token_args(t, rows, P);
+    t.logp = logp; t.entropy = entropy; t.lse = nullptr;
+    t.old_logp = old_logp; t.ref_logp = ref_logp; t.adv_tok = adv_tok;
+    t.clip_lo = params->clip_lo; t.clip_hi = params->clip_hi; t.kl_coef = params->kl_coef;
+    t.ent_coef = params->ent_coef; t.kl_mode = params->kl_mode;
+    for (int k = 0; k < K; ++k)
+        t.norm[k] = params->norm ? params->norm[k] : static_cast<float>(P.counts[k] > 0 ? P.counts[k] : 1);
+    t.coef_a = L.coef_a; t.coef_b = L.coef_b; t.tok_loss = tok_loss;
+    t.inv_sums = L.inv_sums; t.loss = loss; t.metrics = metrics;
+    CUDA_TRY(ctx, launch_finish_forward(t, true, st, &nl));
+
+    __nv_bfloat16* dH = static_cast<__nv_bfloat16*>(dHidden);
+    CUDA_TRY(ctx, launch_zero_masked_rows(L.tok_slot, rows->n_tok, H, dH, st));
+    nl += 1;
+    const long long ldT = L.max_slots;
+    CUDA_TRY(ctx, launch_transpose_bf16(L.hp, H, L.hT, ldT, P.n_slots, H, st));
+    nl += P.n_slots > 0;
+
+    CUtensorMap tm_hp, tm_hT, tm_WT;
+    if (P.n_slots > 0) {
+        if ((rc = make_tmap(ctx, &tm_hp, L.hp, H, P.n_slots, static_cast<uint64_t>(H) * 2, kTileM))) return rc;
+        if ((rc = make_tmap(ctx, &tm_hT, L.hT, P.n_slots, H, static_cast<uint64_t>(ldT) * 2, kTileN))) return rc;
+    }
+    if ((rc = make_tmap(ctx, &tm_WT, L.WT, V, H, static_cast<uint64_t>(V) * 2, kTileN))) return rc;
+
+    for (int k = 0; k < K; ++k) {
+        const int rows_k = P.offsets[k + 1] - P.offsets[k];
+        float* dWk = static_cast<float*>(dW[k]);
+        if (rows_k == 0) {
+            if (!params->accumulate_dW) CUDA_TRY(ctx, cudaMemsetAsync(dWk, 0, sizeof(float) * V * H, st));
+            continue;
+        }
+        const __nv_bfloat16* Wk = static_cast<const __nv_bfloat16*>(rows->W[k]);
+        CUDA_TRY(ctx, launch_transpose_bf16(Wk, H, L.WT, V, V, H, st));
+        nl += 1;
+        CUtensorMap tm_W;
+        if ((rc = make_tmap(ctx, &tm_W, Wk, H, V, static_cast<uint64_t>(H) * 2, kTileN))) return rc;
+
+        for (int c0 = 0; c0 < rows_k; c0 += cr) {
+            const int nc = rows_k - c0 < cr ? rows_k - c0 : cr;          // multiple of kTileM
+            const int slot0 = P.offsets[k] + c0;
+            for (int v0 = 0; v0 < V; v0 += cv) {
+                const int vc = V - v0 < cv ? V - v0 : cv;
+                // (1) recompute the logits of this (rows x vocab) chunk and form dL/dz in bf16
+                GemmArgs g;
+                memset(&g, 0, sizeof(g));
+                g.m_tiles = nc / kTileM; g.n_tiles = (vc + kTileN - 1) / kTileN; g.k_iters = H / kTileK;
+                g.group_m = 16;
+                g.a_row0 = slot0; g.b_row0 = v0; g.m_rows = nc; g.n_cols = vc;
+                g.target_p = L.target_p; g.vocab0 = v0; g.scale = rows->inv_temperature;
+                g.coef_a = L.coef_a; g.coef_b = L.coef_b; g.row_lse = L.row_lse; g.row_ent = L.row_ent;
+                g.G = L.G; g.ldg = cv; g.status = ctx->d_status;
+                CUDA_TRY(ctx, launch_gemm(kEpiLogitGrad, tm_hp, tm_W, g, ctx->sm_count, st));
+                // (2) token-major copy of the chunk for the weight gradient
+                CUDA_TRY(ctx, launch_transpose_bf16(L.G, cv, L.GT, cr, nc, vc, st));
+                // (3) dH_chunk[nc, H] (+)= G[nc, vc] * W[v0:v0+vc, :]
+                CUtensorMap tm_G, tm_GT;
+                if ((rc = make_tmap(ctx, &tm_G, L.G, vc, nc, static_cast<uint64_t>(cv) * 2, kTileM))) return rc;
+                if ((rc = make_tmap(ctx, &tm_GT, L.GT, nc, vc, static_cast<uint64_t>(cr) * 2, kTileM))) return rc;
+                GemmArgs h;
+                memset(&h, 0, sizeof(h));
+                h.m_tiles = nc / kTileM; h.n_tiles = (H + kTileN - 1) / kTileN; h.k_iters = (vc + kTileK - 1) / kTileK;
+                h.group_m = 16;
+                h.a_row0 = 0; h.b_row0 = 0; h.a_k0 = 0; h.b_k0 = v0; h.m_rows = nc; h.n_cols = H;
+                h.C = L.dHc; h.ldc = H; h.beta = v0 > 0; h.status = ctx->d_status;
+                CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, tm_G, tm_WT, h, ctx->sm_count, st));
+                // (4) dW[v0:v0+vc, :] (+)= G^T[vc, nc] * h[rows, :]
+                GemmArgs w;
+                memset(&w, 0, sizeof(w));
+                w.m_tiles = (vc + kTileM - 1) / kTileM; w.n_tiles = (H + kTileN - 1) / kTileN; w.k_iters = nc / kTileK;
+                w.group_m = 16;
+                w.a_row0 = 0; w.b_row0 = 0; w.a_k0 = 0; w.b_k0 = slot0; w.m_rows = vc; w.n_cols = H;
+                w.C = dWk + static_cast<long long>(v0) * H; w.ldc = H;
+                w.beta = (params->accumulate_dW || c0 > 0) ? 1 : 0; w.status = ctx->d_status;
+                CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, tm_GT, tm_hT, w, ctx->sm_count, st));
+                nl += 4;
+            }
+            CUDA_TRY(ctx, launch_store_dhidden(L.dHc, L.slot_tok, slot0, nc, H, dH, st));
+            nl += 1;
+        }
+    }
+    ctx->launches += nl;
+    return UNITY_OK;
+}
+
+}  // extern "C"
