@@ -24,7 +24,8 @@ UNITY_MAX_ROLES = 64
 UNITY_N_METRICS = 8
 
 EXPORTS = ["unity_create", "unity_destroy", "unity_workspace_bytes", "unity_workspace_min_bytes",
-           "unity_check_status", "unity_last_error", "unity_launch_count", "unity_role_advantage",
+           "unity_check_status", "unity_last_error", "unity_launch_count", "unity_set_profiling",
+           "unity_get_profile", "unity_role_advantage",
            "unity_logprob_fwd", "unity_ppo_loss_fwd_bwd"]
 
 
@@ -80,6 +81,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.unity_last_error.restype = C.c_char_p
     lib.unity_launch_count.argtypes = [vp]
     lib.unity_launch_count.restype = i64
+    lib.unity_set_profiling.argtypes = [vp, C.c_int]
+    lib.unity_set_profiling.restype = C.c_int
+    lib.unity_get_profile.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
+    lib.unity_get_profile.restype = C.c_int
     lib.unity_role_advantage.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, f32p,
                                          C.POINTER(unity_adv_params), i64, vp, vp, vp, vp, vp, vp]
     lib.unity_role_advantage.restype = C.c_int
@@ -140,6 +145,21 @@ def unity_check_status(ctx) -> None:
 
 def unity_launch_count(ctx) -> int:
     return int(load_library().unity_launch_count(ctx))
+
+
+PROF_CLASSES = ["fwd_gemm", "grad_gemm", "dh_gemm", "dw_gemm", "transpose"]
+
+
+def unity_set_profiling(ctx, enable: bool) -> None:
+    _raise(ctx, load_library().unity_set_profiling(ctx, 1 if enable else 0))
+
+
+def unity_get_profile(ctx) -> dict:
+    n = len(PROF_CLASSES)
+    ms = (C.c_double * n)()
+    cnt = (C.c_int64 * n)()
+    _raise(ctx, load_library().unity_get_profile(ctx, ms, cnt))
+    return {name: {"ms": float(ms[i]), "launches": int(cnt[i])} for i, name in enumerate(PROF_CLASSES)}
 
 
 def unity_role_advantage(ctx, n_traj: int, n_roles: int, n_groups: int, inv_role, inv_group, inv_traj,
@@ -238,6 +258,12 @@ class Context:
     @property
     def launch_count(self) -> int:
         return unity_launch_count(self.ctx)
+
+    def set_profiling(self, enable: bool):
+        unity_set_profiling(self.ctx, enable)
+
+    def get_profile(self) -> dict:
+        return unity_get_profile(self.ctx)
 
     def role_advantage(self, *a, **kw):
         return unity_role_advantage(self.ctx, *a, **kw)

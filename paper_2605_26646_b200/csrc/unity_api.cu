@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "internal.h"
 
@@ -24,6 +25,11 @@ struct unity_ctx {
     EncodeTiledFn encode;
     long long launches;
     char err[512];
+    // optional per-kernel-class timing (unity_set_profiling): pairs of events around each launch
+    int profiling;
+    std::vector<cudaEvent_t>* ev_pool;
+    std::vector<int>* ev_class;     // class of the i-th recorded pair
+    size_t ev_used;                 // events handed out since the last unity_get_profile
 };
 
 namespace {
@@ -50,6 +56,27 @@ int fail(unity_ctx* ctx, int code, const char* fmt, ...) {
         cudaError_t e_ = (expr);                                                                         \
         if (e_ != cudaSuccess) return fail(ctx, UNITY_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e_)); \
     } while (0)
+
+// Records an event pair around the launches issued during its lifetime when profiling is on.
+struct ProfScope {
+    unity_ctx* c;
+    bool on;
+    ProfScope(unity_ctx* ctx, int cls) : c(ctx), on(ctx->profiling != 0) {
+        if (!on) return;
+        while (c->ev_pool->size() < c->ev_used + 2) {
+            cudaEvent_t e;
+            if (cudaEventCreate(&e) != cudaSuccess) { on = false; return; }
+            c->ev_pool->push_back(e);
+        }
+        c->ev_class->push_back(cls);
+        cudaEventRecord((*c->ev_pool)[c->ev_used], c->stream);
+    }
+    ~ProfScope() {
+        if (!on) return;
+        cudaEventRecord((*c->ev_pool)[c->ev_used + 1], c->stream);
+        c->ev_used += 2;
+    }
+};
 
 struct Bump {
     char* base;
@@ -239,7 +266,10 @@ int forward_sweep(unity_ctx* ctx, const unity_rows* r, RowPlan& P) {
         g.stats = L.stats + P.stats_base[k]; g.stats_pitch = rows_k;
         g.target_p = L.target_p; g.vocab0 = 0; g.scale = r->inv_temperature;
         g.status = ctx->d_status;
-        CUDA_TRY(ctx, launch_gemm(kEpiSoftmaxStats, tmA, tmB, g, ctx->sm_count, st));
+        {
+            ProfScope ps(ctx, UNITY_PROF_FWD_GEMM);
+            CUDA_TRY(ctx, launch_gemm(kEpiSoftmaxStats, tmA, tmB, g, ctx->sm_count, st));
+        }
         nl += 1;
     }
     ctx->launches += nl;
@@ -290,6 +320,8 @@ int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace
         return UNITY_ERR_CUDA;
     }
     c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    c->ev_pool = new (std::nothrow) std::vector<cudaEvent_t>();
+    c->ev_class = new (std::nothrow) std::vector<int>();
     if (cudaMalloc(&c->d_status, 256) != cudaSuccess || cudaMallocHost(&c->h_pinned, 4096) != cudaSuccess ||
         cudaMemset(c->d_status, 0, 256) != cudaSuccess || gemm_set_attributes() != cudaSuccess) {
         if (c->d_status) cudaFree(c->d_status);
@@ -308,6 +340,9 @@ int unity_destroy(unity_ctx* ctx) {
     cudaStreamSynchronize(ctx->stream);
     cudaFree(ctx->d_status);
     cudaFreeHost(ctx->h_pinned);
+    if (ctx->ev_pool) for (cudaEvent_t e : *ctx->ev_pool) cudaEventDestroy(e);
+    delete ctx->ev_pool;
+    delete ctx->ev_class;
     delete ctx;
     return UNITY_OK;
 }
@@ -340,6 +375,31 @@ int unity_check_status(unity_ctx* ctx) {
 const char* unity_last_error(const unity_ctx* ctx) { return ctx ? ctx->err : "null context"; }
 
 int64_t unity_launch_count(const unity_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int unity_set_profiling(unity_ctx* ctx, int enable) {
+    if (!ctx || !ctx->ev_pool || !ctx->ev_class) return UNITY_ERR_INVALID_ARG;
+    ctx->profiling = enable != 0;
+    ctx->ev_used = 0;
+    ctx->ev_class->clear();
+    return UNITY_OK;
+}
+
+int unity_get_profile(unity_ctx* ctx, double* ms, int64_t* launches) {
+    if (!ctx || !ms || !launches || !ctx->ev_pool) return UNITY_ERR_INVALID_ARG;
+    for (int i = 0; i < UNITY_PROF_CLASSES; ++i) { ms[i] = 0.0; launches[i] = 0; }
+    CUDA_TRY(ctx, cudaSetDevice(ctx->device));
+    CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream));
+    for (size_t i = 0; i < ctx->ev_class->size(); ++i) {
+        float t = 0.f;
+        CUDA_TRY(ctx, cudaEventElapsedTime(&t, (*ctx->ev_pool)[2 * i], (*ctx->ev_pool)[2 * i + 1]));
+        const int cls = (*ctx->ev_class)[i];
+        ms[cls] += t;
+        launches[cls] += 1;
+    }
+    ctx->ev_used = 0;
+    ctx->ev_class->clear();
+    return UNITY_OK;
+}
 
 // ------------------------------------------------------------------------------------------------
 int unity_role_advantage(unity_ctx* ctx, int32_t n_inv, int32_t n_traj, int32_t n_roles, int32_t n_groups,
@@ -472,7 +532,10 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
     CUDA_TRY(ctx, launch_zero_masked_rows(L.tok_slot, rows->n_tok, H, dH, st));
     nl += 1;
     const long long ldT = L.max_slots;
-    CUDA_TRY(ctx, launch_transpose_bf16(L.hp, H, L.hT, ldT, P.n_slots, H, st));
+    {
+        ProfScope ps(ctx, UNITY_PROF_TRANSPOSE);
+        CUDA_TRY(ctx, launch_transpose_bf16(L.hp, H, L.hT, ldT, P.n_slots, H, st));
+    }
     nl += P.n_slots > 0;
 
     CUtensorMap tm_hp, tm_hT, tm_WT;
@@ -490,7 +553,10 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
             continue;
         }
         const __nv_bfloat16* Wk = static_cast<const __nv_bfloat16*>(rows->W[k]);
-        CUDA_TRY(ctx, launch_transpose_bf16(Wk, H, L.WT, V, V, H, st));
+        {
+            ProfScope ps(ctx, UNITY_PROF_TRANSPOSE);
+            CUDA_TRY(ctx, launch_transpose_bf16(Wk, H, L.WT, V, V, H, st));
+        }
         nl += 1;
         CUtensorMap tm_W;
         if ((rc = make_tmap(ctx, &tm_W, Wk, H, V, static_cast<uint64_t>(H) * 2, kTileN))) return rc;
@@ -509,9 +575,15 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 g.target_p = L.target_p; g.vocab0 = v0; g.scale = rows->inv_temperature;
                 g.coef_a = L.coef_a; g.coef_b = L.coef_b; g.row_lse = L.row_lse; g.row_ent = L.row_ent;
                 g.G = L.G; g.ldg = cv; g.status = ctx->d_status;
-                CUDA_TRY(ctx, launch_gemm(kEpiLogitGrad, tm_hp, tm_W, g, ctx->sm_count, st));
+                {
+                    ProfScope ps(ctx, UNITY_PROF_GRAD_GEMM);
+                    CUDA_TRY(ctx, launch_gemm(kEpiLogitGrad, tm_hp, tm_W, g, ctx->sm_count, st));
+                }
                 // (2) token-major copy of the chunk for the weight gradient
-                CUDA_TRY(ctx, launch_transpose_bf16(L.G, cv, L.GT, cr, nc, vc, st));
+                {
+                    ProfScope ps(ctx, UNITY_PROF_TRANSPOSE);
+                    CUDA_TRY(ctx, launch_transpose_bf16(L.G, cv, L.GT, cr, nc, vc, st));
+                }
                 // (3) dH_chunk[nc, H] (+)= G[nc, vc] * W[v0:v0+vc, :]
                 CUtensorMap tm_G, tm_GT;
                 if ((rc = make_tmap(ctx, &tm_G, L.G, vc, nc, static_cast<uint64_t>(cv) * 2, kTileM))) return rc;
@@ -522,7 +594,10 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 h.group_m = 16;
                 h.a_row0 = 0; h.b_row0 = 0; h.a_k0 = 0; h.b_k0 = v0; h.m_rows = nc; h.n_cols = H;
                 h.C = L.dHc; h.ldc = H; h.beta = v0 > 0; h.status = ctx->d_status;
-                CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, tm_G, tm_WT, h, ctx->sm_count, st));
+                {
+                    ProfScope ps(ctx, UNITY_PROF_DH_GEMM);
+                    CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, tm_G, tm_WT, h, ctx->sm_count, st));
+                }
                 // (4) dW[v0:v0+vc, :] (+)= G^T[vc, nc] * h[rows, :]
                 GemmArgs w;
                 memset(&w, 0, sizeof(w));
@@ -531,7 +606,10 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 w.a_row0 = 0; w.b_row0 = 0; w.a_k0 = 0; w.b_k0 = slot0; w.m_rows = vc; w.n_cols = H;
                 w.C = dWk + static_cast<long long>(v0) * H; w.ldc = H;
                 w.beta = (params->accumulate_dW || c0 > 0) ? 1 : 0; w.status = ctx->d_status;
-                CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, tm_GT, tm_hT, w, ctx->sm_count, st));
+                {
+                    ProfScope ps(ctx, UNITY_PROF_DW_GEMM);
+                    CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, tm_GT, tm_hT, w, ctx->sm_count, st));
+                }
                 nl += 4;
             }
             CUDA_TRY(ctx, launch_store_dhidden(L.dHc, L.slot_tok, slot0, nc, H, dH, st));
