@@ -1,0 +1,290 @@
+"""GPU parity: libunity (through its C ABI) against the fp64 oracle, element by element, on the same
+seeded inputs.  Sizes span several row tiles, vocabulary tiles and chunks, with ragged tails."""
+import numpy as np
+import pytest
+import torch
+
+import parity_util as pu
+from paper_2605_26646_b200 import binding as ub
+from paper_2605_26646_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def check_forward(g, o, mask):
+    for key in ("logp", "entropy", "lse"):
+        if key in g and key in o:
+            got = g[key].cpu().numpy()
+            assert np.abs(got - o[key]).max() <= pu.TOL_LOGP, key
+            assert np.all(got[~mask] == 0), key + " must be 0 on masked rows"
+
+
+def check_ppo(g, o, w, atol_loss=1e-6):
+    mask = w.tok_mask.numpy() != 0
+    check_forward(g, o, mask)
+    loss = g["loss"].cpu().numpy()
+    assert np.all(np.abs(loss - o["loss"]) <= pu.TOL_LOSS * np.abs(o["loss"]) + atol_loss), (loss, o["loss"])
+    tl = g["tok_loss"].cpu().numpy()
+    assert np.abs(tl - o["tok_loss"]).max() <= pu.TOL_LOGP
+    assert np.all(tl[~mask] == 0)
+    dH = g["dHidden"].float().cpu().numpy()
+    assert np.all(dH[~mask] == 0), "dHidden must be 0 on masked rows"
+    if np.linalg.norm(o["dHidden"]) > 0:
+        assert pu.rel_fro(dH, o["dHidden"]) <= pu.TOL_GRAD
+    else:
+        assert np.abs(dH).max() == 0
+    for k in range(w.K):
+        got = g["dW"][k].cpu().numpy()
+        if o["dW"][k] is None:
+            continue
+        if np.linalg.norm(o["dW"][k]) > 0:
+            assert pu.rel_fro(got, o["dW"][k]) <= pu.TOL_GRAD, f"dW[{k}]"
+        else:
+            assert np.abs(got).max() == 0
+    om = np.concatenate([o["metrics_model"], o["metrics_role"]])
+    gm = g["metrics"].cpu().numpy()
+    assert np.array_equal(gm[:, 0], om[:, 0])                       # valid counts are exact
+    assert np.abs(gm - om).max() <= 1e-3 * max(1.0, np.abs(om[:, 1:]).max())
+
+
+def run_all_stages(w, **ppo_kw):
+    d = pu.DeviceInputs(w)
+    ctx = pu.make_ctx(w)
+    try:
+        ga, oa = pu.gpu_advantage(ctx, w, d), pu.oracle_advantage(w)
+        assert np.abs(ga["adv_inv"].cpu().numpy() - oa["adv_inv"]).max() <= pu.TOL_ADV
+        assert np.abs(ga["adv_tok"].cpu().numpy() - oa["adv_tok"]).max() <= pu.TOL_ADV
+        gl, ol = pu.gpu_logprob(ctx, w, d), pu.oracle_logprob(w)
+        check_forward(gl, ol, w.tok_mask.numpy() != 0)
+        cur = torch.from_numpy(ol["logp"].astype(np.float32))
+        old, ref = cur + w.noise_old, cur + w.noise_ref
+        adv = torch.from_numpy(oa["adv_tok"].astype(np.float32))
+        gp = pu.gpu_ppo(ctx, w, d, old.cuda(), ref.cuda(), adv.cuda(), **ppo_kw)
+        op = pu.oracle_ppo(w, old.numpy(), ref.numpy(), adv.numpy(), **ppo_kw)
+        check_ppo(gp, op, w)
+    finally:
+        ctx.close()
+
+
+# ------------------------------------------------------------------------------------ stage 1
+
+@pytest.mark.parametrize("name", list(wl.CONFIGS))
+def test_advantage_full_size(name):
+    w = wl.make_structure(name)
+    d = pu.DeviceInputs(w)
+    ctx = ub.Context(0, 1 << 22)
+    g, o = pu.gpu_advantage(ctx, w, d), pu.oracle_advantage(w)
+    assert np.abs(g["adv_inv"].cpu().numpy() - o["adv_inv"]).max() <= pu.TOL_ADV
+    assert np.abs(g["adv_tok"].cpu().numpy() - o["adv_tok"]).max() <= pu.TOL_ADV
+    assert np.abs(g["seg_mean"].cpu().numpy() - o["seg_mean"]).max() <= pu.TOL_ADV
+    assert np.abs(g["seg_std"].cpu().numpy() - o["seg_std"]).max() <= pu.TOL_ADV
+    if name == "stress":                       # constant segments give exactly zero
+        seg = (w.inv_group.long() * w.n_roles + w.inv_role.long()).numpy()
+        const = o["seg_std"][seg] == 0
+        assert const.any() and np.all(g["adv_inv"].cpu().numpy()[const] == 0)
+    ctx.close()
+
+
+@pytest.mark.parametrize("ddof,eps,one_group", [(1, 1e-6, False), (0, 0.0, False), (0, 1e-6, True)])
+def test_advantage_variants(ddof, eps, one_group):
+    w = wl.make_structure("search", cut_rows=500, cut_max_len=40)
+    if one_group:                              # role-wise whitening over the whole batch
+        w.inv_group.zero_()
+        w.n_groups = 1
+    w.lam = torch.tensor([[1.0, 0.5, 2.0], [0.0, 1.0, 1.0], [1.5, 1.0, 0.25]])
+    w.r_node = wl.normal(5, 77, w.n_inv)
+    d = pu.DeviceInputs(w)
+    ctx = ub.Context(0, 1 << 22)
+    g, o = pu.gpu_advantage(ctx, w, d, ddof=ddof, eps=eps), pu.oracle_advantage(w, ddof=ddof, eps=eps)
+    assert np.abs(g["adv_inv"].cpu().numpy() - o["adv_inv"]).max() <= pu.TOL_ADV
+    assert np.abs(g["adv_tok"].cpu().numpy() - o["adv_tok"]).max() <= pu.TOL_ADV
+    ctx.close()
+
+
+def test_advantage_null_inputs_unaligned_views_and_empty_batch():
+    import oracle.unity_oracle as orc
+    w = wl.make_structure("rag_qa")
+    d = pu.DeviceInputs(w)
+    ctx = ub.Context(0, 1 << 22)
+    # no turn reward, no mask, default lambda
+    adv_inv = torch.empty(w.n_inv, device="cuda")
+    big = torch.empty(w.n_tok + 3, device="cuda")
+    adv_tok = big[1:1 + w.n_tok]              # 4-byte aligned only: exercises the scalar store path
+    ctx.role_advantage(w.n_traj, w.n_roles, w.n_groups, d.inv_role, d.inv_group, d.inv_traj, d.r_node, None, d.r_traj,
+                       None, 1e-6, 0, d.cu_seqlens, None, adv_inv, adv_tok)
+    ctx.check_status()
+    o = orc.role_advantage(w.inv_role.numpy(), w.inv_group.numpy(), w.inv_traj.numpy(), w.r_node.numpy(), None,
+                           w.r_traj.numpy(), None, w.n_roles, w.n_groups, w.cu_seqlens.numpy(), None)
+    assert np.abs(adv_tok.cpu().numpy() - o["adv_tok"]).max() <= pu.TOL_ADV
+    # invocations without any token
+    cu0 = torch.zeros(w.n_inv + 1, dtype=torch.int64, device="cuda")
+    ctx.role_advantage(w.n_traj, w.n_roles, w.n_groups, d.inv_role, d.inv_group, d.inv_traj, d.r_node, None, d.r_traj,
+                       None, 1e-6, 0, cu0, None, adv_inv, torch.empty(0, device="cuda"))
+    ctx.check_status()
+    assert np.abs(adv_inv.cpu().numpy() - o["adv_inv"]).max() <= pu.TOL_ADV
+    ctx.close()
+
+
+def test_bad_indices_are_flagged_not_fatal():
+    w = wl.make_structure("tiny")
+    w.inv_role[3] = 9                          # role id out of range
+    d = pu.DeviceInputs(w)
+    ctx = ub.Context(0, 1 << 22)
+    adv_inv = torch.empty(w.n_inv, device="cuda")
+    adv_tok = torch.empty(w.n_tok, device="cuda")
+    ctx.role_advantage(w.n_traj, w.n_roles, w.n_groups, d.inv_role, d.inv_group, d.inv_traj, d.r_node, d.r_turn,
+                       d.r_traj, None, 1e-6, 0, d.cu_seqlens, d.tok_mask, adv_inv, adv_tok)
+    with pytest.raises(ub.UnityError) as e:
+        ctx.check_status()
+    assert e.value.code == -7
+    assert adv_inv[3].item() == 0.0
+    ctx.check_status()                         # the status word was cleared
+    ctx.close()
+
+
+# ------------------------------------------------------------------------------------ stages 2 + 3
+
+def test_tiny_full():
+    run_all_stages(wl.make("tiny", device="cuda"))
+
+
+@pytest.mark.parametrize("name", ["rag_qa", "search", "code", "stress"])
+def test_config_parity_cut(name):
+    # same H, V, K, roles and groups as the full configuration; token batch cut to ~300 rows
+    run_all_stages(wl.make(name, device="cuda", cut_rows=300, cut_max_len=64))
+
+
+def small_workload(H, V, rows, role_model=None, K=None, max_len=48, seed_offset=0):
+    w = wl.make_structure("search", cut_rows=rows, cut_max_len=max_len, H=H, V=V, seed_offset=seed_offset)
+    if role_model is not None:
+        w.role_model = torch.tensor(role_model, dtype=torch.int32)
+        w.K = K or int(max(role_model)) + 1
+    return wl.materialize(w, device="cuda")
+
+
+@pytest.mark.parametrize("H,V,rows", [(64, 1000, 150), (128, 4096 + 8, 700), (320, 2048, 129), (256, 520, 40)])
+def test_small_shapes_and_ragged_tails(H, V, rows):
+    # V not a multiple of the 256-wide vocabulary tile, rows not a multiple of the 128-row tile
+    run_all_stages(small_workload(H, V, rows))
+
+
+@pytest.mark.parametrize("kl_mode,ent_coef,clip", [(1, 0.0, (0.2, 0.2)), (2, 0.01, (0.1, 0.3)), (3, 0.02, (0.2, 0.28))])
+def test_kl_modes_entropy_bonus_and_temperature(kl_mode, ent_coef, clip):
+    w = small_workload(256, 3000, 400, seed_offset=kl_mode)
+    w.inv_temperature = 0.7
+    w.noise_old = w.noise_old * 6.0            # log-ratio noise 0.3: many tokens on the clipped branch
+    run_all_stages(w, kl_mode=kl_mode, kl_coef=0.1, ent_coef=ent_coef, clip=clip)
+
+
+def test_model_without_rows_and_three_models():
+    # roles map to models 0 and 1; model 2 is never used: its dW must come back as zeros
+    run_all_stages(small_workload(128, 1024, 300, role_model=[0, 1, 0], K=3))
+
+
+def test_all_rows_masked_and_single_row():
+    w = small_workload(128, 1024, 200)
+    w.tok_mask.zero_()
+    d = pu.DeviceInputs(w)
+    ctx = pu.make_ctx(w)
+    z = torch.zeros(w.n_tok, device="cuda")
+    g = pu.gpu_ppo(ctx, w, d, z, z, z)
+    assert torch.all(g["loss"] == 0) and torch.all(g["dHidden"] == 0) and all(torch.all(x == 0) for x in g["dW"])
+    assert torch.all(g["logp"] == 0) and torch.all(g["tok_loss"] == 0)
+    gl = pu.gpu_logprob(ctx, w, d)
+    assert torch.all(gl["logp"] == 0)
+    ctx.close()
+    w.tok_mask[17] = 1
+    run_all_stages(w)
+
+
+def test_gradient_accumulation_is_additive_and_runs_are_bitwise_reproducible():
+    w = small_workload(256, 2048, 600)
+    d = pu.DeviceInputs(w)
+    ctx = pu.make_ctx(w)
+    ol = pu.oracle_logprob(w)
+    cur = torch.from_numpy(ol["logp"].astype(np.float32))
+    old, ref = (cur + w.noise_old).cuda(), (cur + w.noise_ref).cuda()
+    adv = wl.normal(3, 99, w.n_tok).cuda()
+    full = pu.gpu_ppo(ctx, w, d, old, ref, adv)
+    again = pu.gpu_ppo(ctx, w, d, old, ref, adv)
+    assert torch.equal(full["dHidden"], again["dHidden"]) and torch.equal(full["loss"], again["loss"])
+    assert all(torch.equal(a, b) for a, b in zip(full["dW"], again["dW"]))
+    # two micro-batches (mask halves) with the full-batch norm, accumulated into one dW
+    norm = [max(float(full["metrics"][k, 0].item()), 1.0) for k in range(w.K)]
+    half = w.n_tok // 2
+    mask_a, mask_b = w.tok_mask.clone(), w.tok_mask.clone()
+    mask_a[half:] = 0
+    mask_b[:half] = 0
+    dW = [torch.zeros(w.V, w.H, device="cuda") for _ in range(w.K)]
+    d.tok_mask = mask_a.cuda()
+    ga = pu.gpu_ppo(ctx, w, d, old, ref, adv, norm=norm, accumulate=True, dW=dW)
+    d.tok_mask = mask_b.cuda()
+    gb = pu.gpu_ppo(ctx, w, d, old, ref, adv, norm=norm, accumulate=True, dW=dW)
+    assert torch.allclose(ga["loss"] + gb["loss"], full["loss"], rtol=1e-4, atol=1e-7)
+    for k in range(w.K):
+        assert pu.rel_fro(dW[k].cpu().numpy(), full["dW"][k].cpu().numpy()) <= 1e-3
+    dH_sum = (ga["dHidden"].float() + gb["dHidden"].float()).cpu().numpy()
+    assert pu.rel_fro(dH_sum, full["dHidden"].float().cpu().numpy()) <= 1e-3
+    # column sums of dW over the vocabulary vanish (sum_v dL/dz_v = 0 for every row)
+    for k in range(w.K):
+        col = full["dW"][k].double().sum(0).abs().max().item()
+        assert col <= 1e-2 * full["dW"][k].double().abs().sum(0).max().item() + 1e-9
+    ctx.close()
+
+
+def test_small_workspace_uses_smaller_chunks_and_too_small_is_an_error():
+    w = small_workload(256, 4096, 1500, max_len=200)
+    d = pu.DeviceInputs(w)
+    need = ub.unity_workspace_bytes(w.n_tok, w.H, w.V, w.K, w.n_inv)
+    least = ub.unity_workspace_min_bytes(w.n_tok, w.H, w.V, w.K, w.n_inv)
+    assert least < need
+    ol = pu.oracle_logprob(w)
+    cur = torch.from_numpy(ol["logp"].astype(np.float32))
+    old, ref = cur + w.noise_old, cur + w.noise_ref
+    adv = wl.normal(4, 98, w.n_tok)
+    ctx = ub.Context(0, least)                 # several row chunks and vocabulary chunks
+    gp = pu.gpu_ppo(ctx, w, d, old.cuda(), ref.cuda(), adv.cuda())
+    op = pu.oracle_ppo(w, old.numpy(), ref.numpy(), adv.numpy())
+    check_ppo(gp, op, w)
+    ctx.close()
+    ctx = ub.Context(0, 1 << 16)
+    with pytest.raises(ub.UnityError) as e:
+        pu.gpu_logprob(ctx, w, d)
+    assert e.value.code == -4
+    ctx.close()
+
+
+def test_argument_errors_return_codes():
+    w = small_workload(128, 1024, 100)
+    d = pu.DeviceInputs(w)
+    ctx = pu.make_ctx(w)
+    logp = torch.empty(w.n_tok, device="cuda")
+    args = [d.hidden, d.W, d.cu_seqlens, d.inv_role, w.role_model.tolist(), d.target, d.tok_mask, 1.0, logp]
+    bad_h = torch.empty(w.n_tok, 96, device="cuda", dtype=torch.bfloat16)        # H not a multiple of 64
+    with pytest.raises(ub.UnityError) as e:
+        ctx.logprob_fwd(bad_h, [torch.empty(w.V, 96, device="cuda", dtype=torch.bfloat16)] * w.K, *args[2:])
+    assert e.value.code == -2
+    with pytest.raises(ub.UnityError) as e:                                       # model id outside [0, K)
+        ctx.logprob_fwd(d.hidden, d.W, d.cu_seqlens, d.inv_role, [0, 0, 5], d.target, d.tok_mask, 1.0, logp)
+    assert e.value.code == -1
+    with pytest.raises(ub.UnityError) as e:                                       # non-positive temperature
+        ctx.logprob_fwd(d.hidden, d.W, d.cu_seqlens, d.inv_role, w.role_model.tolist(), d.target, d.tok_mask, 0.0, logp)
+    assert e.value.code == -1
+    odd = torch.empty(w.n_tok * w.H + 8, device="cuda", dtype=torch.bfloat16)[1:1 + w.n_tok * w.H].view(w.n_tok, w.H)
+    with pytest.raises(ub.UnityError) as e:                                       # hidden not 16-byte aligned
+        ctx.logprob_fwd(odd, *args[1:])
+    assert e.value.code == -3
+    # a target outside the vocabulary: flagged, row treated as masked, nothing else disturbed
+    tgt = w.target.clone()
+    row = int(torch.nonzero(w.tok_mask)[5])
+    tgt[row] = w.V + 3
+    ctx.logprob_fwd(d.hidden, d.W, d.cu_seqlens, d.inv_role, w.role_model.tolist(), tgt.cuda(), d.tok_mask, 1.0, logp)
+    with pytest.raises(ub.UnityError) as e:
+        ctx.check_status()
+    assert e.value.code == -7
+    o = pu.oracle_logprob(w)
+    got = logp.cpu().numpy()
+    assert got[row] == 0
+    keep = np.arange(w.n_tok) != row
+    assert np.abs(got[keep] - o["logp"][keep]).max() <= pu.TOL_LOGP
+    ctx.close()
