@@ -1,0 +1,368 @@
+#!/usr/bin/env python
+"""Benchmark of the multi-agent PPO hot path: response tokens/s of one step = role-level advantage +
+fused LM-head log-prob + PPO-clip/KL forward and backward (dHidden, dW), on synthetic data shaped like
+the reflective code-generation workload (H=3584, V=152064, 2 separate models).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload code] [--impl unity|reference]
+
+Prints ONE JSON line (rank 0).  With N > 1 (launched by torch.distributed.run) every rank processes
+its own rollout groups (weak scaling); the only exchange is the all-reduce of the per-model valid-row
+counts before the step and of dW after it.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "response tokens/s, fused LM-head logprob+PPO fwd+bwd; % of bf16 tensor peak"
+UNIT = "tokens/s"
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], tflops_burst=p["bf16_tflops"], tflops_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_sample_run(w, n_rows, old, ref, adv):
+    """Time the fp64 oracle (as it stands) on the first n_rows valid rows of the workload: advantage stage on the
+    whole batch + log-prob / loss / backward on the sample.  Returns (seconds, rows)."""
+    import numpy as np
+    import torch
+    from oracle import unity_oracle as orc
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import parity_util as pu
+    rows = torch.nonzero(w.tok_mask)[:n_rows, 0].numpy()
+    hid_bits = pu.bf16_bits(w.hidden)
+    W_bits = [pu.bf16_bits(x) for x in w.W]
+    t0 = time.perf_counter()
+    pu.oracle_advantage(w)
+    orc.ppo_loss_fwd_bwd(hid_bits, W_bits, w.cu_seqlens.numpy(), w.inv_role.numpy(), w.role_model.numpy(),
+                         w.target.numpy(), w.tok_mask.numpy(), np.asarray(old), np.asarray(ref), np.asarray(adv),
+                         clip_lo=w.clip_lo, clip_hi=w.clip_hi, kl_coef=w.kl_coef, kl_mode=w.kl_mode,
+                         ent_coef=w.ent_coef, inv_temperature=w.inv_temperature, n_roles=w.n_roles, rows=rows)
+    return time.perf_counter() - t0, int(rows.size)
+
+
+def run_reference(args):
+    """The reference arm: the oracle, unmodified, on the host cores, on a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    from paper_2605_26646_b200 import workloads as wl
+    # the same workload definition; hidden rows are only needed for the sampled rows, so a cut keeps host memory small
+    gen_dev = "cuda" if torch.cuda.is_available() else "cpu"      # drawing the inputs is not part of the timed work
+    w = wl.make(args.workload, device=gen_dev, cut_rows=max(args.ref_rows * 2, 256), cut_max_len=128)
+    w.hidden = w.hidden.cpu()
+    w.W = [x.cpu() for x in w.W]
+    n = w.n_tok
+    old = wl.normal(1, 901, n) * 0.05 - 11.0
+    ref = wl.normal(1, 902, n) * 0.05 - 11.0
+    adv = wl.normal(1, 903, n)
+    times = []
+    rows = 0
+    for i in range(args.warmup + args.steps):
+        dt, rows = oracle_sample_run(w, args.ref_rows, old, ref, adv)
+        if i >= args.warmup:
+            times.append(dt)
+    t = sum(times) / len(times)
+    val = rows / t
+    cores = torch.get_num_threads()
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "H": w.H, "V": w.V, "K": w.K, "sample_rows": rows},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"{rows} valid rows of the {args.workload} workload per step, fp64 numpy"},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="code")
+    ap.add_argument("--impl", default="unity", choices=["unity", "reference"])
+    ap.add_argument("--ref-rows", type=int, default=256, help="valid rows per oracle step (reference arm / cpu baseline)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cut-rows", type=int, default=0, help="profile-capture helper: run on a cut of the workload")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.cut_rows == 0:
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2605_26646_b200 import binding as ub
+    from paper_2605_26646_b200 import workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    # ---------------------------------------------------------------- inputs (each rank: its own rollout groups)
+    kw = dict(seed_offset=1000 * rank)
+    if args.cut_rows:
+        kw.update(cut_rows=args.cut_rows)
+    w = wl.make(args.workload, device=dev, **kw)
+    n, H, V, K = w.n_tok, w.H, w.V, w.K
+    d_inv_role, d_inv_group, d_inv_traj = w.inv_role.to(dev), w.inv_group.to(dev), w.inv_traj.to(dev)
+    d_rn, d_rt, d_rj = w.r_node.to(dev), w.r_turn.to(dev), w.r_traj.to(dev)
+    d_cu, d_mask, d_tgt = w.cu_seqlens.to(dev), w.tok_mask.to(dev), w.target.to(dev)
+    role_model = w.role_model.tolist()
+    lam = w.lam.tolist()
+    ws_bytes = ub.unity_workspace_bytes(n, H, V, K, w.n_inv)
+    ctx = ub.Context(local, ws_bytes)
+
+    adv_inv = torch.empty(w.n_inv, device=dev)
+    adv_tok = torch.empty(n, device=dev)
+    logp = torch.empty(n, device=dev)
+    ent = torch.empty(n, device=dev)
+    loss = torch.empty(K, device=dev)
+    metrics = torch.empty((K + w.n_roles) * ub.UNITY_N_METRICS, device=dev)
+    dH = torch.empty(n, H, device=dev, dtype=torch.bfloat16)
+    dW = [torch.empty(V, H, device=dev) for _ in range(K)]
+
+    # current log-probs (stage 2) give the old / reference log-probs of the batch: logp + N(0, 0.05)
+    ctx.logprob_fwd(w.hidden, w.W, d_cu, d_inv_role, role_model, d_tgt, d_mask, w.inv_temperature, logp)
+    ctx.check_status()
+    old = logp + w.noise_old.to(dev)
+    ref = logp + w.noise_ref.to(dev)
+
+    # per-model valid-row counts: the only quantity the ranks must agree on before the step
+    tok_inv = torch.repeat_interleave(torch.arange(w.n_inv), w.cu_seqlens[1:] - w.cu_seqlens[:-1])
+    tok_model = w.role_model[w.inv_role.long()[tok_inv]].long()
+    counts = torch.bincount(tok_model[w.tok_mask != 0], minlength=K).to(torch.float64)
+    n_valid_local = int(counts.sum().item())
+    norm = None
+    n_valid_total = n_valid_local
+    if world > 1:
+        c = counts.to(dev)
+        dist.all_reduce(c)
+        norm = [max(float(x), 1.0) for x in c.tolist()]
+        n_valid_total = int(c.sum().item())
+
+    def step(hid, tgt, msk, o, r):
+        ctx.role_advantage(w.n_traj, w.n_roles, w.n_groups, d_inv_role, d_inv_group, d_inv_traj, d_rn, d_rt, d_rj,
+                           lam, w.adv_eps, w.adv_ddof, d_cu, msk, adv_inv, adv_tok)
+        ctx.ppo_loss_fwd_bwd(hid, w.W, d_cu, d_inv_role, role_model, tgt, msk, w.inv_temperature, w.clip_lo,
+                             w.clip_hi, w.kl_coef, w.kl_mode, w.ent_coef, norm, False, o, r, adv_tok, loss, metrics,
+                             logp, ent, None, dH, dW)
+        if world > 1:
+            for g in dW:
+                dist.all_reduce(g)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step(w.hidden, d_tgt, d_mask, old, ref)
+    ctx.check_status()
+
+    # ---------------------------------------------------------------- timed region (device-resident inputs)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ctx.set_profiling(True)
+    launches0 = ctx.launch_count
+    sync_all()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step(w.hidden, d_tgt, d_mask, old, ref)
+    e1.record()
+    sync_all()
+    ms_total = e0.elapsed_time(e1)
+    launches = ctx.launch_count - launches0
+    prof = ctx.get_profile()
+    ctx.set_profiling(False)
+    clocks = sampler.stop() if rank == 0 else None
+    ctx.check_status()
+    t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    value = n_valid_total / (ms_step * 1e-3)
+
+    # ---------------------------------------------------------------- end to end: host buffers, copies timed
+    e2e = None
+    if not args.no_e2e:
+        h_hid = torch.empty(w.hidden.shape, dtype=w.hidden.dtype, pin_memory=True)
+        h_hid.copy_(w.hidden)
+        h_tgt = w.target.pin_memory()
+        h_msk = w.tok_mask.pin_memory()
+        h_old = torch.empty(n, pin_memory=True)
+        h_old.copy_(old)
+        h_ref = torch.empty(n, pin_memory=True)
+        h_ref.copy_(ref)
+        h_loss = torch.empty(K + metrics.numel(), pin_memory=True)
+        g_hid, g_tgt, g_msk = torch.empty_like(w.hidden), torch.empty_like(d_tgt), torch.empty_like(d_mask)
+        g_old, g_ref = torch.empty_like(old), torch.empty_like(ref)
+        h2d = sum(x.numel() * x.element_size() for x in (h_hid, h_tgt, h_msk, h_old, h_ref))
+        d2h = h_loss.numel() * 4
+
+        def e2e_step():
+            g_hid.copy_(h_hid, non_blocking=True)
+            g_tgt.copy_(h_tgt, non_blocking=True)
+            g_msk.copy_(h_msk, non_blocking=True)
+            g_old.copy_(h_old, non_blocking=True)
+            g_ref.copy_(h_ref, non_blocking=True)
+            step(g_hid, g_tgt, g_msk, g_old, g_ref)
+            h_loss[:K].copy_(loss, non_blocking=True)
+            h_loss[K:].copy_(metrics, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+
+        e2e_step()
+        sync_all()
+        n_e2e = max(1, min(args.steps, 3))
+        e0.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        e1.record()
+        sync_all()
+        t2 = torch.tensor([e0.elapsed_time(e1)], device=dev, dtype=torch.float64)
+        if world > 1:
+            dist.all_reduce(t2, op=dist.ReduceOp.MAX)
+        e2e = {"value": n_valid_total / (float(t2.item()) / n_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": n_e2e}
+        del h_hid, g_hid
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    # ---------------------------------------------------------------- roofline of the dominant kernel class
+    peaks = read_peaks()
+    peak = peaks["tflops_sustained"]           # kernels timed inside a long step: the sustained figure
+    flops_per_tok = 2.0 * H * V                # algorithmic flops of ONE of the four contractions per valid row
+    kern = {}
+    for name in ("fwd_gemm", "grad_gemm", "dh_gemm", "dw_gemm"):
+        p = prof[name]
+        if p["launches"] == 0:
+            continue
+        tf = flops_per_tok * n_valid_local * args.steps / (p["ms"] * 1e-3) / 1e12
+        kern[name] = {"launches": p["launches"], "ms_total": p["ms"], "share_of_step": p["ms"] / ms_total,
+                      "tflops": tf, "frac": tf / peak}
+    kern["transpose"] = {"launches": prof["transpose"]["launches"], "ms_total": prof["transpose"]["ms"],
+                         "share_of_step": prof["transpose"]["ms"] / ms_total}
+    dom = max((k for k in kern if k != "transpose"), key=lambda k: kern[k]["ms_total"])
+    dp = kern[dom]
+    roofline = {"bound": "tensor", "kernel": f"k_gemm<{dom}>", "achieved": dp["tflops"], "peak": peak,
+                "unit": "TFLOP/s", "frac": dp["frac"], "traffic": None,
+                "peak_source": f"{peaks['source']} bf16 GEMM, sustained",
+                "flops_per_launch": flops_per_tok * n_valid_local * args.steps / dp["launches"],
+                "avg_launch_ms": dp["ms_total"] / dp["launches"]}
+    step_tflops_alg = 6.0 * H * V * n_valid_local / (ms_step * 1e-3) / 1e12
+    step_tflops_exe = 8.0 * H * V * n_valid_local / (ms_step * 1e-3) / 1e12
+
+    cpu_baseline = None
+    if not args.no_cpu_baseline:
+        old_h, ref_h, adv_h = old.cpu().numpy(), ref.cpu().numpy(), adv_tok.cpu().numpy()
+        w.hidden = w.hidden.cpu()
+        w.W = [x.cpu() for x in w.W]
+        dt, rows = oracle_sample_run(w, args.ref_rows, old_h, ref_h, adv_h)
+        cpu_baseline = {"value": rows / dt, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+                        "sample": f"{rows} valid rows of the {args.workload} workload (one oracle pass, {dt:.1f} s), fp64 numpy"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": args.workload, "H": H, "V": V, "K": K, "n_roles": w.n_roles, "rows": n,
+                       "valid_rows": n_valid_local, "invocations": w.n_inv,
+                       "l2": "inputs larger than L2 (hidden %.1f GB, W %.1f GB per model)" % (n * H * 2 / 1e9, V * H * 2 / 1e9),
+                       "step": "unity_role_advantage + unity_ppo_loss_fwd_bwd",
+                       "exchange": "none" if world == 1 else "all-reduce of M_k (before) and dW (after)"},
+            "tensor_frac_of_peak_algorithmic_6HV": step_tflops_alg / peak,
+            "tensor_frac_of_peak_executed_8HV": step_tflops_exe / peak,
+            "tensor_frac_of_burst_peak_algorithmic_6HV": step_tflops_alg / peaks["tflops_burst"],
+            "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "kernels": kern,
+            "cpu_baseline": cpu_baseline}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
