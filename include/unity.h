@@ -114,6 +114,36 @@ int unity_role_advantage(unity_ctx* ctx, int32_t n_inv, int32_t n_traj, int32_t 
                          const unity_adv_params* params, int64_t n_tok, const int64_t* cu_seqlens,
                          const uint8_t* tok_mask, float* adv_inv, float* adv_tok, float* seg_mean, float* seg_std);
 
+/* Stage 1 without any allocation (the paper has no counterpart; this exists for deployment reasons).
+ *
+ * Who needs it: hosts that may not call cudaMalloc or create a unity_ctx - a trainer whose framework
+ * allocator already owns all device memory, a plug-in held to a memory budget by its host process, or a
+ * caller that cannot afford the device-wide synchronisation an allocation implies.  The result is the same
+ * as unity_role_advantage's; the per-invocation scratch (combined reward and segment id) sits in a fixed
+ * device array inside the library instead of a workspace, so no context and no workspace are involved and
+ * the call itself performs no cudaMalloc / cudaFree of any kind.
+ *
+ *   device, cuda_stream : GPU to run on (made current by the call) and the stream to enqueue on
+ *   n_inv               : at most UNITY_NOALLOC_MAX_INV, otherwise UNITY_ERR_SHAPE (nothing is launched)
+ *   bad_index_out       : optional DEVICE int32; receives non-zero (stream-ordered, no sync) when a role,
+ *                         group or trajectory id was out of range and its invocation was left out
+ *   err, err_len        : optional HOST buffer that receives a one-line reason when the return is not 0
+ *   every other argument: exactly as in unity_role_advantage
+ * Cost: each GPU that loads the library holds the array (256 B + 8 B * UNITY_NOALLOC_MAX_INV, about 0.5 MiB)
+ * until the process exits.  The first call on a device looks the array's address up once
+ * (cudaGetSymbolAddress); make that first call outside any stream capture.  All calls on a device share the
+ * one array and it keeps the previous call's contents - the call re-initialises what it reads, but two calls
+ * whose kernels can overlap on the GPU (different streams, no ordering between them) race on it: serialise them.
+ */
+#define UNITY_NOALLOC_MAX_INV 65536
+int unity_role_advantage_noalloc(int device, void* cuda_stream, int32_t n_inv, int32_t n_traj, int32_t n_roles,
+                                 int32_t n_groups, const int32_t* inv_role, const int32_t* inv_group,
+                                 const int32_t* inv_traj, const float* r_node, const float* r_turn,
+                                 const float* r_traj, const float* lam, const unity_adv_params* params,
+                                 int64_t n_tok, const int64_t* cu_seqlens, const uint8_t* tok_mask, float* adv_inv,
+                                 float* adv_tok, float* seg_mean, float* seg_std, int32_t* bad_index_out, char* err,
+                                 size_t err_len);
+
 /* ------------------------------------------------------------------------------------------------
  * Shared description of the response-token rows for stages 2 and 3.  Token i belongs to the
  * invocation s with cu_seqlens[s] <= i < cu_seqlens[s+1]; its role is inv_role[s]; the model that

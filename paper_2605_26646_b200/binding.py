@@ -25,7 +25,7 @@ UNITY_N_METRICS = 8
 
 EXPORTS = ["unity_create", "unity_destroy", "unity_workspace_bytes", "unity_workspace_min_bytes",
            "unity_check_status", "unity_last_error", "unity_launch_count", "unity_set_profiling",
-           "unity_get_profile", "unity_role_advantage",
+           "unity_get_profile", "unity_role_advantage", "unity_role_advantage_noalloc",
            "unity_logprob_fwd", "unity_ppo_loss_fwd_bwd"]
 
 
@@ -88,6 +88,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.unity_role_advantage.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, f32p,
                                          C.POINTER(unity_adv_params), i64, vp, vp, vp, vp, vp, vp]
     lib.unity_role_advantage.restype = C.c_int
+    lib.unity_role_advantage_noalloc.argtypes = [C.c_int, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, f32p,
+                                                 C.POINTER(unity_adv_params), i64, vp, vp, vp, vp, vp, vp, vp,
+                                                 C.c_char_p, C.c_size_t]
+    lib.unity_role_advantage_noalloc.restype = C.c_int
     lib.unity_logprob_fwd.argtypes = [vp, C.POINTER(unity_rows), vp, vp, vp]
     lib.unity_logprob_fwd.restype = C.c_int
     lib.unity_ppo_loss_fwd_bwd.argtypes = [vp, C.POINTER(unity_rows), C.POINTER(unity_ppo_params), vp, vp, vp,
@@ -180,6 +184,36 @@ def unity_role_advantage(ctx, n_traj: int, n_roles: int, n_groups: int, inv_role
         _ptr(tok_mask, torch.uint8, "tok_mask"), _ptr(adv_inv, f32, "adv_inv"), _ptr(adv_tok, f32, "adv_tok"),
         _ptr(seg_mean, f32, "seg_mean"), _ptr(seg_std, f32, "seg_std"))
     _raise(ctx, code)
+
+
+UNITY_NOALLOC_MAX_INV = 65536
+
+
+def unity_role_advantage_noalloc(device: int, stream_ptr: int, n_traj: int, n_roles: int, n_groups: int, inv_role,
+                                 inv_group, inv_traj, r_node, r_turn, r_traj, lam: Optional[Sequence[float]],
+                                 eps: float, ddof: int, cu_seqlens, tok_mask, adv_inv, adv_tok, seg_mean=None,
+                                 seg_std=None, bad_index_out=None) -> None:
+    """Context-free, allocation-free form of unity_role_advantage (scratch is a fixed array inside the library;
+    at most UNITY_NOALLOC_MAX_INV invocations).  Same arguments otherwise; `bad_index_out` is an optional int32
+    CUDA tensor of one element."""
+    n_inv = int(inv_role.numel())
+    n_tok = int(adv_tok.numel()) if adv_tok is not None else 0
+    lam_arr = None
+    if lam is not None:
+        flat = [float(x) for row in lam for x in (row if hasattr(row, "__iter__") else [row])]
+        lam_arr = (C.c_float * len(flat))(*flat)
+    p = unity_adv_params(eps, ddof)
+    i32, f32 = torch.int32, torch.float32
+    msg = C.create_string_buffer(256)
+    code = load_library().unity_role_advantage_noalloc(
+        device, stream_ptr, n_inv, n_traj, n_roles, n_groups, _ptr(inv_role, i32, "inv_role"),
+        _ptr(inv_group, i32, "inv_group"), _ptr(inv_traj, i32, "inv_traj"), _ptr(r_node, f32, "r_node"),
+        _ptr(r_turn, f32, "r_turn"), _ptr(r_traj, f32, "r_traj"), lam_arr, C.byref(p), n_tok,
+        _ptr(cu_seqlens, torch.int64, "cu_seqlens"), _ptr(tok_mask, torch.uint8, "tok_mask"),
+        _ptr(adv_inv, f32, "adv_inv"), _ptr(adv_tok, f32, "adv_tok"), _ptr(seg_mean, f32, "seg_mean"),
+        _ptr(seg_std, f32, "seg_std"), _ptr(bad_index_out, i32, "bad_index_out"), msg, 256)
+    if code != UNITY_OK:
+        raise UnityError(code, msg.value.decode())
 
 
 def _make_rows(hidden, W, cu_seqlens, inv_role, role_model, target, tok_mask, inv_temperature, keep):
