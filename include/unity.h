@@ -68,15 +68,14 @@ const char* unity_last_error(const unity_ctx* ctx);
 int64_t unity_launch_count(const unity_ctx* ctx);
 
 /* Measurement hooks (no counterpart in the paper).  With profiling enabled, each tensor-core GEMM launch
- * and each transpose of unity_ppo_loss_fwd_bwd / unity_logprob_fwd is bracketed by a CUDA event pair on
+ * of unity_ppo_loss_fwd_bwd / unity_logprob_fwd is bracketed by a CUDA event pair on
  * the context's stream.  unity_get_profile synchronises the stream, returns per class the summed device
  * time in milliseconds (ms[UNITY_PROF_CLASSES]) and the number of launches, and resets the counters. */
 #define UNITY_PROF_FWD_GEMM 0   /* LM-head GEMM fused with online log-softmax / gather / entropy */
 #define UNITY_PROF_GRAD_GEMM 1  /* logit recompute fused with dL/dz                              */
 #define UNITY_PROF_DH_GEMM 2    /* dHidden chunk GEMM                                            */
 #define UNITY_PROF_DW_GEMM 3    /* dW chunk GEMM                                                 */
-#define UNITY_PROF_TRANSPOSE 4  /* bf16 transposes feeding the K-major operands                  */
-#define UNITY_PROF_CLASSES 5
+#define UNITY_PROF_CLASSES 4
 int unity_set_profiling(unity_ctx* ctx, int enable);
 int unity_get_profile(unity_ctx* ctx, double* ms, int64_t* launches);
 

@@ -151,7 +151,7 @@ def unity_launch_count(ctx) -> int:
     return int(load_library().unity_launch_count(ctx))
 
 
-PROF_CLASSES = ["fwd_gemm", "grad_gemm", "dh_gemm", "dw_gemm", "transpose"]
+PROF_CLASSES = ["fwd_gemm", "grad_gemm", "dh_gemm", "dw_gemm"]
 
 
 def unity_set_profiling(ctx, enable: bool) -> None:

@@ -1,4 +1,5 @@
-// Persistent, warp-specialised bf16 GEMM for sm_100a:  C[m, n] = sum_k A[m, k] * B[n, k].
+// Persistent, warp-specialised bf16 GEMM for sm_100a:  C[m, n] = sum_k A[m, k] * B[n, k], each operand
+// either K-major ([rows, K] in memory) or MN-major ([K, rows] in memory), so no operand is ever transposed in HBM.
 //
 //   warp 0      : TMA producer  - streams 128x64 (A) and 256x64 (B) bf16 slabs into a 4-stage shared-memory ring
 //   warp 1      : MMA issuer    - one thread issues tcgen05.mma (128x256x16) into one of two 256-column TMEM
@@ -75,7 +76,13 @@ __device__ __forceinline__ unsigned pack_bf16(float lo, float hi) {
     return *reinterpret_cast<unsigned*>(&v);
 }
 
-template <int EPI>
+// Operand layouts.  K-major: the operand is stored [rows, K] and a stage holds one box of (rows x 64 K).
+// MN-major: the operand is stored [K, rows] (rows contiguous) and a stage holds rows/64 boxes of (64 rows x 64 K),
+// 8 KiB each, one after the other; the matrix descriptor then has leading byte offset 8 KiB (next 64 rows) and
+// stride byte offset 1 KiB (next 8 values of K), and 16 values of K further is 2 KiB further.
+constexpr int kMnBoxBytes = 64 * kTileK * 2;
+
+template <int EPI, bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs g) {
     extern __shared__ uint8_t smem_raw[];
@@ -125,8 +132,21 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                         if (!ptx::mbar_wait(&empty[stage], phase ^ 1, kWaitBudgetCycles) || *abort_flag) { ok = false; break; }
                         uint8_t* sA = smem + stage * kStageBytes;
                         ptx::mbar_arrive_expect_tx(&full[stage], kStageBytes);
-                        ptx::tma_load_2d(sA, &tmA, &full[stage], g.a_k0 + k * kTileK, a_row);
-                        ptx::tma_load_2d(sA + kABytes, &tmB, &full[stage], g.b_k0 + k * kTileK, b_row);
+                        if (A_MN) {
+#pragma unroll
+                            for (int j = 0; j < kTileM / 64; ++j)
+                                ptx::tma_load_2d(sA + j * kMnBoxBytes, &tmA, &full[stage], a_row + j * 64, g.a_k0 + k * kTileK);
+                        } else {
+                            ptx::tma_load_2d(sA, &tmA, &full[stage], g.a_k0 + k * kTileK, a_row);
+                        }
+                        if (B_MN) {
+#pragma unroll
+                            for (int j = 0; j < kTileN / 64; ++j)
+                                ptx::tma_load_2d(sA + kABytes + j * kMnBoxBytes, &tmB, &full[stage], b_row + j * 64,
+                                                 g.b_k0 + k * kTileK);
+                        } else {
+                            ptx::tma_load_2d(sA + kABytes, &tmB, &full[stage], g.b_k0 + k * kTileK, b_row);
+                        }
                         if (++stage == kStages) { stage = 0; phase ^= 1; }
                     }
                 }
@@ -136,7 +156,7 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = ptx::idesc_bf16_f32(kTileM, kTileN);
+            constexpr uint32_t idesc = ptx::idesc_bf16_f32(kTileM, kTileN) | (A_MN ? (1u << 15) : 0u) | (B_MN ? (1u << 16) : 0u);
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
@@ -150,11 +170,16 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                         if (!ptx::mbar_wait(&full[stage], phase, kWaitBudgetCycles) || *abort_flag) { ok = false; break; }
                         ptx::tc_fence_after();
                         const uint32_t sA = ptx::smem_u32(smem + stage * kStageBytes);
-                        const uint64_t da = ptx::smem_desc_k_sw128(sA);
-                        const uint64_t db = ptx::smem_desc_k_sw128(sA + kABytes);
+                        const uint64_t da = A_MN ? ptx::smem_desc_mn_sw128(sA, kMnBoxBytes) : ptx::smem_desc_k_sw128(sA);
+                        const uint64_t db = B_MN ? ptx::smem_desc_mn_sw128(sA + kABytes, kMnBoxBytes)
+                                                 : ptx::smem_desc_k_sw128(sA + kABytes);
+                        // start-address step (16-byte units) per 16 values of K: 32 B inside a K-major swizzle row,
+                        // 16 rows x 128 B for an MN-major operand
+                        constexpr uint32_t step_a = A_MN ? (16 * 128) >> 4 : 2;
+                        constexpr uint32_t step_b = B_MN ? (16 * 128) >> 4 : 2;
 #pragma unroll
-                        for (int kk = 0; kk < kTileK / 16; ++kk)     // +32 bytes (2 x 16-byte units) per 16 elements of K
-                            ptx::mma_bf16_ss(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (k | kk) != 0 ? 1u : 0u);
+                        for (int kk = 0; kk < kTileK / 16; ++kk)
+                            ptx::mma_bf16_ss(d_tmem, da + step_a * kk, db + step_b * kk, idesc, (k | kk) != 0 ? 1u : 0u);
                         ptx::tc_commit(&empty[stage]);
                         if (++stage == kStages) { stage = 0; phase ^= 1; }
                     }
@@ -309,23 +334,32 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
 
 cudaError_t gemm_set_attributes() {
     cudaError_t e;
-    e = cudaFuncSetAttribute(k_gemm<kEpiSoftmaxStats>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(k_gemm<kEpiSoftmaxStats, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(k_gemm<kEpiLogitGrad>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(k_gemm<kEpiLogitGrad, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(k_gemm<kEpiAccumF32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(k_gemm<kEpiAccumF32, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(k_gemm<kEpiAccumF32, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
 
-cudaError_t launch_gemm(GemmEpilogue epi, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args,
-                        int sm_count, cudaStream_t stream) {
+cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, const CUtensorMap& tmA, const CUtensorMap& tmB,
+                        const GemmArgs& args, int sm_count, cudaStream_t stream) {
     const long long units = epi == kEpiSoftmaxStats ? static_cast<long long>(args.m_tiles) * args.n_splits
                                                     : static_cast<long long>(args.m_tiles) * args.n_tiles;
     if (units <= 0 || args.k_iters <= 0) return cudaSuccess;
     const int grid = static_cast<int>(units < sm_count ? units : sm_count);
     switch (epi) {
-        case kEpiSoftmaxStats: k_gemm<kEpiSoftmaxStats><<<grid, kThreads, kSmemBytes, stream>>>(tmA, tmB, args); break;
-        case kEpiLogitGrad: k_gemm<kEpiLogitGrad><<<grid, kThreads, kSmemBytes, stream>>>(tmA, tmB, args); break;
-        default: k_gemm<kEpiAccumF32><<<grid, kThreads, kSmemBytes, stream>>>(tmA, tmB, args); break;
+        case kEpiSoftmaxStats:
+            k_gemm<kEpiSoftmaxStats, false, false><<<grid, kThreads, kSmemBytes, stream>>>(tmA, tmB, args);
+            break;
+        case kEpiLogitGrad:
+            k_gemm<kEpiLogitGrad, false, false><<<grid, kThreads, kSmemBytes, stream>>>(tmA, tmB, args);
+            break;
+        default:   // fp32 accumulate: B is always MN-major (W or hidden read in place), A is G either way round
+            if (a_mn) k_gemm<kEpiAccumF32, true, true><<<grid, kThreads, kSmemBytes, stream>>>(tmA, tmB, args);
+            else k_gemm<kEpiAccumF32, false, true><<<grid, kThreads, kSmemBytes, stream>>>(tmA, tmB, args);
+            break;
     }
     return cudaGetLastError();
 }

@@ -21,7 +21,7 @@ constexpr int kStatusBadIndex = 1;
 constexpr int kStatusTimeout = 2;
 
 // ----------------------------------------------------------------------------------------------
-// GEMM  C[m, n] = sum_k A[m, k] * B[n, k]   (both operands K-major bf16, fp32 accumulation in TMEM)
+// GEMM  C[m, n] = sum_k A[m, k] * B[n, k]   (bf16 operands, K-major or MN-major, fp32 accumulation in TMEM)
 // ----------------------------------------------------------------------------------------------
 enum GemmEpilogue : int {
     kEpiSoftmaxStats = 0,   // online (max, sum exp, sum exp*z, target logit) per row; nothing of size M x N stored
@@ -57,12 +57,14 @@ struct GemmArgs {
     int* status;
 };
 
-cudaError_t launch_gemm(GemmEpilogue epi, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args,
-                        int sm_count, cudaStream_t stream);
+// a_mn: A is MN-major (only for kEpiAccumF32, whose B operand is always MN-major).  For an MN-major operand
+// a_row0 / b_row0 index the contiguous dimension of its tensor map and a_k0 / b_k0 its rows.
+cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, const CUtensorMap& tmA, const CUtensorMap& tmB,
+                        const GemmArgs& args, int sm_count, cudaStream_t stream);
 cudaError_t gemm_set_attributes();
 
 // ----------------------------------------------------------------------------------------------
-// streaming kernels (advantage, routing, token terms, transposes); each returns the launch error
+// streaming kernels (advantage, routing, token terms); each returns the launch error
 // ----------------------------------------------------------------------------------------------
 struct AdvArgs {
     int n_inv, n_traj, n_roles, n_groups;
@@ -103,10 +105,6 @@ cudaError_t launch_route(const RouteArgs& a, cudaStream_t stream, int* n_launche
 
 cudaError_t launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* target, const int* slot_tok, int n_slots,
                                int H, __nv_bfloat16* hp, int* target_p, cudaStream_t stream);
-
-// out[c, r] = in[r, c] for a bf16 matrix [rows, cols] with row pitch ld_in; out pitch ld_out.
-cudaError_t launch_transpose_bf16(const __nv_bfloat16* in, long long ld_in, __nv_bfloat16* out, long long ld_out,
-                                  int rows, int cols, cudaStream_t stream);
 
 struct TokenArgs {
     int n_slots, n_splits, K, n_roles, n_inv;

@@ -126,7 +126,20 @@ __device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t saddr) {
     d |= static_cast<uint64_t>(2) << 61;                       // layout: 128-byte swizzle
     return d;
 }
-// Instruction descriptor for kind::f16: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
+// MN-major operand (stored [K, rows], rows contiguous), 128-byte swizzle: the stage holds boxes of 64 rows x K,
+// one shared-memory row of 128 B per value of K; `box_bytes` apart lies the box of the next 64 rows (leading
+// byte offset) and 1024 B apart the next group of eight K values (stride byte offset).
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t saddr, uint32_t box_bytes) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((saddr & 0x3FFFF) >> 4);
+    d |= static_cast<uint64_t>(box_bytes >> 4) << 16;
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;
+    d |= static_cast<uint64_t>(1) << 46;
+    d |= static_cast<uint64_t>(2) << 61;
+    return d;
+}
+// Instruction descriptor for kind::f16: bf16 x bf16 -> fp32, M x N tile, both operands K-major
+// (bit 15 / bit 16 set mark A / B as MN-major).
 __host__ __device__ constexpr uint32_t idesc_bf16_f32(int M, int N) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(N >> 3) << 17) |
            (static_cast<uint32_t>(M >> 4) << 24);

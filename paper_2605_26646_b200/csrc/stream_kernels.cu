@@ -1,5 +1,5 @@
 // Streaming (HBM / latency bound) kernels of libunity: role-level advantage, routing of response
-// tokens to their model through the agent-to-model table, row packing, bf16 transposes, per-token PPO
+// tokens to their model through the agent-to-model table, row packing, per-token PPO
 // terms with fixed-order reductions, and the dHidden write-back.  No floating-point atomics anywhere:
 // every reduction has a fixed order, so results are bitwise reproducible.
 #include "internal.h"
@@ -249,34 +249,6 @@ __global__ void k_gather_rows(const __nv_bfloat16* __restrict__ hidden, const in
     if (lane == 0) target_p[slot] = tok >= 0 ? target[tok] : 0;
 }
 
-// 64 x 64 bf16 tile transpose through shared memory; 32-bit accesses on both sides.
-__global__ void k_transpose_bf16(const __nv_bfloat16* __restrict__ in, long long ld_in, __nv_bfloat16* __restrict__ out,
-                                 long long ld_out, int rows, int cols) {
-    __shared__ __nv_bfloat16 tile[64][66];
-    const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;     // 32 x 8 threads
-    for (int rr = ty; rr < 64; rr += 8) {
-        const int r = r0 + rr, c = c0 + tx * 2;
-        __nv_bfloat162 v = __floats2bfloat162_rn(0.f, 0.f);
-        if (r < rows) {
-            if (c + 1 < cols) v = *reinterpret_cast<const __nv_bfloat162*>(in + static_cast<long long>(r) * ld_in + c);
-            else if (c < cols) v.x = in[static_cast<long long>(r) * ld_in + c];
-        }
-        tile[rr][tx * 2] = v.x;
-        tile[rr][tx * 2 + 1] = v.y;
-    }
-    __syncthreads();
-    for (int cc = ty; cc < 64; cc += 8) {
-        const int c = c0 + cc, r = r0 + tx * 2;
-        if (c >= cols) continue;
-        __nv_bfloat162 v;
-        v.x = tile[tx * 2][cc];
-        v.y = tile[tx * 2 + 1][cc];
-        if (r + 1 < rows) *reinterpret_cast<__nv_bfloat162*>(out + static_cast<long long>(c) * ld_out + r) = v;
-        else if (r < rows) out[static_cast<long long>(c) * ld_out + r] = v.x;
-    }
-}
-
 // ------------------------------------------------------------------------------------------------
 // Per-token PPO terms
 // ------------------------------------------------------------------------------------------------
@@ -456,14 +428,6 @@ cudaError_t launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* targe
                                int H, __nv_bfloat16* hp, int* target_p, cudaStream_t stream) {
     if (n_slots == 0) return cudaSuccess;
     k_gather_rows<<<(n_slots + 7) / 8, 256, 0, stream>>>(hidden, target, slot_tok, n_slots, H, hp, target_p);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_transpose_bf16(const __nv_bfloat16* in, long long ld_in, __nv_bfloat16* out, long long ld_out,
-                                  int rows, int cols, cudaStream_t stream) {
-    if (rows == 0 || cols == 0) return cudaSuccess;
-    dim3 grid((cols + 63) / 64, (rows + 63) / 64);
-    k_transpose_bf16<<<grid, 256, 0, stream>>>(in, ld_in, out, ld_out, rows, cols);
     return cudaGetLastError();
 }
 

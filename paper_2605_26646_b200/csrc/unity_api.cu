@@ -35,8 +35,10 @@ struct unity_ctx {
 namespace {
 
 constexpr size_t kAlign = 256;
-constexpr int kChunkRows = 16384;    // token rows per gradient chunk (multiple of kTileM)
-constexpr int kChunkVocab = 8192;    // vocabulary entries per gradient chunk (multiple of kTileN)
+// Gradient chunk: 148 row tiles x 74 vocabulary tiles.  With one CTA per SM (148) every chunk GEMM then runs a
+// whole number of waves: recompute 148 x 74 tiles, dHidden 148 x ceil(H/256), dW 148 x ceil(H/256).
+constexpr int kChunkRows = 148 * kTileM;     // 18944 token rows
+constexpr int kChunkVocab = 74 * kTileN;     // 18944 vocabulary entries
 constexpr int kMinChunkRows = 1024;
 constexpr int kMinChunkVocab = 1024;
 
@@ -97,7 +99,7 @@ struct Layout {
     __nv_bfloat16* hp; int* target_p; float4* stats; float *row_lse, *row_ent, *row_logp;
     // loss + backward
     float *coef_a, *coef_b, *inv_sums;
-    __nv_bfloat16 *hT, *WT, *G, *GT; float* dHc;
+    __nv_bfloat16* G; float* dHc;
     long long max_slots, stats_cap;
     int n_blocks, chunk_rows, chunk_vocab;
     size_t bytes;
@@ -132,10 +134,7 @@ Layout carve(char* base, size_t cap, long long n_tok, int H, int V, int K, int n
         L.coef_a = b.take<float>(L.max_slots);
         L.coef_b = b.take<float>(L.max_slots);
         L.inv_sums = b.take<float>(static_cast<size_t>(n_inv) * 9 + 1);
-        L.hT = b.take<__nv_bfloat16>(static_cast<size_t>(H) * L.max_slots);
-        L.WT = b.take<__nv_bfloat16>(static_cast<size_t>(H) * V);
         L.G = b.take<__nv_bfloat16>(static_cast<size_t>(chunk_rows) * chunk_vocab);
-        L.GT = b.take<__nv_bfloat16>(static_cast<size_t>(chunk_rows) * chunk_vocab);
         L.dHc = b.take<float>(static_cast<size_t>(chunk_rows) * H);
     }
     L.bytes = up(b.off, kAlign);
@@ -152,11 +151,13 @@ int wanted_chunk_vocab(int V) {
     return static_cast<int>(vp < kChunkVocab ? vp : kChunkVocab);
 }
 
+// Tensor map over a row-major bf16 matrix [rows, inner]; boxes are 64 elements (128 B, one swizzle row) wide and
+// box_rows high.  K-major operands use box_rows = tile rows (128 / 256); MN-major operands use 64 (= kTileK).
 int make_tmap(unity_ctx* ctx, CUtensorMap* tm, const void* ptr, uint64_t inner, uint64_t rows, uint64_t pitch_bytes,
               uint32_t box_rows) {
     cuuint64_t dims[2] = {inner, rows};
     cuuint64_t strides[1] = {pitch_bytes};
-    cuuint32_t box[2] = {static_cast<cuuint32_t>(kTileK), box_rows};
+    cuuint32_t box[2] = {64u, box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = ctx->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -268,7 +269,7 @@ int forward_sweep(unity_ctx* ctx, const unity_rows* r, RowPlan& P) {
         g.status = ctx->d_status;
         {
             ProfScope ps(ctx, UNITY_PROF_FWD_GEMM);
-            CUDA_TRY(ctx, launch_gemm(kEpiSoftmaxStats, tmA, tmB, g, ctx->sm_count, st));
+            CUDA_TRY(ctx, launch_gemm(kEpiSoftmaxStats, false, tmA, tmB, g, ctx->sm_count, st));
         }
         nl += 1;
     }
@@ -531,19 +532,14 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
     __nv_bfloat16* dH = static_cast<__nv_bfloat16*>(dHidden);
     CUDA_TRY(ctx, launch_zero_masked_rows(L.tok_slot, rows->n_tok, H, dH, st));
     nl += 1;
-    const long long ldT = L.max_slots;
-    {
-        ProfScope ps(ctx, UNITY_PROF_TRANSPOSE);
-        CUDA_TRY(ctx, launch_transpose_bf16(L.hp, H, L.hT, ldT, P.n_slots, H, st));
-    }
-    nl += P.n_slots > 0;
-
-    CUtensorMap tm_hp, tm_hT, tm_WT;
+    // Operands are read in place: hidden rows and W serve as K-major operands (contraction over H) and as
+    // MN-major operands (contraction over tokens / vocabulary); nothing is transposed in memory.
+    CUtensorMap tm_hp_k, tm_hp_mn;
     if (P.n_slots > 0) {
-        if ((rc = make_tmap(ctx, &tm_hp, L.hp, H, P.n_slots, static_cast<uint64_t>(H) * 2, kTileM))) return rc;
-        if ((rc = make_tmap(ctx, &tm_hT, L.hT, P.n_slots, H, static_cast<uint64_t>(ldT) * 2, kTileN))) return rc;
+        if ((rc = make_tmap(ctx, &tm_hp_k, L.hp, H, P.n_slots, static_cast<uint64_t>(H) * 2, kTileM))) return rc;
+        if ((rc = make_tmap(ctx, &tm_hp_mn, L.hp, H, P.n_slots, static_cast<uint64_t>(H) * 2, kTileK))) return rc;
     }
-    if ((rc = make_tmap(ctx, &tm_WT, L.WT, V, H, static_cast<uint64_t>(V) * 2, kTileN))) return rc;
+    const int h_tiles = (H + kTileN - 1) / kTileN;
 
     for (int k = 0; k < K; ++k) {
         const int rows_k = P.offsets[k + 1] - P.offsets[k];
@@ -553,20 +549,16 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
             continue;
         }
         const __nv_bfloat16* Wk = static_cast<const __nv_bfloat16*>(rows->W[k]);
-        {
-            ProfScope ps(ctx, UNITY_PROF_TRANSPOSE);
-            CUDA_TRY(ctx, launch_transpose_bf16(Wk, H, L.WT, V, V, H, st));
-        }
-        nl += 1;
-        CUtensorMap tm_W;
-        if ((rc = make_tmap(ctx, &tm_W, Wk, H, V, static_cast<uint64_t>(H) * 2, kTileN))) return rc;
+        CUtensorMap tm_W_k, tm_W_mn;
+        if ((rc = make_tmap(ctx, &tm_W_k, Wk, H, V, static_cast<uint64_t>(H) * 2, kTileN))) return rc;
+        if ((rc = make_tmap(ctx, &tm_W_mn, Wk, H, V, static_cast<uint64_t>(H) * 2, kTileK))) return rc;
 
         for (int c0 = 0; c0 < rows_k; c0 += cr) {
             const int nc = rows_k - c0 < cr ? rows_k - c0 : cr;          // multiple of kTileM
             const int slot0 = P.offsets[k] + c0;
             for (int v0 = 0; v0 < V; v0 += cv) {
                 const int vc = V - v0 < cv ? V - v0 : cv;
-                // (1) recompute the logits of this (rows x vocab) chunk and form dL/dz in bf16
+                // (1) recompute the logits of this (rows x vocab) chunk and form dL/dz in bf16: G[nc, vc]
                 GemmArgs g;
                 memset(&g, 0, sizeof(g));
                 g.m_tiles = nc / kTileM; g.n_tiles = (vc + kTileN - 1) / kTileN; g.k_iters = H / kTileK;
@@ -577,40 +569,36 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 g.G = L.G; g.ldg = cv; g.status = ctx->d_status;
                 {
                     ProfScope ps(ctx, UNITY_PROF_GRAD_GEMM);
-                    CUDA_TRY(ctx, launch_gemm(kEpiLogitGrad, tm_hp, tm_W, g, ctx->sm_count, st));
+                    CUDA_TRY(ctx, launch_gemm(kEpiLogitGrad, false, tm_hp_k, tm_W_k, g, ctx->sm_count, st));
                 }
-                // (2) token-major copy of the chunk for the weight gradient
-                {
-                    ProfScope ps(ctx, UNITY_PROF_TRANSPOSE);
-                    CUDA_TRY(ctx, launch_transpose_bf16(L.G, cv, L.GT, cr, nc, vc, st));
-                }
-                // (3) dH_chunk[nc, H] (+)= G[nc, vc] * W[v0:v0+vc, :]
-                CUtensorMap tm_G, tm_GT;
-                if ((rc = make_tmap(ctx, &tm_G, L.G, vc, nc, static_cast<uint64_t>(cv) * 2, kTileM))) return rc;
-                if ((rc = make_tmap(ctx, &tm_GT, L.GT, nc, vc, static_cast<uint64_t>(cr) * 2, kTileM))) return rc;
+                // G viewed as [nc rows, vc]: K-major A for dHidden (contract over vc), MN-major A for dW (rows = K)
+                CUtensorMap tm_G_k, tm_G_mn;
+                if ((rc = make_tmap(ctx, &tm_G_k, L.G, vc, nc, static_cast<uint64_t>(cv) * 2, kTileM))) return rc;
+                if ((rc = make_tmap(ctx, &tm_G_mn, L.G, vc, nc, static_cast<uint64_t>(cv) * 2, kTileK))) return rc;
+                // (2) dH_chunk[nc, H] (+)= G[nc, vc] * W[v0:v0+vc, :]      (B = W, MN-major: rows v are K)
                 GemmArgs h;
                 memset(&h, 0, sizeof(h));
-                h.m_tiles = nc / kTileM; h.n_tiles = (H + kTileN - 1) / kTileN; h.k_iters = (vc + kTileK - 1) / kTileK;
+                h.m_tiles = nc / kTileM; h.n_tiles = h_tiles; h.k_iters = (vc + kTileK - 1) / kTileK;
                 h.group_m = 16;
-                h.a_row0 = 0; h.b_row0 = 0; h.a_k0 = 0; h.b_k0 = v0; h.m_rows = nc; h.n_cols = H;
+                h.a_row0 = 0; h.a_k0 = 0; h.b_row0 = 0; h.b_k0 = v0; h.m_rows = nc; h.n_cols = H;
                 h.C = L.dHc; h.ldc = H; h.beta = v0 > 0; h.status = ctx->d_status;
                 {
                     ProfScope ps(ctx, UNITY_PROF_DH_GEMM);
-                    CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, tm_G, tm_WT, h, ctx->sm_count, st));
+                    CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, false, tm_G_k, tm_W_mn, h, ctx->sm_count, st));
                 }
-                // (4) dW[v0:v0+vc, :] (+)= G^T[vc, nc] * h[rows, :]
+                // (3) dW[v0:v0+vc, :] (+)= G^T[vc, nc] * hidden[slot0:slot0+nc, :]   (both operands MN-major)
                 GemmArgs w;
                 memset(&w, 0, sizeof(w));
-                w.m_tiles = (vc + kTileM - 1) / kTileM; w.n_tiles = (H + kTileN - 1) / kTileN; w.k_iters = nc / kTileK;
+                w.m_tiles = (vc + kTileM - 1) / kTileM; w.n_tiles = h_tiles; w.k_iters = nc / kTileK;
                 w.group_m = 16;
-                w.a_row0 = 0; w.b_row0 = 0; w.a_k0 = 0; w.b_k0 = slot0; w.m_rows = vc; w.n_cols = H;
+                w.a_row0 = 0; w.a_k0 = 0; w.b_row0 = 0; w.b_k0 = slot0; w.m_rows = vc; w.n_cols = H;
                 w.C = dWk + static_cast<long long>(v0) * H; w.ldc = H;
                 w.beta = (params->accumulate_dW || c0 > 0) ? 1 : 0; w.status = ctx->d_status;
                 {
                     ProfScope ps(ctx, UNITY_PROF_DW_GEMM);
-                    CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, tm_GT, tm_hT, w, ctx->sm_count, st));
+                    CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, true, tm_G_mn, tm_hp_mn, w, ctx->sm_count, st));
                 }
-                nl += 4;
+                nl += 3;
             }
             CUDA_TRY(ctx, launch_store_dhidden(L.dHc, L.slot_tok, slot0, nc, H, dH, st));
             nl += 1;
