@@ -154,6 +154,7 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=256, help="valid rows per oracle step (reference arm / cpu baseline)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ctas", default="", help="CTAs per tile for the fwd,grad,dH,dW GEMMs, e.g. 1,1,2,2 (default: library's)")
     ap.add_argument("--cut-rows", type=int, default=0, help="profile-capture helper: run on a cut of the workload")
     args = ap.parse_args()
     if args.warmup < 3 and args.cut_rows == 0:
@@ -189,6 +190,9 @@ def main():
     lam = w.lam.tolist()
     ws_bytes = ub.unity_workspace_bytes(n, H, V, K, w.n_inv)
     ctx = ub.Context(local, ws_bytes)
+    if args.ctas:
+        for option, value in enumerate(int(x) for x in args.ctas.split(",")):
+            ctx.set_option(option, value)
 
     adv_inv = torch.empty(w.n_inv, device=dev)
     adv_tok = torch.empty(n, device=dev)

@@ -77,6 +77,16 @@ int64_t unity_launch_count(const unity_ctx* ctx);
 #define UNITY_PROF_DW_GEMM 3    /* dW chunk GEMM                                                 */
 #define UNITY_PROF_CLASSES 4
 int unity_set_profiling(unity_ctx* ctx, int enable);
+
+/* Tuning knobs (no counterpart in the paper).  Each GEMM class can run with one CTA per 128 x 256 output tile
+ * (value 1) or with a pair of CTAs on neighbouring SMs sharing a 256 x 256 tile (value 2).  Results do not depend
+ * on the choice beyond fp32 summation order inside the tensor core.  Defaults: 1, 2, 2, 2 (measured best on
+ * the H=3584, V=152064 workload; all choices are within a few per cent under the 1 kW power cap). */
+#define UNITY_OPT_CTAS_FWD 0
+#define UNITY_OPT_CTAS_GRAD 1
+#define UNITY_OPT_CTAS_DH 2
+#define UNITY_OPT_CTAS_DW 3
+int unity_set_option(unity_ctx* ctx, int option, int value);
 int unity_get_profile(unity_ctx* ctx, double* ms, int64_t* launches);
 
 /* ------------------------------------------------------------------------------------------------

@@ -25,7 +25,7 @@ UNITY_N_METRICS = 8
 
 EXPORTS = ["unity_create", "unity_destroy", "unity_workspace_bytes", "unity_workspace_min_bytes",
            "unity_check_status", "unity_last_error", "unity_launch_count", "unity_set_profiling",
-           "unity_get_profile", "unity_role_advantage", "unity_role_advantage_noalloc",
+           "unity_get_profile", "unity_set_option", "unity_role_advantage", "unity_role_advantage_noalloc",
            "unity_logprob_fwd", "unity_ppo_loss_fwd_bwd"]
 
 
@@ -83,6 +83,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.unity_launch_count.restype = i64
     lib.unity_set_profiling.argtypes = [vp, C.c_int]
     lib.unity_set_profiling.restype = C.c_int
+    lib.unity_set_option.argtypes = [vp, C.c_int, C.c_int]
+    lib.unity_set_option.restype = C.c_int
     lib.unity_get_profile.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
     lib.unity_get_profile.restype = C.c_int
     lib.unity_role_advantage.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, f32p,
@@ -156,6 +158,13 @@ PROF_CLASSES = ["fwd_gemm", "grad_gemm", "dh_gemm", "dw_gemm"]
 
 def unity_set_profiling(ctx, enable: bool) -> None:
     _raise(ctx, load_library().unity_set_profiling(ctx, 1 if enable else 0))
+
+
+OPT_CTAS = {"fwd_gemm": 0, "grad_gemm": 1, "dh_gemm": 2, "dw_gemm": 3}
+
+
+def unity_set_option(ctx, option: int, value: int) -> None:
+    _raise(ctx, load_library().unity_set_option(ctx, option, value))
 
 
 def unity_get_profile(ctx) -> dict:
@@ -295,6 +304,9 @@ class Context:
 
     def set_profiling(self, enable: bool):
         unity_set_profiling(self.ctx, enable)
+
+    def set_option(self, option: int, value: int):
+        unity_set_option(self.ctx, option, value)
 
     def get_profile(self) -> dict:
         return unity_get_profile(self.ctx)

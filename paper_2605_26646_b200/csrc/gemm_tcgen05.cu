@@ -1,19 +1,29 @@
-// Persistent, warp-specialised bf16 GEMM for sm_100a:  C[m, n] = sum_k A[m, k] * B[n, k], each operand
-// either K-major ([rows, K] in memory) or MN-major ([K, rows] in memory), so no operand is ever transposed in HBM.
+// Persistent, warp-specialised bf16 GEMM for sm_100a:  C[m, n] = sum_k A[m, k] * B[n, k], each operand either
+// K-major ([rows, K] in memory) or MN-major ([K, rows] in memory), so no operand is ever transposed in HBM.
 //
-//   warp 0      : TMA producer  - streams 128x64 (A) and 256x64 (B) bf16 slabs into a 4-stage shared-memory ring
-//   warp 1      : MMA issuer    - one thread issues tcgen05.mma (128x256x16) into one of two 256-column TMEM
-//                                 accumulator stages and commits completion to mbarriers
-//   warps 2..5  : epilogue      - each thread owns one accumulator row (one TMEM lane), drains it 32 columns at
-//                                 a time with tcgen05.ld while the MMA warp already fills the other stage
+// The kernel exists in two forms (template parameter CTAS):
+//   CTAS = 1 : one CTA computes a 128 x 256 output tile (tcgen05.mma.cta_group::1), 4-stage ring of 48 KiB slabs.
+//   CTAS = 2 : two CTAs on neighbouring SMs (a cluster of 2) share one 256 x 256 tile: each loads its own 128 rows
+//              of A and its own 128 of the 256 rows of B (32 KiB per K slab, 6-stage ring) and one
+//              tcgen05.mma.cta_group::2 issued by the even CTA multiplies across both shared memories; each CTA's
+//              tensor memory receives the 128 x 256 accumulator block of its own rows.
+// Per CTA:
+//   warp 0      : TMA producer  - streams its A and B slabs into the shared-memory ring; with CTAS = 2 the bytes of
+//                                 both CTAs are counted on the even CTA's barrier
+//   warp 1      : MMA issuer    - one thread (of the even CTA) issues the MMAs into one of two 256-column
+//                                 accumulator stages and commits completion to the barriers of the CTA(s)
+//   warps 2..5  : epilogue      - each thread owns one accumulator row (one TMEM lane), drains it 32 columns at a
+//                                 time with tcgen05.ld while the MMAs already fill the other stage
 //
 // Three epilogues share the main loop:
 //   softmax statistics : running (max, sum exp, sum exp*z, target logit) per row across a sweep of vocabulary
 //                        tiles; nothing of size rows x vocabulary is ever written
 //   logit gradient     : dL/dz = a*(onehot - p) - b*p*(z - lse + H) in bf16 for a bounded chunk
 //   fp32 accumulate    : C (+)= acc
-// Every mbarrier wait is bounded; on expiry the CTA records a timeout status, all roles leave their loops and
-// the kernel frees its tensor memory and returns.
+// Every mbarrier wait is bounded; on expiry the CTA records a timeout status, all its roles leave their loops, and
+// after a cluster-wide rendezvous the CTA(s) free their tensor memory and return.
+#include <cstring>
+
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -21,54 +31,64 @@ namespace unity {
 
 namespace {
 
-constexpr int kStages = 4;
-constexpr int kABytes = kTileM * kTileK * 2;              // 16 KiB
-constexpr int kBBytes = kTileN * kTileK * 2;              // 32 KiB
-constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kAccStages = 2;
 constexpr int kTmemCols = kAccStages * kTileN;            // 512: all of tensor memory
 constexpr int kBarBytes = 256;
-constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kBarBytes;
 constexpr int kThreads = 192;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kNegBig = -3.0e38f;
+// MN-major operands: a stage holds boxes of 64 rows x 64 K (8 KiB), one after the other.
+constexpr int kMnBoxBytes = 64 * kTileK * 2;
+
+template <int CTAS>
+struct Cfg {
+    static constexpr int kTileRows = kCtaM * CTAS;               // rows of one output tile (128 or 256)
+    static constexpr int kBRows = kTileN / CTAS;                 // rows of B this CTA loads (256 or 128)
+    static constexpr int kABytes = kCtaM * kTileK * 2;           // 16 KiB
+    static constexpr int kBBytes = kBRows * kTileK * 2;          // 32 or 16 KiB
+    static constexpr int kStageBytes = kABytes + kBBytes;        // 48 or 32 KiB
+    static constexpr int kStages = CTAS == 1 ? 4 : 6;
+    static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kBarBytes;
+};
 
 struct Unit {
     int m_tile, n_begin, n_end, split;
 };
 
-// Work decomposition.  Softmax: a unit is (row tile, vocabulary split); groups of `gm` row tiles x all splits
-// are laid out consecutively so that one wave of CTAs shares a small set of A tiles (L2 resident) while the
-// splits stream disjoint parts of B.  Other epilogues: one output tile per unit, m fastest inside groups of
-// `gm` row tiles.
+// Work decomposition over CTA pairs; `it` counts the rounds of a pair's persistent loop.
+// Softmax: a unit is (256-row tile, vocabulary split).  Round `it` works on row-tile group `it` (gm row tiles): pair
+// p takes split p / gm_here of row tile p % gm_here and pairs beyond gm_here * n_splits sit the round out.  All pairs
+// of a round therefore share gm A tiles (L2 resident) and each split's stream of B tiles is fetched from HBM once, by
+// pairs that sweep it in step.  Other epilogues: one 256 x 256 output tile per unit, unit = pair + it * n_pairs, m
+// fastest inside groups of gm row tiles.
+// Returns false when the pair has no more work; `valid` is false for a round the pair sits out.
 template <int EPI>
-__device__ __forceinline__ int num_units(const GemmArgs& g) {
-    return EPI == kEpiSoftmaxStats ? g.m_tiles * g.n_splits : g.m_tiles * g.n_tiles;
-}
-template <int EPI>
-__device__ __forceinline__ Unit get_unit(const GemmArgs& g, int u, int gm) {
-    Unit t;
+__device__ __forceinline__ bool next_unit(const GemmArgs& g, int it, int pair, int n_pairs, int gm, Unit& t, bool& valid) {
     if (EPI == kEpiSoftmaxStats) {
-        const int per_group = gm * g.n_splits;
-        const int grp = u / per_group, r = u - grp * per_group;
-        const int m0 = grp * gm;
+        const int m0 = it * gm;
+        if (m0 >= g.m_tiles) return false;
         const int gm_here = min(gm, g.m_tiles - m0);
-        t.split = r / gm_here;
-        t.m_tile = m0 + (r - t.split * gm_here);
+        valid = pair < gm_here * g.n_splits;
+        t.split = pair / gm_here;
+        t.m_tile = m0 + (pair - t.split * gm_here);
         t.n_begin = t.split * g.tiles_per_split;
         t.n_end = min(t.n_begin + g.tiles_per_split, g.n_tiles);
+        return true;
     } else {
+        const int u = pair + it * n_pairs;
+        if (u >= g.m_tiles * g.n_tiles) return false;
         const int per_group = gm * g.n_tiles;
         const int grp = u / per_group, r = u - grp * per_group;
         const int m0 = grp * gm;
         const int gm_here = min(gm, g.m_tiles - m0);
-        const int nt = r / gm_here;
-        t.m_tile = m0 + (r - nt * gm_here);
-        t.n_begin = nt;
-        t.n_end = nt + 1;
+        const int q = r / gm_here;
+        t.m_tile = m0 + (r - q * gm_here);
         t.split = 0;
+        t.n_begin = q;
+        t.n_end = q + 1;
+        valid = true;
+        return true;
     }
-    return t;
 }
 
 __device__ __forceinline__ unsigned pack_bf16(float lo, float hi) {
@@ -76,76 +96,81 @@ __device__ __forceinline__ unsigned pack_bf16(float lo, float hi) {
     return *reinterpret_cast<unsigned*>(&v);
 }
 
-// Operand layouts.  K-major: the operand is stored [rows, K] and a stage holds one box of (rows x 64 K).
-// MN-major: the operand is stored [K, rows] (rows contiguous) and a stage holds rows/64 boxes of (64 rows x 64 K),
-// 8 KiB each, one after the other; the matrix descriptor then has leading byte offset 8 KiB (next 64 rows) and
-// stride byte offset 1 KiB (next 8 values of K), and 16 values of K further is 2 KiB further.
-constexpr int kMnBoxBytes = 64 * kTileK * 2;
-
-template <int EPI, bool A_MN, bool B_MN>
+template <int EPI, bool A_MN, bool B_MN, int CTAS>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs g) {
+    using C = Cfg<CTAS>;
+    constexpr int kStages = C::kStages, kStageBytes = C::kStageBytes, kABytes = C::kABytes;
     extern __shared__ uint8_t smem_raw[];
+    // the dynamic shared-memory window starts at the same offset in both CTAs of a pair, so all offsets below match
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
-    uint64_t* full = bars;                       // [kStages]  TMA bytes landed
+    uint64_t* full = bars;                       // [kStages]  (even CTA) bytes of both CTAs landed
     uint64_t* empty = bars + kStages;            // [kStages]  MMAs that read the stage have completed
     uint64_t* acc_full = bars + 2 * kStages;     // [2]        accumulator stage complete
-    uint64_t* acc_empty = acc_full + kAccStages; // [2]        accumulator stage drained by the epilogue
+    uint64_t* acc_empty = acc_full + kAccStages; // [2]        (even CTA) stage drained by the epilogues of both CTAs
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + kAccStages);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t cta_rank = CTAS == 2 ? ptx::cluster_ctarank() : 0u;     // 0: issues the MMAs, 1: its peer
+    const int pair = CTAS == 2 ? blockIdx.x >> 1 : blockIdx.x;              // index of this worker (CTA or CTA pair)
+    const int n_pairs = CTAS == 2 ? gridDim.x >> 1 : gridDim.x;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
-        for (int s = 0; s < kAccStages; ++s) { ptx::mbar_init(&acc_full[s], 1); ptx::mbar_init(&acc_empty[s], 4); }
+        for (int s = 0; s < kAccStages; ++s) { ptx::mbar_init(&acc_full[s], 1); ptx::mbar_init(&acc_empty[s], 4 * CTAS); }
         *abort_flag = 0;
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&tmA);
         ptx::prefetch_tensormap(&tmB);
     }
     if (warp == 1) {
-        ptx::tmem_alloc(tmem_slot, kTmemCols);
-        ptx::tmem_relinquish();
+        if (CTAS == 2) { ptx::tmem_alloc_pair(tmem_slot, kTmemCols); ptx::tmem_relinquish_pair(); }
+        else { ptx::tmem_alloc(tmem_slot, kTmemCols); ptx::tmem_relinquish(); }
     }
     ptx::tc_fence_before();
-    __syncthreads();
+    if (CTAS == 2) ptx::cluster_sync_all();   // barriers of both CTAs are initialised before anyone signals across
+    else __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int n_units = num_units<EPI>(g);
     const int gm = max(1, g.group_m);
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------------ TMA producer (both CTAs)
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-                const Unit t = get_unit<EPI>(g, u, gm);
-                const int a_row = g.a_row0 + t.m_tile * kTileM;
+            for (int it = 0; ok; ++it) {
+                Unit t;
+                bool valid;
+                if (!next_unit<EPI>(g, it, pair, n_pairs, gm, t, valid)) break;
+                if (!valid) continue;
+                const int a_row = g.a_row0 + t.m_tile * C::kTileRows + static_cast<int>(cta_rank) * kCtaM;
                 for (int nt = t.n_begin; nt < t.n_end && ok; ++nt) {
-                    const int b_row = g.b_row0 + nt * kTileN;
+                    const int b_row = g.b_row0 + nt * kTileN + static_cast<int>(cta_rank) * C::kBRows;
                     for (int k = 0; k < g.k_iters; ++k) {
                         if (!ptx::mbar_wait(&empty[stage], phase ^ 1, kWaitBudgetCycles) || *abort_flag) { ok = false; break; }
                         uint8_t* sA = smem + stage * kStageBytes;
-                        ptx::mbar_arrive_expect_tx(&full[stage], kStageBytes);
+                        // completion bytes are counted on the barrier of the CTA that issues the MMAs
+                        const uint32_t bar = CTAS == 2 ? ptx::mapa(ptx::smem_u32(&full[stage]), 0) : ptx::smem_u32(&full[stage]);
+                        if (cta_rank == 0) ptx::mbar_arrive_expect_tx(&full[stage], CTAS * kStageBytes);
                         if (A_MN) {
 #pragma unroll
-                            for (int j = 0; j < kTileM / 64; ++j)
-                                ptx::tma_load_2d(sA + j * kMnBoxBytes, &tmA, &full[stage], a_row + j * 64, g.a_k0 + k * kTileK);
+                            for (int j = 0; j < kCtaM / 64; ++j)
+                                ptx::tma_load_2d_on<CTAS>(sA + j * kMnBoxBytes, &tmA, bar, a_row + j * 64, g.a_k0 + k * kTileK);
                         } else {
-                            ptx::tma_load_2d(sA, &tmA, &full[stage], g.a_k0 + k * kTileK, a_row);
+                            ptx::tma_load_2d_on<CTAS>(sA, &tmA, bar, g.a_k0 + k * kTileK, a_row);
                         }
                         if (B_MN) {
 #pragma unroll
-                            for (int j = 0; j < kTileN / 64; ++j)
-                                ptx::tma_load_2d(sA + kABytes + j * kMnBoxBytes, &tmB, &full[stage], b_row + j * 64,
-                                                 g.b_k0 + k * kTileK);
+                            for (int j = 0; j < C::kBRows / 64; ++j)
+                                ptx::tma_load_2d_on<CTAS>(sA + kABytes + j * kMnBoxBytes, &tmB, bar, b_row + j * 64,
+                                                          g.b_k0 + k * kTileK);
                         } else {
-                            ptx::tma_load_2d(sA + kABytes, &tmB, &full[stage], g.b_k0 + k * kTileK, b_row);
+                            ptx::tma_load_2d_on<CTAS>(sA + kABytes, &tmB, bar, g.b_k0 + k * kTileK, b_row);
                         }
                         if (++stage == kStages) { stage = 0; phase ^= 1; }
                     }
@@ -154,14 +179,17 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
             if (!ok) { *abort_flag = 1; atomicOr(g.status, kStatusTimeout); }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = ptx::idesc_bf16_f32(kTileM, kTileN) | (A_MN ? (1u << 15) : 0u) | (B_MN ? (1u << 16) : 0u);
+        // ------------------------------------------------------------------ MMA issuer (even CTA only)
+        if (lane == 0 && cta_rank == 0) {
+            constexpr uint32_t idesc = ptx::idesc_bf16_f32(C::kTileRows, kTileN) | (A_MN ? (1u << 15) : 0u) | (B_MN ? (1u << 16) : 0u);
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-                const Unit t = get_unit<EPI>(g, u, gm);
+            for (int it = 0; ok; ++it) {
+                Unit t;
+                bool valid;
+                if (!next_unit<EPI>(g, it, pair, n_pairs, gm, t, valid)) break;
+                if (!valid) continue;
                 for (int nt = t.n_begin; nt < t.n_end && ok; ++nt) {
                     if (!ptx::mbar_wait(&acc_empty[acc], acc_phase ^ 1, kWaitBudgetCycles) || *abort_flag) { ok = false; break; }
                     ptx::tc_fence_after();
@@ -179,27 +207,30 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                         constexpr uint32_t step_b = B_MN ? (16 * 128) >> 4 : 2;
 #pragma unroll
                         for (int kk = 0; kk < kTileK / 16; ++kk)
-                            ptx::mma_bf16_ss(d_tmem, da + step_a * kk, db + step_b * kk, idesc, (k | kk) != 0 ? 1u : 0u);
-                        ptx::tc_commit(&empty[stage]);
+                            ptx::mma_bf16_ss_on<CTAS>(d_tmem, da + step_a * kk, db + step_b * kk, idesc, (k | kk) != 0 ? 1u : 0u);
+                        ptx::tc_commit_on<CTAS>(&empty[stage]);
                         if (++stage == kStages) { stage = 0; phase ^= 1; }
                     }
                     if (!ok) break;
-                    ptx::tc_commit(&acc_full[acc]);
+                    ptx::tc_commit_on<CTAS>(&acc_full[acc]);
                     if (++acc == kAccStages) { acc = 0; acc_phase ^= 1; }
                 }
             }
             if (!ok) { *abort_flag = 1; atomicOr(g.status, kStatusTimeout); }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue: thread = one row
+        // ------------------------------------------------------------------ epilogue: thread = one row (both CTAs)
         const int quarter = warp & 3;                      // TMEM lanes this warp may touch: 32*quarter ..
-        const int row_in_tile = quarter * 32 + lane;
+        const int row_in_tile = static_cast<int>(cta_rank) * kCtaM + quarter * 32 + lane;
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
-        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-            const Unit t = get_unit<EPI>(g, u, gm);
-            const int row = t.m_tile * kTileM + row_in_tile;        // relative to a_row0
+        for (int it = 0; ok; ++it) {
+            Unit t;
+            bool valid;
+            if (!next_unit<EPI>(g, it, pair, n_pairs, gm, t, valid)) break;
+            if (!valid) continue;
+            const int row = t.m_tile * C::kTileRows + row_in_tile;        // relative to a_row0
             const bool row_ok = row < g.m_rows;
 
             // per-row state
@@ -303,10 +334,13 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                         }
                     }
                 }
-                // release the accumulator stage to the MMA warp
+                // release the accumulator stage to the MMA issuer in the even CTA
                 ptx::tc_fence_before();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&acc_empty[acc]);
+                if (lane == 0) {
+                    if (CTAS == 2) ptx::mbar_arrive_cluster(ptx::mapa(ptx::smem_u32(&acc_empty[acc]), 0));
+                    else ptx::mbar_arrive(&acc_empty[acc]);
+                }
                 if (++acc == kAccStages) { acc = 0; acc_phase ^= 1; }
             }
             if (EPI == kEpiSoftmaxStats && ok && row_ok)
@@ -323,45 +357,80 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
         while (clock64() - t0 < 2000000) { }
     }
     ptx::tc_fence_before();
-    __syncthreads();
+    if (CTAS == 2) ptx::cluster_sync_all();   // neither CTA leaves (or frees tensor memory) while its peer may touch it
+    else __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, kTmemCols);
+        if (CTAS == 2) ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
+        else ptx::tmem_dealloc(tmem_base, kTmemCols);
     }
+}
+
+
+template <int EPI, bool A_MN, bool B_MN, int CTAS>
+cudaError_t set_attr() {
+    return cudaFuncSetAttribute(k_gemm<EPI, A_MN, B_MN, CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                Cfg<CTAS>::kSmemBytes);
+}
+
+template <int EPI, bool A_MN, bool B_MN, int CTAS>
+cudaError_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args, int workers, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(workers * CTAS, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = Cfg<CTAS>::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CTAS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k_gemm<EPI, A_MN, B_MN, CTAS>, tmA, tmB, args);
 }
 
 }  // namespace
 
 cudaError_t gemm_set_attributes() {
     cudaError_t e;
-    e = cudaFuncSetAttribute(k_gemm<kEpiSoftmaxStats, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(k_gemm<kEpiLogitGrad, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(k_gemm<kEpiAccumF32, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(k_gemm<kEpiAccumF32, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if ((e = set_attr<kEpiSoftmaxStats, false, false, 1>()) != cudaSuccess) return e;
+    if ((e = set_attr<kEpiSoftmaxStats, false, false, 2>()) != cudaSuccess) return e;
+    if ((e = set_attr<kEpiLogitGrad, false, false, 1>()) != cudaSuccess) return e;
+    if ((e = set_attr<kEpiLogitGrad, false, false, 2>()) != cudaSuccess) return e;
+    if ((e = set_attr<kEpiAccumF32, false, true, 1>()) != cudaSuccess) return e;
+    if ((e = set_attr<kEpiAccumF32, false, true, 2>()) != cudaSuccess) return e;
+    if ((e = set_attr<kEpiAccumF32, true, true, 1>()) != cudaSuccess) return e;
+    return set_attr<kEpiAccumF32, true, true, 2>();
 }
 
-cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, const CUtensorMap& tmA, const CUtensorMap& tmB,
+int gemm_tile_rows(int ctas) { return kCtaM * ctas; }
+
+cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, int ctas, const CUtensorMap& tmA, const CUtensorMap& tmB,
                         const GemmArgs& args, int sm_count, cudaStream_t stream) {
-    const long long units = epi == kEpiSoftmaxStats ? static_cast<long long>(args.m_tiles) * args.n_splits
-                                                    : static_cast<long long>(args.m_tiles) * args.n_tiles;
-    if (units <= 0 || args.k_iters <= 0) return cudaSuccess;
-    const int grid = static_cast<int>(units < sm_count ? units : sm_count);
+    // softmax: one round handles group_m row tiles x n_splits; other epilogues: plain striding over all tiles
+    const long long units = epi == kEpiSoftmaxStats
+                                ? static_cast<long long>(args.group_m < args.m_tiles ? args.group_m : args.m_tiles) * args.n_splits
+                                : static_cast<long long>(args.m_tiles) * args.n_tiles;
+    if (units <= 0 || args.m_tiles <= 0 || args.k_iters <= 0) return cudaSuccess;
+    const int max_workers = sm_count / ctas;                                   // one CTA per SM
+    const int workers = static_cast<int>(units < max_workers ? units : max_workers);
+    const bool two = ctas == 2;
     switch (epi) {
         case kEpiSoftmaxStats:
-            k_gemm<kEpiSoftmaxStats, false, false><<<grid, kThreads, kSmemBytes, stream>>>(tmA, tmB, args);
-            break;
+            return two ? launch<kEpiSoftmaxStats, false, false, 2>(tmA, tmB, args, workers, stream)
+                       : launch<kEpiSoftmaxStats, false, false, 1>(tmA, tmB, args, workers, stream);
         case kEpiLogitGrad:
-            k_gemm<kEpiLogitGrad, false, false><<<grid, kThreads, kSmemBytes, stream>>>(tmA, tmB, args);
-            break;
+            return two ? launch<kEpiLogitGrad, false, false, 2>(tmA, tmB, args, workers, stream)
+                       : launch<kEpiLogitGrad, false, false, 1>(tmA, tmB, args, workers, stream);
         default:   // fp32 accumulate: B is always MN-major (W or hidden read in place), A is G either way round
-            if (a_mn) k_gemm<kEpiAccumF32, true, true><<<grid, kThreads, kSmemBytes, stream>>>(tmA, tmB, args);
-            else k_gemm<kEpiAccumF32, false, true><<<grid, kThreads, kSmemBytes, stream>>>(tmA, tmB, args);
-            break;
+            if (a_mn)
+                return two ? launch<kEpiAccumF32, true, true, 2>(tmA, tmB, args, workers, stream)
+                           : launch<kEpiAccumF32, true, true, 1>(tmA, tmB, args, workers, stream);
+            return two ? launch<kEpiAccumF32, false, true, 2>(tmA, tmB, args, workers, stream)
+                       : launch<kEpiAccumF32, false, true, 1>(tmA, tmB, args, workers, stream);
     }
-    return cudaGetLastError();
 }
 
 }  // namespace unity

@@ -10,8 +10,11 @@
 
 namespace unity {
 
-constexpr int kTileM = 128;   // rows of the A operand per CTA tile (TMEM lanes)
-constexpr int kTileN = 256;   // rows of the B operand per CTA tile (TMEM columns per accumulator stage)
+constexpr int kTileM = 256;   // rows of one output tile, shared by a pair of CTAs; row groups are padded to this
+constexpr int kCtaM = 128;    // rows of A per CTA of the pair (= TMEM lanes)
+constexpr int kTileN = 256;   // columns of one output tile (TMEM columns per accumulator stage)
+constexpr int kHalfN = 128;   // rows of B loaded by each CTA of the pair
+constexpr int kBoxRows = 128; // rows of a K-major TMA box (A and B alike)
 constexpr int kTileK = 64;    // bf16 elements per shared-memory K slab (one 128-byte swizzle row)
 constexpr int kRouteBlock = 256;          // threads (= tokens) per block in the routing kernels
 constexpr long long kWaitBudgetCycles = 4000000000LL;   // ~2 s: bound of every in-kernel wait
@@ -31,7 +34,7 @@ enum GemmEpilogue : int {
 
 struct GemmArgs {
     // tile grid and coordinates into the tensor maps
-    int m_tiles, n_tiles, k_iters;
+    int m_tiles, n_tiles, k_iters;   // tiles are gemm_tile_rows(ctas) x kTileN
     int group_m;              // row tiles per raster group (consecutive units share these A tiles)
     int a_row0, b_row0;       // first row of A / B (tensor-map coordinates) of tile (0, 0)
     int a_k0, b_k0;           // first K element of A / B
@@ -59,8 +62,11 @@ struct GemmArgs {
 
 // a_mn: A is MN-major (only for kEpiAccumF32, whose B operand is always MN-major).  For an MN-major operand
 // a_row0 / b_row0 index the contiguous dimension of its tensor map and a_k0 / b_k0 its rows.
-cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, const CUtensorMap& tmA, const CUtensorMap& tmB,
+// ctas: 1 = one CTA per 128 x 256 tile, 2 = a CTA pair per 256 x 256 tile; args.m_tiles counts tiles of
+// gemm_tile_rows(ctas) rows.
+cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, int ctas, const CUtensorMap& tmA, const CUtensorMap& tmB,
                         const GemmArgs& args, int sm_count, cudaStream_t stream);
+int gemm_tile_rows(int ctas);
 cudaError_t gemm_set_attributes();
 
 // ----------------------------------------------------------------------------------------------

@@ -30,14 +30,15 @@ struct unity_ctx {
     std::vector<cudaEvent_t>* ev_pool;
     std::vector<int>* ev_class;     // class of the i-th recorded pair
     size_t ev_used;                 // events handed out since the last unity_get_profile
+    int ctas[UNITY_PROF_CLASSES];   // per GEMM class: 1 = single CTA per tile, 2 = CTA pair per tile
 };
 
 namespace {
 
 constexpr size_t kAlign = 256;
-// Gradient chunk: 148 row tiles x 74 vocabulary tiles.  With one CTA per SM (148) every chunk GEMM then runs a
-// whole number of waves: recompute 148 x 74 tiles, dHidden 148 x ceil(H/256), dW 148 x ceil(H/256).
-constexpr int kChunkRows = 148 * kTileM;     // 18944 token rows
+// Gradient chunk: 74 row tiles x 74 vocabulary tiles of 256.  With 74 CTA pairs (148 SMs) every chunk GEMM then runs
+// a whole number of waves: recompute 74 x 74 tiles, dHidden 74 x ceil(H/256), dW 74 x ceil(H/256).
+constexpr int kChunkRows = 74 * kTileM;      // 18944 token rows
 constexpr int kChunkVocab = 74 * kTileN;     // 18944 vocabulary entries
 constexpr int kMinChunkRows = 1024;
 constexpr int kMinChunkVocab = 1024;
@@ -152,7 +153,7 @@ int wanted_chunk_vocab(int V) {
 }
 
 // Tensor map over a row-major bf16 matrix [rows, inner]; boxes are 64 elements (128 B, one swizzle row) wide and
-// box_rows high.  K-major operands use box_rows = tile rows (128 / 256); MN-major operands use 64 (= kTileK).
+// box_rows high.  K-major operands use box_rows = kBoxRows (128); MN-major operands use 64 (= kTileK).
 int make_tmap(unity_ctx* ctx, CUtensorMap* tm, const void* ptr, uint64_t inner, uint64_t rows, uint64_t pitch_bytes,
               uint32_t box_rows) {
     cuuint64_t dims[2] = {inner, rows};
@@ -231,9 +232,11 @@ int forward_sweep(unity_ctx* ctx, const unity_rows* r, RowPlan& P) {
                                      r->H, L.hp, L.target_p, st));
     nl += P.n_slots > 0;
 
+    const int ctas = ctx->ctas[UNITY_PROF_FWD_GEMM];
+    const int tile_rows = gemm_tile_rows(ctas);
     CUtensorMap tmA;
     if (P.n_slots > 0) {
-        int rc = make_tmap(ctx, &tmA, L.hp, r->H, P.n_slots, static_cast<uint64_t>(r->H) * 2, kTileM);
+        int rc = make_tmap(ctx, &tmA, L.hp, r->H, P.n_slots, static_cast<uint64_t>(r->H) * 2, kBoxRows);
         if (rc) return rc;
     }
     const int n_tiles = (r->V + kTileN - 1) / kTileN;
@@ -243,11 +246,18 @@ int forward_sweep(unity_ctx* ctx, const unity_rows* r, RowPlan& P) {
         P.stats_base[k] = sbase;
         const int rows_k = P.offsets[k + 1] - P.offsets[k];
         if (rows_k == 0) continue;
-        const int m_tiles = rows_k / kTileM;
-        int splits = (4 * ctx->sm_count + m_tiles - 1) / m_tiles;
-        if (splits < 4) splits = 4;
+        const int m_tiles = rows_k / tile_rows;
+        // One round of the persistent kernel = gm row tiles x splits vocabulary splits <= number of workers (CTAs
+        // or CTA pairs): gm bounds the hidden rows that must stay L2 resident (a quarter of the workers, about
+        // 4.7 k rows), splits fill the machine.
+        const int n_pairs = ctx->sm_count / ctas;
+        const int gmax = n_pairs / 4 > 0 ? n_pairs / 4 : 1;
+        const int n_grp = (m_tiles + gmax - 1) / gmax;
+        const int gm = (m_tiles + n_grp - 1) / n_grp;
+        int splits = n_pairs / gm;
         if (splits > 32) splits = 32;
         if (splits > n_tiles) splits = n_tiles;
+        if (splits < 1) splits = 1;
         const int tps = (n_tiles + splits - 1) / splits;
         splits = (n_tiles + tps - 1) / tps;
         P.splits[k] = splits;
@@ -255,12 +265,12 @@ int forward_sweep(unity_ctx* ctx, const unity_rows* r, RowPlan& P) {
         if (sbase > L.stats_cap) return fail(ctx, UNITY_ERR_WORKSPACE, "internal: statistics scratch too small");
 
         CUtensorMap tmB;
-        int rc = make_tmap(ctx, &tmB, r->W[k], r->H, r->V, static_cast<uint64_t>(r->H) * 2, kTileN);
+        int rc = make_tmap(ctx, &tmB, r->W[k], r->H, r->V, static_cast<uint64_t>(r->H) * 2, kTileN / ctas);
         if (rc) return rc;
         GemmArgs g;
         memset(&g, 0, sizeof(g));
         g.m_tiles = m_tiles; g.n_tiles = n_tiles; g.k_iters = r->H / kTileK;
-        g.group_m = ctx->sm_count / splits > 0 ? ctx->sm_count / splits : 1;
+        g.group_m = gm;
         g.a_row0 = P.offsets[k]; g.b_row0 = 0; g.a_k0 = 0; g.b_k0 = 0;
         g.m_rows = rows_k; g.n_cols = r->V;
         g.n_splits = splits; g.tiles_per_split = tps;
@@ -269,7 +279,7 @@ int forward_sweep(unity_ctx* ctx, const unity_rows* r, RowPlan& P) {
         g.status = ctx->d_status;
         {
             ProfScope ps(ctx, UNITY_PROF_FWD_GEMM);
-            CUDA_TRY(ctx, launch_gemm(kEpiSoftmaxStats, false, tmA, tmB, g, ctx->sm_count, st));
+            CUDA_TRY(ctx, launch_gemm(kEpiSoftmaxStats, false, ctas, tmA, tmB, g, ctx->sm_count, st));
         }
         nl += 1;
     }
@@ -321,6 +331,10 @@ int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace
         return UNITY_ERR_CUDA;
     }
     c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    c->ctas[UNITY_PROF_FWD_GEMM] = 1;
+    c->ctas[UNITY_PROF_GRAD_GEMM] = 2;
+    c->ctas[UNITY_PROF_DH_GEMM] = 2;
+    c->ctas[UNITY_PROF_DW_GEMM] = 2;
     c->ev_pool = new (std::nothrow) std::vector<cudaEvent_t>();
     c->ev_class = new (std::nothrow) std::vector<int>();
     if (cudaMalloc(&c->d_status, 256) != cudaSuccess || cudaMallocHost(&c->h_pinned, 4096) != cudaSuccess ||
@@ -376,6 +390,16 @@ int unity_check_status(unity_ctx* ctx) {
 const char* unity_last_error(const unity_ctx* ctx) { return ctx ? ctx->err : "null context"; }
 
 int64_t unity_launch_count(const unity_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int unity_set_option(unity_ctx* ctx, int option, int value) {
+    if (!ctx) return UNITY_ERR_INVALID_ARG;
+    if (option >= UNITY_OPT_CTAS_FWD && option <= UNITY_OPT_CTAS_DW) {
+        if (value != 1 && value != 2) return fail(ctx, UNITY_ERR_INVALID_ARG, "CTAs per tile must be 1 or 2");
+        ctx->ctas[option - UNITY_OPT_CTAS_FWD] = value;
+        return UNITY_OK;
+    }
+    return fail(ctx, UNITY_ERR_INVALID_ARG, "unknown option %d", option);
+}
 
 int unity_set_profiling(unity_ctx* ctx, int enable) {
     if (!ctx || !ctx->ev_pool || !ctx->ev_class) return UNITY_ERR_INVALID_ARG;
@@ -536,10 +560,12 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
     // MN-major operands (contraction over tokens / vocabulary); nothing is transposed in memory.
     CUtensorMap tm_hp_k, tm_hp_mn;
     if (P.n_slots > 0) {
-        if ((rc = make_tmap(ctx, &tm_hp_k, L.hp, H, P.n_slots, static_cast<uint64_t>(H) * 2, kTileM))) return rc;
+        if ((rc = make_tmap(ctx, &tm_hp_k, L.hp, H, P.n_slots, static_cast<uint64_t>(H) * 2, kBoxRows))) return rc;
         if ((rc = make_tmap(ctx, &tm_hp_mn, L.hp, H, P.n_slots, static_cast<uint64_t>(H) * 2, kTileK))) return rc;
     }
     const int h_tiles = (H + kTileN - 1) / kTileN;
+    const int c_grad = ctx->ctas[UNITY_PROF_GRAD_GEMM], c_dh = ctx->ctas[UNITY_PROF_DH_GEMM],
+              c_dw = ctx->ctas[UNITY_PROF_DW_GEMM];
 
     for (int k = 0; k < K; ++k) {
         const int rows_k = P.offsets[k + 1] - P.offsets[k];
@@ -550,7 +576,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
         }
         const __nv_bfloat16* Wk = static_cast<const __nv_bfloat16*>(rows->W[k]);
         CUtensorMap tm_W_k, tm_W_mn;
-        if ((rc = make_tmap(ctx, &tm_W_k, Wk, H, V, static_cast<uint64_t>(H) * 2, kTileN))) return rc;
+        if ((rc = make_tmap(ctx, &tm_W_k, Wk, H, V, static_cast<uint64_t>(H) * 2, kTileN / c_grad))) return rc;
         if ((rc = make_tmap(ctx, &tm_W_mn, Wk, H, V, static_cast<uint64_t>(H) * 2, kTileK))) return rc;
 
         for (int c0 = 0; c0 < rows_k; c0 += cr) {
@@ -561,42 +587,42 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 // (1) recompute the logits of this (rows x vocab) chunk and form dL/dz in bf16: G[nc, vc]
                 GemmArgs g;
                 memset(&g, 0, sizeof(g));
-                g.m_tiles = nc / kTileM; g.n_tiles = (vc + kTileN - 1) / kTileN; g.k_iters = H / kTileK;
-                g.group_m = 16;
+                g.m_tiles = nc / gemm_tile_rows(c_grad); g.n_tiles = (vc + kTileN - 1) / kTileN; g.k_iters = H / kTileK;
+                g.group_m = 16 / c_grad;
                 g.a_row0 = slot0; g.b_row0 = v0; g.m_rows = nc; g.n_cols = vc;
                 g.target_p = L.target_p; g.vocab0 = v0; g.scale = rows->inv_temperature;
                 g.coef_a = L.coef_a; g.coef_b = L.coef_b; g.row_lse = L.row_lse; g.row_ent = L.row_ent;
                 g.G = L.G; g.ldg = cv; g.status = ctx->d_status;
                 {
                     ProfScope ps(ctx, UNITY_PROF_GRAD_GEMM);
-                    CUDA_TRY(ctx, launch_gemm(kEpiLogitGrad, false, tm_hp_k, tm_W_k, g, ctx->sm_count, st));
+                    CUDA_TRY(ctx, launch_gemm(kEpiLogitGrad, false, c_grad, tm_hp_k, tm_W_k, g, ctx->sm_count, st));
                 }
                 // G viewed as [nc rows, vc]: K-major A for dHidden (contract over vc), MN-major A for dW (rows = K)
                 CUtensorMap tm_G_k, tm_G_mn;
-                if ((rc = make_tmap(ctx, &tm_G_k, L.G, vc, nc, static_cast<uint64_t>(cv) * 2, kTileM))) return rc;
+                if ((rc = make_tmap(ctx, &tm_G_k, L.G, vc, nc, static_cast<uint64_t>(cv) * 2, kBoxRows))) return rc;
                 if ((rc = make_tmap(ctx, &tm_G_mn, L.G, vc, nc, static_cast<uint64_t>(cv) * 2, kTileK))) return rc;
                 // (2) dH_chunk[nc, H] (+)= G[nc, vc] * W[v0:v0+vc, :]      (B = W, MN-major: rows v are K)
                 GemmArgs h;
                 memset(&h, 0, sizeof(h));
-                h.m_tiles = nc / kTileM; h.n_tiles = h_tiles; h.k_iters = (vc + kTileK - 1) / kTileK;
-                h.group_m = 16;
+                h.m_tiles = nc / gemm_tile_rows(c_dh); h.n_tiles = h_tiles; h.k_iters = (vc + kTileK - 1) / kTileK;
+                h.group_m = 16 / c_dh;
                 h.a_row0 = 0; h.a_k0 = 0; h.b_row0 = 0; h.b_k0 = v0; h.m_rows = nc; h.n_cols = H;
                 h.C = L.dHc; h.ldc = H; h.beta = v0 > 0; h.status = ctx->d_status;
                 {
                     ProfScope ps(ctx, UNITY_PROF_DH_GEMM);
-                    CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, false, tm_G_k, tm_W_mn, h, ctx->sm_count, st));
+                    CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, false, c_dh, tm_G_k, tm_W_mn, h, ctx->sm_count, st));
                 }
                 // (3) dW[v0:v0+vc, :] (+)= G^T[vc, nc] * hidden[slot0:slot0+nc, :]   (both operands MN-major)
                 GemmArgs w;
                 memset(&w, 0, sizeof(w));
-                w.m_tiles = (vc + kTileM - 1) / kTileM; w.n_tiles = h_tiles; w.k_iters = nc / kTileK;
-                w.group_m = 16;
+                w.m_tiles = (vc + gemm_tile_rows(c_dw) - 1) / gemm_tile_rows(c_dw); w.n_tiles = h_tiles; w.k_iters = nc / kTileK;
+                w.group_m = 16 / c_dw;
                 w.a_row0 = 0; w.a_k0 = 0; w.b_row0 = 0; w.b_k0 = slot0; w.m_rows = vc; w.n_cols = H;
                 w.C = dWk + static_cast<long long>(v0) * H; w.ldc = H;
                 w.beta = (params->accumulate_dW || c0 > 0) ? 1 : 0; w.status = ctx->d_status;
                 {
                     ProfScope ps(ctx, UNITY_PROF_DW_GEMM);
-                    CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, true, tm_G_mn, tm_hp_mn, w, ctx->sm_count, st));
+                    CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, true, c_dw, tm_G_mn, tm_hp_mn, w, ctx->sm_count, st));
                 }
                 nl += 3;
             }

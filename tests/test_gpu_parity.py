@@ -47,10 +47,13 @@ def check_ppo(g, o, w, atol_loss=1e-6):
     assert np.abs(gm - om).max() <= 1e-3 * max(1.0, np.abs(om[:, 1:]).max())
 
 
-def run_all_stages(w, **ppo_kw):
+def run_all_stages(w, ctas=None, **ppo_kw):
     d = pu.DeviceInputs(w)
     ctx = pu.make_ctx(w)
     try:
+        if ctas is not None:                       # CTAs per output tile for the four GEMM classes
+            for option, value in enumerate(ctas):
+                ctx.set_option(option, value)
         ga, oa = pu.gpu_advantage(ctx, w, d), pu.oracle_advantage(w)
         assert np.abs(ga["adv_inv"].cpu().numpy() - oa["adv_inv"]).max() <= pu.TOL_ADV
         assert np.abs(ga["adv_tok"].cpu().numpy() - oa["adv_tok"]).max() <= pu.TOL_ADV
@@ -166,6 +169,13 @@ def small_workload(H, V, rows, role_model=None, K=None, max_len=48, seed_offset=
 def test_small_shapes_and_ragged_tails(H, V, rows):
     # V not a multiple of the 256-wide vocabulary tile, rows not a multiple of the 128-row tile
     run_all_stages(small_workload(H, V, rows))
+
+
+@pytest.mark.parametrize("ctas", [(1, 1, 1, 1), (2, 2, 2, 2), (2, 1, 1, 2)])
+def test_single_cta_and_cta_pair_kernels(ctas):
+    # every GEMM class exists as a one-CTA kernel (128-row tiles) and as a CTA-pair kernel (256-row tiles)
+    run_all_stages(small_workload(320, 2048 + 264, 700), ctas=ctas)
+    run_all_stages(wl.make("tiny", device="cuda"), ctas=ctas)
 
 
 @pytest.mark.parametrize("kl_mode,ent_coef,clip", [(1, 0.0, (0.2, 0.2)), (2, 0.01, (0.1, 0.3)), (3, 0.02, (0.2, 0.28))])
