@@ -210,17 +210,18 @@ def main():
     ref = logp + w.noise_ref.to(dev)
 
     # per-model valid-row counts: the only quantity the ranks must agree on before the step
+    from paper_2605_26646_b200 import sharding
     tok_inv = torch.repeat_interleave(torch.arange(w.n_inv), w.cu_seqlens[1:] - w.cu_seqlens[:-1])
     tok_model = w.role_model[w.inv_role.long()[tok_inv]].long()
-    counts = torch.bincount(tok_model[w.tok_mask != 0], minlength=K).to(torch.float64)
+    counts = sharding.local_counts(tok_model, w.tok_mask, K)
     n_valid_local = int(counts.sum().item())
     norm = None
     n_valid_total = n_valid_local
     if world > 1:
-        c = counts.to(dev)
-        dist.all_reduce(c)
-        norm = [max(float(x), 1.0) for x in c.tolist()]
-        n_valid_total = int(c.sum().item())
+        norm = sharding.global_norm(counts.to(dev))
+        tot = torch.tensor([float(n_valid_local)], device=dev, dtype=torch.float64)
+        dist.all_reduce(tot)
+        n_valid_total = int(tot.item())
 
     def step(hid, tgt, msk, o, r):
         ctx.role_advantage(w.n_traj, w.n_roles, w.n_groups, d_inv_role, d_inv_group, d_inv_traj, d_rn, d_rt, d_rj,
@@ -229,8 +230,7 @@ def main():
                              w.clip_hi, w.kl_coef, w.kl_mode, w.ent_coef, norm, False, o, r, adv_tok, loss, metrics,
                              logp, ent, None, dH, dW)
         if world > 1:
-            for g in dW:
-                dist.all_reduce(g)
+            sharding.allreduce_grads(dW)
 
     def sync_all():
         torch.cuda.synchronize()

@@ -210,7 +210,7 @@ def ppo_loss_fwd_bwd(hidden, W, cu_seqlens, inv_role, role_model, target, tok_ma
     cu = np.asarray(cu_seqlens, dtype=np.int64)
     n_tok = int(cu[-1])
     K = len(W)
-    H = np.asarray(hidden).shape[1]
+    H = hidden.shape[1]
     tok_role, tok_model = token_role_model(cu, inv_role, role_model)
     R = int(n_roles if n_roles is not None else np.asarray(role_model).size)
     mask = np.ones(n_tok, bool) if tok_mask is None else (np.asarray(tok_mask) != 0)

@@ -7,4 +7,4 @@ the shared library; the first call into ``binding`` does, and fails loudly if it
 """
 from . import workloads  # noqa: F401
 
-__all__ = ["binding", "build", "workloads"]
+__all__ = ["binding", "build", "sharding", "workloads"]
