@@ -27,6 +27,27 @@ METRIC = "response tokens/s, fused LM-head logprob+PPO fwd+bwd; % of bf16 tensor
 UNIT = "tokens/s"
 
 
+# DRAM traffic of each GEMM class from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum, one launch per
+# class) on a cut of the code workload (profiles/k_gemm_code_cut40k.md), as bytes per logit the launch covers
+# (valid rows x vocabulary columns).  Traffic grows in proportion to the logits covered (same chunk and group sizes),
+# so a full-size launch is estimated as bytes_per_logit x its logits.  Valid only for the kernel source it was taken
+# from: when the hash of gemm_tcgen05.cu differs, the benchmark reports null.
+NCU_TRAFFIC = {"source_sha256_16": "49c0d1fa7357c3b2",
+               "bytes_per_logit": {"fwd_gemm": 1.859, "grad_gemm": 6.99, "dh_gemm": 10.71, "dw_gemm": 10.73}}
+
+
+def ncu_traffic_per_launch(cls: str, logits_per_launch: float):
+    import hashlib
+    src = os.path.join(ROOT, "paper_2605_26646_b200", "csrc", "gemm_tcgen05.cu")
+    try:
+        sha = hashlib.sha256(open(src, "rb").read()).hexdigest()[:16]
+    except OSError:
+        return None
+    if sha != NCU_TRAFFIC["source_sha256_16"] or cls not in NCU_TRAFFIC["bytes_per_logit"]:
+        return None
+    return NCU_TRAFFIC["bytes_per_logit"][cls] * logits_per_launch
+
+
 def read_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -331,7 +352,8 @@ def main():
     dom = max(kern, key=lambda k: kern[k]["ms_total"])
     dp = kern[dom]
     roofline = {"bound": "tensor", "kernel": f"k_gemm<{dom}>", "achieved": dp["tflops"], "peak": peak,
-                "unit": "TFLOP/s", "frac": dp["frac"], "traffic": None,
+                "unit": "TFLOP/s", "frac": dp["frac"],
+                "traffic": ncu_traffic_per_launch(dom, float(V) * n_valid_local * args.steps / dp["launches"]),
                 "peak_source": f"{peaks['source']} bf16 GEMM, sustained",
                 "flops_per_launch": flops_per_tok * n_valid_local * args.steps / dp["launches"],
                 "avg_launch_ms": dp["ms_total"] / dp["launches"]}
