@@ -123,6 +123,18 @@ int unity_role_advantage(unity_ctx* ctx, int32_t n_inv, int32_t n_traj, int32_t 
                          const unity_adv_params* params, int64_t n_tok, const int64_t* cu_seqlens,
                          const uint8_t* tok_mask, float* adv_inv, float* adv_tok, float* seg_mean, float* seg_std);
 
+/* Token-level generalized advantage estimation - the advantage formula printed in paragraph "Advantage
+ * computation and policy evaluation":  A_t = sum_{l=0}^{T-t} (gamma*lambda)^l delta_{t+l},
+ * delta_t = r_t + gamma*V(s_{t+1}) - V(s_t), evaluated per sequence (cu_seqlens) with V = 0 past the last token;
+ * returns[t] = A_t + V(s_t) are the regression targets of the value estimates.  Tokens with tok_mask == 0 are not
+ * part of their sequence (the next token of t is the next unmasked one) and receive 0 in both outputs.
+ *   rewards, values : f32 [n_tok];  tok_mask : u8 [n_tok] or NULL;  gamma, lambda in [0, 1]
+ *   advantages, returns : out f32 [n_tok]
+ * Uses no workspace; fp32 with a fixed evaluation order (bitwise reproducible). */
+int unity_gae(unity_ctx* ctx, int32_t n_inv, int64_t n_tok, const int64_t* cu_seqlens, const float* rewards,
+              const float* values, const uint8_t* tok_mask, float gamma, float lambda, float* advantages,
+              float* returns);
+
 /* Stage 1 without any allocation (the paper has no counterpart; this exists for deployment reasons).
  *
  * Who needs it: hosts that may not call cudaMalloc or create a unity_ctx - a trainer whose framework

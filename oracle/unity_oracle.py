@@ -302,23 +302,26 @@ def ppo_loss_value(hidden, W, cu_seqlens, inv_role, role_model, target, tok_mask
 # token-level generalized advantage estimation (the advantage formula the paper prints)
 # ----------------------------------------------------------------------------------------------
 
-def gae(rewards, values, cu_seqlens, gamma, lam):
+def gae(rewards, values, cu_seqlens, gamma, lam, tok_mask=None):
     """A_t = sum_{l=0}^{T-t} (gamma*lam)^l delta_{t+l},  delta_t = r_t + gamma V(s_{t+1}) - V(s_t),
-    per sequence, with V past the last token taken as 0.  Returns (advantages, returns=A+V)."""
+    per sequence, with V past the last token taken as 0.  Returns (advantages, returns=A+V).
+
+    Tokens with tok_mask == 0 are not part of the sequence: the formula is applied to the remaining tokens of each
+    sequence in order (their "next" token is the next unmasked one) and masked tokens receive 0 in both outputs."""
     r = to_f64(rewards)
     v = to_f64(values)
     cu = np.asarray(cu_seqlens, dtype=np.int64)
+    keep = np.ones(r.shape[0], bool) if tok_mask is None else (np.asarray(tok_mask) != 0)
     A = np.zeros_like(r)
     for s in range(cu.size - 1):
-        lo, hi = int(cu[s]), int(cu[s + 1])
-        T = hi - lo
+        idx = np.arange(int(cu[s]), int(cu[s + 1]))
+        idx = idx[keep[idx]]
+        T = idx.size
         if T == 0:
             continue
-        vs = np.concatenate([v[lo:hi], [0.0]])
-        delta = r[lo:hi] + gamma * vs[1:] - vs[:-1]
+        vs = np.concatenate([v[idx], [0.0]])
+        delta = r[idx] + gamma * vs[1:] - vs[:-1]
+        powers = (gamma * lam) ** np.arange(T)           # (gamma*lam)^l, l = 0 .. T-1
         for t in range(T):
-            acc = 0.0
-            for l in range(T - t):
-                acc += (gamma * lam) ** l * delta[t + l]
-            A[lo + t] = acc
-    return A, A + v
+            A[idx[t]] = (powers[:T - t] * delta[t:]).sum()   # the sum over l written out for this t
+    return A, np.where(keep, A + v, 0.0)

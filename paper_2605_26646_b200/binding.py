@@ -25,7 +25,7 @@ UNITY_N_METRICS = 8
 
 EXPORTS = ["unity_create", "unity_destroy", "unity_workspace_bytes", "unity_workspace_min_bytes",
            "unity_check_status", "unity_last_error", "unity_launch_count", "unity_set_profiling",
-           "unity_get_profile", "unity_set_option", "unity_role_advantage", "unity_role_advantage_noalloc",
+           "unity_get_profile", "unity_set_option", "unity_role_advantage", "unity_gae", "unity_role_advantage_noalloc",
            "unity_logprob_fwd", "unity_ppo_loss_fwd_bwd"]
 
 
@@ -94,6 +94,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
                                                  C.POINTER(unity_adv_params), i64, vp, vp, vp, vp, vp, vp, vp,
                                                  C.c_char_p, C.c_size_t]
     lib.unity_role_advantage_noalloc.restype = C.c_int
+    lib.unity_gae.argtypes = [vp, i32, i64, vp, vp, vp, vp, C.c_float, C.c_float, vp, vp]
+    lib.unity_gae.restype = C.c_int
     lib.unity_logprob_fwd.argtypes = [vp, C.POINTER(unity_rows), vp, vp, vp]
     lib.unity_logprob_fwd.restype = C.c_int
     lib.unity_ppo_loss_fwd_bwd.argtypes = [vp, C.POINTER(unity_rows), C.POINTER(unity_ppo_params), vp, vp, vp,
@@ -192,6 +194,15 @@ def unity_role_advantage(ctx, n_traj: int, n_roles: int, n_groups: int, inv_role
         _ptr(r_traj, f32, "r_traj"), lam_arr, C.byref(p), n_tok, _ptr(cu_seqlens, torch.int64, "cu_seqlens"),
         _ptr(tok_mask, torch.uint8, "tok_mask"), _ptr(adv_inv, f32, "adv_inv"), _ptr(adv_tok, f32, "adv_tok"),
         _ptr(seg_mean, f32, "seg_mean"), _ptr(seg_std, f32, "seg_std"))
+    _raise(ctx, code)
+
+
+def unity_gae(ctx, cu_seqlens, rewards, values, tok_mask, gamma: float, lam: float, advantages, returns) -> None:
+    f32 = torch.float32
+    code = load_library().unity_gae(ctx, int(cu_seqlens.numel()) - 1, int(rewards.numel()),
+                                    _ptr(cu_seqlens, torch.int64, "cu_seqlens"), _ptr(rewards, f32, "rewards"),
+                                    _ptr(values, f32, "values"), _ptr(tok_mask, torch.uint8, "tok_mask"), gamma, lam,
+                                    _ptr(advantages, f32, "advantages"), _ptr(returns, f32, "returns"))
     _raise(ctx, code)
 
 
@@ -313,6 +324,9 @@ class Context:
 
     def role_advantage(self, *a, **kw):
         return unity_role_advantage(self.ctx, *a, **kw)
+
+    def gae(self, *a, **kw):
+        return unity_gae(self.ctx, *a, **kw)
 
     def logprob_fwd(self, *a, **kw):
         return unity_logprob_fwd(self.ctx, *a, **kw)

@@ -4,7 +4,7 @@
 // The kernel exists in two forms (template parameter CTAS):
 //   CTAS = 1 : one CTA computes a 128 x 256 output tile (tcgen05.mma.cta_group::1), 4-stage ring of 48 KiB slabs.
 //   CTAS = 2 : two CTAs on neighbouring SMs (a cluster of 2) share one 256 x 256 tile: each loads its own 128 rows
-//              of A and its own 128 of the 256 rows of B (32 KiB per K slab, 6-stage ring) and one
+//              of A and its own 128 of the 256 rows of B (32 KiB per K slab, 7-stage ring) and one
 //              tcgen05.mma.cta_group::2 issued by the even CTA multiplies across both shared memories; each CTA's
 //              tensor memory receives the 128 x 256 accumulator block of its own rows.
 // Per CTA:
@@ -47,7 +47,7 @@ struct Cfg {
     static constexpr int kABytes = kCtaM * kTileK * 2;           // 16 KiB
     static constexpr int kBBytes = kBRows * kTileK * 2;          // 32 or 16 KiB
     static constexpr int kStageBytes = kABytes + kBBytes;        // 48 or 32 KiB
-    static constexpr int kStages = CTAS == 1 ? 4 : 6;
+    static constexpr int kStages = CTAS == 1 ? 4 : 7;
     static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kBarBytes;
 };
 

@@ -148,4 +148,7 @@ cudaError_t launch_zero_masked_rows(const int* tok_slot, long long n_tok, int H,
 cudaError_t launch_store_dhidden(const float* dHc, const int* slot_tok, int slot0, int n_rows, int H,
                                  __nv_bfloat16* dHidden, cudaStream_t stream);
 
+cudaError_t launch_gae(int n_inv, const int64_t* cu_seqlens, const float* rewards, const float* values,
+                       const uint8_t* tok_mask, float gamma, float lam, float* adv, float* ret, cudaStream_t stream);
+
 }  // namespace unity

@@ -396,6 +396,56 @@ __global__ void k_store_dhidden(const float* __restrict__ dHc, const int* __rest
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Token-level generalized advantage estimation: one warp per sequence, walking it backwards 32 tokens at a time.
+// Inside a chunk the recurrence A_t = delta_t + c*A_next is a composition of affine maps x -> b + a*x, evaluated
+// with a suffix scan over the lanes (masked tokens are the identity map); the value of the next unmasked token
+// comes from a ballot.  Loads and stores are 128-byte coalesced per warp.
+struct GaeArgs {
+    int n_inv;
+    const int64_t* cu_seqlens;
+    const float *rewards, *values;
+    const uint8_t* tok_mask;
+    float gamma, lam;
+    float *adv, *ret;
+};
+
+__global__ void k_gae(GaeArgs a) {
+    const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (s >= a.n_inv) return;
+    const long long lo = a.cu_seqlens[s], hi = a.cu_seqlens[s + 1];
+    const float c = a.gamma * a.lam;
+    float carry_adv = 0.f, carry_val = 0.f;       // A and V of the next unmasked token (0 past the end)
+    for (long long c0 = hi - 32; c0 > lo - 32; c0 -= 32) {
+        const long long t = c0 + lane;
+        const bool in = t >= lo && t < hi;
+        const bool on = in && (a.tok_mask ? a.tok_mask[t] != 0 : true);
+        const float v = on ? a.values[t] : 0.f;
+        const float r = on ? a.rewards[t] : 0.f;
+        const unsigned valid = __ballot_sync(kFull, on);
+        const unsigned above = lane == 31 ? 0u : (valid & (0xffffffffu << (lane + 1)));
+        const int j = above ? __ffs(above) - 1 : 0;
+        const float v_peer = __shfl_sync(kFull, v, j);
+        const float v_next = above ? v_peer : carry_val;
+        const float delta = r + a.gamma * v_next - v;
+        // suffix scan of the maps (ma, mb): result on lane i is the composition of lanes i, i+1, ..., 31
+        float ma = on ? c : 1.f, mb = on ? delta : 0.f;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float pa = __shfl_down_sync(kFull, ma, o), pb = __shfl_down_sync(kFull, mb, o);
+            if (lane + o < 32) { mb = fmaf(ma, pb, mb); ma = ma * pa; }
+        }
+        const float adv = fmaf(ma, carry_adv, mb);
+        if (in) {
+            a.adv[t] = on ? adv : 0.f;
+            a.ret[t] = on ? adv + v : 0.f;
+        }
+        carry_adv = __shfl_sync(kFull, adv, 0);    // lane 0 holds the composition of the whole chunk
+        if (valid) carry_val = __shfl_sync(kFull, v, __ffs(valid) - 1);
+    }
+}
+
 }  // namespace
 
 // ------------------------------------------------------------------------------------------------
@@ -458,6 +508,14 @@ cudaError_t launch_store_dhidden(const float* dHc, const int* slot_tok, int slot
                                  __nv_bfloat16* dHidden, cudaStream_t stream) {
     if (n_rows == 0) return cudaSuccess;
     k_store_dhidden<<<(n_rows + 7) / 8, 256, 0, stream>>>(dHc, slot_tok, slot0, n_rows, H, dHidden);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gae(int n_inv, const int64_t* cu_seqlens, const float* rewards, const float* values,
+                       const uint8_t* tok_mask, float gamma, float lam, float* adv, float* ret, cudaStream_t stream) {
+    if (n_inv == 0) return cudaSuccess;
+    GaeArgs a{n_inv, cu_seqlens, rewards, values, tok_mask, gamma, lam, adv, ret};
+    k_gae<<<(n_inv + 7) / 8, 256, 0, stream>>>(a);
     return cudaGetLastError();
 }
 

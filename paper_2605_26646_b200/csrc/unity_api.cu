@@ -465,6 +465,22 @@ int unity_role_advantage(unity_ctx* ctx, int32_t n_inv, int32_t n_traj, int32_t 
 }
 
 // ------------------------------------------------------------------------------------------------
+int unity_gae(unity_ctx* ctx, int32_t n_inv, int64_t n_tok, const int64_t* cu_seqlens, const float* rewards,
+              const float* values, const uint8_t* tok_mask, float gamma, float lam, float* advantages, float* returns) {
+    if (!ctx) return UNITY_ERR_INVALID_ARG;
+    if (n_inv < 0 || n_tok < 0) return fail(ctx, UNITY_ERR_INVALID_ARG, "negative size");
+    if (n_tok > 0 && (n_inv < 1 || !cu_seqlens || !rewards || !values || !advantages || !returns))
+        return fail(ctx, UNITY_ERR_INVALID_ARG, "cu_seqlens / rewards / values / advantages / returns is NULL or n_inv < 1");
+    if (!(gamma >= 0.f && gamma <= 1.f) || !(lam >= 0.f && lam <= 1.f))
+        return fail(ctx, UNITY_ERR_INVALID_ARG, "gamma and lambda must lie in [0, 1]");
+    if (n_tok == 0) return UNITY_OK;
+    CUDA_TRY(ctx, cudaSetDevice(ctx->device));
+    CUDA_TRY(ctx, launch_gae(n_inv, cu_seqlens, rewards, values, tok_mask, gamma, lam, advantages, returns, ctx->stream));
+    ctx->launches += 1;
+    return UNITY_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
 int unity_logprob_fwd(unity_ctx* ctx, const unity_rows* rows, float* logp, float* entropy, float* lse) {
     int rc = validate_rows(ctx, rows);
     if (rc) return rc;

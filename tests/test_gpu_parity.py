@@ -145,6 +145,35 @@ def test_bad_indices_are_flagged_not_fatal():
     ctx.close()
 
 
+@pytest.mark.parametrize("name,gamma,lam,masked", [("tiny", 1.0, 0.95, True), ("search", 0.99, 0.9, True),
+                                                   ("code", 0.97, 1.0, True), ("stress", 0.9, 0.0, False)])
+def test_gae_full_size(name, gamma, lam, masked):
+    import oracle.unity_oracle as orc
+    w = wl.make_structure(name)                # sequence lengths 0 .. 2048, padded spans, zero-length sequences
+    r = wl.normal(11, 5, w.n_tok)
+    v = wl.normal(11, 6, w.n_tok)
+    mask = w.tok_mask if masked else None
+    ctx = ub.Context(0, 1 << 20)
+    adv = torch.full((w.n_tok,), 7.0, device="cuda")
+    ret = torch.full((w.n_tok,), 7.0, device="cuda")
+    ctx.gae(w.cu_seqlens.cuda(), r.cuda(), v.cuda(), None if mask is None else mask.cuda(), gamma, lam, adv, ret)
+    ctx.check_status()
+    # the oracle evaluates the double sum literally: check the first 400 sequences (all of them for small configs)
+    n_seq = min(w.n_inv, 400)
+    n_chk = int(w.cu_seqlens[n_seq])
+    oa, orr = orc.gae(r.numpy()[:n_chk], v.numpy()[:n_chk], w.cu_seqlens.numpy()[:n_seq + 1], gamma, lam,
+                      None if mask is None else mask.numpy()[:n_chk])
+    scale = max(1.0, float(np.abs(oa).max()))
+    assert np.abs(adv.cpu().numpy()[:n_chk] - oa).max() <= 1e-5 * scale
+    assert np.abs(ret.cpu().numpy()[:n_chk] - orr).max() <= 1e-5 * scale
+    # beyond the checked prefix: masked tokens are zero and returns - advantages reproduces the values
+    a_all, r_all = adv.cpu(), ret.cpu()
+    keep = torch.ones(w.n_tok, dtype=torch.bool) if mask is None else mask != 0
+    assert torch.all(a_all[~keep] == 0) and torch.all(r_all[~keep] == 0)
+    assert torch.allclose((r_all - a_all)[keep], v[keep], atol=1e-5 * scale)
+    ctx.close()
+
+
 # ------------------------------------------------------------------------------------ stages 2 + 3
 
 def test_tiny_full():

@@ -463,3 +463,20 @@ def test_gae_special_cases_and_recursion():
             nxt = v[t + 1] if t + 1 < hi else 0.0
             nxtA = r[t] + gamma * nxt - v[t] + gamma * lam * nxtA
             assert abs(A[t] - nxtA) < 1e-12
+
+
+def test_gae_masked_tokens_are_transparent():
+    rng = np.random.default_rng(9)
+    cu = np.array([0, 7, 12, 12, 20])
+    n = 20
+    r, v = rng.normal(size=n), rng.normal(size=n)
+    mask = (rng.random(n) < 0.6).astype(np.uint8)
+    mask[7:12] = 0                                      # a sequence with no valid token
+    A, ret = orc.gae(r, v, cu, 0.97, 0.9, mask)
+    # removing the masked tokens and running the unmasked formula gives the same numbers
+    keep = mask != 0
+    lens = [int(keep[cu[s]:cu[s + 1]].sum()) for s in range(4)]
+    cu2 = np.concatenate([[0], np.cumsum(lens)])
+    A2, ret2 = orc.gae(r[keep], v[keep], cu2, 0.97, 0.9)
+    assert np.allclose(A[keep], A2, atol=1e-14) and np.allclose(ret[keep], ret2, atol=1e-14)
+    assert np.all(A[~keep] == 0) and np.all(ret[~keep] == 0)
