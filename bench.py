@@ -165,6 +165,54 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def run_micro(args):
+    """Streaming stages at a size where they are HBM-bound rather than launch-bound: role-level advantage
+    (token broadcast) and token-level GAE on 64 Mi tokens.  Prints one JSON line with achieved GB/s against the
+    measured copy bandwidth (algorithmic bytes: mask 1 B + output 4 B per token; rewards, values 8 B + mask 1 B +
+    two outputs 8 B per token)."""
+    import torch
+    from paper_2605_26646_b200 import binding as ub
+    from paper_2605_26646_b200 import workloads as wl
+    dev = torch.device("cuda", 0)
+    n_inv, seq = 1 << 16, 1 << 10
+    n = n_inv * seq
+    R, G = 4, 2048
+    inv_role = wl.randint(3, 1, n_inv, 0, R).to(torch.int32).to(dev)
+    inv_group = (torch.arange(n_inv) // (n_inv // G)).to(torch.int32).to(dev)      # 32 consecutive invocations per group
+    inv_traj = torch.arange(n_inv, dtype=torch.int32, device=dev)
+    r_node = wl.normal(3, 3, n_inv).to(dev)
+    cu = (torch.arange(n_inv + 1, dtype=torch.int64) * seq).to(dev)
+    mask = (torch.rand(n, device=dev) < 0.8).to(torch.uint8)
+    rewards, values = torch.randn(n, device=dev), torch.randn(n, device=dev)
+    adv_inv, adv_tok = torch.empty(n_inv, device=dev), torch.empty(n, device=dev)
+    a_out, r_out = torch.empty(n, device=dev), torch.empty(n, device=dev)
+    ctx = ub.Context(0, 1 << 22)
+    peaks = read_peaks()
+
+    def timed(fn, reps=10):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    t_adv = timed(lambda: ctx.role_advantage(n_inv, R, G, inv_role, inv_group, inv_traj, r_node, None, None, None, 1e-6,
+                                             0, cu, mask, adv_inv, adv_tok))
+    t_gae = timed(lambda: ctx.gae(cu, rewards, values, mask, 0.99, 0.95, a_out, r_out))
+    ctx.check_status()
+    out = {"mode": "micro", "tokens": n, "invocations": n_inv, "peak_hbm_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"],
+           "role_advantage": {"ms": t_adv, "algorithmic_bytes": 5 * n + 28 * n_inv, "gbs": (5 * n + 28 * n_inv) / t_adv / 1e6},
+           "gae": {"ms": t_gae, "algorithmic_bytes": 17 * n, "gbs": 17 * n / t_gae / 1e6}}
+    for k in ("role_advantage", "gae"):
+        out[k]["frac"] = out[k]["gbs"] / peaks["hbm_gbs"]
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -173,6 +221,7 @@ def main():
     ap.add_argument("--workload", default="code")
     ap.add_argument("--impl", default="unity", choices=["unity", "reference"])
     ap.add_argument("--ref-rows", type=int, default=256, help="valid rows per oracle step (reference arm / cpu baseline)")
+    ap.add_argument("--micro", action="store_true", help="measure the streaming stages at an HBM-bound size instead")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ctas", default="", help="CTAs per tile for the fwd,grad,dH,dW GEMMs, e.g. 1,1,2,2 (default: library's)")
@@ -182,6 +231,8 @@ def main():
         args.warmup = 3
     if args.impl == "reference":
         return run_reference(args)
+    if args.micro:
+        return run_micro(args)
 
     import torch
     import torch.distributed as dist

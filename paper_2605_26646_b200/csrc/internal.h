@@ -86,6 +86,7 @@ struct AdvArgs {
     float *adv_inv, *adv_tok, *seg_mean, *seg_std;
     float* r_scratch;   // [n_inv]
     int* seg_scratch;   // [n_inv]
+    int *seg_lo, *seg_hi;   // [n_groups*n_roles] first / last member index (pre-set to INT_MAX-ish / -1), or null
     int* status;
 };
 cudaError_t launch_advantage(const AdvArgs& a, cudaStream_t stream, int* n_launches);

@@ -54,6 +54,7 @@ __global__ void k_adv_combine(AdvArgs a) {
         const float rt = a.r_turn ? a.r_turn[s] : 0.f;
         r = __fadd_rn(__fadd_rn(__fmul_rn(ln, rn), __fmul_rn(lt, rt)), __fmul_rn(lj, rj));
         seg = g * a.n_roles + v;
+        if (a.seg_lo) { atomicMin(&a.seg_lo[seg], s); atomicMax(&a.seg_hi[seg], s); }
     } else {
         atomicOr(a.status, kStatusBadIndex);
     }
@@ -62,49 +63,80 @@ __global__ void k_adv_combine(AdvArgs a) {
     a.adv_inv[s] = 0.f;
 }
 
-// One warp per (group, role) segment.  Three sweeps over the invocation list with 128-bit loads:
-// count + sum -> mean; sum of squared deviations -> sigma; write the members' advantages.
+// One warp per (group, role) segment.  Three sweeps with 128-bit loads over the span of invocation indices that
+// contains the segment's members (recorded by k_adv_combine; rollout groups are normally contiguous, so spans are
+// short and the whole stage is O(n_inv)): count + sum -> mean; sum of squared deviations -> sigma; advantages.
 __global__ void k_adv_segment(AdvArgs a) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     const int n_seg = a.n_groups * a.n_roles;
     if (warp >= n_seg) return;
     const int q = warp;
-    const int n4 = a.n_inv >> 2;
+    int lo = 0, hi = a.n_inv;                       // [lo, hi): invocation indices to look at
+    if (a.seg_lo) { lo = a.seg_lo[q]; hi = a.seg_hi[q] + 1; }
+    if (lo >= hi) {                                 // empty segment
+        if (lane == 0) { if (a.seg_mean) a.seg_mean[q] = 0.f; if (a.seg_std) a.seg_std[q] = 0.f; }
+        return;
+    }
+    const int q0 = lo >> 2, q1 = hi >> 2;           // whole quads [q0, q1); head and tail handled per element
+    const int head_end = min(hi, (q0 << 2) == lo ? lo : (q0 + 1) << 2);
+    const int quad_lo = (q0 << 2) == lo ? q0 : q0 + 1;
+    const int tail_begin = max(head_end, q1 << 2);
     const int4* seg4 = reinterpret_cast<const int4*>(a.seg_scratch);
     const float4* r4 = reinterpret_cast<const float4*>(a.r_scratch);
 
+    // Pivot = reward of the segment's first member.  All sums run over r - pivot, so a segment whose rewards are all
+    // equal gives exactly zero deviations (and zero advantages) whatever the order of the floating-point sums.
+    int first = lo;
+    if (!a.seg_lo) {
+        first = a.n_inv;
+        for (int s = lane; s < a.n_inv; s += 32)
+            if (a.seg_scratch[s] == q) { first = s; break; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) first = min(first, __shfl_xor_sync(kFull, first, o));
+        if (first >= a.n_inv) {                     // empty segment
+            if (lane == 0) { if (a.seg_mean) a.seg_mean[q] = 0.f; if (a.seg_std) a.seg_std[q] = 0.f; }
+            return;
+        }
+    }
+    const float pivot = a.r_scratch[first];
+
     int cnt = 0;
     float sum = 0.f;
-    for (int i = lane; i < n4; i += 32) {
+    for (int s = lo + lane; s < head_end; s += 32)
+        if (a.seg_scratch[s] == q) { cnt++; sum += a.r_scratch[s] - pivot; }
+    for (int i = quad_lo + lane; i < q1; i += 32) {
         const int4 sg = seg4[i];
         if (sg.x == q || sg.y == q || sg.z == q || sg.w == q) {
             const float4 r = r4[i];
-            if (sg.x == q) { cnt++; sum += r.x; }
-            if (sg.y == q) { cnt++; sum += r.y; }
-            if (sg.z == q) { cnt++; sum += r.z; }
-            if (sg.w == q) { cnt++; sum += r.w; }
+            if (sg.x == q) { cnt++; sum += r.x - pivot; }
+            if (sg.y == q) { cnt++; sum += r.y - pivot; }
+            if (sg.z == q) { cnt++; sum += r.z - pivot; }
+            if (sg.w == q) { cnt++; sum += r.w - pivot; }
         }
     }
-    for (int s = (n4 << 2) + lane; s < a.n_inv; s += 32)
-        if (a.seg_scratch[s] == q) { cnt++; sum += a.r_scratch[s]; }
+    for (int s = tail_begin + lane; s < hi; s += 32)
+        if (a.seg_scratch[s] == q) { cnt++; sum += a.r_scratch[s] - pivot; }
     cnt = warp_sum_int(cnt);
     sum = warp_sum(sum);
-    const float mu = cnt > 0 ? sum / static_cast<float>(cnt) : 0.f;
+    const float dmu = cnt > 0 ? sum / static_cast<float>(cnt) : 0.f;     // mean of r - pivot
+    const float mu = pivot + dmu;
 
     float m2 = 0.f;
-    for (int i = lane; i < n4; i += 32) {
+    for (int s = lo + lane; s < head_end; s += 32)
+        if (a.seg_scratch[s] == q) { const float d = (a.r_scratch[s] - pivot) - dmu; m2 += d * d; }
+    for (int i = quad_lo + lane; i < q1; i += 32) {
         const int4 sg = seg4[i];
         if (sg.x == q || sg.y == q || sg.z == q || sg.w == q) {
             const float4 r = r4[i];
-            if (sg.x == q) { const float d = r.x - mu; m2 += d * d; }
-            if (sg.y == q) { const float d = r.y - mu; m2 += d * d; }
-            if (sg.z == q) { const float d = r.z - mu; m2 += d * d; }
-            if (sg.w == q) { const float d = r.w - mu; m2 += d * d; }
+            if (sg.x == q) { const float d = (r.x - pivot) - dmu; m2 += d * d; }
+            if (sg.y == q) { const float d = (r.y - pivot) - dmu; m2 += d * d; }
+            if (sg.z == q) { const float d = (r.z - pivot) - dmu; m2 += d * d; }
+            if (sg.w == q) { const float d = (r.w - pivot) - dmu; m2 += d * d; }
         }
     }
-    for (int s = (n4 << 2) + lane; s < a.n_inv; s += 32)
-        if (a.seg_scratch[s] == q) { const float d = a.r_scratch[s] - mu; m2 += d * d; }
+    for (int s = tail_begin + lane; s < hi; s += 32)
+        if (a.seg_scratch[s] == q) { const float d = (a.r_scratch[s] - pivot) - dmu; m2 += d * d; }
     m2 = warp_sum(m2);
 
     const int dof = cnt - a.ddof;
@@ -115,36 +147,48 @@ __global__ void k_adv_segment(AdvArgs a) {
         if (a.seg_std) a.seg_std[q] = sigma;
     }
     if (cnt == 0) return;
-    for (int s = lane; s < a.n_inv; s += 32)
-        if (a.seg_scratch[s] == q) a.adv_inv[s] = (dof > 0 && denom != 0.f) ? (a.r_scratch[s] - mu) / denom : 0.f;
+    for (int s = lo + lane; s < hi; s += 32)
+        if (a.seg_scratch[s] == q)
+            a.adv_inv[s] = (dof > 0 && denom != 0.f) ? ((a.r_scratch[s] - pivot) - dmu) / denom : 0.f;
 }
 
-// Four tokens per thread: one 32-bit mask load, one 128-bit store.
-__global__ void k_adv_broadcast(AdvArgs a) {
-    const long long i0 = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) * 4;
-    if (i0 >= a.n_tok) return;
-    int s = find_invocation(a.cu_seqlens, a.n_inv, i0);
-    long long end = a.cu_seqlens[s + 1];
-    float adv = a.adv_inv[s];
-    float out[4];
-    const int n = static_cast<int>(min(4LL, a.n_tok - i0));
-    unsigned m4 = 0x01010101u;
+// A block broadcasts rounds x 1024 tokens; in a round each thread handles four consecutive tokens (one 32-bit mask
+// load, one 128-bit store), so every warp instruction covers 128 B of mask and 512 B of output contiguously.
+// The owning invocation is found by binary search once per thread (a chain of dependent loads, amortised over the
+// rounds) and advanced linearly afterwards.
+__global__ void k_adv_broadcast(AdvArgs a, int rounds) {
+    const long long block0 = static_cast<long long>(blockIdx.x) * (blockDim.x * 4) * rounds;
     const bool mask_al = (reinterpret_cast<uintptr_t>(a.tok_mask) & 3) == 0;
     const bool out_al = (reinterpret_cast<uintptr_t>(a.adv_tok) & 15) == 0;
-    if (a.tok_mask) {
-        if (n == 4 && mask_al) m4 = *reinterpret_cast<const unsigned*>(a.tok_mask + i0);
-        else { m4 = 0; for (int j = 0; j < n; ++j) m4 |= static_cast<unsigned>(a.tok_mask[i0 + j]) << (8 * j); }
-    }
+    int s = -1;
+    long long end = 0;
+    float adv = 0.f;
+    for (int round = 0; round < rounds; ++round) {
+        const long long i0 = block0 + (static_cast<long long>(round) * blockDim.x + threadIdx.x) * 4;
+        if (i0 >= a.n_tok) return;
+        if (s < 0) {
+            s = find_invocation(a.cu_seqlens, a.n_inv, i0);
+            end = a.cu_seqlens[s + 1];
+            adv = a.adv_inv[s];
+        }
+        float out[4];
+        const int n = static_cast<int>(min(4LL, a.n_tok - i0));
+        unsigned m4 = 0x01010101u;
+        if (a.tok_mask) {
+            if (n == 4 && mask_al) m4 = *reinterpret_cast<const unsigned*>(a.tok_mask + i0);
+            else { m4 = 0; for (int j = 0; j < n; ++j) m4 |= static_cast<unsigned>(a.tok_mask[i0 + j]) << (8 * j); }
+        }
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const long long i = i0 + j;
-        if (j < n) {
-            while (i >= end && s + 1 < a.n_inv) { ++s; end = a.cu_seqlens[s + 1]; adv = a.adv_inv[s]; }
-            out[j] = ((m4 >> (8 * j)) & 0xffu) ? adv : 0.f;
-        } else out[j] = 0.f;
+        for (int j = 0; j < 4; ++j) {
+            const long long i = i0 + j;
+            if (j < n) {
+                while (i >= end && s + 1 < a.n_inv) { ++s; end = a.cu_seqlens[s + 1]; adv = a.adv_inv[s]; }
+                out[j] = ((m4 >> (8 * j)) & 0xffu) ? adv : 0.f;
+            } else out[j] = 0.f;
+        }
+        if (n == 4 && out_al) *reinterpret_cast<float4*>(a.adv_tok + i0) = make_float4(out[0], out[1], out[2], out[3]);
+        else for (int j = 0; j < n; ++j) a.adv_tok[i0 + j] = out[j];
     }
-    if (n == 4 && out_al) *reinterpret_cast<float4*>(a.adv_tok + i0) = make_float4(out[0], out[1], out[2], out[3]);
-    else for (int j = 0; j < n; ++j) a.adv_tok[i0 + j] = out[j];
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -459,8 +503,12 @@ cudaError_t launch_advantage(const AdvArgs& a, cudaStream_t stream, int* n_launc
         *n_launches += 2;
     }
     if (a.n_tok > 0) {
-        const long long quads = (a.n_tok + 3) / 4;
-        k_adv_broadcast<<<static_cast<unsigned>((quads + 255) / 256), 256, 0, stream>>>(a);
+        // enough blocks to fill the machine (about 8 per SM), at most 32 rounds per block
+        long long rounds = a.n_tok / (1024LL * 148 * 8);
+        rounds = rounds < 1 ? 1 : (rounds > 32 ? 32 : rounds);
+        const long long per_block = 1024 * rounds;
+        k_adv_broadcast<<<static_cast<unsigned>((a.n_tok + per_block - 1) / per_block), 256, 0, stream>>>(
+            a, static_cast<int>(rounds));
         *n_launches += 1;
     }
     return cudaGetLastError();

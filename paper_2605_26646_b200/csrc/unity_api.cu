@@ -449,7 +449,12 @@ int unity_role_advantage(unity_ctx* ctx, int32_t n_inv, int32_t n_traj, int32_t 
     memset(&a, 0, sizeof(a));
     a.r_scratch = b.take<float>(n_inv + 4);
     a.seg_scratch = b.take<int>(n_inv + 4);
+    const size_t n_seg = static_cast<size_t>(n_groups) * n_roles;
+    a.seg_lo = b.take<int>(n_seg);
+    a.seg_hi = b.take<int>(n_seg);
     if (!b.ok) return fail(ctx, UNITY_ERR_WORKSPACE, "workspace too small: need %zu bytes", b.off);
+    CUDA_TRY(ctx, cudaMemsetAsync(a.seg_lo, 0x7f, sizeof(int) * n_seg, ctx->stream));   // 0x7f7f7f7f: above any index
+    CUDA_TRY(ctx, cudaMemsetAsync(a.seg_hi, 0xff, sizeof(int) * n_seg, ctx->stream));   // -1
     a.n_inv = n_inv; a.n_traj = n_traj; a.n_roles = n_roles; a.n_groups = n_groups;
     a.inv_role = inv_role; a.inv_group = inv_group; a.inv_traj = inv_traj;
     a.r_node = r_node; a.r_turn = r_turn; a.r_traj = r_traj;
