@@ -123,6 +123,32 @@ int unity_role_advantage(unity_ctx* ctx, int32_t n_inv, int32_t n_traj, int32_t 
                          const unity_adv_params* params, int64_t n_tok, const int64_t* cu_seqlens,
                          const uint8_t* tok_mask, float* adv_inv, float* adv_tok, float* seg_mean, float* seg_std);
 
+/* Turn-level reward assembly - the step before stage 1 (paragraph "Reward assembly and commitment"), for the
+ * turn-level rules of Section "Workflows and Rewards".  score[j*max_turns + t] is the score after turn t of
+ * trajectory j (answer F1 in the iterative search workflow, verifier pass rate in the reflective code workflow);
+ * n_scores[j] turns of trajectory j have a score.  Each role v has a rule: with u = inv_turn[s] + rules[v].shift,
+ *   UNITY_RULE_ABSOLUTE : r_turn[s] = score[j, u]                 (planner F1(a_0); answer agent F1(a_t))
+ *   UNITY_RULE_MARGINAL : r_turn[s] = score[j, u] - score[j, u-1] (loop agents F1(a_t) - F1(a_{t-1}); code workflow
+ *                         s_0, s_1 - s_0, s_2 - s_1, with shift = 1 for the reflector, which is paid the next
+ *                         round's improvement); the score before the first turn counts as 0
+ *   UNITY_RULE_NONE     : r_turn[s] = 0                           (workflows whose roles share only a final score)
+ * No score at u, or inv_end[s] != 0 (the agent ended the loop), gives 0.  Shared final scores and node-level format
+ * terms need no assembly: they enter stage 1 as r_traj and r_node.
+ *   inv_role, inv_traj, inv_turn : int32 [n_inv];  score : f32 [n_traj*max_turns];  n_scores : int32 [n_traj] or
+ *   NULL (= max_turns);  inv_end : u8 [n_inv] or NULL;  rules : (host) [n_roles];  r_turn : out f32 [n_inv]
+ * An out-of-range role or trajectory id flags UNITY_ERR_BAD_INDEX and yields 0. */
+#define UNITY_RULE_NONE 0
+#define UNITY_RULE_ABSOLUTE 1
+#define UNITY_RULE_MARGINAL 2
+typedef struct {
+    int mode;  /* UNITY_RULE_* */
+    int shift; /* turn offset of the score this role is paid for (0, or 1 for "next round") */
+} unity_reward_rule;
+int unity_reward_assembly(unity_ctx* ctx, int32_t n_inv, int32_t n_traj, int32_t n_roles, int32_t max_turns,
+                          const int32_t* inv_role, const int32_t* inv_traj, const int32_t* inv_turn, const float* score,
+                          const int32_t* n_scores, const uint8_t* inv_end, const unity_reward_rule* rules,
+                          float* r_turn);
+
 /* Token-level generalized advantage estimation - the advantage formula printed in paragraph "Advantage
  * computation and policy evaluation":  A_t = sum_{l=0}^{T-t} (gamma*lambda)^l delta_{t+l},
  * delta_t = r_t + gamma*V(s_{t+1}) - V(s_t), evaluated per sequence (cu_seqlens) with V = 0 past the last token;

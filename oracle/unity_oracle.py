@@ -24,6 +24,10 @@ What each function follows:
   bonus, averaged over valid tokens per model (paragraph "Model-specific updates and
   synchronization": each worker group updates its own actor), and its exact gradient with
   respect to the hidden states and each LM-head matrix.
+* ``reward_assembly`` - the turn-level reward rules of Section "Workflows and Rewards": a role is paid either the
+  score of a turn (Workflow C: planner F1(a_0), answer agent F1(a_t)) or the improvement of the score over the
+  previous turn (Workflow C: F1(a_t) - F1(a_{t-1}) for the loop agents; Workflow D: s_0, s_1 - s_0, s_2 - s_1, the
+  reflector of round i being paid the improvement of round i+1); an agent that ended the loop gets 0.
 * ``gae``             - the generalized-advantage equation printed in the same section
   (A_t = sum_l (gamma lambda)^l delta_{t+l}), evaluated as the literal double sum.
 
@@ -95,6 +99,37 @@ def role_advantage(inv_role, inv_group, inv_traj, r_node, r_turn, r_traj, lam,
         adv_tok[cu[s]:cu[s + 1]] = adv_inv[s]
     adv_tok *= mask
     return dict(r=r, adv_inv=adv_inv, adv_tok=adv_tok, seg_n=seg_n, seg_mean=seg_mean, seg_std=seg_std)
+
+
+# ----------------------------------------------------------------------------------------------
+# turn-level reward assembly (the step before stage 1)
+# ----------------------------------------------------------------------------------------------
+
+RULE_NONE, RULE_ABSOLUTE, RULE_MARGINAL = 0, 1, 2
+
+
+def reward_assembly(inv_role, inv_traj, inv_turn, score, n_scores, rules, inv_end=None):
+    """r_turn per invocation from per-trajectory, per-turn scores.
+
+    ``score[j, t]`` is the score after turn t of trajectory j (answer F1, verifier pass rate); ``n_scores[j]`` turns
+    have a score.  ``rules[v] = (mode, shift)``: with u = turn + shift, mode ABSOLUTE pays score[j, u], mode MARGINAL
+    pays score[j, u] - score[j, u-1] (the score before the first turn counts as 0), mode NONE pays 0.  No score at
+    u (u < 0 or u >= n_scores[j]) pays 0; ``inv_end[s] != 0`` pays 0."""
+    S = len(inv_role)
+    score = to_f64(score)
+    out = np.zeros(S, F64)
+    for s in range(S):
+        mode, shift = rules[int(inv_role[s])]
+        j, u = int(inv_traj[s]), int(inv_turn[s]) + shift
+        if mode == RULE_NONE or u < 0 or u >= int(n_scores[j]):
+            continue
+        if inv_end is not None and inv_end[s]:
+            continue
+        if mode == RULE_ABSOLUTE:
+            out[s] = score[j, u]
+        else:
+            out[s] = score[j, u] - (score[j, u - 1] if u >= 1 else 0.0)
+    return out
 
 
 # ----------------------------------------------------------------------------------------------

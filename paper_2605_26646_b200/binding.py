@@ -25,7 +25,7 @@ UNITY_N_METRICS = 8
 
 EXPORTS = ["unity_create", "unity_destroy", "unity_workspace_bytes", "unity_workspace_min_bytes",
            "unity_check_status", "unity_last_error", "unity_launch_count", "unity_set_profiling",
-           "unity_get_profile", "unity_set_option", "unity_role_advantage", "unity_gae", "unity_role_advantage_noalloc",
+           "unity_get_profile", "unity_set_option", "unity_role_advantage", "unity_reward_assembly", "unity_gae", "unity_role_advantage_noalloc",
            "unity_logprob_fwd", "unity_ppo_loss_fwd_bwd"]
 
 
@@ -37,6 +37,10 @@ class UnityError(RuntimeError):
 
 class unity_adv_params(C.Structure):
     _fields_ = [("eps", C.c_float), ("ddof", C.c_int)]
+
+
+class unity_reward_rule(C.Structure):
+    _fields_ = [("mode", C.c_int), ("shift", C.c_int)]
 
 
 class unity_rows(C.Structure):
@@ -94,6 +98,9 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
                                                  C.POINTER(unity_adv_params), i64, vp, vp, vp, vp, vp, vp, vp,
                                                  C.c_char_p, C.c_size_t]
     lib.unity_role_advantage_noalloc.restype = C.c_int
+    lib.unity_reward_assembly.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp,
+                                          C.POINTER(unity_reward_rule), vp]
+    lib.unity_reward_assembly.restype = C.c_int
     lib.unity_gae.argtypes = [vp, i32, i64, vp, vp, vp, vp, C.c_float, C.c_float, vp, vp]
     lib.unity_gae.restype = C.c_int
     lib.unity_logprob_fwd.argtypes = [vp, C.POINTER(unity_rows), vp, vp, vp]
@@ -194,6 +201,22 @@ def unity_role_advantage(ctx, n_traj: int, n_roles: int, n_groups: int, inv_role
         _ptr(r_traj, f32, "r_traj"), lam_arr, C.byref(p), n_tok, _ptr(cu_seqlens, torch.int64, "cu_seqlens"),
         _ptr(tok_mask, torch.uint8, "tok_mask"), _ptr(adv_inv, f32, "adv_inv"), _ptr(adv_tok, f32, "adv_tok"),
         _ptr(seg_mean, f32, "seg_mean"), _ptr(seg_std, f32, "seg_std"))
+    _raise(ctx, code)
+
+
+RULE_NONE, RULE_ABSOLUTE, RULE_MARGINAL = 0, 1, 2
+
+
+def unity_reward_assembly(ctx, inv_role, inv_traj, inv_turn, score, n_scores, inv_end, rules, r_turn) -> None:
+    """score: f32 CUDA tensor [n_traj, max_turns]; rules: sequence of (mode, shift) per role."""
+    n_traj, max_turns = int(score.shape[0]), int(score.shape[1])
+    arr = (unity_reward_rule * len(rules))(*[unity_reward_rule(int(m), int(sh)) for m, sh in rules])
+    i32 = torch.int32
+    code = load_library().unity_reward_assembly(
+        ctx, int(inv_role.numel()), n_traj, len(rules), max_turns, _ptr(inv_role, i32, "inv_role"),
+        _ptr(inv_traj, i32, "inv_traj"), _ptr(inv_turn, i32, "inv_turn"), _ptr(score, torch.float32, "score"),
+        _ptr(n_scores, i32, "n_scores"), _ptr(inv_end, torch.uint8, "inv_end"), arr,
+        _ptr(r_turn, torch.float32, "r_turn"))
     _raise(ctx, code)
 
 
@@ -324,6 +347,9 @@ class Context:
 
     def role_advantage(self, *a, **kw):
         return unity_role_advantage(self.ctx, *a, **kw)
+
+    def reward_assembly(self, *a, **kw):
+        return unity_reward_assembly(self.ctx, *a, **kw)
 
     def gae(self, *a, **kw):
         return unity_gae(self.ctx, *a, **kw)

@@ -152,4 +152,17 @@ cudaError_t launch_store_dhidden(const float* dHc, const int* slot_tok, int slot
 cudaError_t launch_gae(int n_inv, const int64_t* cu_seqlens, const float* rewards, const float* values,
                        const uint8_t* tok_mask, float gamma, float lam, float* adv, float* ret, cudaStream_t stream);
 
+struct RewardArgs {
+    int n_inv, n_traj, n_roles, max_turns;
+    const int32_t *inv_role, *inv_traj, *inv_turn;
+    const float* score;          // [n_traj, max_turns]
+    const int32_t* n_scores;     // [n_traj] or null (= max_turns)
+    const uint8_t* inv_end;      // [n_inv] or null
+    int mode[UNITY_MAX_ROLES];   // 0 none, 1 absolute, 2 marginal
+    int shift[UNITY_MAX_ROLES];
+    float* r_turn;               // out [n_inv]
+    int* status;
+};
+cudaError_t launch_reward_assembly(const RewardArgs& a, cudaStream_t stream);
+
 }  // namespace unity

@@ -490,6 +490,28 @@ __global__ void k_gae(GaeArgs a) {
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Turn-level reward assembly: one thread per invocation gathers its trajectory's score(s).
+__global__ void k_reward_assembly(RewardArgs a) {
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= a.n_inv) return;
+    float out = 0.f;
+    const int v = a.inv_role[s], j = a.inv_traj[s];
+    if (v < 0 || v >= a.n_roles || j < 0 || j >= a.n_traj) {
+        atomicOr(a.status, kStatusBadIndex);
+    } else {
+        const int mode = a.mode[v];
+        const int u = a.inv_turn[s] + a.shift[v];
+        const int n = min(a.n_scores ? a.n_scores[j] : a.max_turns, a.max_turns);
+        const bool ended = a.inv_end ? a.inv_end[s] != 0 : false;
+        if (mode != 0 && u >= 0 && u < n && !ended) {
+            const float* sc = a.score + static_cast<long long>(j) * a.max_turns;
+            out = mode == 1 ? sc[u] : sc[u] - (u >= 1 ? sc[u - 1] : 0.f);
+        }
+    }
+    a.r_turn[s] = out;
+}
+
 }  // namespace
 
 // ------------------------------------------------------------------------------------------------
@@ -564,6 +586,12 @@ cudaError_t launch_gae(int n_inv, const int64_t* cu_seqlens, const float* reward
     if (n_inv == 0) return cudaSuccess;
     GaeArgs a{n_inv, cu_seqlens, rewards, values, tok_mask, gamma, lam, adv, ret};
     k_gae<<<(n_inv + 7) / 8, 256, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_reward_assembly(const RewardArgs& a, cudaStream_t stream) {
+    if (a.n_inv == 0) return cudaSuccess;
+    k_reward_assembly<<<(a.n_inv + 255) / 256, 256, 0, stream>>>(a);
     return cudaGetLastError();
 }
 

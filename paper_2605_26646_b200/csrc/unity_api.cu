@@ -470,6 +470,35 @@ int unity_role_advantage(unity_ctx* ctx, int32_t n_inv, int32_t n_traj, int32_t 
 }
 
 // ------------------------------------------------------------------------------------------------
+int unity_reward_assembly(unity_ctx* ctx, int32_t n_inv, int32_t n_traj, int32_t n_roles, int32_t max_turns,
+                          const int32_t* inv_role, const int32_t* inv_traj, const int32_t* inv_turn, const float* score,
+                          const int32_t* n_scores, const uint8_t* inv_end, const unity_reward_rule* rules,
+                          float* r_turn) {
+    if (!ctx) return UNITY_ERR_INVALID_ARG;
+    if (n_inv < 0 || n_traj < 0 || max_turns < 1) return fail(ctx, UNITY_ERR_INVALID_ARG, "negative size or max_turns < 1");
+    if (n_roles < 1 || n_roles > UNITY_MAX_ROLES) return fail(ctx, UNITY_ERR_SHAPE, "n_roles=%d outside [1,%d]", n_roles, UNITY_MAX_ROLES);
+    if (!rules) return fail(ctx, UNITY_ERR_INVALID_ARG, "rules is NULL");
+    if (n_inv > 0 && (!inv_role || !inv_traj || !inv_turn || !score || !r_turn))
+        return fail(ctx, UNITY_ERR_INVALID_ARG, "inv_role / inv_traj / inv_turn / score / r_turn is NULL");
+    RewardArgs a;
+    memset(&a, 0, sizeof(a));
+    for (int v = 0; v < n_roles; ++v) {
+        if (rules[v].mode < UNITY_RULE_NONE || rules[v].mode > UNITY_RULE_MARGINAL)
+            return fail(ctx, UNITY_ERR_INVALID_ARG, "rules[%d].mode must be 0, 1 or 2", v);
+        a.mode[v] = rules[v].mode;
+        a.shift[v] = rules[v].shift;
+    }
+    if (n_inv == 0) return UNITY_OK;
+    CUDA_TRY(ctx, cudaSetDevice(ctx->device));
+    a.n_inv = n_inv; a.n_traj = n_traj; a.n_roles = n_roles; a.max_turns = max_turns;
+    a.inv_role = inv_role; a.inv_traj = inv_traj; a.inv_turn = inv_turn; a.score = score; a.n_scores = n_scores;
+    a.inv_end = inv_end; a.r_turn = r_turn; a.status = ctx->d_status;
+    CUDA_TRY(ctx, launch_reward_assembly(a, ctx->stream));
+    ctx->launches += 1;
+    return UNITY_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
 int unity_gae(unity_ctx* ctx, int32_t n_inv, int64_t n_tok, const int64_t* cu_seqlens, const float* rewards,
               const float* values, const uint8_t* tok_mask, float gamma, float lam, float* advantages, float* returns) {
     if (!ctx) return UNITY_ERR_INVALID_ARG;

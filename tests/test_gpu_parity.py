@@ -145,6 +145,27 @@ def test_bad_indices_are_flagged_not_fatal():
     ctx.close()
 
 
+@pytest.mark.parametrize("name,rules", [("code", [(2, 0), (2, 1)]), ("search", [(1, 0), (2, 0), (1, 0)])])
+def test_reward_assembly_full_size(name, rules):
+    import oracle.unity_oracle as orc
+    w = wl.make_structure(name)                # code: coder / reflector deltas; search: planner, searcher, answerer
+    max_turns = int(w.inv_turn.max()) + 1
+    score = wl.uniform(21, 3, w.n_traj * max_turns).float().view(w.n_traj, max_turns)
+    n_scores = (torch.zeros(w.n_traj, dtype=torch.int64).scatter_reduce(0, w.inv_traj.long(), w.inv_turn.long() + 1,
+                                                                        "amax")).to(torch.int32)
+    inv_end = wl.bernoulli(21, 4, w.n_inv, 0.1).to(torch.uint8)
+    ctx = ub.Context(0, 1 << 20)
+    out = torch.full((w.n_inv,), 7.0, device="cuda")
+    ctx.reward_assembly(w.inv_role.cuda(), w.inv_traj.cuda(), w.inv_turn.cuda(), score.cuda(), n_scores.cuda(),
+                        inv_end.cuda(), rules, out)
+    ctx.check_status()
+    ref = orc.reward_assembly(w.inv_role.numpy(), w.inv_traj.numpy(), w.inv_turn.numpy(), score.numpy(),
+                              n_scores.numpy(), rules, inv_end.numpy())
+    assert np.abs(out.cpu().numpy() - ref).max() <= 1e-6
+    assert np.abs(ref).max() > 0 and (ref == 0).any()
+    ctx.close()
+
+
 @pytest.mark.parametrize("name,gamma,lam,masked", [("tiny", 1.0, 0.95, True), ("search", 0.99, 0.9, True),
                                                    ("code", 0.97, 1.0, True), ("stress", 0.9, 0.0, False)])
 def test_gae_full_size(name, gamma, lam, masked):

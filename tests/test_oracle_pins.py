@@ -480,3 +480,31 @@ def test_gae_masked_tokens_are_transparent():
     A2, ret2 = orc.gae(r[keep], v[keep], cu2, 0.97, 0.9)
     assert np.allclose(A[keep], A2, atol=1e-14) and np.allclose(ret[keep], ret2, atol=1e-14)
     assert np.all(A[~keep] == 0) and np.all(ret[~keep] == 0)
+
+
+def test_reward_assembly_follows_the_workflow_rules():
+    # Workflow D (reflective verification loop), scores and expected rewards from the hand fixture
+    rows = np.array([[float(x) for x in line.split()] for line in open(os.path.join(GOLDEN, "workflow_d_rewards.txt"))
+                     if line[0].isdigit()])
+    scores, expect = rows[:, 1:4], rows[:, 4:7]
+    # roles: 0 planner, 1 coder (paid the improvement of their own round), 2 reflector (paid the improvement of the
+    # NEXT round; there is no reflector after the last round)
+    rules = [(orc.RULE_MARGINAL, 0), (orc.RULE_MARGINAL, 0), (orc.RULE_MARGINAL, 1)]
+    inv = [(j, t, v) for j in range(2) for t in range(3) for v in (0, 1, 2) if not (v == 2 and t == 2)]
+    traj, turn, role = (np.array(x) for x in zip(*inv))
+    r = orc.reward_assembly(role, traj, turn, scores, [3, 3], rules)
+    for s, (j, t, v) in enumerate(inv):
+        want = expect[j, t] if v < 2 else expect[j, t + 1]      # r(Reflector_i) = s_{i+1} - s_i
+        assert abs(r[s] - want) < 1e-12
+    # Workflow C (iterative search): planner F1(a_0); answer agent F1(a_t); loop agents F1(a_t) - F1(a_{t-1});
+    # a search agent that outputs <end> gets 0
+    f1 = np.array([[0.25, 0.5, 0.4, 0.9]])
+    rules = [(orc.RULE_ABSOLUTE, 0), (orc.RULE_MARGINAL, 0), (orc.RULE_ABSOLUTE, 0)]      # planner, searcher, answerer
+    role = np.array([0, 1, 2, 1, 2, 1, 2])
+    turn = np.array([0, 1, 1, 2, 2, 3, 3])
+    end = np.array([0, 0, 0, 0, 0, 1, 0])
+    r = orc.reward_assembly(role, np.zeros(7, int), turn, f1, [4], rules, end)
+    assert np.allclose(r, [0.25, 0.25, 0.5, -0.1, 0.4, 0.0, 0.9])
+    # a turn without a score pays nothing, and so does a role without a turn-level rule (Workflows A / B)
+    r = orc.reward_assembly(np.array([1, 0]), np.zeros(2, int), np.array([2, 0]), f1, [2], [(orc.RULE_NONE, 0), (orc.RULE_ABSOLUTE, 0)])
+    assert np.all(r == 0)
