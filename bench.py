@@ -32,8 +32,8 @@ UNIT = "tokens/s"
 # (valid rows x vocabulary columns).  Traffic grows in proportion to the logits covered (same chunk and group sizes),
 # so a full-size launch is estimated as bytes_per_logit x its logits.  Valid only for the kernel source it was taken
 # from: when the hash of gemm_tcgen05.cu differs, the benchmark reports null.
-NCU_TRAFFIC = {"source_sha256_16": "49c0d1fa7357c3b2",
-               "bytes_per_logit": {"fwd_gemm": 1.859, "grad_gemm": 6.99, "dh_gemm": 10.71, "dw_gemm": 10.73}}
+NCU_TRAFFIC = {"source_sha256_16": "2aa4a0f7d9de35b6",
+               "bytes_per_logit": {"fwd_gemm": 1.863, "grad_gemm": 4.734, "dh_gemm": 9.906, "dw_gemm": 9.956}}
 
 
 def ncu_traffic_per_launch(cls: str, logits_per_launch: float):
@@ -225,6 +225,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ctas", default="", help="CTAs per tile for the fwd,grad,dH,dW GEMMs, e.g. 1,1,2,2 (default: library's)")
+    ap.add_argument("--opt", default="", help="library tuning options as id=value,id=value (see UNITY_OPT_* in unity.h)")
     ap.add_argument("--cut-rows", type=int, default=0, help="profile-capture helper: run on a cut of the workload")
     args = ap.parse_args()
     if args.warmup < 3 and args.cut_rows == 0:
@@ -261,7 +262,14 @@ def main():
     role_model = w.role_model.tolist()
     lam = w.lam.tolist()
     ws_bytes = ub.unity_workspace_bytes(n, H, V, K, w.n_inv)
-    ctx = ub.Context(local, ws_bytes)
+    opts = [tuple(int(x) for x in kv.split("=")) for kv in args.opt.split(",") if kv]
+    ws_mult = 1
+    for o, v in opts:
+        if o in (6, 7):
+            ws_mult *= v                       # larger gradient chunks need a larger G / dH scratch
+    ctx = ub.Context(local, ws_bytes + (ws_mult - 1) * (2 * 18944 * 18944 + 4 * 18944 * H) * (2 if ws_mult > 1 else 0))
+    for o, v in opts:
+        ctx.set_option(o, v)
     if args.ctas:
         for option, value in enumerate(int(x) for x in args.ctas.split(",")):
             ctx.set_option(option, value)

@@ -31,6 +31,10 @@ struct unity_ctx {
     std::vector<int>* ev_class;     // class of the i-th recorded pair
     size_t ev_used;                 // events handed out since the last unity_get_profile
     int ctas[UNITY_PROF_CLASSES];   // per GEMM class: 1 = single CTA per tile, 2 = CTA pair per tile
+    int l2_promotion;               // tensor-map L2 promotion: 0 none, 1 64 B, 2 128 B, 3 256 B
+    int chunk_group;                // raster group of the chunk GEMMs, in 128-row tiles
+    int chunk_rows_mult, chunk_vocab_mult;   // gradient chunk = mult x 18944 rows / vocabulary entries
+    int fwd_group;                  // row tiles (128 rows) per round of the forward kernel; 0 = a quarter of the SMs
 };
 
 namespace {
@@ -143,13 +147,13 @@ Layout carve(char* base, size_t cap, long long n_tok, int H, int V, int K, int n
     return L;
 }
 
-int wanted_chunk_rows(long long n_tok, int K) {
-    const long long ms = max_slots_of(n_tok, K);
-    return static_cast<int>(ms < kChunkRows ? ms : kChunkRows);
+int wanted_chunk_rows(long long n_tok, int K, int mult = 1) {
+    const long long ms = max_slots_of(n_tok, K), want = static_cast<long long>(kChunkRows) * mult;
+    return static_cast<int>(ms < want ? ms : want);
 }
-int wanted_chunk_vocab(int V) {
-    const long long vp = static_cast<long long>(up(V, kTileN));
-    return static_cast<int>(vp < kChunkVocab ? vp : kChunkVocab);
+int wanted_chunk_vocab(int V, int mult = 1) {
+    const long long vp = static_cast<long long>(up(V, kTileN)), want = static_cast<long long>(kChunkVocab) * mult;
+    return static_cast<int>(vp < want ? vp : want);
 }
 
 // Tensor map over a row-major bf16 matrix [rows, inner]; boxes are 64 elements (128 B, one swizzle row) wide and
@@ -161,7 +165,7 @@ int make_tmap(unity_ctx* ctx, CUtensorMap* tm, const void* ptr, uint64_t inner, 
     cuuint32_t box[2] = {64u, box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = ctx->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, static_cast<CUtensorMapL2promotion>(ctx->l2_promotion),
                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS)
         return fail(ctx, UNITY_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d): inner=%llu rows=%llu pitch=%llu", (int)r,
@@ -251,7 +255,9 @@ int forward_sweep(unity_ctx* ctx, const unity_rows* r, RowPlan& P) {
         // or CTA pairs): gm bounds the hidden rows that must stay L2 resident (a quarter of the workers, about
         // 4.7 k rows), splits fill the machine.
         const int n_pairs = ctx->sm_count / ctas;
-        const int gmax = n_pairs / 4 > 0 ? n_pairs / 4 : 1;
+        int gmax = ctx->fwd_group > 0 ? ctx->fwd_group / ctas : n_pairs / 4;
+        if (gmax < 1) gmax = 1;
+        if (gmax > n_pairs) gmax = n_pairs;
         const int n_grp = (m_tiles + gmax - 1) / gmax;
         const int gm = (m_tiles + n_grp - 1) / n_grp;
         int splits = n_pairs / gm;
@@ -335,6 +341,11 @@ int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace
     c->ctas[UNITY_PROF_GRAD_GEMM] = 2;
     c->ctas[UNITY_PROF_DH_GEMM] = 2;
     c->ctas[UNITY_PROF_DW_GEMM] = 2;
+    c->l2_promotion = 3;
+    c->chunk_group = 24;
+    c->fwd_group = 0;
+    c->chunk_rows_mult = 1;
+    c->chunk_vocab_mult = 1;
     c->ev_pool = new (std::nothrow) std::vector<cudaEvent_t>();
     c->ev_class = new (std::nothrow) std::vector<int>();
     if (cudaMalloc(&c->d_status, 256) != cudaSuccess || cudaMallocHost(&c->h_pinned, 4096) != cudaSuccess ||
@@ -398,7 +409,12 @@ int unity_set_option(unity_ctx* ctx, int option, int value) {
         ctx->ctas[option - UNITY_OPT_CTAS_FWD] = value;
         return UNITY_OK;
     }
-    return fail(ctx, UNITY_ERR_INVALID_ARG, "unknown option %d", option);
+    if (option == UNITY_OPT_L2_PROMOTION && value >= 0 && value <= 3) { ctx->l2_promotion = value; return UNITY_OK; }
+    if (option == UNITY_OPT_CHUNK_GROUP && value >= 2 && value <= 148) { ctx->chunk_group = value; return UNITY_OK; }
+    if (option == UNITY_OPT_FWD_GROUP && value >= 0 && value <= 148) { ctx->fwd_group = value; return UNITY_OK; }
+    if (option == UNITY_OPT_CHUNK_ROWS && value >= 1 && value <= 8) { ctx->chunk_rows_mult = value; return UNITY_OK; }
+    if (option == UNITY_OPT_CHUNK_VOCAB && value >= 1 && value <= 8) { ctx->chunk_vocab_mult = value; return UNITY_OK; }
+    return fail(ctx, UNITY_ERR_INVALID_ARG, "unknown option %d or value %d out of range", option, value);
 }
 
 int unity_set_profiling(unity_ctx* ctx, int enable) {
@@ -563,7 +579,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
     cudaStream_t st = ctx->stream;
 
     // choose gradient chunk sizes that fit the workspace
-    int cr = wanted_chunk_rows(rows->n_tok, K), cv = wanted_chunk_vocab(V);
+    int cr = wanted_chunk_rows(rows->n_tok, K, ctx->chunk_rows_mult), cv = wanted_chunk_vocab(V, ctx->chunk_vocab_mult);
     RowPlan P;
     bool fits = false;
     while (true) {
@@ -638,7 +654,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 GemmArgs g;
                 memset(&g, 0, sizeof(g));
                 g.m_tiles = nc / gemm_tile_rows(c_grad); g.n_tiles = (vc + kTileN - 1) / kTileN; g.k_iters = H / kTileK;
-                g.group_m = 16 / c_grad;
+                g.group_m = ctx->chunk_group / c_grad > 0 ? ctx->chunk_group / c_grad : 1;
                 g.a_row0 = slot0; g.b_row0 = v0; g.m_rows = nc; g.n_cols = vc;
                 g.target_p = L.target_p; g.vocab0 = v0; g.scale = rows->inv_temperature;
                 g.coef_a = L.coef_a; g.coef_b = L.coef_b; g.row_lse = L.row_lse; g.row_ent = L.row_ent;
@@ -655,7 +671,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 GemmArgs h;
                 memset(&h, 0, sizeof(h));
                 h.m_tiles = nc / gemm_tile_rows(c_dh); h.n_tiles = h_tiles; h.k_iters = (vc + kTileK - 1) / kTileK;
-                h.group_m = 16 / c_dh;
+                h.group_m = ctx->chunk_group / c_dh > 0 ? ctx->chunk_group / c_dh : 1;
                 h.a_row0 = 0; h.a_k0 = 0; h.b_row0 = 0; h.b_k0 = v0; h.m_rows = nc; h.n_cols = H;
                 h.C = L.dHc; h.ldc = H; h.beta = v0 > 0; h.status = ctx->d_status;
                 {
@@ -666,7 +682,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 GemmArgs w;
                 memset(&w, 0, sizeof(w));
                 w.m_tiles = (vc + gemm_tile_rows(c_dw) - 1) / gemm_tile_rows(c_dw); w.n_tiles = h_tiles; w.k_iters = nc / kTileK;
-                w.group_m = 16 / c_dw;
+                w.group_m = ctx->chunk_group / c_dw > 0 ? ctx->chunk_group / c_dw : 1;
                 w.a_row0 = 0; w.a_k0 = 0; w.b_row0 = 0; w.b_k0 = slot0; w.m_rows = vc; w.n_cols = H;
                 w.C = dWk + static_cast<long long>(v0) * H; w.ldc = H;
                 w.beta = (params->accumulate_dW || c0 > 0) ? 1 : 0; w.status = ctx->d_status;
