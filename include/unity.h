@@ -249,6 +249,13 @@ typedef struct {
     float ent_coef;
     const float* norm;      /* (host) f32 [K] or NULL */
     int accumulate_dW;      /* 0: overwrite dW, 1: add to it */
+    /* On-policy shortcut (all three or none; device f32 [n_tok]): logp, entropy and lse that unity_logprob_fwd
+     * returned for THESE weights on THESE rows - e.g. the "old log probabilities" pass of the first PPO epoch, when
+     * the current policy still equals the old one.  The forward sweep over the vocabulary is then skipped (2*H*V of
+     * the 8*H*V flop per token); the backward still recomputes the logits per chunk.  NULL: full computation. */
+    const float* logp_in;
+    const float* entropy_in;
+    const float* lse_in;
 } unity_ppo_params;
 
 int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_ppo_params* params,

@@ -53,7 +53,8 @@ class unity_rows(C.Structure):
 
 class unity_ppo_params(C.Structure):
     _fields_ = [("clip_lo", C.c_float), ("clip_hi", C.c_float), ("kl_coef", C.c_float), ("kl_mode", C.c_int),
-                ("ent_coef", C.c_float), ("norm", C.POINTER(C.c_float)), ("accumulate_dW", C.c_int)]
+                ("ent_coef", C.c_float), ("norm", C.POINTER(C.c_float)), ("accumulate_dW", C.c_int),
+                ("logp_in", C.c_void_p), ("entropy_in", C.c_void_p), ("lse_in", C.c_void_p)]
 
 
 _LIB = None
@@ -289,13 +290,15 @@ def unity_logprob_fwd(ctx, hidden, W, cu_seqlens, inv_role, role_model, target, 
 def unity_ppo_loss_fwd_bwd(ctx, hidden, W, cu_seqlens, inv_role, role_model, target, tok_mask, inv_temperature,
                            clip_lo, clip_hi, kl_coef, kl_mode, ent_coef, norm: Optional[Sequence[float]],
                            accumulate_dW: bool, old_logp, ref_logp, adv_tok, loss, metrics, logp, entropy,
-                           tok_loss, dHidden, dW) -> None:
+                           tok_loss, dHidden, dW, logp_in=None, entropy_in=None, lse_in=None) -> None:
     keep = []
     rows = _make_rows(hidden, W, cu_seqlens, inv_role, role_model, target, tok_mask, inv_temperature, keep)
     norm_arr = None
     if norm is not None:
         norm_arr = (C.c_float * len(norm))(*[float(x) for x in norm])
-    p = unity_ppo_params(clip_lo, clip_hi, kl_coef, kl_mode, ent_coef, norm_arr, 1 if accumulate_dW else 0)
+    f32_ = torch.float32
+    p = unity_ppo_params(clip_lo, clip_hi, kl_coef, kl_mode, ent_coef, norm_arr, 1 if accumulate_dW else 0,
+                         _ptr(logp_in, f32_, "logp_in"), _ptr(entropy_in, f32_, "entropy_in"), _ptr(lse_in, f32_, "lse_in"))
     dWp = (C.c_void_p * len(dW))(*[_ptr(g, torch.float32, "dW") for g in dW])
     f32 = torch.float32
     code = load_library().unity_ppo_loss_fwd_bwd(

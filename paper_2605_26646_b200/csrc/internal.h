@@ -127,6 +127,7 @@ struct TokenArgs {
     // forward outputs (packed and caller order)
     float *row_lse, *row_ent, *row_logp;      // packed [n_slots]
     float *logp, *entropy, *lse;              // caller order [n_tok], nullable
+    const float *logp_in, *entropy_in, *lse_in;   // caller order [n_tok]: results of an earlier forward (or all null)
     // loss part (null for logprob_fwd)
     const float *old_logp, *ref_logp, *adv_tok;
     float clip_lo, clip_hi, kl_coef, ent_coef;

@@ -330,23 +330,29 @@ __global__ void k_finish_rows(TokenArgs a, int with_loss) {
         return;
     }
     const int k = a.tok_model[tok];
-    const long long pitch = a.offsets[k + 1] - a.offsets[k];
-    const float4* st = a.stats + a.stats_base[k] + (slot - a.offsets[k]);
-    const int n_splits = a.model_splits[k];
-    const float c = a.scale * 1.4426950408889634f;    // exp(scale*x) = exp2(c*x)
-    float m = -3.0e38f;
-    for (int j = 0; j < n_splits; ++j) m = fmaxf(m, st[j * pitch].x);
-    float s = 0.f, t = 0.f, zy = -3.0e38f;
-    for (int j = 0; j < n_splits; ++j) {
-        const float4 p = st[j * pitch];
-        const float w = exp2f((p.x - m) * c);
-        s += p.y * w;
-        t += p.z * w;
-        zy = fmaxf(zy, p.w);
+    float lse, ent, logp;
+    if (a.lse_in) {
+        // the caller already evaluated this policy on these rows (unity_logprob_fwd): no forward sweep was run
+        lse = a.lse_in[tok]; ent = a.entropy_in[tok]; logp = a.logp_in[tok];
+    } else {
+        const long long pitch = a.offsets[k + 1] - a.offsets[k];
+        const float4* st = a.stats + a.stats_base[k] + (slot - a.offsets[k]);
+        const int n_splits = a.model_splits[k];
+        const float c = a.scale * 1.4426950408889634f;    // exp(scale*x) = exp2(c*x)
+        float m = -3.0e38f;
+        for (int j = 0; j < n_splits; ++j) m = fmaxf(m, st[j * pitch].x);
+        float s = 0.f, t = 0.f, zy = -3.0e38f;
+        for (int j = 0; j < n_splits; ++j) {
+            const float4 p = st[j * pitch];
+            const float w = exp2f((p.x - m) * c);
+            s += p.y * w;
+            t += p.z * w;
+            zy = fmaxf(zy, p.w);
+        }
+        lse = a.scale * m + logf(s);
+        ent = lse - a.scale * (t / s);
+        logp = a.scale * zy - lse;
     }
-    const float lse = a.scale * m + logf(s);
-    const float ent = lse - a.scale * (t / s);
-    const float logp = a.scale * zy - lse;
     a.row_lse[slot] = lse; a.row_ent[slot] = ent; a.row_logp[slot] = logp;
     if (a.logp) a.logp[tok] = logp;
     if (a.entropy) a.entropy[tok] = ent;

@@ -208,7 +208,7 @@ struct RowPlan {
 };
 
 // Routing, packing and the forward sweep: fills per-split softmax statistics for every packed row.
-int forward_sweep(unity_ctx* ctx, const unity_rows* r, RowPlan& P) {
+int forward_sweep(unity_ctx* ctx, const unity_rows* r, RowPlan& P, bool run_gemm = true) {
     const Layout& L = P.L;
     cudaStream_t st = ctx->stream;
     int nl = 0;
@@ -249,7 +249,7 @@ int forward_sweep(unity_ctx* ctx, const unity_rows* r, RowPlan& P) {
         P.splits[k] = 1;
         P.stats_base[k] = sbase;
         const int rows_k = P.offsets[k + 1] - P.offsets[k];
-        if (rows_k == 0) continue;
+        if (rows_k == 0 || !run_gemm) continue;
         const int m_tiles = rows_k / tile_rows;
         // One round of the persistent kernel = gm row tiles x splits vocabulary splits <= number of workers (CTAs
         // or CTA pairs): gm bounds the hidden rows that must stay L2 resident (a quarter of the workers, about
@@ -603,13 +603,19 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
     if (entropy) CUDA_TRY(ctx, cudaMemsetAsync(entropy, 0, sizeof(float) * rows->n_tok, st));
     if (tok_loss) CUDA_TRY(ctx, cudaMemsetAsync(tok_loss, 0, sizeof(float) * rows->n_tok, st));
 
-    rc = forward_sweep(ctx, rows, P);
+    // On-policy shortcut: when the caller hands in logp / entropy / lse of THESE weights on THESE rows (from
+    // unity_logprob_fwd), the forward sweep over the vocabulary is skipped; the backward still recomputes the logits.
+    const bool have_fwd = params->logp_in && params->entropy_in && params->lse_in;
+    if (!have_fwd && (params->logp_in || params->entropy_in || params->lse_in))
+        return fail(ctx, UNITY_ERR_INVALID_ARG, "logp_in, entropy_in and lse_in must be given together");
+    rc = forward_sweep(ctx, rows, P, !have_fwd);
     if (rc) return rc;
     int nl = 0;
 
     TokenArgs t;
     fill_token_args(t, rows, P);
     t.logp = logp; t.entropy = entropy; t.lse = nullptr;
+    if (have_fwd) { t.logp_in = params->logp_in; t.entropy_in = params->entropy_in; t.lse_in = params->lse_in; }
     t.old_logp = old_logp; t.ref_logp = ref_logp; t.adv_tok = adv_tok;
     t.clip_lo = params->clip_lo; t.clip_hi = params->clip_hi; t.kl_coef = params->kl_coef;
     t.ent_coef = params->ent_coef; t.kl_mode = params->kl_mode;

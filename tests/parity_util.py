@@ -84,7 +84,7 @@ def oracle_logprob(w: wl.Workload, rows=None):
 
 
 def gpu_ppo(ctx: ub.Context, w: wl.Workload, d: DeviceInputs, old, ref, adv, norm=None, accumulate=False, dW=None,
-            kl_mode=None, kl_coef=None, ent_coef=None, clip=None):
+            kl_mode=None, kl_coef=None, ent_coef=None, clip=None, fwd=None):
     K = w.K
     loss = torch.full((K,), 7.0, device="cuda")
     metrics = torch.full(((K + w.n_roles) * ub.UNITY_N_METRICS,), 7.0, device="cuda")
@@ -98,7 +98,8 @@ def gpu_ppo(ctx: ub.Context, w: wl.Workload, d: DeviceInputs, old, ref, adv, nor
     ctx.ppo_loss_fwd_bwd(d.hidden, d.W, d.cu_seqlens, d.inv_role, w.role_model.tolist(), d.target, d.tok_mask,
                          w.inv_temperature, lo, hi, w.kl_coef if kl_coef is None else kl_coef,
                          w.kl_mode if kl_mode is None else kl_mode, w.ent_coef if ent_coef is None else ent_coef,
-                         norm, accumulate, old, ref, adv, loss, metrics, logp, ent, tok_loss, dH, dW)
+                         norm, accumulate, old, ref, adv, loss, metrics, logp, ent, tok_loss, dH, dW,
+                         **({} if fwd is None else dict(logp_in=fwd["logp"], entropy_in=fwd["entropy"], lse_in=fwd["lse"])))
     ctx.check_status()
     return dict(loss=loss, metrics=metrics.view(K + w.n_roles, ub.UNITY_N_METRICS), logp=logp, entropy=ent,
                 tok_loss=tok_loss, dHidden=dH, dW=dW)

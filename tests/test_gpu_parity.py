@@ -236,6 +236,32 @@ def test_kl_modes_entropy_bonus_and_temperature(kl_mode, ent_coef, clip):
     run_all_stages(w, kl_mode=kl_mode, kl_coef=0.1, ent_coef=ent_coef, clip=clip)
 
 
+def test_on_policy_shortcut_reuses_an_earlier_forward():
+    # logp / entropy / lse from unity_logprob_fwd on the same weights replace the forward sweep of the loss call
+    w = small_workload(256, 3000, 500)
+    d = pu.DeviceInputs(w)
+    ctx = pu.make_ctx(w)
+    fwd = pu.gpu_logprob(ctx, w, d)
+    old = fwd["logp"] + w.noise_old.cuda()
+    ref = fwd["logp"] + w.noise_ref.cuda()
+    adv = wl.normal(9, 3, w.n_tok).cuda()
+    full = pu.gpu_ppo(ctx, w, d, old, ref, adv, ent_coef=0.01)
+    launches = ctx.launch_count
+    short = pu.gpu_ppo(ctx, w, d, old, ref, adv, ent_coef=0.01, fwd=fwd)
+    assert ctx.launch_count - launches < launches                         # fewer kernels: no forward GEMM
+    for key in ("loss", "logp", "entropy", "tok_loss", "dHidden"):
+        assert torch.equal(short[key], full[key]), key                    # same statistics in, same bits out
+    assert all(torch.equal(a, b) for a, b in zip(short["dW"], full["dW"]))
+    op = pu.oracle_ppo(w, old.cpu().numpy(), ref.cpu().numpy(), adv.cpu().numpy(), ent_coef=0.01)
+    check_ppo(short, op, w)
+    with pytest.raises(ub.UnityError) as e:                               # all three or none
+        ctx.ppo_loss_fwd_bwd(d.hidden, d.W, d.cu_seqlens, d.inv_role, w.role_model.tolist(), d.target, d.tok_mask, 1.0,
+                             0.2, 0.2, 0.0, 3, 0.0, None, False, old, ref, adv, full["loss"], None, None, None, None,
+                             full["dHidden"], full["dW"], logp_in=fwd["logp"])
+    assert e.value.code == -1
+    ctx.close()
+
+
 def test_model_without_rows_and_three_models():
     # roles map to models 0 and 1; model 2 is never used: its dW must come back as zeros
     run_all_stages(small_workload(128, 1024, 300, role_model=[0, 1, 0], K=3))
