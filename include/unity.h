@@ -80,7 +80,7 @@ int unity_set_profiling(unity_ctx* ctx, int enable);
 
 /* Tuning knobs (no counterpart in the paper).  Each GEMM class can run with one CTA per 128 x 256 output tile
  * (value 1) or with a pair of CTAs on neighbouring SMs sharing a 256 x 256 tile (value 2).  Results do not depend
- * on the choice beyond fp32 summation order inside the tensor core.  Defaults: 1, 2, 2, 2 (measured best on
+ * on the choice beyond fp32 summation order inside the tensor core.  Defaults: 2, 2, 2, 2 (measured best on
  * the H=3584, V=152064 workload; all choices are within a few per cent under the 1 kW power cap). */
 #define UNITY_OPT_CTAS_FWD 0
 #define UNITY_OPT_CTAS_GRAD 1
@@ -91,6 +91,8 @@ int unity_set_profiling(unity_ctx* ctx, int enable);
 #define UNITY_OPT_CHUNK_ROWS 6    /* gradient chunk rows = value x 18944 (default 1; larger needs a larger workspace)   */
 #define UNITY_OPT_CHUNK_VOCAB 7   /* gradient chunk vocabulary entries = value x 18944 (default 1)                      */
 #define UNITY_OPT_FWD_GROUP 8     /* 128-row tiles per round of the forward kernel (default 0 = a quarter of the SMs)   */
+#define UNITY_OPT_FWD_SYNC 9      /* 1 (default): workers of the forward kernel meet at each round start (bounded wait) */
+#define UNITY_OPT_CHUNK_SYNC 10   /* same for the gradient-chunk GEMMs: bit 0 recompute, bit 1 dHidden, bit 2 dW (default 0) */
 int unity_set_option(unity_ctx* ctx, int option, int value);
 int unity_get_profile(unity_ctx* ctx, double* ms, int64_t* launches);
 

@@ -147,6 +147,23 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                 Unit t;
                 bool valid;
                 if (!next_unit<EPI>(g, it, pair, n_pairs, gm, t, valid)) break;
+                if (g.round_counter != nullptr && cta_rank == 0) {
+                    // Soft rendezvous at the start of every round: the workers that share a stream of W tiles stay in
+                    // step only while they start together, and once they drift apart by more than L2 can bridge each
+                    // of them fetches the stream from HBM again.  Purely a performance hint: after a short, bounded
+                    // wait the worker goes on regardless (some CTAs may not be resident yet).
+                    // The counter only ever grows; round_base is its value before this launch (every worker adds one
+                    // per round whether or not it waited, so the host can keep the running total).
+                    atomicAdd(g.round_counter, 1u);
+                    // arrivals expected by the end of this round: every worker (softmax), or every worker that still has
+                    // a tile (the last round of the other epilogues may be partial)
+                    unsigned expect = static_cast<unsigned>(it + 1) * static_cast<unsigned>(n_pairs);
+                    if (EPI != kEpiSoftmaxStats) expect = min(expect, static_cast<unsigned>(g.m_tiles * g.n_tiles));
+                    const unsigned target = g.round_base + expect;
+                    const long long t0 = clock64();
+                    while (static_cast<int>(*reinterpret_cast<volatile unsigned*>(g.round_counter) - target) < 0 &&
+                           clock64() - t0 < 400000) { }
+                }
                 if (!valid) continue;
                 const int a_row = g.a_row0 + t.m_tile * C::kTileRows + static_cast<int>(cta_rank) * kCtaM;
                 for (int nt = t.n_begin; nt < t.n_end && ok; ++nt) {
@@ -414,6 +431,34 @@ cudaError_t gemm_set_attributes() {
 }
 
 int gemm_tile_rows(int ctas) { return kCtaM * ctas; }
+
+namespace {
+// workers and rounds of a launch (must mirror next_unit and launch_gemm)
+void launch_shape(GemmEpilogue epi, int ctas, const GemmArgs& args, int sm_count, int* workers, long long* rounds) {
+    const long long gm = args.group_m < args.m_tiles ? args.group_m : args.m_tiles;
+    const long long units = epi == kEpiSoftmaxStats ? (gm < 1 ? 1 : gm) * args.n_splits
+                                                    : static_cast<long long>(args.m_tiles) * args.n_tiles;
+    const int max_workers = sm_count / ctas;
+    *workers = static_cast<int>(units < max_workers ? units : max_workers);
+    if (units <= 0 || args.m_tiles <= 0 || args.k_iters <= 0) { *workers = 0; *rounds = 0; return; }
+    if (epi == kEpiSoftmaxStats) {
+        const long long g1 = args.group_m < 1 ? 1 : args.group_m;
+        *rounds = (args.m_tiles + g1 - 1) / g1;
+    } else {
+        *rounds = (units + *workers - 1) / *workers;   // workers with a shorter loop stop arriving: see below
+    }
+}
+}  // namespace
+
+unsigned gemm_round_arrivals(GemmEpilogue epi, int ctas, const GemmArgs& args, int sm_count) {
+    int workers; long long rounds;
+    launch_shape(epi, ctas, args, sm_count, &workers, &rounds);
+    if (workers == 0) return 0;
+    if (epi == kEpiSoftmaxStats) return static_cast<unsigned>(rounds * workers);
+    // striding over units: worker p runs ceil((units - p) / workers) rounds
+    const long long units = static_cast<long long>(args.m_tiles) * args.n_tiles;
+    return static_cast<unsigned>(units);
+}
 
 cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, int ctas, const CUtensorMap& tmA, const CUtensorMap& tmB,
                         const GemmArgs& args, int sm_count, cudaStream_t stream) {

@@ -41,6 +41,8 @@ struct GemmArgs {
     int m_rows, n_cols;       // valid extent of C from (a_row0, b_row0): epilogue writes nothing beyond it
     // kEpiSoftmaxStats: a unit is (row tile, vocabulary split); a CTA keeps a unit's running statistics
     int n_splits, tiles_per_split;
+    unsigned* round_counter;  // ever-growing arrival counter (null = no rendezvous between rounds)
+    unsigned round_base;      // its value before this launch
     float4* stats;            // [n_splits][stats_pitch], row relative to a_row0: (max acc, sum e, sum e*acc, target acc)
     long long stats_pitch;
     const int* target_p;      // [rows] packed targets (global vocabulary index), indexed from a_row0 + row
@@ -66,6 +68,8 @@ struct GemmArgs {
 // gemm_tile_rows(ctas) rows.
 cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, int ctas, const CUtensorMap& tmA, const CUtensorMap& tmB,
                         const GemmArgs& args, int sm_count, cudaStream_t stream);
+// Arrivals the launch adds to args.round_counter (rounds x workers); 0 when nothing is launched.
+unsigned gemm_round_arrivals(GemmEpilogue epi, int ctas, const GemmArgs& args, int sm_count);
 int gemm_tile_rows(int ctas);
 cudaError_t gemm_set_attributes();
 

@@ -35,6 +35,9 @@ struct unity_ctx {
     int chunk_group;                // raster group of the chunk GEMMs, in 128-row tiles
     int chunk_rows_mult, chunk_vocab_mult;   // gradient chunk = mult x 18944 rows / vocabulary entries
     int fwd_group;                  // row tiles (128 rows) per round of the forward kernel; 0 = a quarter of the SMs
+    int fwd_sync;                   // 1: workers of the forward kernel meet (softly) at every round start
+    int chunk_sync;                 // bit 0: same for the recompute GEMM, bit 1: dHidden GEMM, bit 2: dW GEMM
+    unsigned round_total;           // arrivals accumulated so far on the rendezvous counter (d_status + 16)
 };
 
 namespace {
@@ -283,6 +286,11 @@ int forward_sweep(unity_ctx* ctx, const unity_rows* r, RowPlan& P, bool run_gemm
         g.stats = L.stats + P.stats_base[k]; g.stats_pitch = rows_k;
         g.target_p = L.target_p; g.vocab0 = 0; g.scale = r->inv_temperature;
         g.status = ctx->d_status;
+        if (ctx->fwd_sync) {
+            g.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
+            g.round_base = ctx->round_total;
+            ctx->round_total += gemm_round_arrivals(kEpiSoftmaxStats, ctas, g, ctx->sm_count);
+        }
         {
             ProfScope ps(ctx, UNITY_PROF_FWD_GEMM);
             CUDA_TRY(ctx, launch_gemm(kEpiSoftmaxStats, false, ctas, tmA, tmB, g, ctx->sm_count, st));
@@ -337,13 +345,15 @@ int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace
         return UNITY_ERR_CUDA;
     }
     c->encode = reinterpret_cast<EncodeTiledFn>(fn);
-    c->ctas[UNITY_PROF_FWD_GEMM] = 1;
+    c->ctas[UNITY_PROF_FWD_GEMM] = 2;
     c->ctas[UNITY_PROF_GRAD_GEMM] = 2;
     c->ctas[UNITY_PROF_DH_GEMM] = 2;
     c->ctas[UNITY_PROF_DW_GEMM] = 2;
     c->l2_promotion = 3;
     c->chunk_group = 24;
     c->fwd_group = 0;
+    c->fwd_sync = 1;
+    c->chunk_sync = 0;
     c->chunk_rows_mult = 1;
     c->chunk_vocab_mult = 1;
     c->ev_pool = new (std::nothrow) std::vector<cudaEvent_t>();
@@ -411,6 +421,8 @@ int unity_set_option(unity_ctx* ctx, int option, int value) {
     }
     if (option == UNITY_OPT_L2_PROMOTION && value >= 0 && value <= 3) { ctx->l2_promotion = value; return UNITY_OK; }
     if (option == UNITY_OPT_CHUNK_GROUP && value >= 2 && value <= 148) { ctx->chunk_group = value; return UNITY_OK; }
+    if (option == UNITY_OPT_FWD_SYNC && (value == 0 || value == 1)) { ctx->fwd_sync = value; return UNITY_OK; }
+    if (option == UNITY_OPT_CHUNK_SYNC && value >= 0 && value <= 7) { ctx->chunk_sync = value; return UNITY_OK; }
     if (option == UNITY_OPT_FWD_GROUP && value >= 0 && value <= 148) { ctx->fwd_group = value; return UNITY_OK; }
     if (option == UNITY_OPT_CHUNK_ROWS && value >= 1 && value <= 8) { ctx->chunk_rows_mult = value; return UNITY_OK; }
     if (option == UNITY_OPT_CHUNK_VOCAB && value >= 1 && value <= 8) { ctx->chunk_vocab_mult = value; return UNITY_OK; }
@@ -665,6 +677,11 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 g.target_p = L.target_p; g.vocab0 = v0; g.scale = rows->inv_temperature;
                 g.coef_a = L.coef_a; g.coef_b = L.coef_b; g.row_lse = L.row_lse; g.row_ent = L.row_ent;
                 g.G = L.G; g.ldg = cv; g.status = ctx->d_status;
+                if (ctx->chunk_sync & 1) {
+                    g.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
+                    g.round_base = ctx->round_total;
+                    ctx->round_total += gemm_round_arrivals(kEpiLogitGrad, c_grad, g, ctx->sm_count);
+                }
                 {
                     ProfScope ps(ctx, UNITY_PROF_GRAD_GEMM);
                     CUDA_TRY(ctx, launch_gemm(kEpiLogitGrad, false, c_grad, tm_hp_k, tm_W_k, g, ctx->sm_count, st));
@@ -680,6 +697,11 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 h.group_m = ctx->chunk_group / c_dh > 0 ? ctx->chunk_group / c_dh : 1;
                 h.a_row0 = 0; h.a_k0 = 0; h.b_row0 = 0; h.b_k0 = v0; h.m_rows = nc; h.n_cols = H;
                 h.C = L.dHc; h.ldc = H; h.beta = v0 > 0; h.status = ctx->d_status;
+                if (ctx->chunk_sync & 2) {
+                    h.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
+                    h.round_base = ctx->round_total;
+                    ctx->round_total += gemm_round_arrivals(kEpiAccumF32, c_dh, h, ctx->sm_count);
+                }
                 {
                     ProfScope ps(ctx, UNITY_PROF_DH_GEMM);
                     CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, false, c_dh, tm_G_k, tm_W_mn, h, ctx->sm_count, st));
@@ -692,6 +714,11 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 w.a_row0 = 0; w.a_k0 = 0; w.b_row0 = 0; w.b_k0 = slot0; w.m_rows = vc; w.n_cols = H;
                 w.C = dWk + static_cast<long long>(v0) * H; w.ldc = H;
                 w.beta = (params->accumulate_dW || c0 > 0) ? 1 : 0; w.status = ctx->d_status;
+                if (ctx->chunk_sync & 4) {
+                    w.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
+                    w.round_base = ctx->round_total;
+                    ctx->round_total += gemm_round_arrivals(kEpiAccumF32, c_dw, w, ctx->sm_count);
+                }
                 {
                     ProfScope ps(ctx, UNITY_PROF_DW_GEMM);
                     CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, true, c_dw, tm_G_mn, tm_hp_mn, w, ctx->sm_count, st));
