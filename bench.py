@@ -32,8 +32,8 @@ UNIT = "tokens/s"
 # (valid rows x vocabulary columns).  Traffic grows in proportion to the logits covered (same chunk and group sizes),
 # so a full-size launch is estimated as bytes_per_logit x its logits.  Valid only for the kernel source it was taken
 # from: when the hash of gemm_tcgen05.cu differs, the benchmark reports null.
-NCU_TRAFFIC = {"source_sha256_16": "2aa4a0f7d9de35b6",
-               "bytes_per_logit": {"fwd_gemm": 1.863, "grad_gemm": 4.734, "dh_gemm": 9.906, "dw_gemm": 9.956}}
+NCU_TRAFFIC = {"source_sha256_16": "6bea9a7ad9088210",
+               "bytes_per_logit": {"fwd_gemm": 2.309, "grad_gemm": 5.054, "dh_gemm": 9.674, "dw_gemm": 9.656}}
 
 
 def ncu_traffic_per_launch(cls: str, logits_per_launch: float):

@@ -92,7 +92,7 @@ int unity_set_profiling(unity_ctx* ctx, int enable);
 #define UNITY_OPT_CHUNK_VOCAB 7   /* gradient chunk vocabulary entries = value x 18944 (default 1)                      */
 #define UNITY_OPT_FWD_GROUP 8     /* 128-row tiles per round of the forward kernel (default 0 = a quarter of the SMs)   */
 #define UNITY_OPT_FWD_SYNC 9      /* 1 (default): workers of the forward kernel meet at each round start (bounded wait) */
-#define UNITY_OPT_CHUNK_SYNC 10   /* same for the gradient-chunk GEMMs: bit 0 recompute, bit 1 dHidden, bit 2 dW (default 0) */
+#define UNITY_OPT_CHUNK_SYNC 10   /* same for the gradient-chunk GEMMs: bit 0 recompute, bit 1 dHidden, bit 2 dW (default 6) */
 int unity_set_option(unity_ctx* ctx, int option, int value);
 int unity_get_profile(unity_ctx* ctx, double* ms, int64_t* launches);
 

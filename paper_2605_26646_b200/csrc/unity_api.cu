@@ -353,7 +353,7 @@ int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace
     c->chunk_group = 24;
     c->fwd_group = 0;
     c->fwd_sync = 1;
-    c->chunk_sync = 0;
+    c->chunk_sync = 6;
     c->chunk_rows_mult = 1;
     c->chunk_vocab_mult = 1;
     c->ev_pool = new (std::nothrow) std::vector<cudaEvent_t>();
