@@ -154,8 +154,13 @@ int wanted_chunk_rows(long long n_tok, int K, int mult = 1) {
     const long long ms = max_slots_of(n_tok, K), want = static_cast<long long>(kChunkRows) * mult;
     return static_cast<int>(ms < want ? ms : want);
 }
+// Columns of the G scratch: a full chunk plus head-room of kTailTiles tiles, so that a short remainder of the
+// vocabulary (V = 152064 is 8 chunks of 18944 plus 512) is absorbed by the last chunk instead of running as a
+// chunk of its own, whose GEMMs would be all epilogue.
+constexpr int kTailTiles = 8;
 int wanted_chunk_vocab(int V, int mult = 1) {
-    const long long vp = static_cast<long long>(up(V, kTileN)), want = static_cast<long long>(kChunkVocab) * mult;
+    const long long vp = static_cast<long long>(up(V, kTileN));
+    const long long want = static_cast<long long>(kChunkVocab) * mult + kTailTiles * kTileN;
     return static_cast<int>(vp < want ? vp : want);
 }
 
@@ -666,8 +671,11 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
         for (int c0 = 0; c0 < rows_k; c0 += cr) {
             const int nc = rows_k - c0 < cr ? rows_k - c0 : cr;          // multiple of kTileM
             const int slot0 = P.offsets[k] + c0;
-            for (int v0 = 0; v0 < V; v0 += cv) {
-                const int vc = V - v0 < cv ? V - v0 : cv;
+            const int tail = kTailTiles * kTileN;
+            const int base = (V > cv && cv > tail + kTileN) ? cv - tail : cv;      // regular chunk width
+            for (int v0 = 0, vc = 0; v0 < V; v0 += vc) {
+                vc = V - v0 < base ? V - v0 : base;
+                if (V - (v0 + vc) <= tail && base < cv) vc = V - v0;               // absorb a short remainder
                 // (1) recompute the logits of this (rows x vocab) chunk and form dL/dz in bf16: G[nc, vc]
                 GemmArgs g;
                 memset(&g, 0, sizeof(g));
