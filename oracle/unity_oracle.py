@@ -360,3 +360,172 @@ def gae(rewards, values, cu_seqlens, gamma, lam, tok_mask=None):
         for t in range(T):
             A[idx[t]] = (powers[:T - t] * delta[t:]).sum()   # the sum over l written out for this t
     return A, np.where(keep, A + v, 0.0)
+
+
+# ----------------------------------------------------------------------------------------------
+# critic side of the update: clipped value loss (paragraph "Model-specific updates and synchronization":
+# each worker group updates its own actor AND critic; "value estimates, returns" are the quantities the
+# paragraph "Advantage computation and policy evaluation" lists for it)
+# ----------------------------------------------------------------------------------------------
+
+def value_loss_fwd_bwd(values, old_values, returns, cu_seqlens, inv_role, role_model, tok_mask=None,
+                       clip_v=0.2, norm=None, K=None):
+    """PPO's clipped value regression, token-mean per model, and its gradient w.r.t. the value estimates.
+
+    v_clip = old_v + clip(v - old_v, -clip_v, +clip_v);  l = 0.5 * max((v - R)^2, (v_clip - R)^2);
+    L_k = (1/M_k) sum over valid tokens of model k of l, M_k = norm[k] if given else max(#valid tokens, 1).
+    The paper prints no value loss; this is the reading fixed for the critic update.  Where the two squares are
+    equal (in particular whenever v is inside the clip range, where v_clip = v) the unclipped branch is taken, so
+    dl/dv = v - R there and 0 where the clipped square is strictly larger (v_clip does not depend on v then).
+    Returns dict(loss[K], M[K], tok_loss[N], dvalues[N], clip_frac[K])."""
+    v = to_f64(values)
+    ov = to_f64(old_values)
+    R = to_f64(returns)
+    n_tok = v.shape[0]
+    if K is None:
+        K = int(np.max(np.asarray(role_model))) + 1 if norm is None else len(norm)
+    _, tok_model = token_role_model(cu_seqlens, inv_role, role_model)
+    mask = np.ones(n_tok, bool) if tok_mask is None else (np.asarray(tok_mask) != 0)
+    d = v - ov
+    # inside the range v_clip IS v (written so, not as ov + (v - ov), which rounds); outside it is the range's end
+    v_clip = np.where(np.abs(d) <= clip_v, v, ov + np.sign(d) * clip_v)
+    sq_u = (v - R) ** 2
+    sq_c = (v_clip - R) ** 2
+    unclipped = sq_u >= sq_c
+    tok = 0.5 * np.where(unclipped, sq_u, sq_c)
+    loss = np.zeros(K, F64)
+    M = np.zeros(K, F64)
+    clip_frac = np.zeros(K, F64)
+    dv = np.zeros(n_tok, F64)
+    for k in range(K):
+        sel = mask & (tok_model == k)
+        cnt = float(sel.sum())
+        M[k] = float(norm[k]) if norm is not None else max(cnt, 1.0)
+        loss[k] = tok[sel].sum() / M[k]
+        clip_frac[k] = (~unclipped[sel]).sum() / max(cnt, 1.0)
+        dv[sel] = np.where(unclipped[sel], v[sel] - R[sel], 0.0) / M[k]
+    return dict(loss=loss, M=M, tok_loss=np.where(mask, tok, 0.0), dvalues=dv, clip_frac=clip_frac)
+
+
+# ----------------------------------------------------------------------------------------------
+# ready-batch construction (Section "Model-Local Buffers": B_i -> D_i^ready may include filtering incomplete
+# trajectories, aligning delayed rewards with token sequences, padding, shuffling and matching the data-parallel
+# configuration of the worker group; batches are built per model instance)
+# ----------------------------------------------------------------------------------------------
+
+_M32 = 0xFFFFFFFF
+
+
+def fmix32(h: int) -> int:
+    """The 32-bit finaliser of MurmurHash3 (public domain, A. Appleby): xor-shift 16, multiply 0x85ebca6b,
+    xor-shift 13, multiply 0xc2b2ae35, xor-shift 16."""
+    h &= _M32
+    h ^= h >> 16
+    h = (h * 0x85EBCA6B) & _M32
+    h ^= h >> 13
+    h = (h * 0xC2B2AE35) & _M32
+    h ^= h >> 16
+    return h
+
+
+def seeded_permutation(n: int, seed: int):
+    """perm[p] for p in [0, n): a seeded bijection of [0, n) built as a 4-round balanced Feistel network on the
+    smallest even-width bit domain that holds n, with cycle walking for values that fall outside [0, n)
+    (Black and Rogaway's construction of ciphers on arbitrary finite domains).  Round keys: key_i =
+    fmix32(seed32 + 0x9E3779B9*(i+1)), seed32 = low word of seed xor high word; round function F(r, i) =
+    fmix32(r xor key_i) truncated to the half width."""
+    if n <= 0:
+        return np.zeros(0, np.int64)
+    bits = max(2, int(n - 1).bit_length())
+    bits += bits & 1
+    half = bits // 2
+    hmask = (1 << half) - 1
+    seed32 = (seed ^ (seed >> 32)) & _M32
+    keys = [fmix32((seed32 + 0x9E3779B9 * (i + 1)) & _M32) for i in range(4)]
+    out = np.zeros(n, np.int64)
+    for p in range(n):
+        x = p
+        while True:
+            left, right = x >> half, x & hmask
+            for i in range(4):
+                left, right = right, left ^ (fmix32(right ^ keys[i]) & hmask)
+            x = (left << half) | right
+            if x < n:
+                break
+        out[p] = x
+    return out
+
+
+def ready_batch_plan(cu_seqlens, inv_role, inv_traj, traj_done, role_model, K, seed, n_parts=1, pad_to=1):
+    """Which invocations of the buffer enter the ready batch, in what order, and where their tokens go.
+
+    Steps, in the paper's order: (1) filter - an invocation is kept when its trajectory is complete
+    (traj_done != 0) and its role maps to a model in [0, K); (2) shuffle - positions p = 0..n_inv-1 are visited
+    in order and position p holds buffer invocation seeded_permutation(n_inv, seed)[p]; (3) per model - kept
+    invocations are listed model by model (each model builds its own batch), in shuffled order inside a model;
+    (4) padding - each kept invocation occupies its length rounded up to a multiple of pad_to; (5) data-parallel
+    split - inside model k, with P_j the padded tokens before invocation j and T_k the model's padded total,
+    invocation j belongs to partition floor(P_j * n_parts / T_k): partitions are contiguous and equal in tokens
+    up to one invocation.
+
+    Returns dict(order[n_kept] buffer indices, out_cu[n_kept+1], model_offsets[K+1] (into order),
+    part_offsets[K*n_parts+1] (into order), n_kept, n_tok)."""
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    n_inv = cu.size - 1
+    perm = seeded_permutation(n_inv, seed)
+    role_model = np.asarray(role_model, dtype=np.int64)
+    per_model = [[] for _ in range(K)]
+    for p in range(n_inv):
+        s = int(perm[p])
+        role, traj = int(inv_role[s]), int(inv_traj[s])
+        if role < 0 or role >= role_model.size or traj < 0 or traj >= len(traj_done):
+            continue
+        k = int(role_model[role])
+        if k < 0 or k >= K or not traj_done[traj]:
+            continue
+        per_model[k].append(s)
+    order, out_cu, model_offsets, part_offsets = [], [0], [0], []
+    for k in range(K):
+        padded = [-(-int(cu[s + 1] - cu[s]) // pad_to) * pad_to for s in per_model[k]]
+        T = sum(padded)
+        P = 0
+        parts = []
+        for s, L in zip(per_model[k], padded):
+            parts.append(min(n_parts - 1, (P * n_parts) // T) if T > 0 else 0)
+            P += L
+            order.append(s)
+            out_cu.append(out_cu[-1] + L)
+        base = model_offsets[-1]
+        for q in range(n_parts):
+            part_offsets.append(base + sum(1 for x in parts if x < q))
+        model_offsets.append(base + len(per_model[k]))
+    part_offsets.append(model_offsets[-1])
+    return dict(order=np.asarray(order, np.int64), out_cu=np.asarray(out_cu, np.int64),
+                model_offsets=np.asarray(model_offsets, np.int64), part_offsets=np.asarray(part_offsets, np.int64),
+                n_kept=len(order), n_tok=out_cu[-1])
+
+
+def ready_batch_gather(src, src_cu, order, out_cu, pad_value):
+    """Token-level tensor of the ready batch: the rows of each kept invocation, then pad rows up to its slot."""
+    src = np.asarray(src)
+    out = np.empty((int(out_cu[-1]),) + src.shape[1:], src.dtype)
+    out[...] = pad_value
+    for j, s in enumerate(order):
+        L = int(src_cu[s + 1] - src_cu[s])
+        out[int(out_cu[j]):int(out_cu[j]) + L] = src[int(src_cu[s]):int(src_cu[s + 1])]
+    return out
+
+
+def align_rewards(r_inv, cu_seqlens, tok_mask=None):
+    """Token-level reward sequence of a delayed (invocation-level) reward: the invocation's reward sits on its last
+    unmasked response token, every other token gets 0 (paragraph "Batch construction": delayed rewards are aligned
+    with the token sequences).  An invocation without an unmasked token has nowhere to put its reward."""
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    r = to_f64(r_inv)
+    out = np.zeros(int(cu[-1]), F64)
+    for s in range(cu.size - 1):
+        for t in range(int(cu[s + 1]) - 1, int(cu[s]) - 1, -1):
+            if tok_mask is None or tok_mask[t]:
+                out[t] = r[s]
+                break
+    return out

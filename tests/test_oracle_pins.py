@@ -508,3 +508,174 @@ def test_reward_assembly_follows_the_workflow_rules():
     # a turn without a score pays nothing, and so does a role without a turn-level rule (Workflows A / B)
     r = orc.reward_assembly(np.array([1, 0]), np.zeros(2, int), np.array([2, 0]), f1, [2], [(orc.RULE_NONE, 0), (orc.RULE_ABSOLUTE, 0)])
     assert np.all(r == 0)
+
+
+# ---------------------------------------------------------------------------- value-loss pins
+
+def value_problem(seed=11, n_inv=7, R=3, K=2, max_len=6):
+    rng = np.random.default_rng(seed)
+    role_model = np.array([v % K for v in range(R)])
+    inv_role = rng.integers(0, R, n_inv)
+    inv_role[:R] = np.arange(R)
+    lens = rng.integers(0, max_len + 1, n_inv)
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    n = int(cu[-1])
+    mask = (rng.random(n) < 0.75).astype(np.uint8)
+    return dict(cu=cu, inv_role=inv_role, role_model=role_model, mask=mask, v=rng.normal(size=n),
+                ov=rng.normal(size=n), R=rng.normal(size=n), K=K)
+
+
+def test_value_loss_without_clipping_is_half_mse_per_model():
+    p = value_problem()
+    out = orc.value_loss_fwd_bwd(p["v"], p["ov"], p["R"], p["cu"], p["inv_role"], p["role_model"], p["mask"],
+                                 clip_v=1e30, K=p["K"])
+    tok_model = p["role_model"][p["inv_role"]][np.repeat(np.arange(len(p["cu"]) - 1), np.diff(p["cu"]))]
+    for k in range(p["K"]):
+        sel = (p["mask"] != 0) & (tok_model == k)
+        assert sel.sum() > 0
+        # numpy's mean of squared errors is the library special case
+        assert abs(out["loss"][k] - 0.5 * np.mean((p["v"][sel] - p["R"][sel]) ** 2)) < 1e-14
+        assert np.allclose(out["dvalues"][sel], (p["v"][sel] - p["R"][sel]) / sel.sum(), atol=1e-15)
+        assert out["clip_frac"][k] == 0
+    assert np.all(out["dvalues"][p["mask"] == 0] == 0) and np.all(out["tok_loss"][p["mask"] == 0] == 0)
+
+
+def test_value_loss_clip_branches_hand_values():
+    # one token per case, old value 0, clip 0.2, a single model:
+    #   v      R      v_clip  (v-R)^2  (v_clip-R)^2   branch      loss     dl/dv
+    #   0.1    1.0    0.1     0.81     0.81           unclipped   0.405    -0.9     (inside the range: tie)
+    #   0.5    1.0    0.2     0.25     0.64           clipped     0.32      0       (moved towards R too far)
+    #   0.5    0.0    0.2     0.25     0.04           unclipped   0.125     0.5     (moved away from R)
+    #  -0.6   -0.1   -0.2     0.25     0.01           unclipped   0.125    -0.5
+    #  -0.6   -1.0   -0.2     0.16     0.64           clipped     0.32      0
+    v = np.array([0.1, 0.5, 0.5, -0.6, -0.6])
+    R = np.array([1.0, 1.0, 0.0, -0.1, -1.0])
+    out = orc.value_loss_fwd_bwd(v, np.zeros(5), R, np.array([0, 5]), np.array([0]), np.array([0]), None, clip_v=0.2)
+    assert np.allclose(out["tok_loss"], [0.405, 0.32, 0.125, 0.125, 0.32], atol=1e-15)
+    assert np.allclose(out["dvalues"] * 5, [-0.9, 0.0, 0.5, -0.5, 0.0], atol=1e-15)
+    assert abs(out["loss"][0] - (0.405 + 0.32 + 0.125 + 0.125 + 0.32) / 5) < 1e-15
+    assert abs(out["clip_frac"][0] - 0.4) < 1e-15
+    # the clipped loss is never below the plain one (pessimistic bound)
+    plain = orc.value_loss_fwd_bwd(v, np.zeros(5), R, np.array([0, 5]), np.array([0]), np.array([0]), None, clip_v=1e30)
+    assert np.all(out["tok_loss"] >= plain["tok_loss"] - 1e-15)
+
+
+def test_value_loss_gradient_matches_autograd_and_finite_differences():
+    p = value_problem(seed=12)
+    norm = [5.0, 3.0]
+    out = orc.value_loss_fwd_bwd(p["v"], p["ov"], p["R"], p["cu"], p["inv_role"], p["role_model"], p["mask"],
+                                 clip_v=0.3, norm=norm)
+    tok_model = torch.from_numpy(p["role_model"][p["inv_role"]][np.repeat(np.arange(len(p["cu"]) - 1), np.diff(p["cu"]))])
+    v = torch.tensor(p["v"], dtype=torch.float64, requires_grad=True)
+    ov, R = torch.from_numpy(p["ov"]), torch.from_numpy(p["R"])
+    vc = ov + torch.clamp(v - ov, -0.3, 0.3)
+    tok = 0.5 * torch.maximum((v - R) ** 2, (vc - R) ** 2) * torch.from_numpy((p["mask"] != 0).astype(np.float64))
+    total = sum(tok[tok_model == k].sum() / norm[k] for k in range(2))
+    total.backward()
+    # inside the clip range the two branches coincide and autograd splits the gradient between them; the sum is the
+    # same number, so the comparison holds everywhere
+    assert np.allclose(out["dvalues"], v.grad.numpy(), atol=1e-14)
+    assert abs(float(total) - out["loss"].sum()) < 1e-14
+    h = 1e-6
+    for i in np.nonzero(p["mask"])[0][:8]:
+        vp, vm = p["v"].copy(), p["v"].copy()
+        vp[i] += h
+        vm[i] -= h
+        f = lambda x: orc.value_loss_fwd_bwd(x, p["ov"], p["R"], p["cu"], p["inv_role"], p["role_model"], p["mask"],
+                                             clip_v=0.3, norm=norm)["loss"].sum()
+        assert abs((f(vp) - f(vm)) / (2 * h) - out["dvalues"][i]) < 1e-8
+
+
+# ---------------------------------------------------------------------------- ready-batch pins
+
+def test_fmix32_published_values_and_permutation_is_a_bijection():
+    # MurmurHash3's finaliser: 0 is its fixed point and 1 maps to 0x514E28B7 (the value quoted with the algorithm)
+    assert orc.fmix32(0) == 0 and orc.fmix32(1) == 0x514E28B7
+    # it is a bijection of 32-bit words (each step is invertible); spot check: no collision among 2^16 inputs
+    assert len({orc.fmix32(x) for x in range(1 << 16)}) == 1 << 16
+    for n in [1, 2, 3, 4, 5, 16, 17, 100, 255, 256, 257, 1000, 4097]:
+        for seed in (0, 1, 20260528, (1 << 63) + 12345):
+            perm = orc.seeded_permutation(n, seed)
+            assert np.array_equal(np.sort(perm), np.arange(n))
+    assert orc.seeded_permutation(0, 3).size == 0
+    # different seeds give different orders, the same seed the same order
+    a, b = orc.seeded_permutation(1000, 1), orc.seeded_permutation(1000, 2)
+    assert not np.array_equal(a, b) and np.array_equal(a, orc.seeded_permutation(1000, 1))
+    # it shuffles: over many seeds, element 0 lands in every quarter of the range about equally often
+    pos = np.array([int(np.nonzero(orc.seeded_permutation(64, s) == 0)[0][0]) for s in range(400)])
+    hist = np.bincount(pos // 16, minlength=4)
+    assert hist.min() > 60 and hist.max() < 140
+    # and neighbours do not stay neighbours
+    assert np.mean(np.abs(np.diff(a)) == 1) < 0.05
+
+
+def batch_problem(seed=3, n_traj=40, R=3, K=2, max_len=9):
+    rng = np.random.default_rng(seed)
+    role_model = np.array([0, 1, 0])
+    inv_traj = np.repeat(np.arange(n_traj), rng.integers(1, 5, n_traj))
+    n_inv = inv_traj.size
+    inv_role = rng.integers(0, R, n_inv)
+    lens = rng.integers(0, max_len + 1, n_inv)
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    done = (rng.random(n_traj) < 0.7).astype(np.uint8)
+    return dict(cu=cu, inv_role=inv_role, inv_traj=inv_traj, done=done, role_model=role_model, K=K, n_inv=n_inv)
+
+
+@pytest.mark.parametrize("n_parts,pad_to", [(1, 1), (4, 1), (3, 8)])
+def test_ready_batch_plan_properties(n_parts, pad_to):
+    p = batch_problem()
+    out = orc.ready_batch_plan(p["cu"], p["inv_role"], p["inv_traj"], p["done"], p["role_model"], p["K"], seed=77,
+                               n_parts=n_parts, pad_to=pad_to)
+    order, out_cu = out["order"], out["out_cu"]
+    # kept set = brute-force filter: complete trajectory (and a role that maps to a model)
+    want = {s for s in range(p["n_inv"]) if p["done"][p["inv_traj"][s]]}
+    assert set(order.tolist()) == want and len(order) == len(want) == out["n_kept"]
+    # model-major: the models of the listed invocations are non-decreasing and match model_offsets
+    models = p["role_model"][p["inv_role"][order]]
+    assert np.all(np.diff(models) >= 0)
+    for k in range(p["K"]):
+        lo, hi = out["model_offsets"][k], out["model_offsets"][k + 1]
+        assert np.all(models[lo:hi] == k) and hi - lo == int((models == k).sum())
+    # inside a model the order is the shuffled order (increasing position in the permutation)
+    position = np.argsort(orc.seeded_permutation(p["n_inv"], 77))
+    for k in range(p["K"]):
+        lo, hi = out["model_offsets"][k], out["model_offsets"][k + 1]
+        assert np.all(np.diff(position[order[lo:hi]]) > 0)
+    # padded slots: each holds its invocation, is a multiple of pad_to, and wastes less than pad_to
+    lens = np.diff(p["cu"])[order]
+    slots = np.diff(out_cu)
+    assert np.all(slots % pad_to == 0) and np.all(slots >= lens) and np.all(slots - lens < pad_to)
+    assert out["n_tok"] == out_cu[-1] == slots.sum()
+    # partitions: contiguous, cover each model's range, and balanced in tokens up to one slot
+    po = out["part_offsets"]
+    assert po.size == p["K"] * n_parts + 1 and np.all(np.diff(po) >= 0) and po[-1] == out["n_kept"]
+    for k in range(p["K"]):
+        assert po[k * n_parts] == out["model_offsets"][k]
+        T = out_cu[out["model_offsets"][k + 1]] - out_cu[out["model_offsets"][k]]
+        for q in range(n_parts):
+            lo, hi = po[k * n_parts + q], po[k * n_parts + q + 1]
+            tokens = out_cu[hi] - out_cu[lo]
+            assert abs(tokens - T / n_parts) <= slots.max()
+
+
+def test_ready_batch_plan_hand_case_gather_and_reward_alignment():
+    # four invocations of lengths 3, 2, 4, 1; trajectory 1 (invocation 2) is incomplete; one model; pad to 4
+    cu = np.array([0, 3, 5, 9, 10])
+    out = orc.ready_batch_plan(cu, [0, 0, 0, 0], [0, 0, 1, 2], [1, 0, 1], [0], 1, seed=5, n_parts=1, pad_to=4)
+    perm = orc.seeded_permutation(4, 5)
+    assert out["order"].tolist() == [s for s in perm.tolist() if s != 2]
+    assert out["out_cu"].tolist() == [0, 4, 8, 12] and out["n_tok"] == 12
+    tok = np.arange(10) + 100
+    g = orc.ready_batch_gather(tok, cu, out["order"], out["out_cu"], -1)
+    for j, s in enumerate(out["order"]):
+        L = cu[s + 1] - cu[s]
+        assert g[4 * j:4 * j + L].tolist() == tok[cu[s]:cu[s + 1]].tolist() and np.all(g[4 * j + L:4 * j + 4] == -1)
+    # delayed rewards: on the last unmasked token of each invocation
+    mask = np.array([1, 1, 0, 1, 1, 0, 0, 0, 0, 1], np.uint8)
+    r = orc.align_rewards([0.5, -1.0, 2.0, 3.0], cu, mask)
+    assert r.tolist() == [0, 0.5, 0, 0, -1.0, 0, 0, 0, 0, 3.0]           # invocation 2 has no unmasked token
+    assert orc.align_rewards([0.5, -1.0, 2.0, 3.0], cu).tolist() == [0, 0, 0.5, 0, -1.0, 0, 0, 0, 2.0, 3.0]
+    # with gamma = lambda = 1 and zero values, GAE of the aligned reward gives every unmasked token its
+    # invocation's reward: the delayed reward reaches the whole response
+    A, _ = orc.gae(r, np.zeros(10), cu, 1.0, 1.0, mask)
+    assert A.tolist() == [0.5, 0.5, 0, -1.0, -1.0, 0, 0, 0, 0, 3.0]
