@@ -168,6 +168,81 @@ int unity_gae(unity_ctx* ctx, int32_t n_inv, int64_t n_tok, const int64_t* cu_se
               const float* values, const uint8_t* tok_mask, float gamma, float lambda, float* advantages,
               float* returns);
 
+/* Critic side of the update (paragraph "Model-specific updates and synchronization": each worker group updates its
+ * own actor and critic; the quantities are the "value estimates" and "returns" of paragraph "Advantage computation
+ * and policy evaluation", returns being unity_gae's second output).  The paper prints no value loss; the one used is
+ * PPO's clipped value regression.  Per valid token, with d = v - old_v:
+ *   v_clip = v if |d| <= clip_v else old_v + sign(d)*clip_v
+ *   l = 0.5 * max((v - R)^2, (v_clip - R)^2)         (equal squares take the unclipped branch)
+ *   loss[k] = (1/M_k) sum_{valid tokens of model k} l ,  M_k = norm[k] if given else max(#valid tokens, 1)
+ *   dvalues[i] = d loss[model(i)] / d v_i = (v - R)/M_k on the unclipped branch, 0 on the clipped one
+ * A token's model is role_model[inv_role[s]] of its invocation s, as in stages 2 and 3.
+ *   values, old_values, returns : f32 [n_tok];  tok_mask : u8 [n_tok] or NULL
+ *   role_model : (host) int32 [n_roles];  norm : (host) f32 [K] or NULL;  clip_v >= 0 (a huge value disables clipping)
+ *   loss : out f32 [K];  clip_frac : out f32 [K] or NULL (share of valid tokens on the clipped branch)
+ *   tok_loss : out f32 [n_tok] or NULL;  dvalues : out f32 [n_tok]; masked tokens receive 0 in both
+ * An out-of-range role or model id flags UNITY_ERR_BAD_INDEX and the invocation's tokens count as masked.
+ * Needs 12 bytes of workspace per invocation.  Deterministic (fixed-order sums, no floating-point atomics). */
+int unity_value_loss_fwd_bwd(unity_ctx* ctx, int32_t n_inv, int32_t n_roles, int32_t K, int64_t n_tok,
+                             const int64_t* cu_seqlens, const int32_t* inv_role, const int32_t* role_model,
+                             const uint8_t* tok_mask, const float* values, const float* old_values,
+                             const float* returns, float clip_v, const float* norm, float* loss, float* clip_frac,
+                             float* tok_loss, float* dvalues);
+
+/* Ready-batch construction - the step between a model-local buffer and the update calls (Section "Model-Local
+ * Buffers": a buffer becomes a ready-to-update batch by filtering incomplete trajectories, aligning delayed rewards
+ * with token sequences, padding, shuffling and matching the data-parallel configuration of the worker group; batches
+ * are built per model).  unity_ready_batch_plan decides WHICH invocations enter, in what order and where their tokens
+ * go; unity_ready_batch_gather then moves any token-level tensor of the buffer into that order.
+ *
+ * Plan.  (1) shuffle: position p = 0..n_inv-1 holds invocation perm(p), perm being a seeded bijection of [0, n_inv):
+ * four balanced Feistel rounds on the smallest even-width bit domain holding n_inv, applied again while the value is
+ * >= n_inv; round function fmix32(right ^ key_i) truncated to the half width, fmix32 = MurmurHash3's 32-bit finaliser,
+ * key_i = fmix32(seed32 + 0x9E3779B9*(i+1)), seed32 = low word of seed xor high word.  (2) filter: an invocation is
+ * kept when traj_done[inv_traj] != 0 and role_model[inv_role] >= 0 (-1 marks a role that is not trained).  (3) kept
+ * invocations are listed model by model, in shuffled order inside a model.  (4) each occupies its length rounded up
+ * to a multiple of pad_to.  (5) inside model k, invocation j with P_j padded tokens of the model before it belongs to
+ * partition min(n_parts-1, P_j*n_parts / T_k), T_k the model's padded total: contiguous partitions, equal in tokens up
+ * to one invocation - one per data-parallel rank or micro-batch.
+ *   cu_seqlens : int64 [n_inv+1];  inv_role, inv_traj : int32 [n_inv];  traj_done : u8 [n_traj]
+ *   role_model : (host) int32 [n_roles], values in [-1, K)
+ *   order          : out int32 [n_inv]: buffer index of the j-th listed invocation; -1 beyond the kept ones
+ *   out_cu_seqlens : out int64 [n_inv+1]: padded token offsets in the ready batch; entries beyond the kept ones
+ *                    repeat the total
+ *   model_offsets  : out int32 [K+1] into order;  part_offsets : out int32 [K*n_parts+1] into order
+ *   totals         : out int64 [2]: kept invocations, padded tokens (read it back to size later calls, or size them
+ *                    by the bounds n_inv and n_tok + n_inv*(pad_to-1))
+ * An out-of-range role or trajectory id drops the invocation and flags UNITY_ERR_BAD_INDEX.  Workspace: about
+ * 5 bytes per invocation + 12*K bytes per 256 invocations.  Integer work only: bit-exact and reproducible. */
+typedef struct {
+    uint64_t seed;
+    int32_t n_parts; /* >= 1, <= 65536 */
+    int32_t pad_to;  /* >= 1 */
+} unity_batch_params;
+int unity_ready_batch_plan(unity_ctx* ctx, int32_t n_inv, int32_t n_traj, int32_t n_roles, int32_t K,
+                           const int64_t* cu_seqlens, const int32_t* inv_role, const int32_t* inv_traj,
+                           const uint8_t* traj_done, const int32_t* role_model, const unity_batch_params* params,
+                           int32_t* order, int64_t* out_cu_seqlens, int32_t* model_offsets, int32_t* part_offsets,
+                           int64_t* totals);
+
+/* Move a token-level tensor (row_bytes bytes per token: 4 for ids / log-probs / values, 1 for masks, 2*H for hidden
+ * rows) from buffer order into the planned order.  The tokens of listed invocation j go to rows out_cu_seqlens[j]..,
+ * followed by pad rows up to out_cu_seqlens[j+1] filled with the pad pattern (pad_bytes in {1,2,4,8} dividing
+ * row_bytes; pad_value NULL = zeros).
+ *   n_inv : size of order;  order, out_cu_seqlens, totals : as written by unity_ready_batch_plan (device)
+ *   src_cu_seqlens : int64 [n_inv+1] of the buffer;  src : buffer tensor;  dst : out, at least totals[1] rows
+ *   src and dst must be aligned to min(16, largest power of two dividing row_bytes), else UNITY_ERR_ALIGNMENT. */
+int unity_ready_batch_gather(unity_ctx* ctx, int32_t n_inv, int64_t n_tok_src, const int32_t* order,
+                             const int64_t* src_cu_seqlens, const int64_t* out_cu_seqlens, const int64_t* totals,
+                             int64_t row_bytes, const void* src, void* dst, const void* pad_value, int32_t pad_bytes);
+
+/* Delayed rewards (paragraph "Batch construction": trajectory-level or delayed rewards are aligned with the token
+ * sequences): tok_reward[t] = r_inv[s] on the last unmasked token of invocation s and 0 on every other token - the
+ * reward sequence unity_gae consumes.  An invocation without an unmasked token has no place for its reward.
+ *   cu_seqlens : int64 [n_inv+1];  tok_mask : u8 [n_tok] or NULL;  r_inv : f32 [n_inv];  tok_reward : out f32 [n_tok] */
+int unity_align_rewards(unity_ctx* ctx, int32_t n_inv, int64_t n_tok, const int64_t* cu_seqlens,
+                        const uint8_t* tok_mask, const float* r_inv, float* tok_reward);
+
 /* Stage 1 without any allocation (the paper has no counterpart; this exists for deployment reasons).
  *
  * Who needs it: hosts that may not call cudaMalloc or create a unity_ctx - a trainer whose framework

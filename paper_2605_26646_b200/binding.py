@@ -25,7 +25,9 @@ UNITY_N_METRICS = 8
 
 EXPORTS = ["unity_create", "unity_destroy", "unity_workspace_bytes", "unity_workspace_min_bytes",
            "unity_check_status", "unity_last_error", "unity_launch_count", "unity_set_profiling",
-           "unity_get_profile", "unity_set_option", "unity_role_advantage", "unity_reward_assembly", "unity_gae", "unity_role_advantage_noalloc",
+           "unity_get_profile", "unity_set_option", "unity_role_advantage", "unity_reward_assembly", "unity_gae", "unity_value_loss_fwd_bwd",
+           "unity_ready_batch_plan", "unity_ready_batch_gather", "unity_align_rewards",
+           "unity_role_advantage_noalloc",
            "unity_logprob_fwd", "unity_ppo_loss_fwd_bwd"]
 
 
@@ -41,6 +43,10 @@ class unity_adv_params(C.Structure):
 
 class unity_reward_rule(C.Structure):
     _fields_ = [("mode", C.c_int), ("shift", C.c_int)]
+
+
+class unity_batch_params(C.Structure):
+    _fields_ = [("seed", C.c_uint64), ("n_parts", C.c_int32), ("pad_to", C.c_int32)]
 
 
 class unity_rows(C.Structure):
@@ -104,6 +110,16 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.unity_reward_assembly.restype = C.c_int
     lib.unity_gae.argtypes = [vp, i32, i64, vp, vp, vp, vp, C.c_float, C.c_float, vp, vp]
     lib.unity_gae.restype = C.c_int
+    lib.unity_value_loss_fwd_bwd.argtypes = [vp, i32, i32, i32, i64, vp, vp, C.POINTER(i32), vp, vp, vp, vp, C.c_float,
+                                             f32p, vp, vp, vp, vp]
+    lib.unity_value_loss_fwd_bwd.restype = C.c_int
+    lib.unity_ready_batch_plan.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, C.POINTER(i32),
+                                           C.POINTER(unity_batch_params), vp, vp, vp, vp, vp]
+    lib.unity_ready_batch_plan.restype = C.c_int
+    lib.unity_ready_batch_gather.argtypes = [vp, i32, i64, vp, vp, vp, vp, i64, vp, vp, vp, i32]
+    lib.unity_ready_batch_gather.restype = C.c_int
+    lib.unity_align_rewards.argtypes = [vp, i32, i64, vp, vp, vp, vp]
+    lib.unity_align_rewards.restype = C.c_int
     lib.unity_logprob_fwd.argtypes = [vp, C.POINTER(unity_rows), vp, vp, vp]
     lib.unity_logprob_fwd.restype = C.c_int
     lib.unity_ppo_loss_fwd_bwd.argtypes = [vp, C.POINTER(unity_rows), C.POINTER(unity_ppo_params), vp, vp, vp,
@@ -227,6 +243,61 @@ def unity_gae(ctx, cu_seqlens, rewards, values, tok_mask, gamma: float, lam: flo
                                     _ptr(cu_seqlens, torch.int64, "cu_seqlens"), _ptr(rewards, f32, "rewards"),
                                     _ptr(values, f32, "values"), _ptr(tok_mask, torch.uint8, "tok_mask"), gamma, lam,
                                     _ptr(advantages, f32, "advantages"), _ptr(returns, f32, "returns"))
+    _raise(ctx, code)
+
+
+def unity_value_loss_fwd_bwd(ctx, cu_seqlens, inv_role, role_model: Sequence[int], K: int, tok_mask, values,
+                             old_values, returns, clip_v: float, norm: Optional[Sequence[float]], loss,
+                             clip_frac=None, tok_loss=None, dvalues=None) -> None:
+    f32 = torch.float32
+    rm = (C.c_int32 * len(role_model))(*[int(x) for x in role_model])
+    norm_arr = None if norm is None else (C.c_float * len(norm))(*[float(x) for x in norm])
+    code = load_library().unity_value_loss_fwd_bwd(
+        ctx, int(inv_role.numel()), len(role_model), K, int(values.numel()),
+        _ptr(cu_seqlens, torch.int64, "cu_seqlens"), _ptr(inv_role, torch.int32, "inv_role"), rm,
+        _ptr(tok_mask, torch.uint8, "tok_mask"), _ptr(values, f32, "values"), _ptr(old_values, f32, "old_values"),
+        _ptr(returns, f32, "returns"), float(clip_v), norm_arr, _ptr(loss, f32, "loss"),
+        _ptr(clip_frac, f32, "clip_frac"), _ptr(tok_loss, f32, "tok_loss"), _ptr(dvalues, f32, "dvalues"))
+    _raise(ctx, code)
+
+
+def unity_ready_batch_plan(ctx, cu_seqlens, inv_role, inv_traj, traj_done, role_model: Sequence[int], K: int,
+                           seed: int, n_parts: int, pad_to: int, order, out_cu_seqlens, model_offsets, part_offsets,
+                           totals) -> None:
+    """order: int32 [n_inv]; out_cu_seqlens: int64 [n_inv+1]; model_offsets: int32 [K+1]; part_offsets: int32
+    [K*n_parts+1]; totals: int64 [2] - all CUDA tensors written by the call."""
+    i32, i64 = torch.int32, torch.int64
+    rm = (C.c_int32 * len(role_model))(*[int(x) for x in role_model])
+    p = unity_batch_params(int(seed) & 0xFFFFFFFFFFFFFFFF, int(n_parts), int(pad_to))
+    code = load_library().unity_ready_batch_plan(
+        ctx, int(inv_role.numel()), int(traj_done.numel()), len(role_model), K, _ptr(cu_seqlens, i64, "cu_seqlens"),
+        _ptr(inv_role, i32, "inv_role"), _ptr(inv_traj, i32, "inv_traj"), _ptr(traj_done, torch.uint8, "traj_done"),
+        rm, C.byref(p), _ptr(order, i32, "order"), _ptr(out_cu_seqlens, i64, "out_cu_seqlens"),
+        _ptr(model_offsets, i32, "model_offsets"), _ptr(part_offsets, i32, "part_offsets"), _ptr(totals, i64, "totals"))
+    _raise(ctx, code)
+
+
+def unity_ready_batch_gather(ctx, order, src_cu_seqlens, out_cu_seqlens, totals, src, dst, pad_value=0) -> None:
+    """src: CUDA tensor [n_tok_src, ...] in buffer order; dst: CUDA tensor [>= totals[1], ...] of the same dtype and
+    trailing shape; pad rows are filled with pad_value."""
+    if src.dtype != dst.dtype or tuple(src.shape[1:]) != tuple(dst.shape[1:]):
+        raise TypeError("src and dst must agree in dtype and trailing shape")
+    row_bytes = src.element_size()
+    for d in src.shape[1:]:
+        row_bytes *= int(d)
+    pad = bytes(torch.tensor([pad_value], dtype=src.dtype).view(torch.uint8).tolist())
+    code = load_library().unity_ready_batch_gather(
+        ctx, int(order.numel()), int(src.shape[0]), _ptr(order, torch.int32, "order"),
+        _ptr(src_cu_seqlens, torch.int64, "src_cu_seqlens"), _ptr(out_cu_seqlens, torch.int64, "out_cu_seqlens"),
+        _ptr(totals, torch.int64, "totals"), row_bytes, _ptr(src, None, "src"), _ptr(dst, None, "dst"), pad, len(pad))
+    _raise(ctx, code)
+
+
+def unity_align_rewards(ctx, cu_seqlens, tok_mask, r_inv, tok_reward) -> None:
+    code = load_library().unity_align_rewards(
+        ctx, int(r_inv.numel()), int(tok_reward.numel()), _ptr(cu_seqlens, torch.int64, "cu_seqlens"),
+        _ptr(tok_mask, torch.uint8, "tok_mask"), _ptr(r_inv, torch.float32, "r_inv"),
+        _ptr(tok_reward, torch.float32, "tok_reward"))
     _raise(ctx, code)
 
 
@@ -356,6 +427,18 @@ class Context:
 
     def gae(self, *a, **kw):
         return unity_gae(self.ctx, *a, **kw)
+
+    def value_loss_fwd_bwd(self, *a, **kw):
+        return unity_value_loss_fwd_bwd(self.ctx, *a, **kw)
+
+    def ready_batch_plan(self, *a, **kw):
+        return unity_ready_batch_plan(self.ctx, *a, **kw)
+
+    def ready_batch_gather(self, *a, **kw):
+        return unity_ready_batch_gather(self.ctx, *a, **kw)
+
+    def align_rewards(self, *a, **kw):
+        return unity_align_rewards(self.ctx, *a, **kw)
 
     def logprob_fwd(self, *a, **kw):
         return unity_logprob_fwd(self.ctx, *a, **kw)

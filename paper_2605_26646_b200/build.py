@@ -9,7 +9,8 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libunity.so")
-SOURCES = ["unity_api.cu", "stream_kernels.cu", "gemm_tcgen05.cu", "noalloc_advantage.cu"]
+SOURCES = ["unity_api.cu", "stream_kernels.cu", "gemm_tcgen05.cu", "batch_kernels.cu",
+           "noalloc_advantage.cu"]
 HEADERS = ["internal.h", "ptx.cuh", os.path.join("..", "..", "include", "unity.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]

@@ -1,0 +1,302 @@
+// Ready-batch construction on the device: the step between a model-local rollout buffer and the update calls.
+//   plan   : seeded shuffle (a Feistel bijection of the position index, so no sort and no random-number state),
+//            filter of invocations whose trajectory is incomplete or whose role is not trained, stable listing per
+//            model, padded token offsets, and a token-balanced split of every model's list into contiguous partitions
+//   gather : moves any token-level tensor of the buffer into the planned order (contiguous block copies + pad fill)
+//   align  : puts a delayed, invocation-level reward on the last unmasked token of its sequence
+// All integer work; every output is a pure function of the inputs (no atomics on results), so it is bit-exact.
+#include <cstring>
+
+#include "internal.h"
+
+namespace unity {
+
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+constexpr int kBatchBlock = 256;
+
+// 32-bit finaliser of MurmurHash3.
+__host__ __device__ __forceinline__ uint32_t fmix32(uint32_t h) {
+    h ^= h >> 16; h *= 0x85ebca6bu; h ^= h >> 13; h *= 0xc2b2ae35u; h ^= h >> 16;
+    return h;
+}
+
+// Position p of the shuffled order holds invocation feistel(p): four balanced Feistel rounds on the smallest
+// even-width bit domain that holds n, re-applied while the value falls outside [0, n) (cycle walking: the map is a
+// bijection of the domain, so the walk from p < n returns to [0, n) after finitely many steps).
+__device__ __forceinline__ int shuffled_index(int p, int n, int half, const uint32_t* key) {
+    const uint32_t hmask = (1u << half) - 1u;
+    uint32_t x = static_cast<uint32_t>(p);
+    do {
+        uint32_t left = x >> half, right = x & hmask;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t f = fmix32(right ^ key[i]) & hmask;
+            const uint32_t nl = right;
+            right = left ^ f;
+            left = nl;
+        }
+        x = (left << half) | right;
+    } while (x >= static_cast<uint32_t>(n));
+    return static_cast<int>(x);
+}
+
+__device__ __forceinline__ long long padded_len(const int64_t* cu, int s, int pad_to) {
+    const long long len = cu[s + 1] - cu[s];
+    return (len + pad_to - 1) / pad_to * pad_to;
+}
+
+// Pass 1: position -> invocation, keep / drop, model; per-block invocation and token counts per model.
+__global__ void k_batch_count(BatchArgs a) {
+    __shared__ int cnt[UNITY_MAX_MODELS];
+    __shared__ unsigned long long tok[UNITY_MAX_MODELS];
+    if (threadIdx.x < UNITY_MAX_MODELS) { cnt[threadIdx.x] = 0; tok[threadIdx.x] = 0ull; }
+    __syncthreads();
+    const int p = blockIdx.x * kBatchBlock + threadIdx.x;
+    if (p < a.n_inv) {
+        const int s = shuffled_index(p, a.n_inv, a.half_bits, a.key);
+        int model = -1;
+        const int role = a.inv_role[s], traj = a.inv_traj[s];
+        if (role < 0 || role >= a.n_roles || traj < 0 || traj >= a.n_traj) {
+            atomicOr(a.status, kStatusBadIndex);
+        } else if (a.traj_done[traj] != 0) {
+            model = a.role_model[role];                 // -1: a role that is not trained
+        }
+        a.pos_inv[p] = s;
+        a.pos_model[p] = static_cast<int8_t>(model);
+        if (model >= 0) {
+            atomicAdd(&cnt[model], 1);                  // integer counts: order does not matter
+            atomicAdd(&tok[model], static_cast<unsigned long long>(padded_len(a.cu_seqlens, s, a.pad_to)));
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < a.K) {
+        a.blk_cnt[blockIdx.x * a.K + threadIdx.x] = cnt[threadIdx.x];
+        a.blk_tok[blockIdx.x * a.K + threadIdx.x] = static_cast<long long>(tok[threadIdx.x]);
+    }
+}
+
+// Pass 2 (one block): exclusive prefix over the blocks, per model, of both counts; model offsets and totals.
+__global__ void k_batch_scan(BatchArgs a) {
+    __shared__ long long part_c[1024];
+    __shared__ long long part_t[1024];
+    __shared__ long long total_c[UNITY_MAX_MODELS], total_t[UNITY_MAX_MODELS];
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int per = (a.n_blocks + nt - 1) / nt;
+    const int b0 = min(tid * per, a.n_blocks), b1 = min(b0 + per, a.n_blocks);
+    for (int k = 0; k < a.K; ++k) {
+        long long sc = 0, st = 0;
+        for (int b = b0; b < b1; ++b) { sc += a.blk_cnt[b * a.K + k]; st += a.blk_tok[b * a.K + k]; }
+        part_c[tid] = sc; part_t[tid] = st;
+        __syncthreads();
+        for (int off = 1; off < nt; off <<= 1) {
+            const long long vc = tid >= off ? part_c[tid - off] : 0, vt = tid >= off ? part_t[tid - off] : 0;
+            __syncthreads();
+            part_c[tid] += vc; part_t[tid] += vt;
+            __syncthreads();
+        }
+        long long rc = part_c[tid] - sc, rt = part_t[tid] - st;
+        if (tid == nt - 1) { total_c[k] = part_c[tid]; total_t[k] = part_t[tid]; }
+        for (int b = b0; b < b1; ++b) {
+            const int c = a.blk_cnt[b * a.K + k];
+            const long long t = a.blk_tok[b * a.K + k];
+            a.blk_cnt[b * a.K + k] = static_cast<int>(rc);
+            a.blk_tok[b * a.K + k] = rt;
+            rc += c; rt += t;
+        }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        long long oc = 0, ot = 0;
+        for (int k = 0; k < a.K; ++k) {
+            a.model_offsets[k] = static_cast<int>(oc);
+            a.model_tok[k] = ot;
+            oc += total_c[k]; ot += total_t[k];
+        }
+        a.model_offsets[a.K] = static_cast<int>(oc);
+        a.model_tok[a.K] = ot;
+        a.totals[0] = oc;
+        a.totals[1] = ot;
+    }
+}
+
+// Pass 3: every kept position finds its place: rank among the kept positions of its model before it (stable), and
+// the padded tokens before it.
+__global__ void k_batch_assign(BatchArgs a) {
+    __shared__ int w_cnt[kBatchBlock / 32];
+    __shared__ long long w_tok[kBatchBlock / 32];
+    const int p = blockIdx.x * kBatchBlock + threadIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int model = p < a.n_inv ? a.pos_model[p] : -1;
+    const int s = p < a.n_inv ? a.pos_inv[p] : 0;
+    const long long len = model >= 0 ? padded_len(a.cu_seqlens, s, a.pad_to) : 0;
+    int my_rank = 0;
+    long long my_tok = 0;
+    for (int k = 0; k < a.K; ++k) {
+        const bool mine = model == k;
+        const unsigned bal = __ballot_sync(kFull, mine);
+        // inclusive warp scan of the token counts of this model's positions
+        long long v = mine ? len : 0;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const long long u = __shfl_up_sync(kFull, v, o);
+            if (lane >= o) v += u;
+        }
+        if (lane == 31) { w_cnt[warp] = __popc(bal); w_tok[warp] = v; }
+        __syncthreads();
+        if (mine) {
+            int rc = __popc(bal & ((1u << lane) - 1u));
+            long long rt = v - len;
+            for (int w = 0; w < warp; ++w) { rc += w_cnt[w]; rt += w_tok[w]; }
+            my_rank = rc;
+            my_tok = rt;
+        }
+        __syncthreads();
+    }
+    if (model < 0) return;
+    const int j = a.model_offsets[model] + a.blk_cnt[blockIdx.x * a.K + model] + my_rank;
+    a.order[j] = s;
+    a.out_cu[j] = a.model_tok[model] + a.blk_tok[blockIdx.x * a.K + model] + my_tok;
+}
+
+// Pass 4: partition boundaries, and the tails of the outputs.  Invocation j of model k, with P_j padded tokens of the
+// model before it, belongs to partition min(n_parts - 1, P_j * n_parts / T_k); partitions are contiguous, so the
+// first member of each is found by comparing neighbours.
+__device__ __forceinline__ int part_of(long long P, long long T, int n_parts) {
+    if (T <= 0) return 0;
+    const long long q = P * n_parts / T;
+    return q < n_parts - 1 ? static_cast<int>(q) : n_parts - 1;
+}
+
+__global__ void k_batch_parts(BatchArgs a) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    const int n_kept = static_cast<int>(a.totals[0]);
+    const long long n_tok = a.totals[1];
+    if (j < a.K * a.n_parts) {                                   // models without a kept invocation
+        const int k = j / a.n_parts;
+        if (a.model_offsets[k + 1] == a.model_offsets[k]) a.part_offsets[j] = a.model_offsets[k];
+    }
+    if (j == 0) a.part_offsets[a.K * a.n_parts] = n_kept;
+    if (j > a.n_inv) return;
+    if (j >= n_kept) {
+        a.out_cu[j] = n_tok;
+        if (j < a.n_inv) a.order[j] = -1;
+        return;
+    }
+    int k = 0;
+    while (k + 1 < a.K && j >= a.model_offsets[k + 1]) ++k;
+    const long long T = a.model_tok[k + 1] - a.model_tok[k];
+    const int mine = part_of(a.out_cu[j] - a.model_tok[k], T, a.n_parts);
+    const int prev = j == a.model_offsets[k] ? -1 : part_of(a.out_cu[j - 1] - a.model_tok[k], T, a.n_parts);
+    for (int q = prev + 1; q <= mine; ++q) a.part_offsets[k * a.n_parts + q] = j;
+    if (j == a.model_offsets[k + 1] - 1)
+        for (int q = mine + 1; q < a.n_parts; ++q) a.part_offsets[k * a.n_parts + q] = j + 1;
+}
+
+// Gather: block (x = kept invocation, strided; y = slice) copies the invocation's contiguous bytes and fills the pad.
+template <typename T>
+__global__ void k_batch_gather(const int* __restrict__ order, const int64_t* __restrict__ src_cu,
+                               const int64_t* __restrict__ out_cu, const long long* __restrict__ totals,
+                               long long units_per_row, const T* __restrict__ src, T* __restrict__ dst, T pad) {
+    const int n_kept = static_cast<int>(totals[0]);
+    for (int j = blockIdx.x; j < n_kept; j += gridDim.x) {
+        const int s = order[j];
+        const long long n_copy = (src_cu[s + 1] - src_cu[s]) * units_per_row;
+        const long long n_slot = (out_cu[j + 1] - out_cu[j]) * units_per_row;
+        const T* from = src + src_cu[s] * units_per_row;
+        T* to = dst + out_cu[j] * units_per_row;
+        const long long stride = static_cast<long long>(gridDim.y) * blockDim.x;
+        for (long long i = static_cast<long long>(blockIdx.y) * blockDim.x + threadIdx.x; i < n_slot; i += stride)
+            to[i] = i < n_copy ? from[i] : pad;
+    }
+}
+
+// Delayed rewards: one warp per invocation walks it backwards; the first unmasked token met takes the reward.
+__global__ void k_align_rewards(int n_inv, const int64_t* __restrict__ cu, const uint8_t* __restrict__ mask,
+                                const float* __restrict__ r_inv, float* __restrict__ tok_reward) {
+    const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (s >= n_inv) return;
+    const long long lo = cu[s], hi = cu[s + 1];
+    const float r = r_inv[s];
+    bool placed = false;
+    for (long long c0 = hi - 32; c0 > lo - 32; c0 -= 32) {
+        const long long t = c0 + lane;
+        const bool in = t >= lo && t < hi;
+        const bool on = in && (mask ? mask[t] != 0 : true);
+        const unsigned valid = __ballot_sync(kFull, on);
+        float out = 0.f;
+        if (!placed && valid) {
+            const int last = 31 - __clz(valid);
+            if (lane == last) out = r;
+            placed = true;
+        }
+        if (in) tok_reward[t] = out;
+    }
+}
+
+template <typename T>
+cudaError_t gather_as(const GatherArgs& g, cudaStream_t stream) {
+    T pad;
+    // the pad pattern, replicated to the width of the copy unit
+    unsigned char bytes[16];
+    for (int i = 0; i < 16; ++i) bytes[i] = g.pad[i % g.pad_bytes];
+    memcpy(&pad, bytes, sizeof(T));
+    const long long units = g.row_bytes / static_cast<long long>(sizeof(T));
+    const int gx = g.n_inv < 4096 ? (g.n_inv > 0 ? g.n_inv : 1) : 4096;
+    // slices per invocation: enough blocks for rows of many bytes, one for per-token scalars
+    long long gy = (g.row_bytes * g.avg_len + 32767) / 32768;
+    gy = gy < 1 ? 1 : (gy > 16 ? 16 : gy);
+    k_batch_gather<T><<<dim3(gx, static_cast<unsigned>(gy)), 256, 0, stream>>>(
+        g.order, g.src_cu, g.out_cu, g.totals, units, static_cast<const T*>(g.src), static_cast<T*>(g.dst), pad);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+void batch_keys(uint64_t seed, int n_inv, BatchArgs* a) {
+    int bits = 2;
+    while (bits < 31 && (1ll << bits) < n_inv) ++bits;
+    bits += bits & 1;
+    a->half_bits = bits / 2;
+    const uint32_t seed32 = static_cast<uint32_t>(seed ^ (seed >> 32));
+    for (int i = 0; i < 4; ++i) a->key[i] = fmix32(seed32 + 0x9E3779B9u * static_cast<uint32_t>(i + 1));
+}
+
+cudaError_t launch_batch_plan(const BatchArgs& a, cudaStream_t stream, int* n_launches) {
+    if (a.n_inv > 0) {
+        k_batch_count<<<a.n_blocks, kBatchBlock, 0, stream>>>(a);
+        *n_launches += 1;
+    }
+    k_batch_scan<<<1, 1024, 0, stream>>>(a);
+    if (a.n_inv > 0) {
+        k_batch_assign<<<a.n_blocks, kBatchBlock, 0, stream>>>(a);
+        *n_launches += 1;
+    }
+    const int n_threads = max(a.n_inv + 1, a.K * a.n_parts);
+    k_batch_parts<<<(n_threads + 255) / 256, 256, 0, stream>>>(a);
+    *n_launches += 2;
+    return cudaGetLastError();
+}
+
+int batch_block() { return kBatchBlock; }
+
+cudaError_t launch_batch_gather(const GatherArgs& g, cudaStream_t stream) {
+    switch (g.unit_bytes) {
+        case 16: return gather_as<uint4>(g, stream);
+        case 8: return gather_as<uint2>(g, stream);
+        case 4: return gather_as<uint32_t>(g, stream);
+        case 2: return gather_as<uint16_t>(g, stream);
+        default: return gather_as<uint8_t>(g, stream);
+    }
+}
+
+cudaError_t launch_align_rewards(int n_inv, const int64_t* cu, const uint8_t* mask, const float* r_inv,
+                                 float* tok_reward, cudaStream_t stream) {
+    if (n_inv == 0) return cudaSuccess;
+    k_align_rewards<<<(n_inv + 7) / 8, 256, 0, stream>>>(n_inv, cu, mask, r_inv, tok_reward);
+    return cudaGetLastError();
+}
+
+}  // namespace unity

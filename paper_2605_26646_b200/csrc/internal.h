@@ -170,4 +170,68 @@ struct RewardArgs {
 };
 cudaError_t launch_reward_assembly(const RewardArgs& a, cudaStream_t stream);
 
+struct ValueArgs {
+    int n_inv, n_roles, K;
+    const int64_t* cu_seqlens;
+    const int32_t* inv_role;
+    int32_t role_model[UNITY_MAX_ROLES];
+    const uint8_t* tok_mask;
+    const float *values, *old_values, *returns;
+    float clip_v;
+    int has_norm;
+    float norm[UNITY_MAX_MODELS];
+    float* inv_sums;    // [n_inv * 3] count, sum of token losses, clipped tokens
+    float* Mk;          // [K] denominators, written by the class reduction
+    float *loss, *clip_frac, *tok_loss, *dvalues;
+    int* status;
+};
+cudaError_t launch_value_loss(const ValueArgs& a, cudaStream_t stream, int* n_launches);
+
+// ----------------------------------------------------------------------------------------------
+// ready-batch construction (batch_kernels.cu)
+// ----------------------------------------------------------------------------------------------
+struct BatchArgs {
+    int n_inv, n_traj, n_roles, K, n_parts, pad_to;
+    int half_bits;               // half width of the Feistel domain
+    uint32_t key[4];             // round keys derived from the seed
+    const int64_t* cu_seqlens;
+    const int32_t *inv_role, *inv_traj;
+    const uint8_t* traj_done;
+    int32_t role_model[UNITY_MAX_ROLES];   // -1: the role's tokens are not trained
+    int n_blocks;                // ceil(n_inv / batch_block())
+    // scratch
+    int* pos_inv;                // [n_inv] invocation at each shuffled position
+    int8_t* pos_model;           // [n_inv] its model, or -1 when dropped
+    int* blk_cnt;                // [n_blocks * K] -> exclusive prefix per model
+    long long* blk_tok;          // [n_blocks * K] same for padded tokens
+    long long* model_tok;        // [K + 1] first padded token of each model
+    // outputs
+    int* order;                  // [n_inv]
+    int64_t* out_cu;             // [n_inv + 1]
+    int* model_offsets;          // [K + 1]
+    int* part_offsets;           // [K * n_parts + 1]
+    long long* totals;           // [2] kept invocations, padded tokens
+    int* status;
+};
+void batch_keys(uint64_t seed, int n_inv, BatchArgs* a);
+int batch_block();
+cudaError_t launch_batch_plan(const BatchArgs& a, cudaStream_t stream, int* n_launches);
+
+struct GatherArgs {
+    int n_inv;                   // upper bound of kept invocations (sizes the grid)
+    const int* order;
+    const int64_t *src_cu, *out_cu;
+    const long long* totals;
+    long long row_bytes;         // bytes per token
+    int unit_bytes;              // copy unit: 1, 2, 4, 8 or 16, dividing row_bytes and the alignment of src / dst
+    long long avg_len;           // mean tokens per invocation (sizes the grid)
+    const void* src;
+    void* dst;
+    unsigned char pad[16];       // pad pattern of pad_bytes bytes
+    int pad_bytes;
+};
+cudaError_t launch_batch_gather(const GatherArgs& g, cudaStream_t stream);
+cudaError_t launch_align_rewards(int n_inv, const int64_t* cu, const uint8_t* mask, const float* r_inv,
+                                 float* tok_reward, cudaStream_t stream);
+
 }  // namespace unity

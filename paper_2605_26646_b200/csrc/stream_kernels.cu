@@ -518,6 +518,82 @@ __global__ void k_reward_assembly(RewardArgs a) {
     a.r_turn[s] = out;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Critic update: clipped value loss.  Three small launches with fixed-order sums: per invocation (one warp each),
+// per model (one warp each), then the gradient with the model's 1/M_k.
+struct ValueTerm {
+    float loss, grad, clipped;
+};
+__device__ __forceinline__ ValueTerm value_term(float v, float ov, float ret, float clip_v) {
+    const float d = v - ov;
+    // inside the range the clipped estimate IS v; outside it is the end of the range
+    const float vc = fabsf(d) <= clip_v ? v : ov + copysignf(clip_v, d);
+    const float eu = v - ret, ec = vc - ret;
+    const float su = eu * eu, sc = ec * ec;
+    const bool unclipped = su >= sc;            // ties take the unclipped branch
+    ValueTerm t;
+    t.loss = 0.5f * (unclipped ? su : sc);
+    t.grad = unclipped ? eu : 0.f;
+    t.clipped = unclipped ? 0.f : 1.f;
+    return t;
+}
+
+__global__ void k_value_inv(ValueArgs a) {
+    const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (s >= a.n_inv) return;
+    const int role = a.inv_role[s];
+    const bool role_ok = role >= 0 && role < a.n_roles && a.role_model[role] >= 0 && a.role_model[role] < a.K;
+    const long long lo = a.cu_seqlens[s], hi = a.cu_seqlens[s + 1];
+    float cnt = 0.f, sum = 0.f, clp = 0.f;
+    for (long long i = lo + lane; i < hi; i += 32) {
+        const bool on = role_ok && (a.tok_mask ? a.tok_mask[i] != 0 : true);
+        float l = 0.f;
+        if (on) {
+            const ValueTerm t = value_term(a.values[i], a.old_values[i], a.returns[i], a.clip_v);
+            l = t.loss; cnt += 1.f; sum += t.loss; clp += t.clipped;
+        }
+        if (a.tok_loss) a.tok_loss[i] = l;
+    }
+    cnt = warp_sum(cnt); sum = warp_sum(sum); clp = warp_sum(clp);
+    if (lane == 0) {
+        if (!role_ok && hi > lo) atomicOr(a.status, kStatusBadIndex);
+        a.inv_sums[s * 3 + 0] = cnt; a.inv_sums[s * 3 + 1] = sum; a.inv_sums[s * 3 + 2] = clp;
+    }
+}
+
+__global__ void k_value_class(ValueArgs a) {
+    const int k = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (k >= a.K) return;
+    float cnt = 0.f, sum = 0.f, clp = 0.f;
+    for (int s = lane; s < a.n_inv; s += 32) {
+        const int role = a.inv_role[s];
+        if (role < 0 || role >= a.n_roles || a.role_model[role] != k) continue;
+        cnt += a.inv_sums[s * 3 + 0]; sum += a.inv_sums[s * 3 + 1]; clp += a.inv_sums[s * 3 + 2];
+    }
+    cnt = warp_sum(cnt); sum = warp_sum(sum); clp = warp_sum(clp);
+    if (lane != 0) return;
+    const float M = a.has_norm ? a.norm[k] : fmaxf(cnt, 1.f);
+    a.Mk[k] = M;
+    a.loss[k] = sum / M;
+    if (a.clip_frac) a.clip_frac[k] = clp / fmaxf(cnt, 1.f);
+}
+
+__global__ void k_value_grad(ValueArgs a) {
+    const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (s >= a.n_inv) return;
+    const int role = a.inv_role[s];
+    const bool role_ok = role >= 0 && role < a.n_roles && a.role_model[role] >= 0 && a.role_model[role] < a.K;
+    const float M = role_ok ? a.Mk[a.role_model[role]] : 1.f;
+    const long long lo = a.cu_seqlens[s], hi = a.cu_seqlens[s + 1];
+    for (long long i = lo + lane; i < hi; i += 32) {
+        const bool on = role_ok && (a.tok_mask ? a.tok_mask[i] != 0 : true);
+        a.dvalues[i] = on ? value_term(a.values[i], a.old_values[i], a.returns[i], a.clip_v).grad / M : 0.f;
+    }
+}
+
 }  // namespace
 
 // ------------------------------------------------------------------------------------------------
@@ -598,6 +674,20 @@ cudaError_t launch_gae(int n_inv, const int64_t* cu_seqlens, const float* reward
 cudaError_t launch_reward_assembly(const RewardArgs& a, cudaStream_t stream) {
     if (a.n_inv == 0) return cudaSuccess;
     k_reward_assembly<<<(a.n_inv + 255) / 256, 256, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_value_loss(const ValueArgs& a, cudaStream_t stream, int* n_launches) {
+    if (a.n_inv > 0) {
+        k_value_inv<<<(a.n_inv + 7) / 8, 256, 0, stream>>>(a);
+        *n_launches += 1;
+    }
+    k_value_class<<<(a.K + 7) / 8, 256, 0, stream>>>(a);
+    *n_launches += 1;
+    if (a.n_inv > 0) {
+        k_value_grad<<<(a.n_inv + 7) / 8, 256, 0, stream>>>(a);
+        *n_launches += 1;
+    }
     return cudaGetLastError();
 }
 

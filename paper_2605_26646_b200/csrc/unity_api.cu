@@ -548,6 +548,131 @@ int unity_gae(unity_ctx* ctx, int32_t n_inv, int64_t n_tok, const int64_t* cu_se
 }
 
 // ------------------------------------------------------------------------------------------------
+int unity_value_loss_fwd_bwd(unity_ctx* ctx, int32_t n_inv, int32_t n_roles, int32_t K, int64_t n_tok,
+                             const int64_t* cu_seqlens, const int32_t* inv_role, const int32_t* role_model,
+                             const uint8_t* tok_mask, const float* values, const float* old_values,
+                             const float* returns, float clip_v, const float* norm, float* loss, float* clip_frac,
+                             float* tok_loss, float* dvalues) {
+    if (!ctx) return UNITY_ERR_INVALID_ARG;
+    if (n_inv < 0 || n_tok < 0) return fail(ctx, UNITY_ERR_INVALID_ARG, "negative size");
+    if (n_roles < 1 || n_roles > UNITY_MAX_ROLES) return fail(ctx, UNITY_ERR_SHAPE, "n_roles=%d outside [1,%d]", n_roles, UNITY_MAX_ROLES);
+    if (K < 1 || K > UNITY_MAX_MODELS) return fail(ctx, UNITY_ERR_SHAPE, "K=%d outside [1,%d]", K, UNITY_MAX_MODELS);
+    if (!role_model || !loss) return fail(ctx, UNITY_ERR_INVALID_ARG, "role_model / loss is NULL");
+    if (!(clip_v >= 0.f)) return fail(ctx, UNITY_ERR_INVALID_ARG, "clip_v must be >= 0");
+    if (n_inv > 0 && (!cu_seqlens || !inv_role)) return fail(ctx, UNITY_ERR_INVALID_ARG, "cu_seqlens / inv_role is NULL");
+    if (n_tok > 0 && (n_inv < 1 || !values || !old_values || !returns || !dvalues))
+        return fail(ctx, UNITY_ERR_INVALID_ARG, "values / old_values / returns / dvalues is NULL or n_inv < 1");
+    ValueArgs a;
+    memset(&a, 0, sizeof(a));
+    for (int k = 0; k < K; ++k) {
+        if (norm && !(norm[k] > 0.f)) return fail(ctx, UNITY_ERR_INVALID_ARG, "norm[%d] must be > 0", k);
+        if (norm) a.norm[k] = norm[k];
+    }
+    for (int v = 0; v < n_roles; ++v) a.role_model[v] = role_model[v];
+    CUDA_TRY(ctx, cudaSetDevice(ctx->device));
+    Bump b{ctx->ws, 0, ctx->ws_bytes, true};
+    a.Mk = b.take<float>(UNITY_MAX_MODELS);
+    a.inv_sums = b.take<float>(static_cast<size_t>(n_inv) * 3 + 4);
+    if (!b.ok) return fail(ctx, UNITY_ERR_WORKSPACE, "workspace too small: need %zu bytes", b.off);
+    a.n_inv = n_inv; a.n_roles = n_roles; a.K = K;
+    a.cu_seqlens = cu_seqlens; a.inv_role = inv_role; a.tok_mask = tok_mask;
+    a.values = values; a.old_values = old_values; a.returns = returns;
+    a.clip_v = clip_v; a.has_norm = norm != nullptr;
+    a.loss = loss; a.clip_frac = clip_frac; a.tok_loss = tok_loss; a.dvalues = dvalues;
+    a.status = ctx->d_status;
+    int nl = 0;
+    CUDA_TRY(ctx, launch_value_loss(a, ctx->stream, &nl));
+    ctx->launches += nl;
+    return UNITY_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+int unity_ready_batch_plan(unity_ctx* ctx, int32_t n_inv, int32_t n_traj, int32_t n_roles, int32_t K,
+                           const int64_t* cu_seqlens, const int32_t* inv_role, const int32_t* inv_traj,
+                           const uint8_t* traj_done, const int32_t* role_model, const unity_batch_params* params,
+                           int32_t* order, int64_t* out_cu_seqlens, int32_t* model_offsets, int32_t* part_offsets,
+                           int64_t* totals) {
+    if (!ctx) return UNITY_ERR_INVALID_ARG;
+    if (n_inv < 0 || n_traj < 0) return fail(ctx, UNITY_ERR_INVALID_ARG, "negative size");
+    if (n_roles < 1 || n_roles > UNITY_MAX_ROLES) return fail(ctx, UNITY_ERR_SHAPE, "n_roles=%d outside [1,%d]", n_roles, UNITY_MAX_ROLES);
+    if (K < 1 || K > UNITY_MAX_MODELS) return fail(ctx, UNITY_ERR_SHAPE, "K=%d outside [1,%d]", K, UNITY_MAX_MODELS);
+    if (!params || !role_model || !out_cu_seqlens || !model_offsets || !part_offsets || !totals)
+        return fail(ctx, UNITY_ERR_INVALID_ARG, "params / role_model / out_cu_seqlens / model_offsets / part_offsets / totals is NULL");
+    if (params->n_parts < 1 || params->n_parts > 65536 || params->pad_to < 1)
+        return fail(ctx, UNITY_ERR_INVALID_ARG, "n_parts must lie in [1, 65536] and pad_to must be >= 1");
+    if (n_inv > 0 && (!cu_seqlens || !inv_role || !inv_traj || !traj_done || !order))
+        return fail(ctx, UNITY_ERR_INVALID_ARG, "cu_seqlens / inv_role / inv_traj / traj_done / order is NULL");
+    BatchArgs a;
+    memset(&a, 0, sizeof(a));
+    for (int v = 0; v < n_roles; ++v) {
+        if (role_model[v] < -1 || role_model[v] >= K) return fail(ctx, UNITY_ERR_INVALID_ARG, "role_model[%d]=%d outside [-1,%d)", v, role_model[v], K);
+        a.role_model[v] = role_model[v];
+    }
+    CUDA_TRY(ctx, cudaSetDevice(ctx->device));
+    a.n_inv = n_inv; a.n_traj = n_traj; a.n_roles = n_roles; a.K = K;
+    a.n_parts = params->n_parts; a.pad_to = params->pad_to;
+    batch_keys(params->seed, n_inv, &a);
+    a.n_blocks = (n_inv + batch_block() - 1) / batch_block();
+    Bump b{ctx->ws, 0, ctx->ws_bytes, true};
+    a.model_tok = b.take<long long>(UNITY_MAX_MODELS + 1);
+    a.pos_inv = b.take<int>(n_inv);
+    a.pos_model = b.take<int8_t>(n_inv);
+    a.blk_cnt = b.take<int>(static_cast<size_t>(a.n_blocks) * K);
+    a.blk_tok = b.take<long long>(static_cast<size_t>(a.n_blocks) * K);
+    if (!b.ok) return fail(ctx, UNITY_ERR_WORKSPACE, "workspace too small: need %zu bytes", b.off);
+    a.cu_seqlens = cu_seqlens; a.inv_role = inv_role; a.inv_traj = inv_traj; a.traj_done = traj_done;
+    a.order = order; a.out_cu = out_cu_seqlens; a.model_offsets = model_offsets; a.part_offsets = part_offsets;
+    a.totals = reinterpret_cast<long long*>(totals);
+    a.status = ctx->d_status;
+    int nl = 0;
+    CUDA_TRY(ctx, launch_batch_plan(a, ctx->stream, &nl));
+    ctx->launches += nl;
+    return UNITY_OK;
+}
+
+int unity_ready_batch_gather(unity_ctx* ctx, int32_t n_inv, int64_t n_tok_src, const int32_t* order,
+                             const int64_t* src_cu_seqlens, const int64_t* out_cu_seqlens, const int64_t* totals,
+                             int64_t row_bytes, const void* src, void* dst, const void* pad_value, int32_t pad_bytes) {
+    if (!ctx) return UNITY_ERR_INVALID_ARG;
+    if (n_inv < 0 || n_tok_src < 0 || row_bytes < 1) return fail(ctx, UNITY_ERR_INVALID_ARG, "negative size or row_bytes < 1");
+    if (pad_bytes != 1 && pad_bytes != 2 && pad_bytes != 4 && pad_bytes != 8)
+        return fail(ctx, UNITY_ERR_INVALID_ARG, "pad_bytes must be 1, 2, 4 or 8");
+    if (row_bytes % pad_bytes) return fail(ctx, UNITY_ERR_INVALID_ARG, "pad_bytes must divide row_bytes");
+    if (n_inv == 0) return UNITY_OK;
+    if (!order || !src_cu_seqlens || !out_cu_seqlens || !totals || !dst || (n_tok_src > 0 && !src))
+        return fail(ctx, UNITY_ERR_INVALID_ARG, "order / src_cu_seqlens / out_cu_seqlens / totals / src / dst is NULL");
+    int unit = 16;
+    while (unit > 1 && row_bytes % unit) unit >>= 1;
+    if (unit < pad_bytes || (reinterpret_cast<uintptr_t>(src) % unit) || (reinterpret_cast<uintptr_t>(dst) % unit))
+        return fail(ctx, UNITY_ERR_ALIGNMENT, "src / dst must be aligned to %d bytes for rows of %lld bytes", unit,
+                    static_cast<long long>(row_bytes));
+    GatherArgs g;
+    memset(&g, 0, sizeof(g));
+    g.n_inv = n_inv; g.order = order; g.src_cu = src_cu_seqlens; g.out_cu = out_cu_seqlens;
+    g.totals = reinterpret_cast<const long long*>(totals);
+    g.row_bytes = row_bytes; g.unit_bytes = unit; g.avg_len = n_tok_src / n_inv + 1;
+    g.src = src; g.dst = dst; g.pad_bytes = pad_bytes;
+    if (pad_value) memcpy(g.pad, pad_value, pad_bytes);
+    CUDA_TRY(ctx, cudaSetDevice(ctx->device));
+    CUDA_TRY(ctx, launch_batch_gather(g, ctx->stream));
+    ctx->launches += 1;
+    return UNITY_OK;
+}
+
+int unity_align_rewards(unity_ctx* ctx, int32_t n_inv, int64_t n_tok, const int64_t* cu_seqlens,
+                        const uint8_t* tok_mask, const float* r_inv, float* tok_reward) {
+    if (!ctx) return UNITY_ERR_INVALID_ARG;
+    if (n_inv < 0 || n_tok < 0) return fail(ctx, UNITY_ERR_INVALID_ARG, "negative size");
+    if (n_inv > 0 && (!cu_seqlens || !r_inv)) return fail(ctx, UNITY_ERR_INVALID_ARG, "cu_seqlens / r_inv is NULL");
+    if (n_tok > 0 && (n_inv < 1 || !tok_reward)) return fail(ctx, UNITY_ERR_INVALID_ARG, "tok_reward is NULL or n_inv < 1");
+    if (n_inv == 0) return UNITY_OK;
+    CUDA_TRY(ctx, cudaSetDevice(ctx->device));
+    CUDA_TRY(ctx, launch_align_rewards(n_inv, cu_seqlens, tok_mask, r_inv, tok_reward, ctx->stream));
+    ctx->launches += 1;
+    return UNITY_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
 int unity_logprob_fwd(unity_ctx* ctx, const unity_rows* rows, float* logp, float* entropy, float* lse) {
     int rc = validate_rows(ctx, rows);
     if (rc) return rc;

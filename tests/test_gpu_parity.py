@@ -195,6 +195,47 @@ def test_gae_full_size(name, gamma, lam, masked):
     ctx.close()
 
 
+@pytest.mark.parametrize("name,clip_v,with_norm,masked", [("tiny", 0.2, False, True), ("search", 0.3, True, True),
+                                                          ("code", 1e30, False, True), ("rag_qa", 0.1, False, False)])
+def test_value_loss_full_size(name, clip_v, with_norm, masked):
+    import oracle.unity_oracle as orc
+    w = wl.make_structure(name)
+    v = wl.normal(12, 1, w.n_tok)
+    ov = v + 0.25 * wl.normal(12, 2, w.n_tok)
+    ret = v + wl.normal(12, 3, w.n_tok)
+    mask = w.tok_mask if masked else None
+    norm = [float(1000 + 37 * k) for k in range(w.K)] if with_norm else None
+    ctx = ub.Context(0, 1 << 20)
+    loss = torch.full((w.K,), 7.0, device="cuda")
+    frac = torch.full((w.K,), 7.0, device="cuda")
+    tok = torch.full((w.n_tok,), 7.0, device="cuda")
+    dv = torch.full((w.n_tok,), 7.0, device="cuda")
+    ctx.value_loss_fwd_bwd(w.cu_seqlens.cuda(), w.inv_role.cuda(), w.role_model.tolist(), w.K,
+                           None if mask is None else mask.cuda(), v.cuda(), ov.cuda(), ret.cuda(), clip_v, norm, loss,
+                           frac, tok, dv)
+    ctx.check_status()
+    o = orc.value_loss_fwd_bwd(v.numpy(), ov.numpy(), ret.numpy(), w.cu_seqlens.numpy(), w.inv_role.numpy(),
+                               w.role_model.numpy(), None if mask is None else mask.numpy(), clip_v=clip_v, norm=norm,
+                               K=w.K)
+    assert np.all(np.abs(loss.cpu().numpy() - o["loss"]) <= pu.TOL_LOSS * np.abs(o["loss"]) + 1e-7)
+    assert np.abs(frac.cpu().numpy() - o["clip_frac"]).max() <= 1e-4
+    assert np.abs(tok.cpu().numpy() - o["tok_loss"]).max() <= 1e-5 * max(1.0, float(o["tok_loss"].max()))
+    # the branch is a comparison of two squares: where they agree to rounding either side may win, and the
+    # gradient jumps there; such tokens (a handful in a million) are compared against both branches
+    vd, ovd, rd = (x.numpy().astype(np.float64) for x in (v, ov, ret))
+    d = vd - ovd
+    vc = np.where(np.abs(d) <= clip_v, vd, ovd + np.sign(d) * clip_v)
+    su, sc = (vd - rd) ** 2, (vc - rd) ** 2
+    near = (np.abs(su - sc) <= 1e-5 * np.maximum(su, sc)) & (np.abs(d) > clip_v)
+    assert near.sum() <= 1e-4 * w.n_tok + 2
+    g = dv.cpu().numpy().astype(np.float64)
+    scale = np.abs(o["dvalues"]).max()
+    assert np.abs(g - o["dvalues"])[~near].max() <= 1e-5 * scale
+    keep = np.ones(w.n_tok, bool) if mask is None else mask.numpy() != 0
+    assert np.all(g[~keep] == 0) and np.all(tok.cpu().numpy()[~keep] == 0)
+    ctx.close()
+
+
 # ------------------------------------------------------------------------------------ stages 2 + 3
 
 def test_tiny_full():
