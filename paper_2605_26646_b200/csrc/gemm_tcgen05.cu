@@ -15,6 +15,12 @@
 //   warps 2..5  : epilogue      - each thread owns one accumulator row (one TMEM lane), drains it 32 columns at a
 //                                 time with tcgen05.ld while the MMAs already fill the other stage
 //
+// The fp32-accumulate epilogue also exists with 512-column tiles (template parameter NB = 2, CTA pairs only): two
+// N = 256 MMAs per K step fill all of tensor memory as ONE accumulator stage, so a K slab of A is loaded once for
+// twice the columns (a quarter less operand traffic from L2 and DRAM).  The epilogue then does not overlap the next
+// tile's MMAs, which is affordable only because these GEMMs contract over a whole gradient chunk (hundreds of K
+// slabs per tile); it adds into C with fire-and-forget vector reductions instead of load-add-store.
+//
 // Three epilogues share the main loop:
 //   softmax statistics : running (max, sum exp, sum exp*z, target logit) per row across a sweep of vocabulary
 //                        tiles; nothing of size rows x vocabulary is ever written
@@ -31,8 +37,7 @@ namespace unity {
 
 namespace {
 
-constexpr int kAccStages = 2;
-constexpr int kTmemCols = kAccStages * kTileN;            // 512: all of tensor memory
+constexpr int kTmemCols = 2 * kTileN;                     // 512: all of tensor memory (two stages of 256 or one of 512)
 constexpr int kBarBytes = 256;
 constexpr int kThreads = 192;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -40,14 +45,16 @@ constexpr float kNegBig = -3.0e38f;
 // MN-major operands: a stage holds boxes of 64 rows x 64 K (8 KiB), one after the other.
 constexpr int kMnBoxBytes = 64 * kTileK * 2;
 
-template <int CTAS>
+template <int CTAS, int NB = 1>
 struct Cfg {
     static constexpr int kTileRows = kCtaM * CTAS;               // rows of one output tile (128 or 256)
-    static constexpr int kBRows = kTileN / CTAS;                 // rows of B this CTA loads (256 or 128)
+    static constexpr int kTileCols = kTileN * NB;                // columns of one output tile (256 or 512)
+    static constexpr int kAccStages = 2 / NB;                    // accumulator stages in tensor memory
+    static constexpr int kBRows = kTileN / CTAS;                 // rows of B this CTA loads per 256-column block
     static constexpr int kABytes = kCtaM * kTileK * 2;           // 16 KiB
-    static constexpr int kBBytes = kBRows * kTileK * 2;          // 32 or 16 KiB
-    static constexpr int kStageBytes = kABytes + kBBytes;        // 48 or 32 KiB
-    static constexpr int kStages = CTAS == 1 ? 4 : 7;
+    static constexpr int kBBytes = kBRows * kTileK * 2;          // 32 or 16 KiB per 256-column block
+    static constexpr int kStageBytes = kABytes + NB * kBBytes;   // 48 or 32 KiB
+    static constexpr int kStages = (CTAS == 1 || NB == 2) ? 4 : 7;
     static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kBarBytes;
 };
 
@@ -96,11 +103,13 @@ __device__ __forceinline__ unsigned pack_bf16(float lo, float hi) {
     return *reinterpret_cast<unsigned*>(&v);
 }
 
-template <int EPI, bool A_MN, bool B_MN, int CTAS>
+template <int EPI, bool A_MN, bool B_MN, int CTAS, int NB = 1>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs g) {
-    using C = Cfg<CTAS>;
-    constexpr int kStages = C::kStages, kStageBytes = C::kStageBytes, kABytes = C::kABytes;
+    using C = Cfg<CTAS, NB>;
+    constexpr int kStages = C::kStages, kStageBytes = C::kStageBytes, kABytes = C::kABytes, kBBytes = C::kBBytes;
+    constexpr int kAccStages = C::kAccStages, kTileCols = C::kTileCols;
+    static_assert(NB == 1 || (EPI == kEpiAccumF32 && CTAS == 2), "512-column tiles: fp32-accumulate epilogue, CTA pairs");
     extern __shared__ uint8_t smem_raw[];
     // the dynamic shared-memory window starts at the same offset in both CTAs of a pair, so all offsets below match
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -167,7 +176,7 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                 if (!valid) continue;
                 const int a_row = g.a_row0 + t.m_tile * C::kTileRows + static_cast<int>(cta_rank) * kCtaM;
                 for (int nt = t.n_begin; nt < t.n_end && ok; ++nt) {
-                    const int b_row = g.b_row0 + nt * kTileN + static_cast<int>(cta_rank) * C::kBRows;
+                    const int b_row = g.b_row0 + nt * kTileCols + static_cast<int>(cta_rank) * C::kBRows;
                     for (int k = 0; k < g.k_iters; ++k) {
                         if (!ptx::mbar_wait(&empty[stage], phase ^ 1, kWaitBudgetCycles) || *abort_flag) { ok = false; break; }
                         uint8_t* sA = smem + stage * kStageBytes;
@@ -181,13 +190,17 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                         } else {
                             ptx::tma_load_2d_on<CTAS>(sA, &tmA, bar, g.a_k0 + k * kTileK, a_row);
                         }
-                        if (B_MN) {
 #pragma unroll
-                            for (int j = 0; j < C::kBRows / 64; ++j)
-                                ptx::tma_load_2d_on<CTAS>(sA + kABytes + j * kMnBoxBytes, &tmB, bar, b_row + j * 64,
-                                                          g.b_k0 + k * kTileK);
-                        } else {
-                            ptx::tma_load_2d_on<CTAS>(sA + kABytes, &tmB, bar, g.b_k0 + k * kTileK, b_row);
+                        for (int nb = 0; nb < NB; ++nb) {          // one block of B rows per 256 output columns
+                            uint8_t* sB = sA + kABytes + nb * kBBytes;
+                            if (B_MN) {
+#pragma unroll
+                                for (int j = 0; j < C::kBRows / 64; ++j)
+                                    ptx::tma_load_2d_on<CTAS>(sB + j * kMnBoxBytes, &tmB, bar, b_row + nb * kTileN + j * 64,
+                                                              g.b_k0 + k * kTileK);
+                            } else {
+                                ptx::tma_load_2d_on<CTAS>(sB, &tmB, bar, g.b_k0 + k * kTileK, b_row + nb * kTileN);
+                            }
                         }
                         if (++stage == kStages) { stage = 0; phase ^= 1; }
                     }
@@ -214,7 +227,7 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                 for (int nt = t.n_begin; nt < t.n_end && ok; ++nt) {
                     if (!ptx::mbar_wait(&acc_empty[acc], acc_phase ^ 1, kWaitBudgetCycles) || *abort_flag) { ok = false; break; }
                     ptx::tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + acc * kTileN;
+                    const uint32_t d_tmem = tmem_base + acc * kTileCols;
                     for (int k = 0; k < g.k_iters; ++k) {
                         if (!ready && !ptx::mbar_wait(&full[stage], phase, kWaitBudgetCycles)) { ok = false; break; }
                         ptx::tc_fence_after();
@@ -229,9 +242,15 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                         // 16 rows x 128 B for an MN-major operand
                         constexpr uint32_t step_a = A_MN ? (16 * 128) >> 4 : 2;
                         constexpr uint32_t step_b = B_MN ? (16 * 128) >> 4 : 2;
+                        // the shared-memory descriptor counts addresses in 16-byte units
 #pragma unroll
-                        for (int kk = 0; kk < kTileK / 16; ++kk)
-                            ptx::mma_bf16_ss_on<CTAS>(d_tmem, da + step_a * kk, db + step_b * kk, idesc, (k | kk) != 0 ? 1u : 0u);
+                        for (int nb = 0; nb < NB; ++nb) {
+#pragma unroll
+                            for (int kk = 0; kk < kTileK / 16; ++kk)
+                                ptx::mma_bf16_ss_on<CTAS>(d_tmem + nb * kTileN, da + step_a * kk,
+                                                          db + static_cast<uint64_t>(nb * (kBBytes >> 4)) + step_b * kk, idesc,
+                                                          (k | kk) != 0 ? 1u : 0u);
+                        }
                         ptx::tc_commit_on<CTAS>(&empty[stage]);
                         stage = next_stage;
                         phase = next_phase;
@@ -276,10 +295,10 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
             for (int nt = t.n_begin; nt < t.n_end && ok; ++nt) {
                 if (!ptx::mbar_wait(&acc_full[acc], acc_phase, kWaitBudgetCycles) || *abort_flag) { ok = false; break; }
                 ptx::tc_fence_after();
-                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kTileN;
-                const int col0 = nt * kTileN;
+                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kTileCols;
+                const int col0 = nt * kTileCols;
 #pragma unroll 1
-                for (int c = 0; c < kTileN / 32; ++c) {
+                for (int c = 0; c < kTileCols / 32; ++c) {
                     const int cbase = col0 + c * 32;
                     if (cbase >= g.n_cols) break;               // uniform across the CTA
                     uint32_t rr[32];
@@ -349,6 +368,12 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                             for (int q = 0; q < 8; ++q) {
                                 if (q * 4 < n_here) {
                                     float4 o = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                                    if (NB == 2 && g.beta) {
+                                        // one owner per element per launch and launches are stream-ordered, so the
+                                        // sum is the same single rounded addition as load-add-store
+                                        ptx::red_add_v4_f32(dst + q * 4, o);
+                                        continue;
+                                    }
                                     if (g.beta) {
                                         const float4 old = *reinterpret_cast<const float4*>(dst + q * 4);
                                         o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
@@ -392,19 +417,19 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
 }
 
 
-template <int EPI, bool A_MN, bool B_MN, int CTAS>
+template <int EPI, bool A_MN, bool B_MN, int CTAS, int NB = 1>
 cudaError_t set_attr() {
-    return cudaFuncSetAttribute(k_gemm<EPI, A_MN, B_MN, CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                Cfg<CTAS>::kSmemBytes);
+    return cudaFuncSetAttribute(k_gemm<EPI, A_MN, B_MN, CTAS, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                Cfg<CTAS, NB>::kSmemBytes);
 }
 
-template <int EPI, bool A_MN, bool B_MN, int CTAS>
+template <int EPI, bool A_MN, bool B_MN, int CTAS, int NB = 1>
 cudaError_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args, int workers, cudaStream_t stream) {
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(workers * CTAS, 1, 1);
     cfg.blockDim = dim3(kThreads, 1, 1);
-    cfg.dynamicSmemBytes = Cfg<CTAS>::kSmemBytes;
+    cfg.dynamicSmemBytes = Cfg<CTAS, NB>::kSmemBytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -413,7 +438,7 @@ cudaError_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArg
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, k_gemm<EPI, A_MN, B_MN, CTAS>, tmA, tmB, args);
+    return cudaLaunchKernelEx(&cfg, k_gemm<EPI, A_MN, B_MN, CTAS, NB>, tmA, tmB, args);
 }
 
 }  // namespace
@@ -427,10 +452,13 @@ cudaError_t gemm_set_attributes() {
     if ((e = set_attr<kEpiAccumF32, false, true, 1>()) != cudaSuccess) return e;
     if ((e = set_attr<kEpiAccumF32, false, true, 2>()) != cudaSuccess) return e;
     if ((e = set_attr<kEpiAccumF32, true, true, 1>()) != cudaSuccess) return e;
-    return set_attr<kEpiAccumF32, true, true, 2>();
+    if ((e = set_attr<kEpiAccumF32, true, true, 2>()) != cudaSuccess) return e;
+    if ((e = set_attr<kEpiAccumF32, false, true, 2, 2>()) != cudaSuccess) return e;
+    return set_attr<kEpiAccumF32, true, true, 2, 2>();
 }
 
 int gemm_tile_rows(int ctas) { return kCtaM * ctas; }
+int gemm_tile_cols(bool wide) { return wide ? 2 * kTileN : kTileN; }
 
 namespace {
 // workers and rounds of a launch (must mirror next_unit and launch_gemm)
@@ -461,7 +489,7 @@ unsigned gemm_round_arrivals(GemmEpilogue epi, int ctas, const GemmArgs& args, i
 }
 
 cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, int ctas, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                        const GemmArgs& args, int sm_count, cudaStream_t stream) {
+                        const GemmArgs& args, int sm_count, cudaStream_t stream, bool wide) {
     // softmax: one round handles group_m row tiles x n_splits; other epilogues: plain striding over all tiles
     const long long units = epi == kEpiSoftmaxStats
                                 ? static_cast<long long>(args.group_m < args.m_tiles ? args.group_m : args.m_tiles) * args.n_splits
@@ -478,6 +506,9 @@ cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, int ctas, const CUtensorMap
             return two ? launch<kEpiLogitGrad, false, false, 2>(tmA, tmB, args, workers, stream)
                        : launch<kEpiLogitGrad, false, false, 1>(tmA, tmB, args, workers, stream);
         default:   // fp32 accumulate: B is always MN-major (W or hidden read in place), A is G either way round
+            if (wide && two)
+                return a_mn ? launch<kEpiAccumF32, true, true, 2, 2>(tmA, tmB, args, workers, stream)
+                            : launch<kEpiAccumF32, false, true, 2, 2>(tmA, tmB, args, workers, stream);
             if (a_mn)
                 return two ? launch<kEpiAccumF32, true, true, 2>(tmA, tmB, args, workers, stream)
                            : launch<kEpiAccumF32, true, true, 1>(tmA, tmB, args, workers, stream);

@@ -66,11 +66,13 @@ struct GemmArgs {
 // a_row0 / b_row0 index the contiguous dimension of its tensor map and a_k0 / b_k0 its rows.
 // ctas: 1 = one CTA per 128 x 256 tile, 2 = a CTA pair per 256 x 256 tile; args.m_tiles counts tiles of
 // gemm_tile_rows(ctas) rows.
+// wide: 512-column output tiles (kEpiAccumF32 with ctas = 2 only); args.n_tiles then counts tiles of 512 columns.
 cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, int ctas, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                        const GemmArgs& args, int sm_count, cudaStream_t stream);
+                        const GemmArgs& args, int sm_count, cudaStream_t stream, bool wide = false);
 // Arrivals the launch adds to args.round_counter (rounds x workers); 0 when nothing is launched.
 unsigned gemm_round_arrivals(GemmEpilogue epi, int ctas, const GemmArgs& args, int sm_count);
 int gemm_tile_rows(int ctas);
+int gemm_tile_cols(bool wide);
 cudaError_t gemm_set_attributes();
 
 // ----------------------------------------------------------------------------------------------

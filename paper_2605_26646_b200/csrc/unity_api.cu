@@ -32,11 +32,12 @@ struct unity_ctx {
     size_t ev_used;                 // events handed out since the last unity_get_profile
     int ctas[UNITY_PROF_CLASSES];   // per GEMM class: 1 = single CTA per tile, 2 = CTA pair per tile
     int l2_promotion;               // tensor-map L2 promotion: 0 none, 1 64 B, 2 128 B, 3 256 B
-    int chunk_group;                // raster group of the chunk GEMMs, in 128-row tiles
+    int chunk_group[3];             // raster group of the recompute / dHidden / dW chunk GEMMs, in 128-row tiles
     int chunk_rows_mult, chunk_vocab_mult;   // gradient chunk = mult x 18944 rows / vocabulary entries
     int fwd_group;                  // row tiles (128 rows) per round of the forward kernel; 0 = a quarter of the SMs
     int fwd_sync;                   // 1: workers of the forward kernel meet (softly) at every round start
     int chunk_sync;                 // bit 0: same for the recompute GEMM, bit 1: dHidden GEMM, bit 2: dW GEMM
+    int wide_acc;                   // 1: dHidden / dW chunk GEMMs use 512-column tiles (CTA pairs only)
     unsigned round_total;           // arrivals accumulated so far on the rendezvous counter (d_status + 16)
 };
 
@@ -355,12 +356,13 @@ int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace
     c->ctas[UNITY_PROF_DH_GEMM] = 2;
     c->ctas[UNITY_PROF_DW_GEMM] = 2;
     c->l2_promotion = 3;
-    c->chunk_group = 24;
+    c->chunk_group[0] = c->chunk_group[1] = c->chunk_group[2] = 32;
     c->fwd_group = 0;
     c->fwd_sync = 1;
     c->chunk_sync = 6;
     c->chunk_rows_mult = 1;
     c->chunk_vocab_mult = 1;
+    c->wide_acc = 1;
     c->ev_pool = new (std::nothrow) std::vector<cudaEvent_t>();
     c->ev_class = new (std::nothrow) std::vector<int>();
     if (cudaMalloc(&c->d_status, 256) != cudaSuccess || cudaMallocHost(&c->h_pinned, 4096) != cudaSuccess ||
@@ -425,12 +427,20 @@ int unity_set_option(unity_ctx* ctx, int option, int value) {
         return UNITY_OK;
     }
     if (option == UNITY_OPT_L2_PROMOTION && value >= 0 && value <= 3) { ctx->l2_promotion = value; return UNITY_OK; }
-    if (option == UNITY_OPT_CHUNK_GROUP && value >= 2 && value <= 148) { ctx->chunk_group = value; return UNITY_OK; }
+    if (option == UNITY_OPT_CHUNK_GROUP && value >= 2 && value <= 148) {
+        ctx->chunk_group[0] = ctx->chunk_group[1] = ctx->chunk_group[2] = value;
+        return UNITY_OK;
+    }
+    if (option >= UNITY_OPT_GROUP_GRAD && option <= UNITY_OPT_GROUP_DW && value >= 2 && value <= 148) {
+        ctx->chunk_group[option - UNITY_OPT_GROUP_GRAD] = value;
+        return UNITY_OK;
+    }
     if (option == UNITY_OPT_FWD_SYNC && (value == 0 || value == 1)) { ctx->fwd_sync = value; return UNITY_OK; }
     if (option == UNITY_OPT_CHUNK_SYNC && value >= 0 && value <= 7) { ctx->chunk_sync = value; return UNITY_OK; }
     if (option == UNITY_OPT_FWD_GROUP && value >= 0 && value <= 148) { ctx->fwd_group = value; return UNITY_OK; }
     if (option == UNITY_OPT_CHUNK_ROWS && value >= 1 && value <= 8) { ctx->chunk_rows_mult = value; return UNITY_OK; }
     if (option == UNITY_OPT_CHUNK_VOCAB && value >= 1 && value <= 8) { ctx->chunk_vocab_mult = value; return UNITY_OK; }
+    if (option == UNITY_OPT_WIDE_ACC && (value == 0 || value == 1)) { ctx->wide_acc = value; return UNITY_OK; }
     return fail(ctx, UNITY_ERR_INVALID_ARG, "unknown option %d or value %d out of range", option, value);
 }
 
@@ -777,7 +787,10 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
         if ((rc = make_tmap(ctx, &tm_hp_k, L.hp, H, P.n_slots, static_cast<uint64_t>(H) * 2, kBoxRows))) return rc;
         if ((rc = make_tmap(ctx, &tm_hp_mn, L.hp, H, P.n_slots, static_cast<uint64_t>(H) * 2, kTileK))) return rc;
     }
-    const int h_tiles = (H + kTileN - 1) / kTileN;
+    const bool wide_dh = ctx->wide_acc && ctx->ctas[UNITY_PROF_DH_GEMM] == 2;
+    const bool wide_dw = ctx->wide_acc && ctx->ctas[UNITY_PROF_DW_GEMM] == 2;
+    const int h_tiles_dh = (H + gemm_tile_cols(wide_dh) - 1) / gemm_tile_cols(wide_dh);
+    const int h_tiles_dw = (H + gemm_tile_cols(wide_dw) - 1) / gemm_tile_cols(wide_dw);
     const int c_grad = ctx->ctas[UNITY_PROF_GRAD_GEMM], c_dh = ctx->ctas[UNITY_PROF_DH_GEMM],
               c_dw = ctx->ctas[UNITY_PROF_DW_GEMM];
 
@@ -805,7 +818,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 GemmArgs g;
                 memset(&g, 0, sizeof(g));
                 g.m_tiles = nc / gemm_tile_rows(c_grad); g.n_tiles = (vc + kTileN - 1) / kTileN; g.k_iters = H / kTileK;
-                g.group_m = ctx->chunk_group / c_grad > 0 ? ctx->chunk_group / c_grad : 1;
+                g.group_m = ctx->chunk_group[0] / c_grad > 0 ? ctx->chunk_group[0] / c_grad : 1;
                 g.a_row0 = slot0; g.b_row0 = v0; g.m_rows = nc; g.n_cols = vc;
                 g.target_p = L.target_p; g.vocab0 = v0; g.scale = rows->inv_temperature;
                 g.coef_a = L.coef_a; g.coef_b = L.coef_b; g.row_lse = L.row_lse; g.row_ent = L.row_ent;
@@ -826,8 +839,8 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 // (2) dH_chunk[nc, H] (+)= G[nc, vc] * W[v0:v0+vc, :]      (B = W, MN-major: rows v are K)
                 GemmArgs h;
                 memset(&h, 0, sizeof(h));
-                h.m_tiles = nc / gemm_tile_rows(c_dh); h.n_tiles = h_tiles; h.k_iters = (vc + kTileK - 1) / kTileK;
-                h.group_m = ctx->chunk_group / c_dh > 0 ? ctx->chunk_group / c_dh : 1;
+                h.m_tiles = nc / gemm_tile_rows(c_dh); h.n_tiles = h_tiles_dh; h.k_iters = (vc + kTileK - 1) / kTileK;
+                h.group_m = ctx->chunk_group[1] / c_dh > 0 ? ctx->chunk_group[1] / c_dh : 1;
                 h.a_row0 = 0; h.a_k0 = 0; h.b_row0 = 0; h.b_k0 = v0; h.m_rows = nc; h.n_cols = H;
                 h.C = L.dHc; h.ldc = H; h.beta = v0 > 0; h.status = ctx->d_status;
                 if (ctx->chunk_sync & 2) {
@@ -837,13 +850,13 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 }
                 {
                     ProfScope ps(ctx, UNITY_PROF_DH_GEMM);
-                    CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, false, c_dh, tm_G_k, tm_W_mn, h, ctx->sm_count, st));
+                    CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, false, c_dh, tm_G_k, tm_W_mn, h, ctx->sm_count, st, wide_dh));
                 }
                 // (3) dW[v0:v0+vc, :] (+)= G^T[vc, nc] * hidden[slot0:slot0+nc, :]   (both operands MN-major)
                 GemmArgs w;
                 memset(&w, 0, sizeof(w));
-                w.m_tiles = (vc + gemm_tile_rows(c_dw) - 1) / gemm_tile_rows(c_dw); w.n_tiles = h_tiles; w.k_iters = nc / kTileK;
-                w.group_m = ctx->chunk_group / c_dw > 0 ? ctx->chunk_group / c_dw : 1;
+                w.m_tiles = (vc + gemm_tile_rows(c_dw) - 1) / gemm_tile_rows(c_dw); w.n_tiles = h_tiles_dw; w.k_iters = nc / kTileK;
+                w.group_m = ctx->chunk_group[2] / c_dw > 0 ? ctx->chunk_group[2] / c_dw : 1;
                 w.a_row0 = 0; w.a_k0 = 0; w.b_row0 = 0; w.b_k0 = slot0; w.m_rows = vc; w.n_cols = H;
                 w.C = dWk + static_cast<long long>(v0) * H; w.ldc = H;
                 w.beta = (params->accumulate_dW || c0 > 0) ? 1 : 0; w.status = ctx->d_status;
@@ -854,7 +867,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 }
                 {
                     ProfScope ps(ctx, UNITY_PROF_DW_GEMM);
-                    CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, true, c_dw, tm_G_mn, tm_hp_mn, w, ctx->sm_count, st));
+                    CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, true, c_dw, tm_G_mn, tm_hp_mn, w, ctx->sm_count, st, wide_dw));
                 }
                 nl += 3;
             }

@@ -47,13 +47,15 @@ def check_ppo(g, o, w, atol_loss=1e-6):
     assert np.abs(gm - om).max() <= 1e-3 * max(1.0, np.abs(om[:, 1:]).max())
 
 
-def run_all_stages(w, ctas=None, **ppo_kw):
+def run_all_stages(w, ctas=None, options=(), **ppo_kw):
     d = pu.DeviceInputs(w)
     ctx = pu.make_ctx(w)
     try:
         if ctas is not None:                       # CTAs per output tile for the four GEMM classes
             for option, value in enumerate(ctas):
                 ctx.set_option(option, value)
+        for option, value in options:
+            ctx.set_option(option, value)
         ga, oa = pu.gpu_advantage(ctx, w, d), pu.oracle_advantage(w)
         assert np.abs(ga["adv_inv"].cpu().numpy() - oa["adv_inv"]).max() <= pu.TOL_ADV
         assert np.abs(ga["adv_tok"].cpu().numpy() - oa["adv_tok"]).max() <= pu.TOL_ADV
@@ -267,6 +269,14 @@ def test_single_cta_and_cta_pair_kernels(ctas):
     # every GEMM class exists as a one-CTA kernel (128-row tiles) and as a CTA-pair kernel (256-row tiles)
     run_all_stages(small_workload(320, 2048 + 264, 700), ctas=ctas)
     run_all_stages(wl.make("tiny", device="cuda"), ctas=ctas)
+
+
+@pytest.mark.parametrize("wide", [0, 1])
+def test_accumulate_gemms_with_256_and_512_column_tiles(wide):
+    # the dHidden / dW chunk GEMMs of CTA pairs exist with 256 x 256 tiles (two accumulator stages) and with
+    # 256 x 512 tiles (one stage, reductions into C); H = 320 and 832 leave ragged column tails in both
+    for H, V, rows in [(320, 2048 + 264, 700), (832, 1536, 300)]:
+        run_all_stages(small_workload(H, V, rows), ctas=(2, 2, 2, 2), options=[(11, wide)])
 
 
 @pytest.mark.parametrize("kl_mode,ent_coef,clip", [(1, 0.0, (0.2, 0.2)), (2, 0.01, (0.1, 0.3)), (3, 0.02, (0.2, 0.28))])
