@@ -58,6 +58,8 @@ int unity_destroy(unity_ctx* ctx);
  * workspace still works down to unity_workspace_min_bytes (smaller gradient chunks). */
 size_t unity_workspace_bytes(int64_t n_tok, int32_t H, int32_t V, int32_t K, int32_t n_inv);
 size_t unity_workspace_min_bytes(int64_t n_tok, int32_t H, int32_t V, int32_t K, int32_t n_inv);
+/* Scratch bytes that leave room for the logit stash of UNITY_OPT_LOGIT_STASH. */
+size_t unity_workspace_bytes_stash(int64_t n_tok, int32_t H, int32_t V, int32_t K, int32_t n_inv);
 
 /* Synchronise the stream, return the sticky device status (UNITY_OK, UNITY_ERR_BAD_INDEX,
  * UNITY_ERR_TIMEOUT or UNITY_ERR_CUDA) and clear it. */
@@ -97,6 +99,12 @@ int unity_set_profiling(unity_ctx* ctx, int enable);
 #define UNITY_OPT_GROUP_GRAD 12   /* raster group of the recompute GEMM alone, in 128-row tiles                           */
 #define UNITY_OPT_GROUP_DH 13     /* ... of the dHidden GEMM                                                               */
 #define UNITY_OPT_GROUP_DW 14     /* ... of the dW GEMM                                                                    */
+#define UNITY_OPT_LOGIT_STASH 15  /* 0 (default): the backward recomputes the logits per vocabulary chunk.  1: the loss call
+                                     runs its forward block by block of 18432 rows and keeps the block's scaled logits in
+                                     bf16 (rows x V, about 6 GB at V = 152064, sized by unity_workspace_bytes_stash); the
+                                     backward turns them into dL/dz in place.  Executed work drops from 8 to 6 H V flop per
+                                     token; the full n_tok x V logits still never exist.  Ignored (recompute) when the
+                                     workspace has no room or the on-policy shortcut is used. */
 int unity_set_option(unity_ctx* ctx, int option, int value);
 int unity_get_profile(unity_ctx* ctx, double* ms, int64_t* launches);
 

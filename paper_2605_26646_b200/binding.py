@@ -24,6 +24,7 @@ UNITY_MAX_ROLES = 64
 UNITY_N_METRICS = 8
 
 EXPORTS = ["unity_create", "unity_destroy", "unity_workspace_bytes", "unity_workspace_min_bytes",
+           "unity_workspace_bytes_stash",
            "unity_check_status", "unity_last_error", "unity_launch_count", "unity_set_profiling",
            "unity_get_profile", "unity_set_option", "unity_role_advantage", "unity_reward_assembly", "unity_gae", "unity_value_loss_fwd_bwd",
            "unity_ready_batch_plan", "unity_ready_batch_gather", "unity_align_rewards",
@@ -83,7 +84,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.unity_create.restype = C.c_int
     lib.unity_destroy.argtypes = [vp]
     lib.unity_destroy.restype = C.c_int
-    for fn in (lib.unity_workspace_bytes, lib.unity_workspace_min_bytes):
+    for fn in (lib.unity_workspace_bytes, lib.unity_workspace_min_bytes, lib.unity_workspace_bytes_stash):
         fn.argtypes = [i64, i32, i32, i32, i32]
         fn.restype = C.c_size_t
     lib.unity_check_status.argtypes = [vp]
@@ -156,6 +157,13 @@ def unity_workspace_bytes(n_tok: int, H: int, V: int, K: int, n_inv: int) -> int
 
 def unity_workspace_min_bytes(n_tok: int, H: int, V: int, K: int, n_inv: int) -> int:
     return int(load_library().unity_workspace_min_bytes(n_tok, H, V, K, n_inv))
+
+
+def unity_workspace_bytes_stash(n_tok: int, H: int, V: int, K: int, n_inv: int) -> int:
+    return int(load_library().unity_workspace_bytes_stash(n_tok, H, V, K, n_inv))
+
+
+OPT_LOGIT_STASH = 15
 
 
 def unity_create(device: int, stream_ptr: int, workspace: torch.Tensor) -> C.c_void_p:

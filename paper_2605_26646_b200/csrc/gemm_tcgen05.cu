@@ -334,6 +334,23 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
 #pragma unroll
                             for (int j = 0; j < 32; ++j) if (j == jt) z_tgt = v[j];
                         }
+                        if (g.Z != nullptr && row_ok) {
+                            // keep the scaled logits of this bounded block of rows (bf16), grouped by vocabulary
+                            // chunk, for a backward pass that does not recompute them
+                            int zc = cbase / g.z_chunk_cols;
+                            zc = zc < g.z_chunks - 1 ? zc : g.z_chunks - 1;
+                            __nv_bfloat16* dst = g.Z + zc * g.z_chunk_stride + static_cast<long long>(row) * g.ldz +
+                                                 (cbase - zc * g.z_chunk_cols);
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                if (q * 8 < n_here)
+                                    *reinterpret_cast<uint4*>(dst + q * 8) = make_uint4(
+                                        pack_bf16(v[8 * q] * g.scale, v[8 * q + 1] * g.scale),
+                                        pack_bf16(v[8 * q + 2] * g.scale, v[8 * q + 3] * g.scale),
+                                        pack_bf16(v[8 * q + 4] * g.scale, v[8 * q + 5] * g.scale),
+                                        pack_bf16(v[8 * q + 6] * g.scale, v[8 * q + 7] * g.scale));
+                            }
+                        }
                     } else if (EPI == kEpiLogitGrad) {
                         // G = -p*(a + b*(z - lse + H)) (+ a at the target), z = scale*acc, p = exp(z - lse)
                         const float shift = -lse * kLog2e;

@@ -48,6 +48,10 @@ struct GemmArgs {
     const int* target_p;      // [rows] packed targets (global vocabulary index), indexed from a_row0 + row
     int vocab0;               // global vocabulary index of B row b_row0
     float scale;              // inv_temperature (softmax) / unused otherwise
+    __nv_bfloat16* Z;         // optional stash of the scaled logits (null = none): chunk zc holds columns
+    long long ldz;            //   [zc * z_chunk_cols, ...) of every row, row pitch ldz, chunks z_chunk_stride apart;
+    long long z_chunk_stride; //   the last of the z_chunks chunks also takes the columns beyond it
+    int z_chunk_cols, z_chunks;
     // kEpiLogitGrad
     const float* coef_a;      // [rows] dL/dlogp * scale, packed order
     const float* coef_b;      // [rows] dL/dentropy * scale
@@ -120,6 +124,7 @@ cudaError_t launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* targe
                                int H, __nv_bfloat16* hp, int* target_p, cudaStream_t stream);
 
 struct TokenArgs {
+    int slot_begin;            // k_finish_rows works on slots [slot_begin, n_slots)
     int n_slots, n_splits, K, n_roles, n_inv;
     long long n_tok;
     const float4* stats;       // per model: base stats_base[k], pitch = padded rows of the model
@@ -149,6 +154,20 @@ struct TokenArgs {
     float* metrics;            // [(K + n_roles) * 8] nullable
 };
 cudaError_t launch_finish_forward(const TokenArgs& a, bool with_loss, cudaStream_t stream, int* n_launches);
+// the two halves of the above: per-row terms for slots [a.slot_begin, a.n_slots), and the loss / metric reductions
+cudaError_t launch_finish_rows(const TokenArgs& a, bool with_loss, cudaStream_t stream, int* n_launches);
+cudaError_t launch_loss_reduce(const TokenArgs& a, cudaStream_t stream, int* n_launches);
+
+// In place, for a block of rows x cols (row pitch ld) of stashed scaled logits z: z <- dL/dz =
+// -p*(a + b*(z - lse + H)) (+ a at the target), p = exp(z - lse); per-row vectors are indexed from `row0`.
+struct LogitGradArgs {
+    __nv_bfloat16* Z;
+    long long ld;
+    int rows, cols, row0, vocab0;
+    const int* target_p;
+    const float *coef_a, *coef_b, *row_lse, *row_ent;
+};
+cudaError_t launch_logit_grad_inplace(const LogitGradArgs& a, cudaStream_t stream);
 
 cudaError_t launch_zero_masked_rows(const int* tok_slot, long long n_tok, int H, __nv_bfloat16* dHidden,
                                     cudaStream_t stream);

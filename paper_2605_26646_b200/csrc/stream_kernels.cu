@@ -321,7 +321,7 @@ __device__ __forceinline__ PpoTerms ppo_terms(float logp, float ent, float old_l
 
 // One thread per packed row: merge the vocabulary splits, form lse / entropy / logp, then the loss terms.
 __global__ void k_finish_rows(TokenArgs a, int with_loss) {
-    const int slot = blockIdx.x * blockDim.x + threadIdx.x;
+    const int slot = a.slot_begin + blockIdx.x * blockDim.x + threadIdx.x;
     if (slot >= a.n_slots) return;
     const int tok = a.slot_tok[slot];
     if (tok < 0) {
@@ -416,6 +416,34 @@ __global__ void k_class_reduce(TokenArgs a) {
         for (int j = 1; j < 8; ++j) m[j] = acc[j] / dn;
     }
     if (c < a.K) a.loss[c] = acc[8] / a.norm[c];
+}
+
+// Stashed logits -> logit gradients, in place.  A thread converts eight consecutive bf16 values (one 128-bit load and
+// store); a warp covers 512 contiguous bytes of a row.  Streaming: 2 B read + 2 B written per logit.
+__global__ void k_logit_grad_inplace(LogitGradArgs a) {
+    const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * 8;
+    if (c0 >= a.cols) return;
+    for (int r = blockIdx.y; r < a.rows; r += gridDim.y) {
+        const int slot = a.row0 + r;
+        const float ca = a.coef_a[slot], cb = a.coef_b[slot], lse = a.row_lse[slot];
+        const float hl = a.row_ent[slot] - lse;
+        const int tgt = a.target_p[slot] - a.vocab0;
+        uint4* ptr = reinterpret_cast<uint4*>(a.Z + static_cast<long long>(r) * a.ld + c0);
+        uint4 raw = *ptr;
+        __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&raw);
+        const float shift = -lse * 1.4426950408889634f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float2 z = __bfloat1622float2(h2[j]);
+            const float p0 = exp2f(fmaf(z.x, 1.4426950408889634f, shift));
+            const float p1 = exp2f(fmaf(z.y, 1.4426950408889634f, shift));
+            float g0 = -p0 * fmaf(cb, z.x + hl, ca), g1 = -p1 * fmaf(cb, z.y + hl, ca);
+            if (c0 + 2 * j == tgt) g0 += ca;
+            if (c0 + 2 * j + 1 == tgt) g1 += ca;
+            h2[j] = __floats2bfloat162_rn(g0, g1);
+        }
+        *ptr = raw;
+    }
 }
 
 __global__ void k_zero_masked_rows(const int* __restrict__ tok_slot, long long n_tok, int H,
@@ -633,19 +661,37 @@ cudaError_t launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* targe
     return cudaGetLastError();
 }
 
+cudaError_t launch_finish_rows(const TokenArgs& a, bool with_loss, cudaStream_t stream, int* n_launches) {
+    const int n = a.n_slots - a.slot_begin;
+    if (n > 0) {
+        k_finish_rows<<<(n + 255) / 256, 256, 0, stream>>>(a, with_loss ? 1 : 0);
+        *n_launches += 1;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_loss_reduce(const TokenArgs& a, cudaStream_t stream, int* n_launches) {
+    if (a.n_inv > 0) {
+        k_inv_reduce<<<(a.n_inv + 7) / 8, 256, 0, stream>>>(a);
+        *n_launches += 1;
+    }
+    k_class_reduce<<<(a.K + a.n_roles + 7) / 8, 256, 0, stream>>>(a);
+    *n_launches += 1;
+    return cudaGetLastError();
+}
+
 cudaError_t launch_finish_forward(const TokenArgs& a, bool with_loss, cudaStream_t stream, int* n_launches) {
-    if (a.n_slots > 0) {
-        k_finish_rows<<<(a.n_slots + 255) / 256, 256, 0, stream>>>(a, with_loss ? 1 : 0);
-        *n_launches += 1;
-    }
-    if (with_loss) {
-        if (a.n_inv > 0) {
-            k_inv_reduce<<<(a.n_inv + 7) / 8, 256, 0, stream>>>(a);
-            *n_launches += 1;
-        }
-        k_class_reduce<<<(a.K + a.n_roles + 7) / 8, 256, 0, stream>>>(a);
-        *n_launches += 1;
-    }
+    cudaError_t e = launch_finish_rows(a, with_loss, stream, n_launches);
+    if (e != cudaSuccess || !with_loss) return e;
+    return launch_loss_reduce(a, stream, n_launches);
+}
+
+cudaError_t launch_logit_grad_inplace(const LogitGradArgs& a, cudaStream_t stream) {
+    if (a.rows <= 0 || a.cols <= 0) return cudaSuccess;
+    // a block covers 2048 columns of one row; y walks the rows (grid-stride, the y extent is limited to 65535)
+    const unsigned gx = static_cast<unsigned>((a.cols + 2047) / 2048);
+    const unsigned gy = static_cast<unsigned>(a.rows < 32768 ? a.rows : 32768);
+    k_logit_grad_inplace<<<dim3(gx, gy), 256, 0, stream>>>(a);
     return cudaGetLastError();
 }
 

@@ -37,6 +37,7 @@ struct unity_ctx {
     int fwd_group;                  // row tiles (128 rows) per round of the forward kernel; 0 = a quarter of the SMs
     int fwd_sync;                   // 1: workers of the forward kernel meet (softly) at every round start
     int chunk_sync;                 // bit 0: same for the recompute GEMM, bit 1: dHidden GEMM, bit 2: dW GEMM
+    int logit_stash;                // 1: the loss call keeps the logits of one row block instead of recomputing them
     int wide_acc;                   // 1: dHidden / dW chunk GEMMs use 512-column tiles (CTA pairs only)
     unsigned round_total;           // arrivals accumulated so far on the rendezvous counter (d_status + 16)
 };
@@ -117,8 +118,9 @@ struct Layout {
 long long max_slots_of(long long n_tok, int K) { return static_cast<long long>(up(n_tok, kTileM)) + static_cast<long long>(kTileM) * K; }
 
 // Carve the workspace.  chunk_rows / chunk_vocab are the wanted gradient chunk sizes (0 = forward only).
+// z_chunks > 0: the G scratch holds that many vocabulary chunks side by side (the logit stash of one row block).
 Layout carve(char* base, size_t cap, long long n_tok, int H, int V, int K, int n_inv, int chunk_rows, int chunk_vocab,
-             bool* fits) {
+             bool* fits, int z_chunks = 0) {
     Layout L;
     memset(&L, 0, sizeof(L));
     Bump b{base, 0, cap, true};
@@ -143,7 +145,7 @@ Layout carve(char* base, size_t cap, long long n_tok, int H, int V, int K, int n
         L.coef_a = b.take<float>(L.max_slots);
         L.coef_b = b.take<float>(L.max_slots);
         L.inv_sums = b.take<float>(static_cast<size_t>(n_inv) * 9 + 1);
-        L.G = b.take<__nv_bfloat16>(static_cast<size_t>(chunk_rows) * chunk_vocab);
+        L.G = b.take<__nv_bfloat16>(static_cast<size_t>(chunk_rows) * chunk_vocab * (z_chunks > 0 ? z_chunks : 1));
         L.dHc = b.take<float>(static_cast<size_t>(chunk_rows) * H);
     }
     L.bytes = up(b.off, kAlign);
@@ -164,6 +166,23 @@ int wanted_chunk_vocab(int V, int mult = 1) {
     const long long want = static_cast<long long>(kChunkVocab) * mult + kTailTiles * kTileN;
     return static_cast<int>(vp < want ? vp : want);
 }
+
+// Regular width of a vocabulary chunk and the number of chunks: all chunks but the last are `base` wide, the last one
+// also takes a remainder of up to kTailTiles tiles (its width stays <= cv).
+void vocab_chunks(int V, int cv, int* base_out, int* n_out) {
+    const int tail = kTailTiles * kTileN;
+    const int base = (V > cv && cv > tail + kTileN) ? cv - tail : cv;
+    int n = 0;
+    for (int v0 = 0, vc = 0; v0 < V; v0 += vc, ++n) {
+        vc = V - v0 < base ? V - v0 : base;
+        if (V - (v0 + vc) <= tail && base < cv) vc = V - v0;
+    }
+    *base_out = base;
+    *n_out = n;
+}
+// Row block of the logit stash: 72 row tiles, so that the forward kernel's rounds (18 row tiles x 4 vocabulary splits
+// on 74 CTA pairs) are whole.
+constexpr int kStashRows = 72 * kTileM;
 
 // Tensor map over a row-major bf16 matrix [rows, inner]; boxes are 64 elements (128 B, one swizzle row) wide and
 // box_rows high.  K-major operands use box_rows = kBoxRows (128); MN-major operands use 64 (= kTileK).
@@ -216,6 +235,71 @@ struct RowPlan {
     int n_slots;
 };
 
+// Shape of one forward launch over `rows` packed rows (a multiple of the row tile): row tiles per round and
+// vocabulary splits.  One round of the persistent kernel = gm row tiles x splits vocabulary splits <= number of
+// workers (CTAs or CTA pairs): gm bounds the hidden rows that must stay L2 resident (a quarter of the workers, about
+// 4.7 k rows), splits fill the machine.
+void forward_shape(const unity_ctx* ctx, int V, int rows, int* gm_out, int* splits_out, int* tps_out) {
+    const int ctas = ctx->ctas[UNITY_PROF_FWD_GEMM];
+    const int m_tiles = rows / gemm_tile_rows(ctas);
+    const int n_tiles = (V + kTileN - 1) / kTileN;
+    const int n_pairs = ctx->sm_count / ctas;
+    int gmax = ctx->fwd_group > 0 ? ctx->fwd_group / ctas : n_pairs / 4;
+    if (gmax < 1) gmax = 1;
+    if (gmax > n_pairs) gmax = n_pairs;
+    const int n_grp = (m_tiles + gmax - 1) / gmax;
+    const int gm = n_grp > 0 ? (m_tiles + n_grp - 1) / n_grp : 1;
+    int splits = n_pairs / (gm > 0 ? gm : 1);
+    if (splits > 32) splits = 32;
+    if (splits > n_tiles) splits = n_tiles;
+    if (splits < 1) splits = 1;
+    const int tps = (n_tiles + splits - 1) / splits;
+    *gm_out = gm > 0 ? gm : 1;
+    *splits_out = (n_tiles + tps - 1) / tps;
+    *tps_out = tps;
+}
+int forward_splits(const unity_ctx* ctx, int V, int rows) {
+    int gm, splits, tps;
+    forward_shape(ctx, V, rows, &gm, &splits, &tps);
+    return splits;
+}
+
+// Optional stash of the scaled logits written by the forward kernel (see GemmArgs::Z).
+struct ZStash {
+    __nv_bfloat16* Z;
+    long long ldz, chunk_stride;
+    int chunk_cols, chunks;
+};
+
+// LM-head GEMM + online softmax statistics for packed rows [slot0, slot0 + rows) of one model; statistics go to
+// stats[split * rows + (slot - slot0)].
+int launch_forward(unity_ctx* ctx, const unity_rows* r, int slot0, int rows, float4* stats, const int* target_p,
+                   const CUtensorMap& tmA, const CUtensorMap& tmB, const ZStash* z, int* splits_out) {
+    const int ctas = ctx->ctas[UNITY_PROF_FWD_GEMM];
+    int gm, splits, tps;
+    forward_shape(ctx, r->V, rows, &gm, &splits, &tps);
+    *splits_out = splits;
+    GemmArgs g;
+    memset(&g, 0, sizeof(g));
+    g.m_tiles = rows / gemm_tile_rows(ctas); g.n_tiles = (r->V + kTileN - 1) / kTileN; g.k_iters = r->H / kTileK;
+    g.group_m = gm;
+    g.a_row0 = slot0; g.b_row0 = 0; g.a_k0 = 0; g.b_k0 = 0;
+    g.m_rows = rows; g.n_cols = r->V;
+    g.n_splits = splits; g.tiles_per_split = tps;
+    g.stats = stats; g.stats_pitch = rows;
+    g.target_p = target_p; g.vocab0 = 0; g.scale = r->inv_temperature;
+    g.status = ctx->d_status;
+    if (z) { g.Z = z->Z; g.ldz = z->ldz; g.z_chunk_stride = z->chunk_stride; g.z_chunk_cols = z->chunk_cols; g.z_chunks = z->chunks; }
+    if (ctx->fwd_sync) {
+        g.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
+        g.round_base = ctx->round_total;
+        ctx->round_total += gemm_round_arrivals(kEpiSoftmaxStats, ctas, g, ctx->sm_count);
+    }
+    ProfScope ps(ctx, UNITY_PROF_FWD_GEMM);
+    CUDA_TRY(ctx, launch_gemm(kEpiSoftmaxStats, false, ctas, tmA, tmB, g, ctx->sm_count, ctx->stream));
+    return UNITY_OK;
+}
+
 // Routing, packing and the forward sweep: fills per-split softmax statistics for every packed row.
 int forward_sweep(unity_ctx* ctx, const unity_rows* r, RowPlan& P, bool run_gemm = true) {
     const Layout& L = P.L;
@@ -245,62 +329,25 @@ int forward_sweep(unity_ctx* ctx, const unity_rows* r, RowPlan& P, bool run_gemm
                                      r->H, L.hp, L.target_p, st));
     nl += P.n_slots > 0;
 
-    const int ctas = ctx->ctas[UNITY_PROF_FWD_GEMM];
-    const int tile_rows = gemm_tile_rows(ctas);
     CUtensorMap tmA;
     if (P.n_slots > 0) {
         int rc = make_tmap(ctx, &tmA, L.hp, r->H, P.n_slots, static_cast<uint64_t>(r->H) * 2, kBoxRows);
         if (rc) return rc;
     }
-    const int n_tiles = (r->V + kTileN - 1) / kTileN;
     long long sbase = 0;
     for (int k = 0; k < r->K; ++k) {
         P.splits[k] = 1;
         P.stats_base[k] = sbase;
         const int rows_k = P.offsets[k + 1] - P.offsets[k];
         if (rows_k == 0 || !run_gemm) continue;
-        const int m_tiles = rows_k / tile_rows;
-        // One round of the persistent kernel = gm row tiles x splits vocabulary splits <= number of workers (CTAs
-        // or CTA pairs): gm bounds the hidden rows that must stay L2 resident (a quarter of the workers, about
-        // 4.7 k rows), splits fill the machine.
-        const int n_pairs = ctx->sm_count / ctas;
-        int gmax = ctx->fwd_group > 0 ? ctx->fwd_group / ctas : n_pairs / 4;
-        if (gmax < 1) gmax = 1;
-        if (gmax > n_pairs) gmax = n_pairs;
-        const int n_grp = (m_tiles + gmax - 1) / gmax;
-        const int gm = (m_tiles + n_grp - 1) / n_grp;
-        int splits = n_pairs / gm;
-        if (splits > 32) splits = 32;
-        if (splits > n_tiles) splits = n_tiles;
-        if (splits < 1) splits = 1;
-        const int tps = (n_tiles + splits - 1) / splits;
-        splits = (n_tiles + tps - 1) / tps;
-        P.splits[k] = splits;
-        sbase += static_cast<long long>(splits) * rows_k;
-        if (sbase > L.stats_cap) return fail(ctx, UNITY_ERR_WORKSPACE, "internal: statistics scratch too small");
-
         CUtensorMap tmB;
-        int rc = make_tmap(ctx, &tmB, r->W[k], r->H, r->V, static_cast<uint64_t>(r->H) * 2, kTileN / ctas);
+        int rc = make_tmap(ctx, &tmB, r->W[k], r->H, r->V, static_cast<uint64_t>(r->H) * 2, kTileN / ctx->ctas[UNITY_PROF_FWD_GEMM]);
         if (rc) return rc;
-        GemmArgs g;
-        memset(&g, 0, sizeof(g));
-        g.m_tiles = m_tiles; g.n_tiles = n_tiles; g.k_iters = r->H / kTileK;
-        g.group_m = gm;
-        g.a_row0 = P.offsets[k]; g.b_row0 = 0; g.a_k0 = 0; g.b_k0 = 0;
-        g.m_rows = rows_k; g.n_cols = r->V;
-        g.n_splits = splits; g.tiles_per_split = tps;
-        g.stats = L.stats + P.stats_base[k]; g.stats_pitch = rows_k;
-        g.target_p = L.target_p; g.vocab0 = 0; g.scale = r->inv_temperature;
-        g.status = ctx->d_status;
-        if (ctx->fwd_sync) {
-            g.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
-            g.round_base = ctx->round_total;
-            ctx->round_total += gemm_round_arrivals(kEpiSoftmaxStats, ctas, g, ctx->sm_count);
-        }
-        {
-            ProfScope ps(ctx, UNITY_PROF_FWD_GEMM);
-            CUDA_TRY(ctx, launch_gemm(kEpiSoftmaxStats, false, ctas, tmA, tmB, g, ctx->sm_count, st));
-        }
+        if (sbase + static_cast<long long>(forward_splits(ctx, r->V, rows_k)) * rows_k > L.stats_cap)
+            return fail(ctx, UNITY_ERR_WORKSPACE, "internal: statistics scratch too small");
+        rc = launch_forward(ctx, r, P.offsets[k], rows_k, L.stats + sbase, L.target_p, tmA, tmB, nullptr, &P.splits[k]);
+        if (rc) return rc;
+        sbase += static_cast<long long>(P.splits[k]) * rows_k;
         nl += 1;
     }
     ctx->launches += nl;
@@ -363,6 +410,7 @@ int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace
     c->chunk_rows_mult = 1;
     c->chunk_vocab_mult = 1;
     c->wide_acc = 1;
+    c->logit_stash = 0;
     c->ev_pool = new (std::nothrow) std::vector<cudaEvent_t>();
     c->ev_class = new (std::nothrow) std::vector<int>();
     if (cudaMalloc(&c->d_status, 256) != cudaSuccess || cudaMallocHost(&c->h_pinned, 4096) != cudaSuccess ||
@@ -393,6 +441,18 @@ int unity_destroy(unity_ctx* ctx) {
 size_t unity_workspace_bytes(int64_t n_tok, int32_t H, int32_t V, int32_t K, int32_t n_inv) {
     if (n_tok < 0 || H <= 0 || V <= 0 || K <= 0 || n_inv < 0) return 0;
     return carve(nullptr, ~size_t(0), n_tok, H, V, K, n_inv, wanted_chunk_rows(n_tok, K), wanted_chunk_vocab(V), nullptr).bytes;
+}
+
+size_t unity_workspace_bytes_stash(int64_t n_tok, int32_t H, int32_t V, int32_t K, int32_t n_inv) {
+    if (n_tok < 0 || H <= 0 || V <= 0 || K <= 0 || n_inv < 0) return 0;
+    int cr = wanted_chunk_rows(n_tok, K);
+    if (cr > kStashRows) cr = kStashRows;
+    const int cv = wanted_chunk_vocab(V);
+    int base, n;
+    vocab_chunks(V, cv, &base, &n);
+    const size_t a = carve(nullptr, ~size_t(0), n_tok, H, V, K, n_inv, cr, cv, nullptr, n).bytes;
+    const size_t b = unity_workspace_bytes(n_tok, H, V, K, n_inv);
+    return a > b ? a : b;
 }
 
 size_t unity_workspace_min_bytes(int64_t n_tok, int32_t H, int32_t V, int32_t K, int32_t n_inv) {
@@ -440,6 +500,7 @@ int unity_set_option(unity_ctx* ctx, int option, int value) {
     if (option == UNITY_OPT_FWD_GROUP && value >= 0 && value <= 148) { ctx->fwd_group = value; return UNITY_OK; }
     if (option == UNITY_OPT_CHUNK_ROWS && value >= 1 && value <= 8) { ctx->chunk_rows_mult = value; return UNITY_OK; }
     if (option == UNITY_OPT_CHUNK_VOCAB && value >= 1 && value <= 8) { ctx->chunk_vocab_mult = value; return UNITY_OK; }
+    if (option == UNITY_OPT_LOGIT_STASH && (value == 0 || value == 1)) { ctx->logit_stash = value; return UNITY_OK; }
     if (option == UNITY_OPT_WIDE_ACC && (value == 0 || value == 1)) { ctx->wide_acc = value; return UNITY_OK; }
     return fail(ctx, UNITY_ERR_INVALID_ARG, "unknown option %d or value %d out of range", option, value);
 }
@@ -730,11 +791,28 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
     CUDA_TRY(ctx, cudaSetDevice(ctx->device));
     cudaStream_t st = ctx->stream;
 
+    // On-policy shortcut: when the caller hands in logp / entropy / lse of THESE weights on THESE rows (from
+    // unity_logprob_fwd), the forward sweep over the vocabulary is skipped; the backward still recomputes the logits.
+    const bool have_fwd = params->logp_in && params->entropy_in && params->lse_in;
+    if (!have_fwd && (params->logp_in || params->entropy_in || params->lse_in))
+        return fail(ctx, UNITY_ERR_INVALID_ARG, "logp_in, entropy_in and lse_in must be given together");
+
     // choose gradient chunk sizes that fit the workspace
     int cr = wanted_chunk_rows(rows->n_tok, K, ctx->chunk_rows_mult), cv = wanted_chunk_vocab(V, ctx->chunk_vocab_mult);
     RowPlan P;
     bool fits = false;
-    while (true) {
+    // Logit stash: the forward runs block by block of rows and keeps the block's scaled logits (bf16, one slab per
+    // vocabulary chunk); the backward turns each slab into dL/dz in place instead of recomputing the logits.
+    bool stash = ctx->logit_stash && !have_fwd;
+    int z_base = 0, z_chunks = 0;
+    if (stash) {
+        const int cr_s = cr < kStashRows ? cr : kStashRows, cv_s = wanted_chunk_vocab(V);
+        vocab_chunks(V, cv_s, &z_base, &z_chunks);
+        P.L = carve(ctx->ws, ctx->ws_bytes, rows->n_tok, H, V, K, rows->n_inv, cr_s, cv_s, &fits, z_chunks);
+        if (fits) { cr = cr_s; cv = cv_s; }
+        else stash = false;                     // workspace without room for the stash: recompute instead
+    }
+    while (!stash) {
         P.L = carve(ctx->ws, ctx->ws_bytes, rows->n_tok, H, V, K, rows->n_inv, cr, cv, &fits);
         if (fits) break;
         if (cr > kMinChunkRows && cr >= cv) cr = static_cast<int>(up(cr / 2, kTileM));
@@ -755,12 +833,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
     if (entropy) CUDA_TRY(ctx, cudaMemsetAsync(entropy, 0, sizeof(float) * rows->n_tok, st));
     if (tok_loss) CUDA_TRY(ctx, cudaMemsetAsync(tok_loss, 0, sizeof(float) * rows->n_tok, st));
 
-    // On-policy shortcut: when the caller hands in logp / entropy / lse of THESE weights on THESE rows (from
-    // unity_logprob_fwd), the forward sweep over the vocabulary is skipped; the backward still recomputes the logits.
-    const bool have_fwd = params->logp_in && params->entropy_in && params->lse_in;
-    if (!have_fwd && (params->logp_in || params->entropy_in || params->lse_in))
-        return fail(ctx, UNITY_ERR_INVALID_ARG, "logp_in, entropy_in and lse_in must be given together");
-    rc = forward_sweep(ctx, rows, P, !have_fwd);
+    rc = forward_sweep(ctx, rows, P, !have_fwd && !stash);
     if (rc) return rc;
     int nl = 0;
 
@@ -775,7 +848,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
         t.norm[k] = params->norm ? params->norm[k] : static_cast<float>(P.counts[k] > 0 ? P.counts[k] : 1);
     t.coef_a = L.coef_a; t.coef_b = L.coef_b; t.tok_loss = tok_loss;
     t.inv_sums = L.inv_sums; t.loss = loss; t.metrics = metrics;
-    CUDA_TRY(ctx, launch_finish_forward(t, true, st, &nl));
+    if (!stash) CUDA_TRY(ctx, launch_finish_forward(t, true, st, &nl));
 
     __nv_bfloat16* dH = static_cast<__nv_bfloat16*>(dHidden);
     CUDA_TRY(ctx, launch_zero_masked_rows(L.tok_slot, rows->n_tok, H, dH, st));
@@ -802,18 +875,33 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
             continue;
         }
         const __nv_bfloat16* Wk = static_cast<const __nv_bfloat16*>(rows->W[k]);
-        CUtensorMap tm_W_k, tm_W_mn;
+        CUtensorMap tm_W_k, tm_W_mn, tm_W_f;
         if ((rc = make_tmap(ctx, &tm_W_k, Wk, H, V, static_cast<uint64_t>(H) * 2, kTileN / c_grad))) return rc;
+        if (stash && (rc = make_tmap(ctx, &tm_W_f, Wk, H, V, static_cast<uint64_t>(H) * 2, kTileN / ctx->ctas[UNITY_PROF_FWD_GEMM]))) return rc;
         if ((rc = make_tmap(ctx, &tm_W_mn, Wk, H, V, static_cast<uint64_t>(H) * 2, kTileK))) return rc;
 
         for (int c0 = 0; c0 < rows_k; c0 += cr) {
             const int nc = rows_k - c0 < cr ? rows_k - c0 : cr;          // multiple of kTileM
             const int slot0 = P.offsets[k] + c0;
+            if (stash) {
+                // forward over this block of rows, keeping its logits; then the per-row loss terms of the block
+                const ZStash z{L.G, cv, static_cast<long long>(cr) * cv, z_base, z_chunks};
+                int splits = 1;
+                if ((rc = launch_forward(ctx, rows, slot0, nc, L.stats, L.target_p, tm_hp_k, tm_W_f, &z, &splits))) return rc;
+                TokenArgs tc = t;
+                tc.slot_begin = slot0; tc.n_slots = slot0 + nc;
+                tc.offsets[k] = slot0; tc.offsets[k + 1] = slot0 + nc;
+                tc.stats_base[k] = 0; tc.model_splits[k] = splits;
+                CUDA_TRY(ctx, launch_finish_rows(tc, true, st, &nl));
+                nl += 1;
+            }
             const int tail = kTailTiles * kTileN;
             const int base = (V > cv && cv > tail + kTileN) ? cv - tail : cv;      // regular chunk width
-            for (int v0 = 0, vc = 0; v0 < V; v0 += vc) {
+            int ci = 0;
+            for (int v0 = 0, vc = 0; v0 < V; v0 += vc, ++ci) {
                 vc = V - v0 < base ? V - v0 : base;
                 if (V - (v0 + vc) <= tail && base < cv) vc = V - v0;               // absorb a short remainder
+                __nv_bfloat16* Gc = stash ? L.G + static_cast<long long>(ci) * cr * cv : L.G;
                 // (1) recompute the logits of this (rows x vocab) chunk and form dL/dz in bf16: G[nc, vc]
                 GemmArgs g;
                 memset(&g, 0, sizeof(g));
@@ -823,19 +911,27 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 g.target_p = L.target_p; g.vocab0 = v0; g.scale = rows->inv_temperature;
                 g.coef_a = L.coef_a; g.coef_b = L.coef_b; g.row_lse = L.row_lse; g.row_ent = L.row_ent;
                 g.G = L.G; g.ldg = cv; g.status = ctx->d_status;
-                if (ctx->chunk_sync & 1) {
+                if (!stash && (ctx->chunk_sync & 1)) {
                     g.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
                     g.round_base = ctx->round_total;
                     ctx->round_total += gemm_round_arrivals(kEpiLogitGrad, c_grad, g, ctx->sm_count);
                 }
-                {
+                if (stash) {
+                    LogitGradArgs lg;
+                    memset(&lg, 0, sizeof(lg));
+                    lg.Z = Gc; lg.ld = cv; lg.rows = nc; lg.cols = vc; lg.row0 = slot0; lg.vocab0 = v0;
+                    lg.target_p = L.target_p; lg.coef_a = L.coef_a; lg.coef_b = L.coef_b;
+                    lg.row_lse = L.row_lse; lg.row_ent = L.row_ent;
+                    ProfScope ps(ctx, UNITY_PROF_GRAD_GEMM);
+                    CUDA_TRY(ctx, launch_logit_grad_inplace(lg, st));
+                } else {
                     ProfScope ps(ctx, UNITY_PROF_GRAD_GEMM);
                     CUDA_TRY(ctx, launch_gemm(kEpiLogitGrad, false, c_grad, tm_hp_k, tm_W_k, g, ctx->sm_count, st));
                 }
                 // G viewed as [nc rows, vc]: K-major A for dHidden (contract over vc), MN-major A for dW (rows = K)
                 CUtensorMap tm_G_k, tm_G_mn;
-                if ((rc = make_tmap(ctx, &tm_G_k, L.G, vc, nc, static_cast<uint64_t>(cv) * 2, kBoxRows))) return rc;
-                if ((rc = make_tmap(ctx, &tm_G_mn, L.G, vc, nc, static_cast<uint64_t>(cv) * 2, kTileK))) return rc;
+                if ((rc = make_tmap(ctx, &tm_G_k, Gc, vc, nc, static_cast<uint64_t>(cv) * 2, kBoxRows))) return rc;
+                if ((rc = make_tmap(ctx, &tm_G_mn, Gc, vc, nc, static_cast<uint64_t>(cv) * 2, kTileK))) return rc;
                 // (2) dH_chunk[nc, H] (+)= G[nc, vc] * W[v0:v0+vc, :]      (B = W, MN-major: rows v are K)
                 GemmArgs h;
                 memset(&h, 0, sizeof(h));
@@ -875,6 +971,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
             nl += 1;
         }
     }
+    if (stash) CUDA_TRY(ctx, launch_loss_reduce(t, st, &nl));
     ctx->launches += nl;
     return UNITY_OK;
 }

@@ -25,9 +25,9 @@ def rel_fro(a: np.ndarray, b: np.ndarray) -> float:
     return num / den if den > 0 else num
 
 
-def make_ctx(w: wl.Workload, extra: int = 0) -> ub.Context:
-    need = ub.unity_workspace_bytes(w.n_tok, w.H, w.V, w.K, w.n_inv)
-    return ub.Context(0, need + extra)
+def make_ctx(w: wl.Workload, extra: int = 0, stash: bool = False) -> ub.Context:
+    size = ub.unity_workspace_bytes_stash if stash else ub.unity_workspace_bytes
+    return ub.Context(0, size(w.n_tok, w.H, w.V, w.K, w.n_inv) + extra)
 
 
 def dev(t, device="cuda"):

@@ -49,7 +49,7 @@ def check_ppo(g, o, w, atol_loss=1e-6):
 
 def run_all_stages(w, ctas=None, options=(), **ppo_kw):
     d = pu.DeviceInputs(w)
-    ctx = pu.make_ctx(w)
+    ctx = pu.make_ctx(w, stash=(ub.OPT_LOGIT_STASH, 1) in list(options))
     try:
         if ctas is not None:                       # CTAs per output tile for the four GEMM classes
             for option, value in enumerate(ctas):
@@ -277,6 +277,19 @@ def test_accumulate_gemms_with_256_and_512_column_tiles(wide):
     # 256 x 512 tiles (one stage, reductions into C); H = 320 and 832 leave ragged column tails in both
     for H, V, rows in [(320, 2048 + 264, 700), (832, 1536, 300)]:
         run_all_stages(small_workload(H, V, rows), ctas=(2, 2, 2, 2), options=[(11, wide)])
+
+
+@pytest.mark.parametrize("name", ["tiny", "rag_qa", "code", "stress"])
+def test_logit_stash_instead_of_recompute(name):
+    # the loss call keeps the scaled logits of a row block in bf16 and turns them into dL/dz in place; same outputs
+    # within the same tolerances (V = 151936 ends in a half tile; the cuts span all eight vocabulary chunks)
+    w = wl.make(name, device="cuda") if name == "tiny" else wl.make(name, device="cuda", cut_rows=300, cut_max_len=64)
+    run_all_stages(w, options=[(ub.OPT_LOGIT_STASH, 1)])
+
+
+def test_logit_stash_small_shapes_and_entropy_bonus():
+    for H, V, rows in [(320, 2048 + 264, 700), (64, 1000, 150)]:
+        run_all_stages(small_workload(H, V, rows), options=[(ub.OPT_LOGIT_STASH, 1)], ent_coef=0.02, kl_mode=2)
 
 
 @pytest.mark.parametrize("kl_mode,ent_coef,clip", [(1, 0.0, (0.2, 0.2)), (2, 0.01, (0.1, 0.3)), (3, 0.02, (0.2, 0.28))])
