@@ -264,11 +264,12 @@ def main():
     # room for the optional logit stash too (reported as an extra; the headline step never uses it)
     ws_bytes = max(ub.unity_workspace_bytes(n, H, V, K, w.n_inv), ub.unity_workspace_bytes_stash(n, H, V, K, w.n_inv))
     opts = [tuple(int(x) for x in kv.split("=")) for kv in args.opt.split(",") if kv]
-    ws_mult = 1
-    for o, v in opts:
-        if o in (6, 7):
-            ws_mult *= v                       # larger gradient chunks need a larger G / dH scratch
-    ctx = ub.Context(local, ws_bytes + (ws_mult - 1) * (2 * 18944 * 18944 + 4 * 18944 * H) * (2 if ws_mult > 1 else 0))
+    extra = 0
+    mults = {6: 2, 7: 2}
+    mults.update({o: v for o, v in opts if o in (6, 7)})
+    if (mults[6], mults[7]) != (2, 2):         # non-default gradient chunks need their own G / dH scratch
+        extra = 2 * mults[6] * 18944 * (mults[7] * 18944 + 2048) + 4 * mults[6] * 18944 * H
+    ctx = ub.Context(local, ws_bytes + extra)
     for o, v in opts:
         ctx.set_option(o, v)
     if args.ctas:

@@ -49,6 +49,9 @@ constexpr size_t kAlign = 256;
 // a whole number of waves: recompute 74 x 74 tiles, dHidden 74 x ceil(H/256), dW 74 x ceil(H/256).
 constexpr int kChunkRows = 74 * kTileM;      // 18944 token rows
 constexpr int kChunkVocab = 74 * kTileN;     // 18944 vocabulary entries
+// A gradient chunk spans kDefaultChunkMult x kDefaultChunkMult such blocks by default: the dHidden / dW GEMMs then
+// contract over twice as many vocabulary entries / rows per output tile and read-modify-write their outputs half as often.
+constexpr int kDefaultChunkMult = 2;
 constexpr int kMinChunkRows = 1024;
 constexpr int kMinChunkVocab = 1024;
 
@@ -407,8 +410,8 @@ int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace
     c->fwd_group = 0;
     c->fwd_sync = 1;
     c->chunk_sync = 6;
-    c->chunk_rows_mult = 1;
-    c->chunk_vocab_mult = 1;
+    c->chunk_rows_mult = kDefaultChunkMult;
+    c->chunk_vocab_mult = kDefaultChunkMult;
     c->wide_acc = 1;
     c->logit_stash = 0;
     c->ev_pool = new (std::nothrow) std::vector<cudaEvent_t>();
@@ -440,14 +443,15 @@ int unity_destroy(unity_ctx* ctx) {
 
 size_t unity_workspace_bytes(int64_t n_tok, int32_t H, int32_t V, int32_t K, int32_t n_inv) {
     if (n_tok < 0 || H <= 0 || V <= 0 || K <= 0 || n_inv < 0) return 0;
-    return carve(nullptr, ~size_t(0), n_tok, H, V, K, n_inv, wanted_chunk_rows(n_tok, K), wanted_chunk_vocab(V), nullptr).bytes;
+    return carve(nullptr, ~size_t(0), n_tok, H, V, K, n_inv, wanted_chunk_rows(n_tok, K, kDefaultChunkMult),
+                 wanted_chunk_vocab(V, kDefaultChunkMult), nullptr).bytes;
 }
 
 size_t unity_workspace_bytes_stash(int64_t n_tok, int32_t H, int32_t V, int32_t K, int32_t n_inv) {
     if (n_tok < 0 || H <= 0 || V <= 0 || K <= 0 || n_inv < 0) return 0;
     int cr = wanted_chunk_rows(n_tok, K);
     if (cr > kStashRows) cr = kStashRows;
-    const int cv = wanted_chunk_vocab(V);
+    const int cv = wanted_chunk_vocab(V, kDefaultChunkMult);
     int base, n;
     vocab_chunks(V, cv, &base, &n);
     const size_t a = carve(nullptr, ~size_t(0), n_tok, H, V, K, n_inv, cr, cv, nullptr, n).bytes;
@@ -806,7 +810,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
     bool stash = ctx->logit_stash && !have_fwd;
     int z_base = 0, z_chunks = 0;
     if (stash) {
-        const int cr_s = cr < kStashRows ? cr : kStashRows, cv_s = wanted_chunk_vocab(V);
+        const int cr_s = cr < kStashRows ? cr : kStashRows, cv_s = wanted_chunk_vocab(V, ctx->chunk_vocab_mult);
         vocab_chunks(V, cv_s, &z_base, &z_chunks);
         P.L = carve(ctx->ws, ctx->ws_bytes, rows->n_tok, H, V, K, rows->n_inv, cr_s, cv_s, &fits, z_chunks);
         if (fits) { cr = cr_s; cv = cv_s; }
@@ -902,20 +906,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 vc = V - v0 < base ? V - v0 : base;
                 if (V - (v0 + vc) <= tail && base < cv) vc = V - v0;               // absorb a short remainder
                 __nv_bfloat16* Gc = stash ? L.G + static_cast<long long>(ci) * cr * cv : L.G;
-                // (1) recompute the logits of this (rows x vocab) chunk and form dL/dz in bf16: G[nc, vc]
-                GemmArgs g;
-                memset(&g, 0, sizeof(g));
-                g.m_tiles = nc / gemm_tile_rows(c_grad); g.n_tiles = (vc + kTileN - 1) / kTileN; g.k_iters = H / kTileK;
-                g.group_m = ctx->chunk_group[0] / c_grad > 0 ? ctx->chunk_group[0] / c_grad : 1;
-                g.a_row0 = slot0; g.b_row0 = v0; g.m_rows = nc; g.n_cols = vc;
-                g.target_p = L.target_p; g.vocab0 = v0; g.scale = rows->inv_temperature;
-                g.coef_a = L.coef_a; g.coef_b = L.coef_b; g.row_lse = L.row_lse; g.row_ent = L.row_ent;
-                g.G = L.G; g.ldg = cv; g.status = ctx->d_status;
-                if (!stash && (ctx->chunk_sync & 1)) {
-                    g.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
-                    g.round_base = ctx->round_total;
-                    ctx->round_total += gemm_round_arrivals(kEpiLogitGrad, c_grad, g, ctx->sm_count);
-                }
+                // (1) dL/dz of this (rows x vocab) chunk in bf16: G[nc, vc]
                 if (stash) {
                     LogitGradArgs lg;
                     memset(&lg, 0, sizeof(lg));
@@ -924,9 +915,34 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                     lg.row_lse = L.row_lse; lg.row_ent = L.row_ent;
                     ProfScope ps(ctx, UNITY_PROF_GRAD_GEMM);
                     CUDA_TRY(ctx, launch_logit_grad_inplace(lg, st));
+                    nl += 1;
                 } else {
-                    ProfScope ps(ctx, UNITY_PROF_GRAD_GEMM);
-                    CUDA_TRY(ctx, launch_gemm(kEpiLogitGrad, false, c_grad, tm_hp_k, tm_W_k, g, ctx->sm_count, st));
+                    // recompute the logits.  Whatever the chunk size, one launch covers at most kChunkRows x
+                    // (kChunkVocab + tail) of it: the kernel re-reads its W block once per group of row tiles, and
+                    // that block has to stay small enough for the group's hidden rows to survive in L2 meanwhile.
+                    for (int r0 = 0; r0 < nc; r0 += kChunkRows) {
+                        const int nr = nc - r0 < kChunkRows ? nc - r0 : kChunkRows;
+                        for (int q0 = 0, qc = 0; q0 < vc; q0 += qc) {
+                            qc = vc - q0 < kChunkVocab ? vc - q0 : kChunkVocab;
+                            if (vc - (q0 + qc) <= tail) qc = vc - q0;
+                            GemmArgs g;
+                            memset(&g, 0, sizeof(g));
+                            g.m_tiles = nr / gemm_tile_rows(c_grad); g.n_tiles = (qc + kTileN - 1) / kTileN; g.k_iters = H / kTileK;
+                            g.group_m = ctx->chunk_group[0] / c_grad > 0 ? ctx->chunk_group[0] / c_grad : 1;
+                            g.a_row0 = slot0 + r0; g.b_row0 = v0 + q0; g.m_rows = nr; g.n_cols = qc;
+                            g.target_p = L.target_p; g.vocab0 = v0 + q0; g.scale = rows->inv_temperature;
+                            g.coef_a = L.coef_a; g.coef_b = L.coef_b; g.row_lse = L.row_lse; g.row_ent = L.row_ent;
+                            g.G = Gc + static_cast<long long>(r0) * cv + q0; g.ldg = cv; g.status = ctx->d_status;
+                            if (ctx->chunk_sync & 1) {
+                                g.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
+                                g.round_base = ctx->round_total;
+                                ctx->round_total += gemm_round_arrivals(kEpiLogitGrad, c_grad, g, ctx->sm_count);
+                            }
+                            ProfScope ps(ctx, UNITY_PROF_GRAD_GEMM);
+                            CUDA_TRY(ctx, launch_gemm(kEpiLogitGrad, false, c_grad, tm_hp_k, tm_W_k, g, ctx->sm_count, st));
+                            nl += 1;
+                        }
+                    }
                 }
                 // G viewed as [nc rows, vc]: K-major A for dHidden (contract over vc), MN-major A for dW (rows = K)
                 CUtensorMap tm_G_k, tm_G_mn;
@@ -965,7 +981,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                     ProfScope ps(ctx, UNITY_PROF_DW_GEMM);
                     CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, true, c_dw, tm_G_mn, tm_hp_mn, w, ctx->sm_count, st, wide_dw));
                 }
-                nl += 3;
+                nl += 2;
             }
             CUDA_TRY(ctx, launch_store_dhidden(L.dHc, L.slot_tok, slot0, nc, H, dH, st));
             nl += 1;
