@@ -291,6 +291,19 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                 ent = g.row_ent[g.a_row0 + row];
             }
             const float c2 = g.scale * kLog2e;
+            // per-row constants of the logit-gradient epilogue (see there)
+            float gshift = 0.f, gA = 0.f, gB = 0.f;
+            unsigned gsign = 0u;
+            if (EPI == kEpiLogitGrad) {
+                gshift = -lse * kLog2e;
+                if (!g.has_ent) {
+                    gshift += __log2f(fabsf(ca));              // -inf for a == 0: every exp2 below gives 0
+                    gsign = ca > 0.f ? 0x80008000u : 0u;
+                } else {
+                    gA = -fmaf(cb, ent - lse, ca);
+                    gB = -cb * g.scale;
+                }
+            }
 
             for (int nt = t.n_begin; nt < t.n_end && ok; ++nt) {
                 if (!ptx::mbar_wait(&acc_full[acc], acc_phase, kWaitBudgetCycles) || *abort_flag) { ok = false; break; }
@@ -352,22 +365,37 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                             }
                         }
                     } else if (EPI == kEpiLogitGrad) {
-                        // G = -p*(a + b*(z - lse + H)) (+ a at the target), z = scale*acc, p = exp(z - lse)
-                        const float shift = -lse * kLog2e;
-                        const float hl = ent - lse;
+                        // G = -p*(a + b*(z - lse + H)) (+ a at the target), z = scale*acc, p = exp(z - lse), written
+                        // with as few instructions per logit as possible (the epilogue shares issue slots and power
+                        // with the MMAs of the next tile):
+                        //   b == 0 for the whole launch:  |G| = exp2(acc*c2 + (shift + log2|a|)), sign(G) = -sign(a)
+                        //                                 -> one FMA and one exp2 per logit, sign set on the packed pair
+                        //   otherwise:                    G = p * (A + B*acc), A = -(a + b*(H - lse)), B = -b*scale
                         unsigned packed[16];
+                        if (!g.has_ent) {
 #pragma unroll
-                        for (int j = 0; j < 32; j += 2) {
-                            float o[2];
+                            for (int j = 0; j < 32; j += 2)
+                                packed[j >> 1] = pack_bf16(exp2f(fmaf(v[j], c2, gshift)), exp2f(fmaf(v[j + 1], c2, gshift))) ^ gsign;
+                        } else {
 #pragma unroll
-                            for (int q = 0; q < 2; ++q) {
-                                const float z = v[j + q] * g.scale;
-                                const float p = exp2f(fmaf(z, kLog2e, shift));
-                                float gg = -p * fmaf(cb, z + hl, ca);
-                                if (cbase + j + q == tgt) gg += ca;
-                                o[q] = gg;
-                            }
-                            packed[j >> 1] = pack_bf16(o[0], o[1]);
+                            for (int j = 0; j < 32; j += 2)
+                                packed[j >> 1] = pack_bf16(exp2f(fmaf(v[j], c2, gshift)) * fmaf(gB, v[j], gA),
+                                                           exp2f(fmaf(v[j + 1], c2, gshift)) * fmaf(gB, v[j + 1], gA));
+                        }
+                        const int jt = tgt - cbase;
+                        if (jt >= 0 && jt < 32) {                 // the target logit of this row: add a (rare branch)
+                            float vt = 0.f;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) if (j == jt) vt = v[j];
+                            const float z = vt * g.scale;
+                            const float pt = exp2f(fmaf(z, kLog2e, -lse * kLog2e));
+                            const float gt = fmaf(-pt, fmaf(cb, z + (ent - lse), ca), ca);
+                            const unsigned bits = static_cast<unsigned>(__bfloat16_as_ushort(__float2bfloat16_rn(gt)));
+                            const unsigned keep = (jt & 1) ? 0x0000ffffu : 0xffff0000u;
+                            const unsigned put = (jt & 1) ? (bits << 16) : bits;
+                            const int jp = jt >> 1;
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) packed[j] = (j == jp) ? ((packed[j] & keep) | put) : packed[j];
                         }
                         if (row_ok) {
                             __nv_bfloat16* dst = g.G + static_cast<long long>(row) * g.ldg + cbase;

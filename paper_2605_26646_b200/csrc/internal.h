@@ -55,6 +55,7 @@ struct GemmArgs {
     // kEpiLogitGrad
     const float* coef_a;      // [rows] dL/dlogp * scale, packed order
     const float* coef_b;      // [rows] dL/dentropy * scale
+    int has_ent;              // 0: every coef_b of the launch is zero (no entropy term): shorter epilogue
     const float* row_lse;     // [rows]
     const float* row_ent;     // [rows]
     __nv_bfloat16* G;         // [m_rows, ldg] chunk-local

@@ -932,6 +932,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                             g.a_row0 = slot0 + r0; g.b_row0 = v0 + q0; g.m_rows = nr; g.n_cols = qc;
                             g.target_p = L.target_p; g.vocab0 = v0 + q0; g.scale = rows->inv_temperature;
                             g.coef_a = L.coef_a; g.coef_b = L.coef_b; g.row_lse = L.row_lse; g.row_ent = L.row_ent;
+                            g.has_ent = params->ent_coef != 0.f;
                             g.G = Gc + static_cast<long long>(r0) * cv + q0; g.ldg = cv; g.status = ctx->d_status;
                             if (ctx->chunk_sync & 1) {
                                 g.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
