@@ -278,7 +278,8 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
             const bool row_ok = row < g.m_rows;
 
             // per-row state
-            float run_m = kNegBig, run_s = 0.f, run_t = 0.f, z_tgt = kNegBig;
+            float run_m = kNegBig, z_tgt = kNegBig;
+            uint64_t run_s2 = 0ull, run_t2 = 0ull;           // (even, odd) partial sums of e and e*v
             int tgt = -1;
             float ca = 0.f, cb = 0.f, lse = 0.f, ent = 0.f;
             if (EPI == kEpiSoftmaxStats || EPI == kEpiLogitGrad) {
@@ -327,20 +328,27 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
 #pragma unroll
                             for (int j = 0; j < 32; ++j) if (j >= n_here) v[j] = kNegBig;
                         }
-                        float cm = v[0];
+                        float cm = ptx::max3(v[0], v[1], v[2]);
 #pragma unroll
-                        for (int j = 1; j < 32; ++j) cm = fmaxf(cm, v[j]);
+                        for (int j = 3; j < 31; j += 2) cm = ptx::max3(cm, v[j], v[j + 1]);
+                        cm = fmaxf(cm, v[31]);
                         const float new_m = fmaxf(run_m, cm);
-                        const float resc = exp2f((run_m - new_m) * c2);
-                        run_s *= resc;
-                        run_t *= resc;
+                        const float resc = ptx::ex2((run_m - new_m) * c2);
+                        const uint64_t resc2 = ptx::pack2(resc, resc);
+                        run_s2 = ptx::mul2(run_s2, resc2);
+                        run_t2 = ptx::mul2(run_t2, resc2);
                         run_m = new_m;
                         const float shift = -new_m * c2;
+                        const uint64_t shift2 = ptx::pack2(shift, shift), c22 = ptx::pack2(c2, c2);
+                        // two logits per instruction: e = 2^(v*c2 + shift); sum e; sum e*v (even / odd partial sums)
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const float e = exp2f(fmaf(v[j], c2, shift));
-                            run_s += e;
-                            run_t = fmaf(e, v[j], run_t);
+                        for (int j = 0; j < 32; j += 2) {
+                            const uint64_t x = ptx::pack2(v[j], v[j + 1]);
+                            float a0, a1;
+                            ptx::unpack2(ptx::fma2(x, c22, shift2), a0, a1);
+                            const uint64_t e = ptx::pack2(ptx::ex2(a0), ptx::ex2(a1));
+                            run_s2 = ptx::add2(run_s2, e);
+                            run_t2 = ptx::fma2(e, x, run_t2);
                         }
                         const int jt = tgt - cbase;
                         if (jt >= 0 && jt < 32) {
@@ -372,15 +380,24 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                         //                                 -> one FMA and one exp2 per logit, sign set on the packed pair
                         //   otherwise:                    G = p * (A + B*acc), A = -(a + b*(H - lse)), B = -b*scale
                         unsigned packed[16];
+                        const uint64_t c22 = ptx::pack2(c2, c2), gshift2 = ptx::pack2(gshift, gshift);
                         if (!g.has_ent) {
 #pragma unroll
-                            for (int j = 0; j < 32; j += 2)
-                                packed[j >> 1] = pack_bf16(exp2f(fmaf(v[j], c2, gshift)), exp2f(fmaf(v[j + 1], c2, gshift))) ^ gsign;
+                            for (int j = 0; j < 32; j += 2) {
+                                float a0, a1;
+                                ptx::unpack2(ptx::fma2(ptx::pack2(v[j], v[j + 1]), c22, gshift2), a0, a1);
+                                packed[j >> 1] = pack_bf16(ptx::ex2(a0), ptx::ex2(a1)) ^ gsign;
+                            }
                         } else {
+                            const uint64_t gA2 = ptx::pack2(gA, gA), gB2 = ptx::pack2(gB, gB);
 #pragma unroll
-                            for (int j = 0; j < 32; j += 2)
-                                packed[j >> 1] = pack_bf16(exp2f(fmaf(v[j], c2, gshift)) * fmaf(gB, v[j], gA),
-                                                           exp2f(fmaf(v[j + 1], c2, gshift)) * fmaf(gB, v[j + 1], gA));
+                            for (int j = 0; j < 32; j += 2) {
+                                const uint64_t x = ptx::pack2(v[j], v[j + 1]);
+                                float a0, a1, o0, o1;
+                                ptx::unpack2(ptx::fma2(x, c22, gshift2), a0, a1);
+                                ptx::unpack2(ptx::mul2(ptx::pack2(ptx::ex2(a0), ptx::ex2(a1)), ptx::fma2(gB2, x, gA2)), o0, o1);
+                                packed[j >> 1] = pack_bf16(o0, o1);
+                            }
                         }
                         const int jt = tgt - cbase;
                         if (jt >= 0 && jt < 32) {                 // the target logit of this row: add a (rare branch)
@@ -388,7 +405,7 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
 #pragma unroll
                             for (int j = 0; j < 32; ++j) if (j == jt) vt = v[j];
                             const float z = vt * g.scale;
-                            const float pt = exp2f(fmaf(z, kLog2e, -lse * kLog2e));
+                            const float pt = ptx::ex2(fmaf(z, kLog2e, -lse * kLog2e));
                             const float gt = fmaf(-pt, fmaf(cb, z + (ent - lse), ca), ca);
                             const unsigned bits = static_cast<unsigned>(__bfloat16_as_ushort(__float2bfloat16_rn(gt)));
                             const unsigned keep = (jt & 1) ? 0x0000ffffu : 0xffff0000u;
@@ -438,8 +455,12 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                 }
                 if (++acc == kAccStages) { acc = 0; acc_phase ^= 1; }
             }
-            if (EPI == kEpiSoftmaxStats && ok && row_ok)
-                g.stats[t.split * g.stats_pitch + row] = make_float4(run_m, run_s, run_t, z_tgt);
+            if (EPI == kEpiSoftmaxStats && ok && row_ok) {
+                float s0, s1, t0, t1;
+                ptx::unpack2(run_s2, s0, s1);
+                ptx::unpack2(run_t2, t0, t1);
+                g.stats[t.split * g.stats_pitch + row] = make_float4(run_m, s0 + s1, t0 + t1, z_tgt);
+            }
         }
         if (!ok) { *abort_flag = 1; atomicOr(g.status, kStatusTimeout); }
     }
