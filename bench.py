@@ -28,12 +28,12 @@ UNIT = "tokens/s"
 
 
 # DRAM traffic of each GEMM class from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum, one launch per
-# class) on a cut of the code workload (profiles/k_gemm_code_cut40k.md), as bytes per logit the launch covers
+# class) on a cut of the code workload (profiles/k_gemm_code_cut90k.md), as bytes per logit the launch covers
 # (valid rows x vocabulary columns).  Traffic grows in proportion to the logits covered (same chunk and group sizes),
 # so a full-size launch is estimated as bytes_per_logit x its logits.  Valid only for the kernel source it was taken
 # from: when the hash of gemm_tcgen05.cu differs, the benchmark reports null.
-NCU_TRAFFIC = {"source_sha256_16": "6bea9a7ad9088210",
-               "bytes_per_logit": {"fwd_gemm": 2.309, "grad_gemm": 5.054, "dh_gemm": 9.674, "dw_gemm": 9.656}}
+NCU_TRAFFIC = {"source_sha256_16": "4741a1195a8a1476",
+               "bytes_per_logit": {"fwd_gemm": 1.776, "grad_gemm": 4.480, "dh_gemm": 6.756, "dw_gemm": 6.749}}
 
 
 def ncu_traffic_per_launch(cls: str, logits_per_launch: float):
