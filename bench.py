@@ -166,10 +166,11 @@ def run_reference(args):
 
 
 def run_micro(args):
-    """Streaming stages at a size where they are HBM-bound rather than launch-bound: role-level advantage
-    (token broadcast) and token-level GAE on 64 Mi tokens.  Prints one JSON line with achieved GB/s against the
-    measured copy bandwidth (algorithmic bytes: mask 1 B + output 4 B per token; rewards, values 8 B + mask 1 B +
-    two outputs 8 B per token)."""
+    """Streaming stages at a size where they are HBM-bound rather than launch-bound, on 64 Mi tokens: role-level
+    advantage (token broadcast), token-level GAE, clipped value loss, delayed-reward alignment and the ready-batch
+    gather.  Prints one JSON line with achieved GB/s against the measured copy bandwidth.  Algorithmic bytes per token:
+    advantage mask 1 + output 4; GAE rewards, values 8 + mask 1 + two outputs 8; value loss three inputs 12 + mask 1 +
+    gradient 4; alignment mask 1 + output 4; gather 2 x row bytes."""
     import torch
     from paper_2605_26646_b200 import binding as ub
     from paper_2605_26646_b200 import workloads as wl
@@ -204,11 +205,30 @@ def run_micro(args):
     t_adv = timed(lambda: ctx.role_advantage(n_inv, R, G, inv_role, inv_group, inv_traj, r_node, None, None, None, 1e-6,
                                              0, cu, mask, adv_inv, adv_tok))
     t_gae = timed(lambda: ctx.gae(cu, rewards, values, mask, 0.99, 0.95, a_out, r_out))
+    vloss = torch.empty(R, device=dev)
+    t_val = timed(lambda: ctx.value_loss_fwd_bwd(cu, inv_role, list(range(R)), R, mask, values, rewards, r_out, 0.2, None,
+                                                 vloss, None, None, a_out))
+    t_aln = timed(lambda: ctx.align_rewards(cu, mask, r_node, a_out))
+    # ready batch: plan over all invocations (80 % of the trajectories complete), then gather a 4-byte token tensor
+    done = (torch.rand(n_inv, device=dev) < 0.8).to(torch.uint8)
+    order = torch.empty(n_inv, dtype=torch.int32, device=dev)
+    out_cu = torch.empty(n_inv + 1, dtype=torch.int64, device=dev)
+    m_off = torch.empty(R + 1, dtype=torch.int32, device=dev)
+    p_off = torch.empty(R * 8 + 1, dtype=torch.int32, device=dev)
+    totals = torch.empty(2, dtype=torch.int64, device=dev)
+    t_plan = timed(lambda: ctx.ready_batch_plan(cu, inv_role, inv_traj, done, list(range(R)), R, 7, 8, 1, order, out_cu,
+                                                m_off, p_off, totals))
+    t_gat = timed(lambda: ctx.ready_batch_gather(order, cu, out_cu, totals, rewards, r_out, 0.0))
+    kept_tok = int(totals[1].item())
     ctx.check_status()
     out = {"mode": "micro", "tokens": n, "invocations": n_inv, "peak_hbm_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"],
            "role_advantage": {"ms": t_adv, "algorithmic_bytes": 5 * n + 28 * n_inv, "gbs": (5 * n + 28 * n_inv) / t_adv / 1e6},
-           "gae": {"ms": t_gae, "algorithmic_bytes": 17 * n, "gbs": 17 * n / t_gae / 1e6}}
-    for k in ("role_advantage", "gae"):
+           "gae": {"ms": t_gae, "algorithmic_bytes": 17 * n, "gbs": 17 * n / t_gae / 1e6},
+           "value_loss": {"ms": t_val, "algorithmic_bytes": 17 * n, "gbs": 17 * n / t_val / 1e6},
+           "align_rewards": {"ms": t_aln, "algorithmic_bytes": 5 * n, "gbs": 5 * n / t_aln / 1e6},
+           "ready_batch_gather_f32": {"ms": t_gat, "algorithmic_bytes": 8 * kept_tok, "gbs": 8 * kept_tok / t_gat / 1e6},
+           "ready_batch_plan": {"ms": t_plan, "note": "latency-bound: four small launches over the invocations"}}
+    for k in ("role_advantage", "gae", "value_loss", "align_rewards", "ready_batch_gather_f32"):
         out[k]["frac"] = out[k]["gbs"] / peaks["hbm_gbs"]
     print(json.dumps(out), flush=True)
 

@@ -201,9 +201,10 @@ struct ValueArgs {
     const float *values, *old_values, *returns;
     float clip_v;
     int has_norm;
+    int vec_ok;         // token arrays 16-byte aligned and the mask 4-byte aligned: 128-bit accesses allowed
     float norm[UNITY_MAX_MODELS];
     float* inv_sums;    // [n_inv * 3] count, sum of token losses, clipped tokens
-    float* Mk;          // [K] denominators, written by the class reduction
+    float* Mk;          // [2 * UNITY_MAX_MODELS] denominators M_k, then max(valid tokens, 1) per model
     float *loss, *clip_frac, *tok_loss, *dvalues;
     int* status;
 };

@@ -547,8 +547,8 @@ __global__ void k_reward_assembly(RewardArgs a) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// Critic update: clipped value loss.  Three small launches with fixed-order sums: per invocation (one warp each),
-// per model (one warp each), then the gradient with the model's 1/M_k.
+// Critic update: clipped value loss.  The token data is read once: a first pass over the mask bytes alone gives the
+// denominators M_k, the main pass then forms loss terms and gradients; all sums have a fixed order.
 struct ValueTerm {
     float loss, grad, clipped;
 };
@@ -566,49 +566,70 @@ __device__ __forceinline__ ValueTerm value_term(float v, float ov, float ret, fl
     return t;
 }
 
-__global__ void k_value_inv(ValueArgs a) {
+// (1) valid tokens per invocation (mask bytes only).
+__global__ void k_value_count(ValueArgs a) {
     const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (s >= a.n_inv) return;
     const int role = a.inv_role[s];
     const bool role_ok = role >= 0 && role < a.n_roles && a.role_model[role] >= 0 && a.role_model[role] < a.K;
     const long long lo = a.cu_seqlens[s], hi = a.cu_seqlens[s + 1];
-    float cnt = 0.f, sum = 0.f, clp = 0.f;
-    for (long long i = lo + lane; i < hi; i += 32) {
-        const bool on = role_ok && (a.tok_mask ? a.tok_mask[i] != 0 : true);
-        float l = 0.f;
-        if (on) {
-            const ValueTerm t = value_term(a.values[i], a.old_values[i], a.returns[i], a.clip_v);
-            l = t.loss; cnt += 1.f; sum += t.loss; clp += t.clipped;
+    int cnt = 0;
+    if (role_ok) {
+        if (a.tok_mask == nullptr) {
+            cnt = lane == 0 ? static_cast<int>(hi - lo) : 0;
+        } else {
+            // bytes up to the next 16-byte boundary one by one, then 16 mask bytes per lane and load, then the rest
+            const uintptr_t addr = reinterpret_cast<uintptr_t>(a.tok_mask) + static_cast<uintptr_t>(lo);
+            const long long head_end = min(hi, lo + static_cast<long long>((16 - (addr & 15)) & 15));
+            for (long long i = lo + lane; i < head_end; i += 32) cnt += a.tok_mask[i] != 0;
+            const long long n_vec = (hi - head_end) >> 4;
+            const uint4* mv = reinterpret_cast<const uint4*>(a.tok_mask + head_end);
+            for (long long q = lane; q < n_vec; q += 32) {
+                const uint4 m = mv[q];
+                cnt += (__popc(__vcmpne4(m.x, 0u)) + __popc(__vcmpne4(m.y, 0u)) + __popc(__vcmpne4(m.z, 0u)) +
+                        __popc(__vcmpne4(m.w, 0u))) >> 3;
+            }
+            for (long long i = head_end + (n_vec << 4) + lane; i < hi; i += 32) cnt += a.tok_mask[i] != 0;
         }
-        if (a.tok_loss) a.tok_loss[i] = l;
     }
-    cnt = warp_sum(cnt); sum = warp_sum(sum); clp = warp_sum(clp);
+    cnt = warp_sum_int(cnt);
     if (lane == 0) {
         if (!role_ok && hi > lo) atomicOr(a.status, kStatusBadIndex);
-        a.inv_sums[s * 3 + 0] = cnt; a.inv_sums[s * 3 + 1] = sum; a.inv_sums[s * 3 + 2] = clp;
+        a.inv_sums[s * 3 + 0] = static_cast<float>(cnt);
     }
 }
 
-__global__ void k_value_class(ValueArgs a) {
-    const int k = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
-    if (k >= a.K) return;
-    float cnt = 0.f, sum = 0.f, clp = 0.f;
-    for (int s = lane; s < a.n_inv; s += 32) {
+// Fixed-order sum over the 1024 threads of a block: lanes, then the 32 warp totals.
+__device__ __forceinline__ float block_sum_1024(float v, float* sh) {
+    v = warp_sum(v);
+    __syncthreads();                                   // sh may still be read from an earlier call
+    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float t = 0.f;
+    if (threadIdx.x < 32) t = warp_sum(sh[threadIdx.x]);
+    return t;                                          // valid in warp 0
+}
+
+// (2) denominators M_k (one block of 1024 threads per model, fixed order).
+__global__ void k_value_norm(ValueArgs a) {
+    __shared__ float sh[32];
+    const int k = blockIdx.x;
+    float cnt = 0.f;
+    for (int s = threadIdx.x; s < a.n_inv; s += 1024) {
         const int role = a.inv_role[s];
         if (role < 0 || role >= a.n_roles || a.role_model[role] != k) continue;
-        cnt += a.inv_sums[s * 3 + 0]; sum += a.inv_sums[s * 3 + 1]; clp += a.inv_sums[s * 3 + 2];
+        cnt += a.inv_sums[s * 3 + 0];
     }
-    cnt = warp_sum(cnt); sum = warp_sum(sum); clp = warp_sum(clp);
-    if (lane != 0) return;
-    const float M = a.has_norm ? a.norm[k] : fmaxf(cnt, 1.f);
-    a.Mk[k] = M;
-    a.loss[k] = sum / M;
-    if (a.clip_frac) a.clip_frac[k] = clp / fmaxf(cnt, 1.f);
+    cnt = block_sum_1024(cnt, sh);
+    if (threadIdx.x == 0) {
+        a.Mk[k] = a.has_norm ? a.norm[k] : fmaxf(cnt, 1.f);
+        a.Mk[UNITY_MAX_MODELS + k] = fmaxf(cnt, 1.f);
+    }
 }
 
-__global__ void k_value_grad(ValueArgs a) {
+// (3) the one pass over the token data: loss terms, gradient (already divided by M_k), per-invocation sums.
+__global__ void k_value_main(ValueArgs a) {
     const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (s >= a.n_inv) return;
@@ -616,10 +637,64 @@ __global__ void k_value_grad(ValueArgs a) {
     const bool role_ok = role >= 0 && role < a.n_roles && a.role_model[role] >= 0 && a.role_model[role] < a.K;
     const float M = role_ok ? a.Mk[a.role_model[role]] : 1.f;
     const long long lo = a.cu_seqlens[s], hi = a.cu_seqlens[s + 1];
-    for (long long i = lo + lane; i < hi; i += 32) {
+    float sum = 0.f, clp = 0.f;
+    auto one = [&](long long i) {
         const bool on = role_ok && (a.tok_mask ? a.tok_mask[i] != 0 : true);
-        a.dvalues[i] = on ? value_term(a.values[i], a.old_values[i], a.returns[i], a.clip_v).grad / M : 0.f;
+        float l = 0.f, gr = 0.f;
+        if (on) {
+            const ValueTerm t = value_term(a.values[i], a.old_values[i], a.returns[i], a.clip_v);
+            l = t.loss; gr = t.grad / M; sum += t.loss; clp += t.clipped;
+        }
+        a.dvalues[i] = gr;
+        if (a.tok_loss) a.tok_loss[i] = l;
+    };
+    if (!a.vec_ok) {
+        for (long long i = lo + lane; i < hi; i += 32) one(i);
+    } else {
+        // tokens up to a multiple of four one by one, then four tokens per lane with 128-bit accesses, then the rest
+        const long long head_end = min(hi, (lo + 3) & ~3LL);
+        for (long long i = lo + lane; i < head_end; i += 32) one(i);
+        const long long n_quad = (hi - head_end) >> 2;
+        for (long long q = lane; q < n_quad; q += 32) {
+            const long long i = head_end + (q << 2);
+            const float4 v = *reinterpret_cast<const float4*>(a.values + i);
+            const float4 ov = *reinterpret_cast<const float4*>(a.old_values + i);
+            const float4 rt = *reinterpret_cast<const float4*>(a.returns + i);
+            const unsigned m4 = a.tok_mask ? *reinterpret_cast<const unsigned*>(a.tok_mask + i) : 0x01010101u;
+            const float vv[4] = {v.x, v.y, v.z, v.w}, oo[4] = {ov.x, ov.y, ov.z, ov.w}, rr[4] = {rt.x, rt.y, rt.z, rt.w};
+            float g4[4], l4[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                g4[j] = 0.f; l4[j] = 0.f;
+                if (role_ok && ((m4 >> (8 * j)) & 0xffu)) {
+                    const ValueTerm t = value_term(vv[j], oo[j], rr[j], a.clip_v);
+                    l4[j] = t.loss; g4[j] = t.grad / M; sum += t.loss; clp += t.clipped;
+                }
+            }
+            *reinterpret_cast<float4*>(a.dvalues + i) = make_float4(g4[0], g4[1], g4[2], g4[3]);
+            if (a.tok_loss) *reinterpret_cast<float4*>(a.tok_loss + i) = make_float4(l4[0], l4[1], l4[2], l4[3]);
+        }
+        for (long long i = head_end + (n_quad << 2) + lane; i < hi; i += 32) one(i);
     }
+    sum = warp_sum(sum); clp = warp_sum(clp);
+    if (lane == 0) { a.inv_sums[s * 3 + 1] = sum; a.inv_sums[s * 3 + 2] = clp; }
+}
+
+// (4) loss and clip fraction per model (one block per model).
+__global__ void k_value_class(ValueArgs a) {
+    __shared__ float sh[32];
+    const int k = blockIdx.x;
+    float sum = 0.f, clp = 0.f;
+    for (int s = threadIdx.x; s < a.n_inv; s += 1024) {
+        const int role = a.inv_role[s];
+        if (role < 0 || role >= a.n_roles || a.role_model[role] != k) continue;
+        sum += a.inv_sums[s * 3 + 1]; clp += a.inv_sums[s * 3 + 2];
+    }
+    sum = block_sum_1024(sum, sh);
+    clp = block_sum_1024(clp, sh);
+    if (threadIdx.x != 0) return;
+    a.loss[k] = sum / a.Mk[k];
+    if (a.clip_frac) a.clip_frac[k] = clp / a.Mk[UNITY_MAX_MODELS + k];
 }
 
 }  // namespace
@@ -724,16 +799,12 @@ cudaError_t launch_reward_assembly(const RewardArgs& a, cudaStream_t stream) {
 }
 
 cudaError_t launch_value_loss(const ValueArgs& a, cudaStream_t stream, int* n_launches) {
-    if (a.n_inv > 0) {
-        k_value_inv<<<(a.n_inv + 7) / 8, 256, 0, stream>>>(a);
-        *n_launches += 1;
-    }
-    k_value_class<<<(a.K + 7) / 8, 256, 0, stream>>>(a);
-    *n_launches += 1;
-    if (a.n_inv > 0) {
-        k_value_grad<<<(a.n_inv + 7) / 8, 256, 0, stream>>>(a);
-        *n_launches += 1;
-    }
+    const int gi = (a.n_inv + 7) / 8;
+    if (a.n_inv > 0) { k_value_count<<<gi, 256, 0, stream>>>(a); *n_launches += 1; }
+    k_value_norm<<<a.K, 1024, 0, stream>>>(a);
+    if (a.n_inv > 0) { k_value_main<<<gi, 256, 0, stream>>>(a); *n_launches += 1; }
+    k_value_class<<<a.K, 1024, 0, stream>>>(a);
+    *n_launches += 2;
     return cudaGetLastError();
 }
 

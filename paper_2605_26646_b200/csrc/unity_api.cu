@@ -646,13 +646,16 @@ int unity_value_loss_fwd_bwd(unity_ctx* ctx, int32_t n_inv, int32_t n_roles, int
     for (int v = 0; v < n_roles; ++v) a.role_model[v] = role_model[v];
     CUDA_TRY(ctx, cudaSetDevice(ctx->device));
     Bump b{ctx->ws, 0, ctx->ws_bytes, true};
-    a.Mk = b.take<float>(UNITY_MAX_MODELS);
+    a.Mk = b.take<float>(2 * UNITY_MAX_MODELS);
     a.inv_sums = b.take<float>(static_cast<size_t>(n_inv) * 3 + 4);
     if (!b.ok) return fail(ctx, UNITY_ERR_WORKSPACE, "workspace too small: need %zu bytes", b.off);
     a.n_inv = n_inv; a.n_roles = n_roles; a.K = K;
     a.cu_seqlens = cu_seqlens; a.inv_role = inv_role; a.tok_mask = tok_mask;
     a.values = values; a.old_values = old_values; a.returns = returns;
     a.clip_v = clip_v; a.has_norm = norm != nullptr;
+    a.vec_ok = ((reinterpret_cast<uintptr_t>(values) | reinterpret_cast<uintptr_t>(old_values) |
+                 reinterpret_cast<uintptr_t>(returns) | reinterpret_cast<uintptr_t>(dvalues) |
+                 reinterpret_cast<uintptr_t>(tok_loss)) & 15) == 0 && (reinterpret_cast<uintptr_t>(tok_mask) & 3) == 0;
     a.loss = loss; a.clip_frac = clip_frac; a.tok_loss = tok_loss; a.dvalues = dvalues;
     a.status = ctx->d_status;
     int nl = 0;

@@ -238,6 +238,25 @@ def test_value_loss_full_size(name, clip_v, with_norm, masked):
     ctx.close()
 
 
+def test_value_loss_unaligned_views_take_the_scalar_path():
+    import oracle.unity_oracle as orc
+    w = wl.make_structure("rag_qa")
+    n = w.n_tok
+    v, ov, ret = wl.normal(13, 1, n), wl.normal(13, 2, n), wl.normal(13, 3, n)
+    pad = lambda t: torch.cat([torch.zeros(1, dtype=t.dtype), t]).cuda()[1:]       # data pointer off by one element
+    ctx = ub.Context(0, 1 << 20)
+    loss = torch.empty(w.K, device="cuda")
+    dv = torch.full((n + 1,), 7.0, device="cuda")[1:]
+    ctx.value_loss_fwd_bwd(w.cu_seqlens.cuda(), w.inv_role.cuda(), w.role_model.tolist(), w.K, pad(w.tok_mask), pad(v),
+                           pad(ov), pad(ret), 0.5, None, loss, None, None, dv)
+    ctx.check_status()
+    o = orc.value_loss_fwd_bwd(v.numpy(), ov.numpy(), ret.numpy(), w.cu_seqlens.numpy(), w.inv_role.numpy(),
+                               w.role_model.numpy(), w.tok_mask.numpy(), clip_v=0.5, K=w.K)
+    assert np.all(np.abs(loss.cpu().numpy() - o["loss"]) <= pu.TOL_LOSS * np.abs(o["loss"]))
+    assert np.abs(dv.cpu().numpy() - o["dvalues"]).max() <= 1e-5 * np.abs(o["dvalues"]).max() + 1e-9
+    ctx.close()
+
+
 # ------------------------------------------------------------------------------------ stages 2 + 3
 
 def test_tiny_full():
