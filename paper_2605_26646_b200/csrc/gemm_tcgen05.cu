@@ -362,14 +362,19 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                             zc = zc < g.z_chunks - 1 ? zc : g.z_chunks - 1;
                             __nv_bfloat16* dst = g.Z + zc * g.z_chunk_stride + static_cast<long long>(row) * g.ldz +
                                                  (cbase - zc * g.z_chunk_cols);
+                            unsigned zp[16];
 #pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                if (q * 8 < n_here)
-                                    *reinterpret_cast<uint4*>(dst + q * 8) = make_uint4(
-                                        pack_bf16(v[8 * q] * g.scale, v[8 * q + 1] * g.scale),
-                                        pack_bf16(v[8 * q + 2] * g.scale, v[8 * q + 3] * g.scale),
-                                        pack_bf16(v[8 * q + 4] * g.scale, v[8 * q + 5] * g.scale),
-                                        pack_bf16(v[8 * q + 6] * g.scale, v[8 * q + 7] * g.scale));
+                            for (int j = 0; j < 16; ++j) zp[j] = pack_bf16(v[2 * j] * g.scale, v[2 * j + 1] * g.scale);
+                            if (n_here == 32 && g.g_wide_store) {
+                                ptx::st_global_v8(dst, zp[0], zp[1], zp[2], zp[3], zp[4], zp[5], zp[6], zp[7]);
+                                ptx::st_global_v8(dst + 16, zp[8], zp[9], zp[10], zp[11], zp[12], zp[13], zp[14], zp[15]);
+                            } else {
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    if (q * 8 < n_here)
+                                        *reinterpret_cast<uint4*>(dst + q * 8) =
+                                            make_uint4(zp[4 * q], zp[4 * q + 1], zp[4 * q + 2], zp[4 * q + 3]);
+                                }
                             }
                         }
                     } else if (EPI == kEpiLogitGrad) {
@@ -416,11 +421,19 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                         }
                         if (row_ok) {
                             __nv_bfloat16* dst = g.G + static_cast<long long>(row) * g.ldg + cbase;
+                            if (n_here == 32 && g.g_wide_store) {
+                                // two full 32-byte sectors per thread instead of four half sectors
+                                ptx::st_global_v8(dst, packed[0], packed[1], packed[2], packed[3], packed[4], packed[5],
+                                                  packed[6], packed[7]);
+                                ptx::st_global_v8(dst + 16, packed[8], packed[9], packed[10], packed[11], packed[12],
+                                                  packed[13], packed[14], packed[15]);
+                            } else {
 #pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                if (q * 8 < n_here)
-                                    *reinterpret_cast<uint4*>(dst + q * 8) =
-                                        make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                                for (int q = 0; q < 4; ++q) {
+                                    if (q * 8 < n_here)
+                                        *reinterpret_cast<uint4*>(dst + q * 8) =
+                                            make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                                }
                             }
                         }
                     } else {

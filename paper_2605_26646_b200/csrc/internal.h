@@ -60,6 +60,7 @@ struct GemmArgs {
     const float* row_ent;     // [rows]
     __nv_bfloat16* G;         // [m_rows, ldg] chunk-local
     long long ldg;
+    int g_wide_store;         // G and ldg allow 32-byte aligned row segments: 256-bit stores
     // kEpiAccumF32
     float* C;
     long long ldc;

@@ -119,6 +119,14 @@ __device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
     return r;
 }
 
+// 256-bit store: eight 32-bit words to a 32-byte aligned global address (one full sector per thread and instruction).
+__device__ __forceinline__ void st_global_v8(void* addr, unsigned r0, unsigned r1, unsigned r2, unsigned r3, unsigned r4,
+                                             unsigned r5, unsigned r6, unsigned r7) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(addr), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(r4), "r"(r5), "r"(r6), "r"(r7)
+                 : "memory");
+}
+
 // Fire-and-forget vector reduction: four consecutive floats at a 16-byte aligned global address += v.
 __device__ __forceinline__ void red_add_v4_f32(float* addr, float4 v) {
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};"

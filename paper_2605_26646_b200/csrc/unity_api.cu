@@ -292,7 +292,11 @@ int launch_forward(unity_ctx* ctx, const unity_rows* r, int slot0, int rows, flo
     g.stats = stats; g.stats_pitch = rows;
     g.target_p = target_p; g.vocab0 = 0; g.scale = r->inv_temperature;
     g.status = ctx->d_status;
-    if (z) { g.Z = z->Z; g.ldz = z->ldz; g.z_chunk_stride = z->chunk_stride; g.z_chunk_cols = z->chunk_cols; g.z_chunks = z->chunks; }
+    if (z) {
+        g.Z = z->Z; g.ldz = z->ldz; g.z_chunk_stride = z->chunk_stride; g.z_chunk_cols = z->chunk_cols; g.z_chunks = z->chunks;
+        g.g_wide_store = (reinterpret_cast<uintptr_t>(z->Z) % 32 == 0) && (z->ldz * 2 % 32 == 0) && (z->chunk_stride * 2 % 32 == 0) &&
+                         (z->chunk_cols * 2 % 32 == 0);
+    }
     if (ctx->fwd_sync) {
         g.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
         g.round_base = ctx->round_total;
@@ -937,6 +941,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                             g.coef_a = L.coef_a; g.coef_b = L.coef_b; g.row_lse = L.row_lse; g.row_ent = L.row_ent;
                             g.has_ent = params->ent_coef != 0.f;
                             g.G = Gc + static_cast<long long>(r0) * cv + q0; g.ldg = cv; g.status = ctx->d_status;
+                            g.g_wide_store = (reinterpret_cast<uintptr_t>(g.G) % 32 == 0) && (g.ldg * 2 % 32 == 0);
                             if (ctx->chunk_sync & 1) {
                                 g.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
                                 g.round_base = ctx->round_total;
