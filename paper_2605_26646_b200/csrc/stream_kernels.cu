@@ -418,31 +418,42 @@ __global__ void k_class_reduce(TokenArgs a) {
     if (c < a.K) a.loss[c] = acc[8] / a.norm[c];
 }
 
-// Stashed logits -> logit gradients, in place.  A thread converts eight consecutive bf16 values (one 128-bit load and
-// store); a warp covers 512 contiguous bytes of a row.  Streaming: 2 B read + 2 B written per logit.
-__global__ void k_logit_grad_inplace(LogitGradArgs a) {
-    const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * 8;
-    if (c0 >= a.cols) return;
+// Stashed logits -> logit gradients, in place.  A block converts 8192 consecutive columns of one row: every thread
+// first issues its four 128-bit loads (4 KiB apart, so each warp access covers 512 contiguous bytes), then converts
+// and stores them.  Streaming: 2 B read + 2 B written per logit.
+constexpr int kGradVecs = 4;
+__global__ void __launch_bounds__(256) k_logit_grad_inplace(LogitGradArgs a) {
+    const int c_first = blockIdx.x * (256 * 8 * kGradVecs) + threadIdx.x * 8;
     for (int r = blockIdx.y; r < a.rows; r += gridDim.y) {
         const int slot = a.row0 + r;
+        uint4* row = reinterpret_cast<uint4*>(a.Z + static_cast<long long>(r) * a.ld);
+        uint4 raw[kGradVecs];
+#pragma unroll
+        for (int u = 0; u < kGradVecs; ++u) {
+            const int c0 = c_first + u * 2048;
+            if (c0 < a.cols) raw[u] = row[c0 >> 3];
+        }
         const float ca = a.coef_a[slot], cb = a.coef_b[slot], lse = a.row_lse[slot];
         const float hl = a.row_ent[slot] - lse;
         const int tgt = a.target_p[slot] - a.vocab0;
-        uint4* ptr = reinterpret_cast<uint4*>(a.Z + static_cast<long long>(r) * a.ld + c0);
-        uint4 raw = *ptr;
-        __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&raw);
         const float shift = -lse * 1.4426950408889634f;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const float2 z = __bfloat1622float2(h2[j]);
-            const float p0 = exp2f(fmaf(z.x, 1.4426950408889634f, shift));
-            const float p1 = exp2f(fmaf(z.y, 1.4426950408889634f, shift));
-            float g0 = -p0 * fmaf(cb, z.x + hl, ca), g1 = -p1 * fmaf(cb, z.y + hl, ca);
-            if (c0 + 2 * j == tgt) g0 += ca;
-            if (c0 + 2 * j + 1 == tgt) g1 += ca;
-            h2[j] = __floats2bfloat162_rn(g0, g1);
+        for (int u = 0; u < kGradVecs; ++u) {
+            const int c0 = c_first + u * 2048;
+            if (c0 >= a.cols) continue;
+            __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&raw[u]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float2 z = __bfloat1622float2(h2[j]);
+                const float p0 = exp2f(fmaf(z.x, 1.4426950408889634f, shift));
+                const float p1 = exp2f(fmaf(z.y, 1.4426950408889634f, shift));
+                float g0 = -p0 * fmaf(cb, z.x + hl, ca), g1 = -p1 * fmaf(cb, z.y + hl, ca);
+                if (c0 + 2 * j == tgt) g0 += ca;
+                if (c0 + 2 * j + 1 == tgt) g1 += ca;
+                h2[j] = __floats2bfloat162_rn(g0, g1);
+            }
+            row[c0 >> 3] = raw[u];
         }
-        *ptr = raw;
     }
 }
 
@@ -763,8 +774,8 @@ cudaError_t launch_finish_forward(const TokenArgs& a, bool with_loss, cudaStream
 
 cudaError_t launch_logit_grad_inplace(const LogitGradArgs& a, cudaStream_t stream) {
     if (a.rows <= 0 || a.cols <= 0) return cudaSuccess;
-    // a block covers 2048 columns of one row; y walks the rows (grid-stride, the y extent is limited to 65535)
-    const unsigned gx = static_cast<unsigned>((a.cols + 2047) / 2048);
+    // a block covers 8192 columns of one row; y walks the rows (grid-stride, the y extent is limited to 65535)
+    const unsigned gx = static_cast<unsigned>((a.cols + 8191) / 8192);
     const unsigned gy = static_cast<unsigned>(a.rows < 32768 ? a.rows : 32768);
     k_logit_grad_inplace<<<dim3(gx, gy), 256, 0, stream>>>(a);
     return cudaGetLastError();
