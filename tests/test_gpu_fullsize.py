@@ -29,11 +29,15 @@ class DeviceRows:
         return pu.bf16_bits(self.t[torch.as_tensor(np.asarray(idx), device=self.t.device)])
 
 
-@pytest.mark.parametrize("name,n_sample,chunk_rows", [("rag_qa", 192, 1200), ("search", 96, 1000), ("code", 96, 1000), ("stress", 64, 600)])
-def test_full_size_sampled_parity(name, n_sample, chunk_rows):
+@pytest.mark.parametrize("name,n_sample,chunk_rows,stash", [("rag_qa", 192, 1200, False), ("search", 96, 1000, False),
+                                                            ("code", 96, 1000, False), ("stress", 64, 600, False),
+                                                            ("rag_qa", 192, 1200, True), ("stress", 64, 600, True)])
+def test_full_size_sampled_parity(name, n_sample, chunk_rows, stash):
     w = wl.make(name, device="cuda")
     d = pu.DeviceInputs(w)
-    ctx = pu.make_ctx(w)
+    ctx = pu.make_ctx(w, stash=stash)
+    if stash:          # logit stash instead of the recompute GEMM: several row blocks per model at these sizes
+        ctx.set_option(ub.OPT_LOGIT_STASH, 1)
     K, n = w.K, w.n_tok
     role_model = w.role_model.tolist()
     mask_np = w.tok_mask.numpy() != 0
