@@ -191,6 +191,32 @@ __global__ void k_adv_broadcast(AdvArgs a, int rounds) {
     }
 }
 
+// The same broadcast with one warp per invocation, for batches of long invocations: no search; after the tokens up to
+// the next multiple of 16, every lane handles 16 tokens per step (one 128-bit mask load, four 128-bit stores).
+__global__ void k_adv_broadcast_inv(AdvArgs a) {
+    const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (s >= a.n_inv) return;
+    const long long lo = a.cu_seqlens[s], hi = a.cu_seqlens[s + 1];
+    const float adv = a.adv_inv[s];
+    const long long head_end = min(hi, (lo + 15) & ~15LL);
+    for (long long i = lo + lane; i < head_end; i += 32) a.adv_tok[i] = (a.tok_mask == nullptr || a.tok_mask[i]) ? adv : 0.f;
+    const long long n_vec = (hi - head_end) >> 4;
+    for (long long q = lane; q < n_vec; q += 32) {
+        const long long i = head_end + (q << 4);
+        uint4 m = make_uint4(0x01010101u, 0x01010101u, 0x01010101u, 0x01010101u);
+        if (a.tok_mask) m = *reinterpret_cast<const uint4*>(a.tok_mask + i);
+        const unsigned w[4] = {m.x, m.y, m.z, m.w};
+        float4* out = reinterpret_cast<float4*>(a.adv_tok + i);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            out[j] = make_float4((w[j] & 0xffu) ? adv : 0.f, (w[j] & 0xff00u) ? adv : 0.f, (w[j] & 0xff0000u) ? adv : 0.f,
+                                 (w[j] & 0xff000000u) ? adv : 0.f);
+    }
+    for (long long i = head_end + (n_vec << 4) + lane; i < hi; i += 32)
+        a.adv_tok[i] = (a.tok_mask == nullptr || a.tok_mask[i]) ? adv : 0.f;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Routing: stable partition of the valid tokens by model id (count, scan, assign)
 // ------------------------------------------------------------------------------------------------
@@ -535,6 +561,95 @@ __global__ void k_gae(GaeArgs a) {
     }
 }
 
+// The same recurrence with four tokens per lane (128 tokens per warp step, 128-bit accesses; chunks are aligned to
+// absolute token indices that are multiples of 128, tokens outside the sequence count as masked).  Inside a lane the
+// four maps are composed one after the other; across lanes by the suffix scan; then every token's advantage follows
+// from the advantage entering its lane.
+__global__ void k_gae_vec(GaeArgs a) {
+    const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (s >= a.n_inv) return;
+    const long long lo = a.cu_seqlens[s], hi = a.cu_seqlens[s + 1];
+    if (hi <= lo) return;
+    const float c = a.gamma * a.lam;
+    float carry_adv = 0.f, carry_val = 0.f;
+    for (long long c0 = ((hi - 1) >> 7) << 7; c0 + 128 > lo; c0 -= 128) {
+        const long long t0 = c0 + 4 * lane;
+        float v[4] = {0.f, 0.f, 0.f, 0.f}, r[4] = {0.f, 0.f, 0.f, 0.f};
+        unsigned m4 = 0u;
+        const bool whole = t0 >= lo && t0 + 4 <= hi;
+        if (whole) {
+            const float4 vv = *reinterpret_cast<const float4*>(a.values + t0);
+            const float4 rr = *reinterpret_cast<const float4*>(a.rewards + t0);
+            v[0] = vv.x; v[1] = vv.y; v[2] = vv.z; v[3] = vv.w;
+            r[0] = rr.x; r[1] = rr.y; r[2] = rr.z; r[3] = rr.w;
+            m4 = a.tok_mask ? *reinterpret_cast<const unsigned*>(a.tok_mask + t0) : 0x01010101u;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const long long t = t0 + j;
+                if (t >= lo && t < hi) {
+                    v[j] = a.values[t]; r[j] = a.rewards[t];
+                    if (a.tok_mask ? a.tok_mask[t] != 0 : true) m4 |= 0x01u << (8 * j);
+                }
+            }
+        }
+        bool on[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) on[j] = ((m4 >> (8 * j)) & 0xffu) != 0;
+        const bool any = m4 != 0u;
+        // value of the first unmasked token of the lanes above (or of the chunks above)
+        float first_v = 0.f;
+#pragma unroll
+        for (int j = 3; j >= 0; --j) if (on[j]) first_v = v[j];
+        const unsigned valid = __ballot_sync(kFull, any);
+        const unsigned above = lane == 31 ? 0u : (valid & (0xffffffffu << (lane + 1)));
+        const float v_peer = __shfl_sync(kFull, first_v, above ? __ffs(above) - 1 : 0);
+        float v_next = above ? v_peer : carry_val;
+        // the lane's tokens from the last to the first: token j maps the advantage entering the lane, x, to pb[j] + pa[j]*x
+        float pa[4], pb[4];
+        float ma = 1.f, mb = 0.f;
+#pragma unroll
+        for (int j = 3; j >= 0; --j) {
+            if (on[j]) {
+                const float delta = r[j] + a.gamma * v_next - v[j];
+                mb = fmaf(c, mb, delta);
+                ma = ma * c;
+                v_next = v[j];
+            }
+            pa[j] = ma; pb[j] = mb;
+        }
+        // suffix scan of the lane maps: lane i ends with the composition of lanes i .. 31
+        float sa = ma, sb = mb;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float qa = __shfl_down_sync(kFull, sa, o), qb = __shfl_down_sync(kFull, sb, o);
+            if (lane + o < 32) { sb = fmaf(sa, qb, sb); sa = sa * qa; }
+        }
+        const float at_lane = fmaf(sa, carry_adv, sb);            // advantage at this lane's first unmasked token
+        const float from_above = __shfl_down_sync(kFull, at_lane, 1);
+        const float x = lane == 31 ? carry_adv : from_above;      // advantage entering this lane
+        float adv[4], ret[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            adv[j] = on[j] ? fmaf(pa[j], x, pb[j]) : 0.f;
+            ret[j] = on[j] ? adv[j] + v[j] : 0.f;
+        }
+        if (whole) {
+            *reinterpret_cast<float4*>(a.adv + t0) = make_float4(adv[0], adv[1], adv[2], adv[3]);
+            *reinterpret_cast<float4*>(a.ret + t0) = make_float4(ret[0], ret[1], ret[2], ret[3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const long long t = t0 + j;
+                if (t >= lo && t < hi) { a.adv[t] = adv[j]; a.ret[t] = ret[j]; }
+            }
+        }
+        carry_adv = __shfl_sync(kFull, at_lane, 0);
+        if (valid) carry_val = __shfl_sync(kFull, first_v, __ffs(valid) - 1);
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Turn-level reward assembly: one thread per invocation gathers its trajectory's score(s).
 __global__ void k_reward_assembly(RewardArgs a) {
@@ -720,7 +835,12 @@ cudaError_t launch_advantage(const AdvArgs& a, cudaStream_t stream, int* n_launc
         k_adv_segment<<<(n_seg + 7) / 8, 256, 0, stream>>>(a);
         *n_launches += 2;
     }
-    if (a.n_tok > 0) {
+    const bool aligned = (reinterpret_cast<uintptr_t>(a.tok_mask) & 15) == 0 && (reinterpret_cast<uintptr_t>(a.adv_tok) & 15) == 0;
+    if (a.n_tok > 0 && aligned && a.n_tok / a.n_inv >= 128 && a.n_inv >= 1024) {
+        // long invocations, and enough of them to fill the machine: one warp each
+        k_adv_broadcast_inv<<<(a.n_inv + 7) / 8, 256, 0, stream>>>(a);
+        *n_launches += 1;
+    } else if (a.n_tok > 0) {
         // enough blocks to fill the machine (about 8 per SM), at most 32 rounds per block
         long long rounds = a.n_tok / (1024LL * 148 * 8);
         rounds = rounds < 1 ? 1 : (rounds > 32 ? 32 : rounds);
@@ -799,7 +919,12 @@ cudaError_t launch_gae(int n_inv, const int64_t* cu_seqlens, const float* reward
                        const uint8_t* tok_mask, float gamma, float lam, float* adv, float* ret, cudaStream_t stream) {
     if (n_inv == 0) return cudaSuccess;
     GaeArgs a{n_inv, cu_seqlens, rewards, values, tok_mask, gamma, lam, adv, ret};
-    k_gae<<<(n_inv + 7) / 8, 256, 0, stream>>>(a);
+    const uintptr_t al = reinterpret_cast<uintptr_t>(rewards) | reinterpret_cast<uintptr_t>(values) |
+                         reinterpret_cast<uintptr_t>(adv) | reinterpret_cast<uintptr_t>(ret);
+    if ((al & 15) == 0 && (reinterpret_cast<uintptr_t>(tok_mask) & 3) == 0)
+        k_gae_vec<<<(n_inv + 7) / 8, 256, 0, stream>>>(a);
+    else
+        k_gae<<<(n_inv + 7) / 8, 256, 0, stream>>>(a);
     return cudaGetLastError();
 }
 

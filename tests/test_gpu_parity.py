@@ -238,6 +238,23 @@ def test_value_loss_full_size(name, clip_v, with_norm, masked):
     ctx.close()
 
 
+def test_gae_unaligned_views_take_the_scalar_path():
+    import oracle.unity_oracle as orc
+    w = wl.make_structure("rag_qa")
+    n = w.n_tok
+    r, v = wl.normal(14, 1, n), wl.normal(14, 2, n)
+    pad = lambda t: torch.cat([torch.zeros(1, dtype=t.dtype), t]).cuda()[1:]       # data pointer off by one element
+    ctx = ub.Context(0, 1 << 20)
+    adv = torch.full((n + 1,), 7.0, device="cuda")[1:]
+    ret = torch.full((n + 1,), 7.0, device="cuda")[1:]
+    ctx.gae(w.cu_seqlens.cuda(), pad(r), pad(v), pad(w.tok_mask), 0.98, 0.9, adv, ret)
+    ctx.check_status()
+    oa, orr = orc.gae(r.numpy(), v.numpy(), w.cu_seqlens.numpy(), 0.98, 0.9, w.tok_mask.numpy())
+    scale = max(1.0, float(np.abs(oa).max()))
+    assert np.abs(adv.cpu().numpy() - oa).max() <= 1e-5 * scale and np.abs(ret.cpu().numpy() - orr).max() <= 1e-5 * scale
+    ctx.close()
+
+
 def test_value_loss_unaligned_views_take_the_scalar_path():
     import oracle.unity_oracle as orc
     w = wl.make_structure("rag_qa")
