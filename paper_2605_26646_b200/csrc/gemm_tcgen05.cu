@@ -68,6 +68,7 @@ struct Unit {
 // of a round therefore share gm A tiles (L2 resident) and each split's stream of B tiles is fetched from HBM once, by
 // pairs that sweep it in step.  Other epilogues: one 256 x 256 output tile per unit, unit = pair + it * n_pairs, m
 // fastest inside groups of gm row tiles.
+// Other epilogues, continued: the column order alternates from one group of row tiles to the next.
 // Returns false when the pair has no more work; `valid` is false for a round the pair sits out.
 template <int EPI>
 __device__ __forceinline__ bool next_unit(const GemmArgs& g, int it, int pair, int n_pairs, int gm, Unit& t, bool& valid) {
@@ -91,8 +92,10 @@ __device__ __forceinline__ bool next_unit(const GemmArgs& g, int it, int pair, i
         const int q = r / gm_here;
         t.m_tile = m0 + (r - q * gm_here);
         t.split = 0;
-        t.n_begin = q;
-        t.n_end = q + 1;
+        // odd groups walk the columns backwards: the B tiles a group ends with are the ones the next group starts
+        // with, while they are still in L2
+        t.n_begin = (grp & 1) ? g.n_tiles - 1 - q : q;
+        t.n_end = t.n_begin + 1;
         valid = true;
         return true;
     }
