@@ -105,6 +105,9 @@ int unity_set_profiling(unity_ctx* ctx, int enable);
                                      backward turns them into dL/dz in place.  Executed work drops from 8 to 6 H V flop per
                                      token; the full n_tok x V logits still never exist.  Ignored (recompute) when the
                                      workspace has no room or the on-policy shortcut is used. */
+#define UNITY_OPT_L2_HINTS_FWD 16 /* 16..19: L2 eviction policy of the forward / recompute / dHidden / dW GEMM: value =
+                                     A-operand loads | B-operand loads << 2 | logit-gradient stores << 4, each 0 normal,
+                                     1 evict first, 2 evict last (defaults 6, 22, 0, 0: measured +0.3-0.7 % on the first two) */
 int unity_set_option(unity_ctx* ctx, int option, int value);
 int unity_get_profile(unity_ctx* ctx, double* ms, int64_t* launches);
 

@@ -155,6 +155,7 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
+            const uint64_t pol_a = ptx::l2_policy(g.l2_hints & 3), pol_b = ptx::l2_policy((g.l2_hints >> 2) & 3);
             for (int it = 0; ok; ++it) {
                 Unit t;
                 bool valid;
@@ -189,9 +190,9 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                         if (A_MN) {
 #pragma unroll
                             for (int j = 0; j < kCtaM / 64; ++j)
-                                ptx::tma_load_2d_on<CTAS>(sA + j * kMnBoxBytes, &tmA, bar, a_row + j * 64, g.a_k0 + k * kTileK);
+                                ptx::tma_load_2d_hint_on<CTAS>(sA + j * kMnBoxBytes, &tmA, bar, a_row + j * 64, g.a_k0 + k * kTileK, pol_a);
                         } else {
-                            ptx::tma_load_2d_on<CTAS>(sA, &tmA, bar, g.a_k0 + k * kTileK, a_row);
+                            ptx::tma_load_2d_hint_on<CTAS>(sA, &tmA, bar, g.a_k0 + k * kTileK, a_row, pol_a);
                         }
 #pragma unroll
                         for (int nb = 0; nb < NB; ++nb) {          // one block of B rows per 256 output columns
@@ -199,10 +200,10 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                             if (B_MN) {
 #pragma unroll
                                 for (int j = 0; j < C::kBRows / 64; ++j)
-                                    ptx::tma_load_2d_on<CTAS>(sB + j * kMnBoxBytes, &tmB, bar, b_row + nb * kTileN + j * 64,
-                                                              g.b_k0 + k * kTileK);
+                                    ptx::tma_load_2d_hint_on<CTAS>(sB + j * kMnBoxBytes, &tmB, bar, b_row + nb * kTileN + j * 64,
+                                                                   g.b_k0 + k * kTileK, pol_b);
                             } else {
-                                ptx::tma_load_2d_on<CTAS>(sB, &tmB, bar, g.b_k0 + k * kTileK, b_row + nb * kTileN);
+                                ptx::tma_load_2d_hint_on<CTAS>(sB, &tmB, bar, g.b_k0 + k * kTileK, b_row + nb * kTileN, pol_b);
                             }
                         }
                         if (++stage == kStages) { stage = 0; phase ^= 1; }
@@ -272,6 +273,7 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
+        const uint64_t pol_st = ptx::l2_policy((g.l2_hints >> 4) & 3);
         for (int it = 0; ok; ++it) {
             Unit t;
             bool valid;
@@ -426,10 +428,10 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                             __nv_bfloat16* dst = g.G + static_cast<long long>(row) * g.ldg + cbase;
                             if (n_here == 32 && g.g_wide_store) {
                                 // two full 32-byte sectors per thread instead of four half sectors
-                                ptx::st_global_v8(dst, packed[0], packed[1], packed[2], packed[3], packed[4], packed[5],
-                                                  packed[6], packed[7]);
-                                ptx::st_global_v8(dst + 16, packed[8], packed[9], packed[10], packed[11], packed[12],
-                                                  packed[13], packed[14], packed[15]);
+                                ptx::st_global_v8_hint(dst, packed[0], packed[1], packed[2], packed[3], packed[4], packed[5],
+                                                       packed[6], packed[7], pol_st);
+                                ptx::st_global_v8_hint(dst + 16, packed[8], packed[9], packed[10], packed[11], packed[12],
+                                                       packed[13], packed[14], packed[15], pol_st);
                             } else {
 #pragma unroll
                                 for (int q = 0; q < 4; ++q) {

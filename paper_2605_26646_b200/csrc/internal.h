@@ -65,6 +65,7 @@ struct GemmArgs {
     float* C;
     long long ldc;
     int beta;                 // 0: overwrite, 1: add to C
+    int l2_hints;             // L2 eviction policy (0 normal, 1 first, 2 last): bits 0-1 A loads, 2-3 B loads, 4-5 G stores
     int* status;
 };
 

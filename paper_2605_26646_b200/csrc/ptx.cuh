@@ -241,6 +241,40 @@ __device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
         : "memory");
 }
 
+// L2 eviction policies for loads and stores that carry a cache hint: 0 normal, 1 evict first, 2 evict last.
+__device__ __forceinline__ uint64_t l2_policy(int kind) {
+    uint64_t p;
+    if (kind == 1) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    else if (kind == 2) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    else asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void st_global_v8_hint(void* addr, unsigned r0, unsigned r1, unsigned r2, unsigned r3,
+                                                  unsigned r4, unsigned r5, unsigned r6, unsigned r7, uint64_t policy) {
+    asm volatile("st.global.L2::cache_hint.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8}, %9;"
+                 ::"l"(addr), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(r4), "r"(r5), "r"(r6), "r"(r7), "l"(policy)
+                 : "memory");
+}
+// 2-D tiled load with an L2 cache hint; CTAS = 2: completion bytes go to the barrier (cluster address) of the pair's
+// leading CTA.
+template <int CTAS>
+__device__ __forceinline__ void tma_load_2d_hint_on(void* smem_dst, const void* tmap, uint32_t bar_addr, int32_t x, int32_t y,
+                                                    uint64_t policy) {
+    if (CTAS == 2) {
+        asm volatile(
+            "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+            "[%0], [%1, {%3, %4}], [%2], %5;"
+            ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar_addr), "r"(x), "r"(y), "l"(policy)
+            : "memory");
+    } else {
+        asm volatile(
+            "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+            "[%0], [%1, {%3, %4}], [%2], %5;"
+            ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar_addr), "r"(x), "r"(y), "l"(policy)
+            : "memory");
+    }
+}
+
 // Forms selected by the number of CTAs that cooperate on a tile (1, or 2 = a CTA pair).
 template <int CTAS>
 __device__ __forceinline__ void tma_load_2d_on(void* smem_dst, const void* tmap, uint32_t bar_addr, int32_t x, int32_t y) {

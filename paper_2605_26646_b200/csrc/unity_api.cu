@@ -38,6 +38,7 @@ struct unity_ctx {
     int fwd_sync;                   // 1: workers of the forward kernel meet (softly) at every round start
     int chunk_sync;                 // bit 0: same for the recompute GEMM, bit 1: dHidden GEMM, bit 2: dW GEMM
     int logit_stash;                // 1: the loss call keeps the logits of one row block instead of recomputing them
+    int l2_hints[UNITY_PROF_CLASSES]; // per GEMM class: GemmArgs::l2_hints
     int wide_acc;                   // 1: dHidden / dW chunk GEMMs use 512-column tiles (CTA pairs only)
     unsigned round_total;           // arrivals accumulated so far on the rendezvous counter (d_status + 16)
 };
@@ -292,6 +293,7 @@ int launch_forward(unity_ctx* ctx, const unity_rows* r, int slot0, int rows, flo
     g.stats = stats; g.stats_pitch = rows;
     g.target_p = target_p; g.vocab0 = 0; g.scale = r->inv_temperature;
     g.status = ctx->d_status;
+    g.l2_hints = ctx->l2_hints[UNITY_PROF_FWD_GEMM];
     if (z) {
         g.Z = z->Z; g.ldz = z->ldz; g.z_chunk_stride = z->chunk_stride; g.z_chunk_cols = z->chunk_cols; g.z_chunks = z->chunks;
         g.g_wide_store = (reinterpret_cast<uintptr_t>(z->Z) % 32 == 0) && (z->ldz * 2 % 32 == 0) && (z->chunk_stride * 2 % 32 == 0) &&
@@ -417,6 +419,12 @@ int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace
     c->chunk_rows_mult = kDefaultChunkMult;
     c->chunk_vocab_mult = kDefaultChunkMult;
     c->wide_acc = 1;
+    // forward / recompute: the round's hidden rows are kept (evict last) while the W stream passes (evict first); the
+    // logit-gradient chunk is written evict-first, it is far larger than L2 and not read again by the same kernel
+    c->l2_hints[UNITY_PROF_FWD_GEMM] = 2 | (1 << 2);
+    c->l2_hints[UNITY_PROF_GRAD_GEMM] = 2 | (1 << 2) | (1 << 4);
+    c->l2_hints[UNITY_PROF_DH_GEMM] = 0;
+    c->l2_hints[UNITY_PROF_DW_GEMM] = 0;
     c->logit_stash = 0;
     c->ev_pool = new (std::nothrow) std::vector<cudaEvent_t>();
     c->ev_class = new (std::nothrow) std::vector<int>();
@@ -509,6 +517,10 @@ int unity_set_option(unity_ctx* ctx, int option, int value) {
     if (option == UNITY_OPT_CHUNK_ROWS && value >= 1 && value <= 8) { ctx->chunk_rows_mult = value; return UNITY_OK; }
     if (option == UNITY_OPT_CHUNK_VOCAB && value >= 1 && value <= 8) { ctx->chunk_vocab_mult = value; return UNITY_OK; }
     if (option == UNITY_OPT_LOGIT_STASH && (value == 0 || value == 1)) { ctx->logit_stash = value; return UNITY_OK; }
+    if (option >= UNITY_OPT_L2_HINTS_FWD && option < UNITY_OPT_L2_HINTS_FWD + UNITY_PROF_CLASSES && value >= 0 && value < 64) {
+        ctx->l2_hints[option - UNITY_OPT_L2_HINTS_FWD] = value;
+        return UNITY_OK;
+    }
     if (option == UNITY_OPT_WIDE_ACC && (value == 0 || value == 1)) { ctx->wide_acc = value; return UNITY_OK; }
     return fail(ctx, UNITY_ERR_INVALID_ARG, "unknown option %d or value %d out of range", option, value);
 }
@@ -940,6 +952,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                             g.target_p = L.target_p; g.vocab0 = v0 + q0; g.scale = rows->inv_temperature;
                             g.coef_a = L.coef_a; g.coef_b = L.coef_b; g.row_lse = L.row_lse; g.row_ent = L.row_ent;
                             g.has_ent = params->ent_coef != 0.f;
+                            g.l2_hints = ctx->l2_hints[UNITY_PROF_GRAD_GEMM];
                             g.G = Gc + static_cast<long long>(r0) * cv + q0; g.ldg = cv; g.status = ctx->d_status;
                             g.g_wide_store = (reinterpret_cast<uintptr_t>(g.G) % 32 == 0) && (g.ldg * 2 % 32 == 0);
                             if (ctx->chunk_sync & 1) {
@@ -964,6 +977,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 h.group_m = ctx->chunk_group[1] / c_dh > 0 ? ctx->chunk_group[1] / c_dh : 1;
                 h.a_row0 = 0; h.a_k0 = 0; h.b_row0 = 0; h.b_k0 = v0; h.m_rows = nc; h.n_cols = H;
                 h.C = L.dHc; h.ldc = H; h.beta = v0 > 0; h.status = ctx->d_status;
+                h.l2_hints = ctx->l2_hints[UNITY_PROF_DH_GEMM];
                 if (ctx->chunk_sync & 2) {
                     h.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
                     h.round_base = ctx->round_total;
@@ -981,6 +995,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 w.a_row0 = 0; w.a_k0 = 0; w.b_row0 = 0; w.b_k0 = slot0; w.m_rows = vc; w.n_cols = H;
                 w.C = dWk + static_cast<long long>(v0) * H; w.ldc = H;
                 w.beta = (params->accumulate_dW || c0 > 0) ? 1 : 0; w.status = ctx->d_status;
+                w.l2_hints = ctx->l2_hints[UNITY_PROF_DW_GEMM];
                 if (ctx->chunk_sync & 4) {
                     w.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
                     w.round_base = ctx->round_total;
