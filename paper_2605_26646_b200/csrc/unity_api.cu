@@ -184,7 +184,7 @@ void vocab_chunks(int V, int cv, int* base_out, int* n_out) {
     *base_out = base;
     *n_out = n;
 }
-// Row block of the logit stash: 72 row tiles, so that the forward kernel's rounds (18 row tiles x 4 vocabulary splits
+// Row block of the logit stash: 72 row tiles, so that the forward kernel's rounds (24 row tiles x 3 vocabulary splits
 // on 74 CTA pairs) are whole.
 constexpr int kStashRows = 72 * kTileM;
 
@@ -241,8 +241,8 @@ struct RowPlan {
 
 // Shape of one forward launch over `rows` packed rows (a multiple of the row tile): row tiles per round and
 // vocabulary splits.  One round of the persistent kernel = gm row tiles x splits vocabulary splits <= number of
-// workers (CTAs or CTA pairs): gm bounds the hidden rows that must stay L2 resident (a quarter of the workers, about
-// 4.7 k rows), splits fill the machine.
+// workers (CTAs or CTA pairs): gm bounds the hidden rows that must stay L2 resident (48 tiles of 128 rows by default:
+// 6 k rows, 44 MB at H = 3584, loaded with an evict-last hint), splits fill the machine.
 void forward_shape(const unity_ctx* ctx, int V, int rows, int* gm_out, int* splits_out, int* tps_out) {
     const int ctas = ctx->ctas[UNITY_PROF_FWD_GEMM];
     const int m_tiles = rows / gemm_tile_rows(ctas);
@@ -413,7 +413,7 @@ int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace
     c->ctas[UNITY_PROF_DW_GEMM] = 2;
     c->l2_promotion = 3;
     c->chunk_group[0] = c->chunk_group[1] = c->chunk_group[2] = 32;
-    c->fwd_group = 0;
+    c->fwd_group = 48;
     c->fwd_sync = 1;
     c->chunk_sync = 6;
     c->chunk_rows_mult = kDefaultChunkMult;
