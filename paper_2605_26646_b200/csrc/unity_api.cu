@@ -251,12 +251,22 @@ void forward_shape(const unity_ctx* ctx, int V, int rows, int* gm_out, int* spli
     int gmax = ctx->fwd_group > 0 ? ctx->fwd_group / ctas : n_pairs / 4;
     if (gmax < 1) gmax = 1;
     if (gmax > n_pairs) gmax = n_pairs;
-    const int n_grp = (m_tiles + gmax - 1) / gmax;
-    const int gm = n_grp > 0 ? (m_tiles + n_grp - 1) / n_grp : 1;
-    int splits = n_pairs / (gm > 0 ? gm : 1);
-    if (splits > 32) splits = 32;
-    if (splits > n_tiles) splits = n_tiles;
-    if (splits < 1) splits = 1;
+    // Among round sizes from two thirds of gmax up to gmax, take the one with the least work per worker: rounds x
+    // vocabulary tiles per split (a batch whose row tiles do not divide well would otherwise idle part of the machine
+    // or run a nearly empty last round); ties go to the larger round, which streams W less often.
+    int gm = 1, splits = 1;
+    long long best = -1;
+    const int cand_min = m_tiles <= gmax ? 1 : (2 * gmax + 2) / 3;      // few row tiles: any round size is L2-safe
+    for (int cand = gmax; cand >= cand_min; --cand) {
+        const int c = cand < m_tiles ? cand : (m_tiles > 0 ? m_tiles : 1);
+        int sp = n_pairs / c;
+        if (sp > 32) sp = 32;
+        if (sp > n_tiles) sp = n_tiles;
+        if (sp < 1) sp = 1;
+        const long long rounds = (m_tiles + c - 1) / c;
+        const long long cost = rounds * ((n_tiles + sp - 1) / sp);
+        if (best < 0 || cost < best) { best = cost; gm = c; splits = sp; }
+    }
     const int tps = (n_tiles + splits - 1) / splits;
     *gm_out = gm > 0 ? gm : 1;
     *splits_out = (n_tiles + tps - 1) / tps;
