@@ -367,6 +367,18 @@ def test_model_without_rows_and_three_models():
     run_all_stages(small_workload(128, 1024, 300, role_model=[0, 1, 0], K=3))
 
 
+def test_sixteen_models_and_sixty_four_roles():
+    # the limits of the interface: UNITY_MAX_MODELS models, UNITY_MAX_ROLES roles (most groups x role segments are tiny)
+    w = wl.make_structure("search", cut_rows=1500, cut_max_len=32, H=128, V=1024 + 72)
+    R, K = ub.UNITY_MAX_ROLES, ub.UNITY_MAX_MODELS
+    s = torch.arange(w.n_inv)
+    w.inv_role = ((w.inv_role.long() + 3 * (s % 22)) % R).to(torch.int32)
+    w.n_roles, w.K = R, K
+    w.role_model = (torch.arange(R) % K).to(torch.int32)
+    w.lam = torch.ones(R, 3)
+    run_all_stages(wl.materialize(w, device="cuda"))
+
+
 def test_all_rows_masked_and_single_row():
     w = small_workload(128, 1024, 200)
     w.tok_mask.zero_()
