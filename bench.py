@@ -397,6 +397,34 @@ def main():
         shortcut = {"value": n_valid_total / (float(t3.item()) / 2 * 1e-3), "unit": UNIT, "steps": 2,
                     "note": "loss call given logp/entropy/lse of unity_logprob_fwd (first PPO epoch): forward sweep skipped"}
 
+    # ---------------------------------------------------------------- extras: the log-prob call alone, and one iteration
+    # A PPO iteration of a worker group evaluates old and reference log-probs before the update: advantage +
+    # 2 x unity_logprob_fwd + unity_ppo_loss_fwd_bwd.
+    fwd_extra = iter_extra = None
+    if not args.no_e2e:
+        def fwd_call():
+            ctx.logprob_fwd(w.hidden, w.W, d_cu, d_inv_role, role_model, d_tgt, d_mask, w.inv_temperature, logp, ent, lse0)
+        fwd_call()
+        sync_all()
+        e0.record()
+        for _ in range(2):
+            fwd_call()
+        e1.record()
+        sync_all()
+        t_f = e0.elapsed_time(e1) / 2
+        e0.record()
+        fwd_call()
+        fwd_call()
+        step(w.hidden, d_tgt, d_mask, old, ref)
+        e1.record()
+        sync_all()
+        t_i = e0.elapsed_time(e1)
+        ctx.check_status()
+        fwd_extra = {"value": n_valid_local / (t_f * 1e-3), "unit": UNIT, "ms": t_f,
+                     "tflops": 2.0 * H * V * n_valid_local / (t_f * 1e-3) / 1e12, "note": "unity_logprob_fwd alone (this rank)"}
+        iter_extra = {"value": n_valid_local / (t_i * 1e-3), "unit": UNIT, "ms": t_i,
+                      "note": "advantage + 2 x unity_logprob_fwd (old, reference) + unity_ppo_loss_fwd_bwd (this rank)"}
+
     # ---------------------------------------------------------------- extra (not the headline): logit stash
     # The loss call keeps the bf16 logits of one block of 18432 rows (about 6 GB) and turns them into dL/dz in place
     # instead of recomputing them: 6*H*V executed flop per token.  Same outputs within the parity tolerances.
@@ -528,7 +556,8 @@ def main():
             "tensor_frac_of_peak_executed_8HV": step_tflops_exe / peak,
             "tensor_frac_of_burst_peak_algorithmic_6HV": step_tflops_alg / peaks["tflops_burst"],
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "kernels": kern,
-            "on_policy_shortcut": shortcut, "logit_stash": stash_extra, "cpu_baseline": cpu_baseline}
+            "on_policy_shortcut": shortcut, "logit_stash": stash_extra, "logprob_fwd": fwd_extra, "iteration": iter_extra,
+            "cpu_baseline": cpu_baseline}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
