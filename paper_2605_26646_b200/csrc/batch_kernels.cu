@@ -207,33 +207,62 @@ __global__ void k_batch_gather(const int* __restrict__ order, const int64_t* __r
         const T* from = src + src_cu[s] * units_per_row;
         T* to = dst + out_cu[j] * units_per_row;
         const long long stride = static_cast<long long>(gridDim.y) * blockDim.x;
-        for (long long i = static_cast<long long>(blockIdx.y) * blockDim.x + threadIdx.x; i < n_slot; i += stride)
-            to[i] = i < n_copy ? from[i] : pad;
+        // four units per thread and step, loads issued before the stores
+        for (long long i = static_cast<long long>(blockIdx.y) * blockDim.x + threadIdx.x; i < n_slot; i += 4 * stride) {
+            T v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const long long q = i + u * stride;
+                v[u] = q < n_copy ? from[q] : pad;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const long long q = i + u * stride;
+                if (q < n_slot) to[q] = v[u];
+            }
+        }
     }
 }
 
-// Delayed rewards: one warp per invocation walks it backwards; the first unmasked token met takes the reward.
+// Delayed rewards: one warp per invocation.  The sequence is zero-filled front to back, 16 tokens per lane and step
+// (one 128-bit mask load, four 128-bit stores) once the index is a multiple of 16; every lane remembers the last
+// unmasked token it saw, the warp takes the maximum, and after the warp's stores are ordered that token gets the reward.
 __global__ void k_align_rewards(int n_inv, const int64_t* __restrict__ cu, const uint8_t* __restrict__ mask,
-                                const float* __restrict__ r_inv, float* __restrict__ tok_reward) {
+                                const float* __restrict__ r_inv, float* __restrict__ tok_reward, int vec_ok) {
     const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (s >= n_inv) return;
     const long long lo = cu[s], hi = cu[s + 1];
-    const float r = r_inv[s];
-    bool placed = false;
-    for (long long c0 = hi - 32; c0 > lo - 32; c0 -= 32) {
-        const long long t = c0 + lane;
-        const bool in = t >= lo && t < hi;
-        const bool on = in && (mask ? mask[t] != 0 : true);
-        const unsigned valid = __ballot_sync(kFull, on);
-        float out = 0.f;
-        if (!placed && valid) {
-            const int last = 31 - __clz(valid);
-            if (lane == last) out = r;
-            placed = true;
-        }
-        if (in) tok_reward[t] = out;
+    long long last = -1;
+    const long long head_end = vec_ok ? min(hi, (lo + 15) & ~15LL) : hi;
+    for (long long t = lo + lane; t < head_end; t += 32) {
+        tok_reward[t] = 0.f;
+        if (mask == nullptr || mask[t]) last = t;
     }
+    const long long n_vec = (hi - head_end) >> 4;
+    for (long long q = lane; q < n_vec; q += 32) {
+        const long long t = head_end + (q << 4);
+        float4* out = reinterpret_cast<float4*>(tok_reward + t);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) out[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (mask == nullptr) {
+            last = t + 15;
+        } else {
+            const uint4 m = *reinterpret_cast<const uint4*>(mask + t);
+            const unsigned w[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (w[j]) last = t + 4 * j + ((31 - __clz(__vcmpne4(w[j], 0u))) >> 3);   // highest non-zero byte
+        }
+    }
+    for (long long t = head_end + (n_vec << 4) + lane; t < hi; t += 32) {
+        tok_reward[t] = 0.f;
+        if (mask == nullptr || mask[t]) last = t;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) last = max(last, __shfl_xor_sync(kFull, last, o));
+    __syncwarp();                                   // the zero stores of all lanes are ordered before the reward's
+    if (lane == 0 && last >= 0) tok_reward[last] = r_inv[s];
 }
 
 template <typename T>
@@ -295,7 +324,8 @@ cudaError_t launch_batch_gather(const GatherArgs& g, cudaStream_t stream) {
 cudaError_t launch_align_rewards(int n_inv, const int64_t* cu, const uint8_t* mask, const float* r_inv,
                                  float* tok_reward, cudaStream_t stream) {
     if (n_inv == 0) return cudaSuccess;
-    k_align_rewards<<<(n_inv + 7) / 8, 256, 0, stream>>>(n_inv, cu, mask, r_inv, tok_reward);
+    const int vec_ok = (reinterpret_cast<uintptr_t>(mask) & 15) == 0 && (reinterpret_cast<uintptr_t>(tok_reward) & 15) == 0;
+    k_align_rewards<<<(n_inv + 7) / 8, 256, 0, stream>>>(n_inv, cu, mask, r_inv, tok_reward, vec_ok);
     return cudaGetLastError();
 }
 

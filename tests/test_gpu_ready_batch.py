@@ -116,3 +116,24 @@ def test_align_rewards_full_size(name, masked):
     want = orc.align_rewards(r.numpy(), w.cu_seqlens.numpy(), None if mask is None else mask.numpy())
     assert np.array_equal(out.cpu().numpy().astype(np.float64), want)
     ctx.close()
+
+
+def test_align_rewards_unaligned_views_and_all_masked_sequences():
+    w = wl.make_structure("rag_qa")
+    r = wl.normal(33, 1, w.n_inv)
+    mask = w.tok_mask.clone()
+    lo, hi = int(w.cu_seqlens[5]), int(w.cu_seqlens[6])
+    mask[lo:hi] = 0                                            # a sequence without any unmasked token drops its reward
+    ctx = ub.Context(0, 1 << 20)
+    m_dev = torch.cat([torch.zeros(1, dtype=torch.uint8), mask]).cuda()[1:]          # pointers off by one element
+    out = torch.full((w.n_tok + 1,), 7.0, device="cuda")[1:]
+    ctx.align_rewards(w.cu_seqlens.cuda(), m_dev, r.cuda(), out)
+    ctx.check_status()
+    want = orc.align_rewards(r.numpy(), w.cu_seqlens.numpy(), mask.numpy())
+    assert np.array_equal(out.cpu().numpy().astype(np.float64), want) and np.all(want[lo:hi] == 0)
+    # the aligned path on the same data
+    out2 = torch.full((w.n_tok,), 7.0, device="cuda")
+    ctx.align_rewards(w.cu_seqlens.cuda(), mask.cuda(), r.cuda(), out2)
+    ctx.check_status()
+    assert np.array_equal(out2.cpu().numpy().astype(np.float64), want)
+    ctx.close()
