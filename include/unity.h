@@ -94,7 +94,7 @@ int unity_set_profiling(unity_ctx* ctx, int enable);
 #define UNITY_OPT_CHUNK_VOCAB 7   /* gradient chunk vocabulary entries = value x 18944 (default 2)                      */
 #define UNITY_OPT_FWD_GROUP 8     /* 128-row tiles per round of the forward kernel (default 48; 0 = a quarter of the SMs) */
 #define UNITY_OPT_FWD_SYNC 9      /* 1 (default): workers of the forward kernel meet at each round start (bounded wait) */
-#define UNITY_OPT_CHUNK_SYNC 10   /* same for the gradient-chunk GEMMs: bit 0 recompute, bit 1 dHidden, bit 2 dW (default 6) */
+#define UNITY_OPT_CHUNK_SYNC 10   /* same for the gradient-chunk GEMMs: bit 0 recompute, bit 1 dHidden, bit 2 dW (default 7) */
 #define UNITY_OPT_WIDE_ACC 11     /* 1 (default): the dHidden / dW chunk GEMMs of CTA pairs use 256 x 512 output tiles    */
 #define UNITY_OPT_GROUP_GRAD 12   /* raster group of the recompute GEMM alone, in 128-row tiles                           */
 #define UNITY_OPT_GROUP_DH 13     /* ... of the dHidden GEMM                                                               */

@@ -425,7 +425,7 @@ int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace
     c->chunk_group[0] = c->chunk_group[1] = c->chunk_group[2] = 32;
     c->fwd_group = 48;
     c->fwd_sync = 1;
-    c->chunk_sync = 6;
+    c->chunk_sync = 7;
     c->chunk_rows_mult = kDefaultChunkMult;
     c->chunk_vocab_mult = kDefaultChunkMult;
     c->wide_acc = 1;
