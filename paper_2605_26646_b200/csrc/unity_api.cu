@@ -893,10 +893,19 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
         if ((rc = make_tmap(ctx, &tm_hp_k, L.hp, H, P.n_slots, static_cast<uint64_t>(H) * 2, kBoxRows))) return rc;
         if ((rc = make_tmap(ctx, &tm_hp_mn, L.hp, H, P.n_slots, static_cast<uint64_t>(H) * 2, kTileK))) return rc;
     }
-    const bool wide_dh = ctx->wide_acc && ctx->ctas[UNITY_PROF_DH_GEMM] == 2;
-    const bool wide_dw = ctx->wide_acc && ctx->ctas[UNITY_PROF_DW_GEMM] == 2;
-    const int h_tiles_dh = (H + gemm_tile_cols(wide_dh) - 1) / gemm_tile_cols(wide_dh);
-    const int h_tiles_dw = (H + gemm_tile_cols(wide_dw) - 1) / gemm_tile_cols(wide_dw);
+    // 512-column tiles unless 256-column tiles waste clearly less of this launch: the share of executed MMA work that
+    // is useful = (H / padded columns) x (tiles / tiles rounded up to whole waves of CTA pairs); the wide form gets a
+    // 4 % bonus for its lower operand traffic.
+    const int n_workers = ctx->sm_count / 2;
+    auto pick_wide = [&](int cls, int m_tiles) {
+        if (!ctx->wide_acc || ctx->ctas[cls] != 2) return false;
+        auto useful = [&](int cols) {
+            const long long nt = (H + cols - 1) / cols, tiles = nt * m_tiles;
+            const long long waves = (tiles + n_workers - 1) / n_workers;
+            return (static_cast<double>(H) / (nt * cols)) * (static_cast<double>(tiles) / (waves * n_workers));
+        };
+        return m_tiles <= 0 || 1.04 * useful(2 * kTileN) >= useful(kTileN);
+    };
     const int c_grad = ctx->ctas[UNITY_PROF_GRAD_GEMM], c_dh = ctx->ctas[UNITY_PROF_DH_GEMM],
               c_dw = ctx->ctas[UNITY_PROF_DW_GEMM];
 
@@ -983,7 +992,9 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 // (2) dH_chunk[nc, H] (+)= G[nc, vc] * W[v0:v0+vc, :]      (B = W, MN-major: rows v are K)
                 GemmArgs h;
                 memset(&h, 0, sizeof(h));
-                h.m_tiles = nc / gemm_tile_rows(c_dh); h.n_tiles = h_tiles_dh; h.k_iters = (vc + kTileK - 1) / kTileK;
+                const bool wide_dh = pick_wide(UNITY_PROF_DH_GEMM, nc / gemm_tile_rows(c_dh));
+                h.m_tiles = nc / gemm_tile_rows(c_dh); h.n_tiles = (H + gemm_tile_cols(wide_dh) - 1) / gemm_tile_cols(wide_dh);
+                h.k_iters = (vc + kTileK - 1) / kTileK;
                 h.group_m = ctx->chunk_group[1] / c_dh > 0 ? ctx->chunk_group[1] / c_dh : 1;
                 h.a_row0 = 0; h.a_k0 = 0; h.b_row0 = 0; h.b_k0 = v0; h.m_rows = nc; h.n_cols = H;
                 h.C = L.dHc; h.ldc = H; h.beta = v0 > 0; h.status = ctx->d_status;
@@ -1000,7 +1011,9 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 // (3) dW[v0:v0+vc, :] (+)= G^T[vc, nc] * hidden[slot0:slot0+nc, :]   (both operands MN-major)
                 GemmArgs w;
                 memset(&w, 0, sizeof(w));
-                w.m_tiles = (vc + gemm_tile_rows(c_dw) - 1) / gemm_tile_rows(c_dw); w.n_tiles = h_tiles_dw; w.k_iters = nc / kTileK;
+                w.m_tiles = (vc + gemm_tile_rows(c_dw) - 1) / gemm_tile_rows(c_dw);
+                const bool wide_dw = pick_wide(UNITY_PROF_DW_GEMM, w.m_tiles);
+                w.n_tiles = (H + gemm_tile_cols(wide_dw) - 1) / gemm_tile_cols(wide_dw); w.k_iters = nc / kTileK;
                 w.group_m = ctx->chunk_group[2] / c_dw > 0 ? ctx->chunk_group[2] / c_dw : 1;
                 w.a_row0 = 0; w.a_k0 = 0; w.b_row0 = 0; w.b_k0 = slot0; w.m_rows = vc; w.n_cols = H;
                 w.C = dWk + static_cast<long long>(v0) * H; w.ldc = H;
