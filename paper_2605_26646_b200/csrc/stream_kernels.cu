@@ -761,7 +761,7 @@ __global__ void k_value_main(ValueArgs a) {
     if (s >= a.n_inv) return;
     const int role = a.inv_role[s];
     const bool role_ok = role >= 0 && role < a.n_roles && a.role_model[role] >= 0 && a.role_model[role] < a.K;
-    const float M = role_ok ? a.Mk[a.role_model[role]] : 1.f;
+    const float inv_M = 1.f / (role_ok ? a.Mk[a.role_model[role]] : 1.f);
     const long long lo = a.cu_seqlens[s], hi = a.cu_seqlens[s + 1];
     float sum = 0.f, clp = 0.f;
     auto one = [&](long long i) {
@@ -769,7 +769,7 @@ __global__ void k_value_main(ValueArgs a) {
         float l = 0.f, gr = 0.f;
         if (on) {
             const ValueTerm t = value_term(a.values[i], a.old_values[i], a.returns[i], a.clip_v);
-            l = t.loss; gr = t.grad / M; sum += t.loss; clp += t.clipped;
+            l = t.loss; gr = t.grad * inv_M; sum += t.loss; clp += t.clipped;
         }
         a.dvalues[i] = gr;
         if (a.tok_loss) a.tok_loss[i] = l;
@@ -794,7 +794,7 @@ __global__ void k_value_main(ValueArgs a) {
                 g4[j] = 0.f; l4[j] = 0.f;
                 if (role_ok && ((m4 >> (8 * j)) & 0xffu)) {
                     const ValueTerm t = value_term(vv[j], oo[j], rr[j], a.clip_v);
-                    l4[j] = t.loss; g4[j] = t.grad / M; sum += t.loss; clp += t.clipped;
+                    l4[j] = t.loss; g4[j] = t.grad * inv_M; sum += t.loss; clp += t.clipped;
                 }
             }
             *reinterpret_cast<float4*>(a.dvalues + i) = make_float4(g4[0], g4[1], g4[2], g4[3]);
