@@ -137,3 +137,32 @@ def test_align_rewards_unaligned_views_and_all_masked_sequences():
     ctx.check_status()
     assert np.array_equal(out2.cpu().numpy().astype(np.float64), want)
     ctx.close()
+
+
+def test_ready_batch_many_partitions_sixteen_models_and_zero_length_invocations():
+    # more partitions than invocations per model (most are empty), the largest model count, invocations of length 0
+    w = wl.make_structure("search", cut_rows=2000, cut_max_len=40)      # most invocations keep no tokens at all
+    R, K = ub.UNITY_MAX_ROLES, ub.UNITY_MAX_MODELS
+    s = torch.arange(w.n_inv)
+    inv_role = ((w.inv_role.long() + 3 * (s % 22)) % R).to(torch.int32)
+    role_model = [(v * 7) % K if v % 5 else -1 for v in range(R)]      # every fifth role is not trained
+    done = (wl.uniform(34, 1, w.n_traj) < 0.6).to(torch.uint8)
+    n_parts, pad_to, seed = 300, 32, 123456789
+    ctx = ub.Context(0, 1 << 22)
+    order = torch.full((w.n_inv,), 7, dtype=torch.int32, device="cuda")
+    out_cu = torch.full((w.n_inv + 1,), 7, dtype=torch.int64, device="cuda")
+    mo = torch.full((K + 1,), 7, dtype=torch.int32, device="cuda")
+    po = torch.full((K * n_parts + 1,), 7, dtype=torch.int32, device="cuda")
+    totals = torch.full((2,), 7, dtype=torch.int64, device="cuda")
+    ctx.ready_batch_plan(w.cu_seqlens.cuda(), inv_role.cuda(), w.inv_traj.cuda(), done.cuda(), role_model, K, seed,
+                         n_parts, pad_to, order, out_cu, mo, po, totals)
+    ctx.check_status()
+    o = orc.ready_batch_plan(w.cu_seqlens.numpy(), inv_role.numpy(), w.inv_traj.numpy(), done.numpy(), role_model, K,
+                             seed, n_parts=n_parts, pad_to=pad_to)
+    n_kept = o["n_kept"]
+    assert totals.tolist() == [n_kept, o["n_tok"]] and n_kept > 0
+    assert np.array_equal(order.cpu().numpy()[:n_kept], o["order"])
+    assert np.array_equal(out_cu.cpu().numpy()[:n_kept + 1], o["out_cu"])
+    assert np.array_equal(mo.cpu().numpy(), o["model_offsets"])
+    assert np.array_equal(po.cpu().numpy(), o["part_offsets"])
+    ctx.close()
