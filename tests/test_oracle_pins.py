@@ -679,3 +679,114 @@ def test_ready_batch_plan_hand_case_gather_and_reward_alignment():
     # invocation's reward: the delayed reward reaches the whole response
     A, _ = orc.gae(r, np.zeros(10), cu, 1.0, 1.0, mask)
     assert A.tolist() == [0.5, 0.5, 0, -1.0, -1.0, 0, 0, 0, 0, 3.0]
+
+
+# ---------------------------------------------------------------------------- metric records (per model / per role)
+# Section "Parameter Sharing in the System": role identity and agent-level metrics are kept even when roles share
+# parameters; paragraph "Batch construction": role identifiers are preserved for role-specific analysis.
+
+METRIC_NAMES = ["n", "pg", "kl", "entropy", "clip_frac", "ratio", "logp", "adv"]
+
+
+def brute_force_records(p, cur_logp, cur_ent, old, ref, adv, lo, hi, kl_mode, keys, n_classes):
+    """The eight numbers of every class, token by token with python scalars; `keys[i]` is the class of token i.
+    Independent of the oracle's own per-token intermediates: it starts from the (separately pinned) log-probs and
+    entropies and restates each quantity's definition."""
+    acc = [[0.0] * 8 for _ in range(n_classes)]
+    for i in range(len(cur_logp)):
+        if not p["tok_mask"][i]:
+            continue
+        c = int(keys[i])
+        ratio = math.exp(cur_logp[i] - old[i])
+        un = -ratio * adv[i]
+        cl = -min(max(ratio, 1.0 - lo), 1.0 + hi) * adv[i]
+        d = ref[i] - cur_logp[i]
+        kl = {1: -d, 2: 0.5 * d * d, 3: math.exp(d) - d - 1.0}[kl_mode]
+        row = [1.0, max(un, cl), kl, cur_ent[i], 1.0 if cl > un else 0.0, ratio, cur_logp[i], adv[i]]
+        for j in range(8):
+            acc[c][j] += row[j]
+    out = np.zeros((n_classes, 8))
+    for c in range(n_classes):
+        n = acc[c][0]
+        out[c, 0] = n
+        for j in range(1, 8):
+            out[c, j] = acc[c][j] / max(n, 1.0)
+    return out
+
+
+@pytest.mark.parametrize("K,R,role_model,kl_mode", [(1, 2, [0, 0], 3), (2, 3, [0, 0, 1], 3), (2, 3, [0, 0, 1], 2),
+                                                   (2, 4, [1, 0, 1, 0], 1)])
+def test_metric_records_match_brute_force_per_model_and_per_role(K, R, role_model, kl_mode):
+    p = tiny_problem(seed=40 + R, n_inv=16, H=8, V=12, K=K, R=R, max_len=6, mask_p=0.7)
+    p["role_model"] = np.array(role_model)
+    f = fwd(p)
+    rng = np.random.default_rng(5)
+    N = f["logp"].size
+    old = f["logp"] + 0.3 * rng.normal(size=N)           # wide ratios: both clip branches occur
+    ref = f["logp"] + 0.2 * rng.normal(size=N)
+    adv = rng.normal(size=N) + 0.3
+    lo, hi = 0.2, 0.3
+    out = ppo(p, old, ref, adv, clip_lo=lo, clip_hi=hi, kl_coef=0.1, kl_mode=kl_mode, ent_coef=0.01, n_roles=R)
+    tok_inv = np.repeat(np.arange(len(p["inv_role"])), np.diff(p["cu_seqlens"]))
+    tok_role = p["inv_role"][tok_inv]
+    tok_model = p["role_model"][tok_role]
+    bm = brute_force_records(p, f["logp"], f["entropy"], old, ref, adv, lo, hi, kl_mode, tok_model, K)
+    br = brute_force_records(p, f["logp"], f["entropy"], old, ref, adv, lo, hi, kl_mode, tok_role, R)
+    assert out["metrics_model"].shape == (K, 8) and out["metrics_role"].shape == (R, 8)
+    assert np.abs(out["metrics_model"] - bm).max() < 1e-12
+    assert np.abs(out["metrics_role"] - br).max() < 1e-12
+    # the fixture must be able to tell columns and classes apart: no two columns and no two roles coincide, both
+    # clip branches occur, and roles that share a model still have different records
+    assert 0.0 < br[:, 4].max() and br[:, 4].min() < 1.0
+    for a in range(8):
+        for b in range(a + 1, 8):
+            assert np.abs(br[:, a] - br[:, b]).max() > 1e-3, (METRIC_NAMES[a], METRIC_NAMES[b])
+    shared = [v for v in range(R) if role_model.count(role_model[v]) > 1]
+    assert len(shared) >= 2 and np.abs(br[shared[0], 1:] - br[shared[1], 1:]).max() > 1e-3
+    # per-model counts are the sums of their roles' counts; per-model means are the count-weighted role means
+    for k in range(K):
+        roles_k = [v for v in range(R) if role_model[v] == k]
+        n_k = sum(br[v, 0] for v in roles_k)
+        assert out["metrics_model"][k, 0] == n_k
+        for j in range(1, 8):
+            assert abs(out["metrics_model"][k, j] - sum(br[v, 0] * br[v, j] for v in roles_k) / max(n_k, 1.0)) < 1e-12
+
+
+def test_metric_records_closed_form_columns():
+    """Every column gets a different known value: W = 0 makes logp = -ln V and entropy = ln V on every row; old =
+    logp - delta makes the ratio e^delta (inside the clip range, so nothing is clipped); ref = logp + d0 makes
+    the k3 term e^d0 - d0 - 1; a constant advantage c makes the surrogate -c e^delta."""
+    V, c, delta, d0 = 16, 0.75, 0.1, 0.3
+    p = tiny_problem(seed=50, n_inv=10, V=V, K=2, R=3)
+    p["role_model"] = np.array([0, 0, 1])
+    p["W"] = [np.zeros_like(w) for w in p["W"]]
+    N = p["hidden"].shape[0]
+    lp = np.full(N, -math.log(V))
+    out = ppo(p, lp - delta, lp + d0, np.full(N, c), kl_coef=0.1, kl_mode=3, ent_coef=0.0, n_roles=3)
+    valid = p["tok_mask"] != 0
+    tok_inv = np.repeat(np.arange(10), np.diff(p["cu_seqlens"]))
+    tok_role = p["inv_role"][tok_inv]
+    expect = [None, -c * math.exp(delta), math.exp(d0) - d0 - 1.0, math.log(V), 0.0, math.exp(delta), -math.log(V), c]
+    for v in range(3):
+        rec = out["metrics_role"][v]
+        assert rec[0] == float((valid & (tok_role == v)).sum()) and rec[0] > 0
+        for j in range(1, 8):
+            assert abs(rec[j] - expect[j]) < 1e-13, METRIC_NAMES[j]
+    for k, roles_k in enumerate([(0, 1), (2,)]):
+        rec = out["metrics_model"][k]
+        assert rec[0] == float((valid & np.isin(tok_role, roles_k)).sum())
+        for j in range(1, 8):
+            assert abs(rec[j] - expect[j]) < 1e-13, METRIC_NAMES[j]
+
+
+def test_metric_record_of_a_role_without_valid_tokens_is_zero():
+    p = tiny_problem(seed=51, n_inv=9, K=1, R=3)
+    p["role_model"] = np.array([0, 0, 0])
+    tok_inv = np.repeat(np.arange(9), np.diff(p["cu_seqlens"]))
+    p["tok_mask"][p["inv_role"][tok_inv] == 1] = 0            # role 1 present but fully masked
+    p["inv_role"][p["inv_role"] == 2] = 0                     # role 2 never invoked
+    cur = fwd(p)["logp"]
+    out = ppo(p, cur, cur, np.ones(cur.size), n_roles=3)
+    assert np.all(out["metrics_role"][1] == 0) and np.all(out["metrics_role"][2] == 0)
+    assert out["metrics_role"][0, 0] == out["metrics_model"][0, 0] == float((p["tok_mask"] != 0).sum())
+    assert np.abs(out["metrics_role"][0] - out["metrics_model"][0]).max() == 0
