@@ -116,8 +116,7 @@ def oracle_sample_run(w, n_rows, old, ref, adv):
     import numpy as np
     import torch
     from oracle import unity_oracle as orc
-    sys.path.insert(0, os.path.join(ROOT, "tests"))
-    import parity_util as pu
+    import parity_harness as pu
     rows = torch.nonzero(w.tok_mask)[:n_rows, 0].numpy()
     hid_bits = pu.bf16_bits(w.hidden)
     W_bits = [pu.bf16_bits(x) for x in w.W]
@@ -128,6 +127,22 @@ def oracle_sample_run(w, n_rows, old, ref, adv):
                          clip_lo=w.clip_lo, clip_hi=w.clip_hi, kl_coef=w.kl_coef, kl_mode=w.kl_mode,
                          ent_coef=w.ent_coef, inv_temperature=w.inv_temperature, n_roles=w.n_roles, rows=rows)
     return time.perf_counter() - t0, int(rows.size)
+
+
+def oracle_tiny_run():
+    """Time the fp64 oracle on the tiny configuration at full size: advantage, log-prob and loss forward + backward.
+    Returns (seconds, valid rows)."""
+    import numpy as np
+    import torch
+    import parity_harness as pu
+    from paper_2605_26646_b200 import workloads as wl
+    w = wl.make("tiny")
+    t0 = time.perf_counter()
+    oa = pu.oracle_advantage(w)
+    ol = pu.oracle_logprob(w)
+    cur = torch.from_numpy(ol["logp"].astype(np.float32))
+    pu.oracle_ppo(w, (cur + w.noise_old).numpy(), (cur + w.noise_ref).numpy(), oa["adv_tok"].astype(np.float32))
+    return time.perf_counter() - t0, int((w.tok_mask != 0).sum().item())
 
 
 def run_reference(args):
@@ -165,12 +180,12 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
-def run_micro(args):
+def measure_streaming():
     """Streaming stages at a size where they are HBM-bound rather than launch-bound, on 64 Mi tokens: role-level
     advantage (token broadcast), token-level GAE, clipped value loss, delayed-reward alignment and the ready-batch
     gather.  Prints one JSON line with achieved GB/s against the measured copy bandwidth.  Algorithmic bytes per token:
     advantage mask 1 + output 4; GAE rewards, values 8 + mask 1 + two outputs 8; value loss three inputs 12 + mask 1 +
-    gradient 4; alignment mask 1 + output 4; gather 2 x row bytes."""
+    gradient 4; alignment mask 1 + output 4; gather 2 x row bytes.  Returns the table as a dict."""
     import torch
     from paper_2605_26646_b200 import binding as ub
     from paper_2605_26646_b200 import workloads as wl
@@ -230,7 +245,182 @@ def run_micro(args):
            "ready_batch_plan": {"ms": t_plan, "note": "latency-bound: four small launches over the invocations"}}
     for k in ("role_advantage", "gae", "value_loss", "align_rewards", "ready_batch_gather_f32"):
         out[k]["frac"] = out[k]["gbs"] / peaks["hbm_gbs"]
-    print(json.dumps(out), flush=True)
+    ctx.close()
+    return out
+
+
+def run_micro(args):
+    print(json.dumps(measure_streaming()), flush=True)
+
+
+class Job:
+    """One configuration set up for timing: seeded inputs resident on the device, a context with its workspace, output
+    buffers, and `step()` = unity_role_advantage + unity_ppo_loss_fwd_bwd (+ the dW all-reduce when world > 1)."""
+
+    def __init__(self, workload, dev, rank=0, world=1, stash_room=False, opts=(), ctas=(), cut_rows=0):
+        import torch
+        import torch.distributed as dist
+        from paper_2605_26646_b200 import binding as ub
+        from paper_2605_26646_b200 import sharding
+        from paper_2605_26646_b200 import workloads as wl
+        self.world, self.dev = world, dev
+        kw = dict(seed_offset=1000 * rank)
+        if cut_rows:
+            kw.update(cut_rows=cut_rows)
+        w = self.w = wl.make(workload, device=dev, **kw)
+        n, H, V, K = w.n_tok, w.H, w.V, w.K
+        self.d_inv_role, self.d_inv_group, self.d_inv_traj = w.inv_role.to(dev), w.inv_group.to(dev), w.inv_traj.to(dev)
+        self.d_rn, self.d_rt, self.d_rj = w.r_node.to(dev), w.r_turn.to(dev), w.r_traj.to(dev)
+        self.d_cu, self.d_mask, self.d_tgt = w.cu_seqlens.to(dev), w.tok_mask.to(dev), w.target.to(dev)
+        self.role_model = w.role_model.tolist()
+        self.lam = w.lam.tolist()
+        ws_bytes = ub.unity_workspace_bytes(n, H, V, K, w.n_inv)
+        if stash_room:      # room for the optional logit stash too (reported as an extra; the headline step never uses it)
+            ws_bytes = max(ws_bytes, ub.unity_workspace_bytes_stash(n, H, V, K, w.n_inv))
+        extra = 0
+        mults = {6: 2, 7: 2}
+        mults.update({o: v for o, v in opts if o in (6, 7)})
+        if (mults[6], mults[7]) != (2, 2):         # non-default gradient chunks need their own G / dH scratch
+            extra = 2 * mults[6] * 18944 * (mults[7] * 18944 + 2048) + 4 * mults[6] * 18944 * H
+        ctx = self.ctx = ub.Context(dev.index, ws_bytes + extra)
+        for o, v in opts:
+            ctx.set_option(o, v)
+        for option, value in enumerate(ctas):
+            ctx.set_option(option, value)
+
+        self.adv_inv = torch.empty(w.n_inv, device=dev)
+        self.adv_tok = torch.empty(n, device=dev)
+        self.logp = torch.empty(n, device=dev)
+        self.ent = torch.empty(n, device=dev)
+        self.loss = torch.empty(K, device=dev)
+        self.metrics = torch.empty((K + w.n_roles) * ub.UNITY_N_METRICS, device=dev)
+        self.dH = torch.empty(n, H, device=dev, dtype=torch.bfloat16)
+        self.dW = [torch.empty(V, H, device=dev) for _ in range(K)]
+
+        # current log-probs (stage 2) give the old / reference log-probs of the batch: logp + N(0, 0.05)
+        self.lse0 = torch.empty(n, device=dev)
+        ctx.logprob_fwd(w.hidden, w.W, self.d_cu, self.d_inv_role, self.role_model, self.d_tgt, self.d_mask,
+                        w.inv_temperature, self.logp, self.ent, self.lse0)
+        ctx.check_status()
+        self.logp0, self.ent0 = self.logp.clone(), self.ent.clone()
+        self.old = self.logp + w.noise_old.to(dev)
+        self.ref = self.logp + w.noise_ref.to(dev)
+
+        # per-model valid-row counts: the only quantity the ranks must agree on before the step
+        tok_inv = torch.repeat_interleave(torch.arange(w.n_inv), w.cu_seqlens[1:] - w.cu_seqlens[:-1])
+        tok_model = w.role_model[w.inv_role.long()[tok_inv]].long()
+        counts = sharding.local_counts(tok_model, w.tok_mask, K)
+        self.n_valid_local = int(counts.sum().item())
+        self.norm = None
+        self.n_valid_total = self.n_valid_local
+        if world > 1:
+            self.norm = sharding.global_norm(counts.to(dev))
+            tot = torch.tensor([float(self.n_valid_local)], device=dev, dtype=torch.float64)
+            dist.all_reduce(tot)
+            self.n_valid_total = int(tot.item())
+
+    def step(self, hid=None, tgt=None, msk=None, o=None, r=None):
+        from paper_2605_26646_b200 import sharding
+        w, ctx = self.w, self.ctx
+        hid = w.hidden if hid is None else hid
+        tgt = self.d_tgt if tgt is None else tgt
+        msk = self.d_mask if msk is None else msk
+        o = self.old if o is None else o
+        r = self.ref if r is None else r
+        ctx.role_advantage(w.n_traj, w.n_roles, w.n_groups, self.d_inv_role, self.d_inv_group, self.d_inv_traj,
+                           self.d_rn, self.d_rt, self.d_rj, self.lam, w.adv_eps, w.adv_ddof, self.d_cu, msk,
+                           self.adv_inv, self.adv_tok)
+        ctx.ppo_loss_fwd_bwd(hid, w.W, self.d_cu, self.d_inv_role, self.role_model, tgt, msk, w.inv_temperature,
+                             w.clip_lo, w.clip_hi, w.kl_coef, w.kl_mode, w.ent_coef, self.norm, False, o, r,
+                             self.adv_tok, self.loss, self.metrics, self.logp, self.ent, None, self.dH, self.dW)
+        if self.world > 1:
+            sharding.allreduce_grads(self.dW)
+
+    def sync_all(self):
+        import torch
+        import torch.distributed as dist
+        torch.cuda.synchronize()
+        if self.world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def measure(self, steps, warmup, sample_clocks=True):
+        """`warmup` untimed steps, then `steps` steps between CUDA events (barrier + synchronize on both sides, maximum
+        over ranks), SM clocks sampled meanwhile and every GEMM launch bracketed by the library's own event pairs."""
+        import torch
+        import torch.distributed as dist
+        ctx = self.ctx
+        for _ in range(warmup):
+            self.step()
+        ctx.check_status()
+        sampler = ClockSampler(self.dev.index)
+        if sample_clocks:
+            sampler.start()
+        ctx.set_profiling(True)
+        launches0 = ctx.launch_count
+        self.sync_all()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            self.step()
+        e1.record()
+        self.sync_all()
+        ms_total = e0.elapsed_time(e1)
+        launches = ctx.launch_count - launches0
+        prof = ctx.get_profile()
+        ctx.set_profiling(False)
+        clocks = sampler.stop() if sample_clocks else None
+        ctx.check_status()
+        t = torch.tensor([ms_total], device=self.dev, dtype=torch.float64)
+        if self.world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step = float(t.item()) / steps
+        return dict(ms_total=ms_total, ms_step=ms_step, value=self.n_valid_total / (ms_step * 1e-3), launches=launches,
+                    prof=prof, clocks=clocks)
+
+    def kernel_table(self, prof, steps, ms_total, peak):
+        """Per GEMM class: launches, summed device time, share of the timed region, TFLOP/s (2 H V flop per valid row
+        and class) and its fraction of `peak`."""
+        w = self.w
+        kern = {}
+        for name in ("fwd_gemm", "grad_gemm", "dh_gemm", "dw_gemm"):
+            p = prof[name]
+            if p["launches"] == 0:
+                continue
+            tf = 2.0 * w.H * w.V * self.n_valid_local * steps / (p["ms"] * 1e-3) / 1e12
+            kern[name] = {"launches": p["launches"], "ms_total": p["ms"], "share_of_step": p["ms"] / ms_total,
+                          "tflops": tf, "frac": tf / peak}
+        return kern
+
+    def close(self):
+        self.ctx.close()
+
+
+def measure_other_workload(name, dev, peaks, min_seconds=1.5, max_steps=60):
+    """A short leg of another configuration with the headline's call sequence: 3 warm-ups, then at least 5 steps (more
+    for a configuration whose step takes milliseconds, so that the clock sampler sees the leg)."""
+    job = Job(name, dev)
+    job.step()
+    job.sync_all()
+    import torch
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    job.step()
+    e1.record()
+    job.sync_all()
+    steps = int(min(max_steps, max(5, min_seconds * 1e3 / max(e0.elapsed_time(e1), 1e-3))))
+    m = job.measure(steps, 3)
+    w = job.w
+    alg = 6.0 * w.H * w.V * job.n_valid_local / (m["ms_step"] * 1e-3) / 1e12
+    kern = job.kernel_table(m["prof"], steps, m["ms_total"], peaks["tflops_sustained"])
+    out = {"value": m["value"], "unit": UNIT, "ms_per_step": m["ms_step"], "steps": steps, "warmup": 3 + 2,
+           "H": w.H, "V": w.V, "K": w.K, "rows": w.n_tok, "valid_rows": job.n_valid_local, "invocations": w.n_inv,
+           "tensor_frac_of_burst_peak_algorithmic_6HV": alg / peaks["tflops_burst"],
+           "tensor_frac_of_peak_algorithmic_6HV": alg / peaks["tflops_sustained"],
+           "tflops_per_class": {k: v["tflops"] for k, v in kern.items()}, "gpu_launches": int(m["launches"]),
+           "clocks": m["clocks"]}
+    job.close()
+    return out
 
 
 def main():
@@ -271,105 +461,26 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     # ---------------------------------------------------------------- inputs (each rank: its own rollout groups)
-    kw = dict(seed_offset=1000 * rank)
-    if args.cut_rows:
-        kw.update(cut_rows=args.cut_rows)
-    w = wl.make(args.workload, device=dev, **kw)
-    n, H, V, K = w.n_tok, w.H, w.V, w.K
-    d_inv_role, d_inv_group, d_inv_traj = w.inv_role.to(dev), w.inv_group.to(dev), w.inv_traj.to(dev)
-    d_rn, d_rt, d_rj = w.r_node.to(dev), w.r_turn.to(dev), w.r_traj.to(dev)
-    d_cu, d_mask, d_tgt = w.cu_seqlens.to(dev), w.tok_mask.to(dev), w.target.to(dev)
-    role_model = w.role_model.tolist()
-    lam = w.lam.tolist()
-    # room for the optional logit stash too (reported as an extra; the headline step never uses it)
-    ws_bytes = max(ub.unity_workspace_bytes(n, H, V, K, w.n_inv), ub.unity_workspace_bytes_stash(n, H, V, K, w.n_inv))
     opts = [tuple(int(x) for x in kv.split("=")) for kv in args.opt.split(",") if kv]
-    extra = 0
-    mults = {6: 2, 7: 2}
-    mults.update({o: v for o, v in opts if o in (6, 7)})
-    if (mults[6], mults[7]) != (2, 2):         # non-default gradient chunks need their own G / dH scratch
-        extra = 2 * mults[6] * 18944 * (mults[7] * 18944 + 2048) + 4 * mults[6] * 18944 * H
-    ctx = ub.Context(local, ws_bytes + extra)
-    for o, v in opts:
-        ctx.set_option(o, v)
-    if args.ctas:
-        for option, value in enumerate(int(x) for x in args.ctas.split(",")):
-            ctx.set_option(option, value)
-
-    adv_inv = torch.empty(w.n_inv, device=dev)
-    adv_tok = torch.empty(n, device=dev)
-    logp = torch.empty(n, device=dev)
-    ent = torch.empty(n, device=dev)
-    loss = torch.empty(K, device=dev)
-    metrics = torch.empty((K + w.n_roles) * ub.UNITY_N_METRICS, device=dev)
-    dH = torch.empty(n, H, device=dev, dtype=torch.bfloat16)
-    dW = [torch.empty(V, H, device=dev) for _ in range(K)]
-
-    # current log-probs (stage 2) give the old / reference log-probs of the batch: logp + N(0, 0.05)
-    lse0 = torch.empty(n, device=dev)
-    ctx.logprob_fwd(w.hidden, w.W, d_cu, d_inv_role, role_model, d_tgt, d_mask, w.inv_temperature, logp, ent, lse0)
-    ctx.check_status()
-    logp0, ent0 = logp.clone(), ent.clone()
-    old = logp + w.noise_old.to(dev)
-    ref = logp + w.noise_ref.to(dev)
-
-    # per-model valid-row counts: the only quantity the ranks must agree on before the step
-    from paper_2605_26646_b200 import sharding
-    tok_inv = torch.repeat_interleave(torch.arange(w.n_inv), w.cu_seqlens[1:] - w.cu_seqlens[:-1])
-    tok_model = w.role_model[w.inv_role.long()[tok_inv]].long()
-    counts = sharding.local_counts(tok_model, w.tok_mask, K)
-    n_valid_local = int(counts.sum().item())
-    norm = None
-    n_valid_total = n_valid_local
-    if world > 1:
-        norm = sharding.global_norm(counts.to(dev))
-        tot = torch.tensor([float(n_valid_local)], device=dev, dtype=torch.float64)
-        dist.all_reduce(tot)
-        n_valid_total = int(tot.item())
-
-    def step(hid, tgt, msk, o, r):
-        ctx.role_advantage(w.n_traj, w.n_roles, w.n_groups, d_inv_role, d_inv_group, d_inv_traj, d_rn, d_rt, d_rj,
-                           lam, w.adv_eps, w.adv_ddof, d_cu, msk, adv_inv, adv_tok)
-        ctx.ppo_loss_fwd_bwd(hid, w.W, d_cu, d_inv_role, role_model, tgt, msk, w.inv_temperature, w.clip_lo,
-                             w.clip_hi, w.kl_coef, w.kl_mode, w.ent_coef, norm, False, o, r, adv_tok, loss, metrics,
-                             logp, ent, None, dH, dW)
-        if world > 1:
-            sharding.allreduce_grads(dW)
-
-    def sync_all():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-            torch.cuda.synchronize()
-
-    for _ in range(args.warmup):
-        step(w.hidden, d_tgt, d_mask, old, ref)
-    ctx.check_status()
+    ctas = [int(x) for x in args.ctas.split(",")] if args.ctas else []
+    job = Job(args.workload, dev, rank, world, stash_room=True, opts=opts, ctas=ctas, cut_rows=args.cut_rows)
+    w, ctx = job.w, job.ctx
+    n, H, V, K = w.n_tok, w.H, w.V, w.K
+    d_inv_role, d_inv_group, d_inv_traj = job.d_inv_role, job.d_inv_group, job.d_inv_traj
+    d_rn, d_rt, d_rj = job.d_rn, job.d_rt, job.d_rj
+    d_cu, d_mask, d_tgt = job.d_cu, job.d_mask, job.d_tgt
+    role_model, lam, norm = job.role_model, job.lam, job.norm
+    adv_inv, adv_tok, logp, ent, loss, metrics, dH, dW = (job.adv_inv, job.adv_tok, job.logp, job.ent, job.loss,
+                                                          job.metrics, job.dH, job.dW)
+    logp0, ent0, lse0, old, ref = job.logp0, job.ent0, job.lse0, job.old, job.ref
+    n_valid_local, n_valid_total = job.n_valid_local, job.n_valid_total
+    step, sync_all = job.step, job.sync_all
 
     # ---------------------------------------------------------------- timed region (device-resident inputs)
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    ctx.set_profiling(True)
-    launches0 = ctx.launch_count
-    sync_all()
+    m = job.measure(args.steps, args.warmup, sample_clocks=(rank == 0))
+    ms_total, ms_step, value, launches, prof, clocks = (m["ms_total"], m["ms_step"], m["value"], m["launches"],
+                                                         m["prof"], m["clocks"])
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(args.steps):
-        step(w.hidden, d_tgt, d_mask, old, ref)
-    e1.record()
-    sync_all()
-    ms_total = e0.elapsed_time(e1)
-    launches = ctx.launch_count - launches0
-    prof = ctx.get_profile()
-    ctx.set_profiling(False)
-    clocks = sampler.stop() if rank == 0 else None
-    ctx.check_status()
-    t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
-    value = n_valid_total / (ms_step * 1e-3)
 
     # ---------------------------------------------------------------- extra (not the headline): on-policy shortcut
     # First PPO epoch: the current policy equals the old one, so the statistics of the log-prob pass are handed in
@@ -516,14 +627,7 @@ def main():
     peaks = read_peaks()
     peak = peaks["tflops_sustained"]           # kernels timed inside a long step: the sustained figure
     flops_per_tok = 2.0 * H * V                # algorithmic flops of ONE of the four contractions per valid row
-    kern = {}
-    for name in ("fwd_gemm", "grad_gemm", "dh_gemm", "dw_gemm"):
-        p = prof[name]
-        if p["launches"] == 0:
-            continue
-        tf = flops_per_tok * n_valid_local * args.steps / (p["ms"] * 1e-3) / 1e12
-        kern[name] = {"launches": p["launches"], "ms_total": p["ms"], "share_of_step": p["ms"] / ms_total,
-                      "tflops": tf, "frac": tf / peak}
+    kern = job.kernel_table(prof, args.steps, ms_total, peak)
     dom = max(kern, key=lambda k: kern[k]["ms_total"])
     dp = kern[dom]
     roofline = {"bound": "tensor", "kernel": f"k_gemm<{dom}>", "achieved": dp["tflops"], "peak": peak,
@@ -543,6 +647,21 @@ def main():
         dt, rows = oracle_sample_run(w, args.ref_rows, old_h, ref_h, adv_h)
         cpu_baseline = {"value": rows / dt, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
                         "sample": f"{rows} valid rows of the {args.workload} workload (one oracle pass, {dt:.1f} s), fp64 numpy"}
+        # and the smallest configuration at full size: advantage, log-prob and loss forward + backward on every row
+        dt_t, rows_t = oracle_tiny_run()
+        cpu_baseline["tiny_full_size"] = {"value": rows_t / dt_t, "unit": UNIT, "seconds": dt_t,
+                                          "sample": f"all {rows_t} valid rows of the tiny workload, all three calls"}
+
+    # ---------------------------------------------------------------- the other configurations and the streaming stages
+    # Short legs with the same call sequence (1 GPU only).
+    other = streaming = None
+    if world == 1 and not args.no_e2e and not args.cut_rows:
+        job.close()                                   # releases the workspace; the other tensors are small beside 180 GB
+        torch.cuda.empty_cache()
+        other = {name: measure_other_workload(name, dev, peaks)
+                 for name in ("rag_qa", "search", "stress", "code") if name != args.workload}
+        torch.cuda.empty_cache()
+        streaming = measure_streaming()
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
@@ -557,7 +676,7 @@ def main():
             "tensor_frac_of_burst_peak_algorithmic_6HV": step_tflops_alg / peaks["tflops_burst"],
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "kernels": kern,
             "on_policy_shortcut": shortcut, "logit_stash": stash_extra, "logprob_fwd": fwd_extra, "iteration": iter_extra,
-            "cpu_baseline": cpu_baseline}
+            "other_workloads": other, "streaming": streaming, "cpu_baseline": cpu_baseline}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()

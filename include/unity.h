@@ -54,6 +54,10 @@ typedef struct unity_ctx unity_ctx;
 int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace, size_t workspace_bytes);
 int unity_destroy(unity_ctx* ctx);
 
+/* Scratch bytes sufficient for every call on batches of up to n_tok tokens of K models with these H and V,
+ * whatever the number of invocations (it assumes n_inv <= n_tok and includes the bounded logit-gradient chunk).
+ * Equal to unity_workspace_bytes(n_tok, H, V, K, n_tok); callers that know n_inv can ask for less below. */
+size_t unity_workspace_hint(int64_t n_tok, int32_t H, int32_t V, int32_t K);
 /* Scratch bytes that make every call with these sizes run with full-size chunks.  A smaller
  * workspace still works down to unity_workspace_min_bytes (smaller gradient chunks). */
 size_t unity_workspace_bytes(int64_t n_tok, int32_t H, int32_t V, int32_t K, int32_t n_inv);
@@ -108,6 +112,13 @@ int unity_set_profiling(unity_ctx* ctx, int enable);
 #define UNITY_OPT_L2_HINTS_FWD 16 /* 16..19: L2 eviction policy of the forward / recompute / dHidden / dW GEMM: value =
                                      A-operand loads | B-operand loads << 2 | logit-gradient stores << 4, each 0 normal,
                                      1 evict first, 2 evict last (defaults 6, 22, 0, 0: measured +0.3-0.7 % on the first two) */
+#define UNITY_OPT_WAIT_KCYCLES 20  /* bound of every in-kernel wait in thousands of SM clocks (default 4 000 000, about 2 s); when
+                                     it runs out the kernel records UNITY_ERR_TIMEOUT, frees its tensor memory and returns */
+#define UNITY_OPT_TEST_DROP_SLAB 21 /* TEST HOOK for the timeout path; accepted only while UNITY_OPT_WAIT_KCYCLES <= 1000.
+                                     value = 1 + UNITY_PROF_* class: in that class's launches every worker's TMA producer
+                                     leaves out one K slab of its first tile, so the waits behind it expire, the launch
+                                     returns within milliseconds and unity_check_status reports UNITY_ERR_TIMEOUT (outputs
+                                     of that call are undefined).  0 switches it off, and so does a larger wait bound. */
 int unity_set_option(unity_ctx* ctx, int option, int value);
 int unity_get_profile(unity_ctx* ctx, double* ms, int64_t* launches);
 

@@ -23,7 +23,7 @@ UNITY_MAX_MODELS = 16
 UNITY_MAX_ROLES = 64
 UNITY_N_METRICS = 8
 
-EXPORTS = ["unity_create", "unity_destroy", "unity_workspace_bytes", "unity_workspace_min_bytes",
+EXPORTS = ["unity_create", "unity_destroy", "unity_workspace_hint", "unity_workspace_bytes", "unity_workspace_min_bytes",
            "unity_workspace_bytes_stash",
            "unity_check_status", "unity_last_error", "unity_launch_count", "unity_set_profiling",
            "unity_get_profile", "unity_set_option", "unity_role_advantage", "unity_reward_assembly", "unity_gae", "unity_value_loss_fwd_bwd",
@@ -87,6 +87,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     for fn in (lib.unity_workspace_bytes, lib.unity_workspace_min_bytes, lib.unity_workspace_bytes_stash):
         fn.argtypes = [i64, i32, i32, i32, i32]
         fn.restype = C.c_size_t
+    lib.unity_workspace_hint.argtypes = [i64, i32, i32, i32]
+    lib.unity_workspace_hint.restype = C.c_size_t
     lib.unity_check_status.argtypes = [vp]
     lib.unity_check_status.restype = C.c_int
     lib.unity_last_error.argtypes = [vp]
@@ -151,6 +153,10 @@ def _raise(ctx, code: int):
 # ------------------------------------------------------------------------------------------------
 # functions with the names of the C entry points
 # ------------------------------------------------------------------------------------------------
+def unity_workspace_hint(n_tok: int, H: int, V: int, K: int) -> int:
+    return int(load_library().unity_workspace_hint(n_tok, H, V, K))
+
+
 def unity_workspace_bytes(n_tok: int, H: int, V: int, K: int, n_inv: int) -> int:
     return int(load_library().unity_workspace_bytes(n_tok, H, V, K, n_inv))
 
@@ -164,6 +170,8 @@ def unity_workspace_bytes_stash(n_tok: int, H: int, V: int, K: int, n_inv: int) 
 
 
 OPT_LOGIT_STASH = 15
+OPT_WAIT_KCYCLES = 20
+OPT_TEST_DROP_SLAB = 21
 
 
 def unity_create(device: int, stream_ptr: int, workspace: torch.Tensor) -> C.c_void_p:

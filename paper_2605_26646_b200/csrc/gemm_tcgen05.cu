@@ -182,7 +182,12 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                 for (int nt = t.n_begin; nt < t.n_end && ok; ++nt) {
                     const int b_row = g.b_row0 + nt * kTileCols + static_cast<int>(cta_rank) * C::kBRows;
                     for (int k = 0; k < g.k_iters; ++k) {
-                        if (!ptx::mbar_wait(&empty[stage], phase ^ 1, kWaitBudgetCycles) || *abort_flag) { ok = false; break; }
+                        if (!ptx::mbar_wait(&empty[stage], phase ^ 1, g.wait_budget) || *abort_flag) { ok = false; break; }
+                        if (g.test_drop_slab && it == 0 && nt == t.n_begin && k == (g.k_iters > 1 ? 1 : 0)) {
+                            // test hook: this slab never arrives; the MMA issuer's wait for it must run out
+                            if (++stage == kStages) { stage = 0; phase ^= 1; }
+                            continue;
+                        }
                         uint8_t* sA = smem + stage * kStageBytes;
                         // completion bytes are counted on the barrier of the CTA that issues the MMAs
                         const uint32_t bar = CTAS == 2 ? ptx::mapa(ptx::smem_u32(&full[stage]), 0) : ptx::smem_u32(&full[stage]);
@@ -229,11 +234,11 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                 if (!next_unit<EPI>(g, it, pair, n_pairs, gm, t, valid)) break;
                 if (!valid) continue;
                 for (int nt = t.n_begin; nt < t.n_end && ok; ++nt) {
-                    if (!ptx::mbar_wait(&acc_empty[acc], acc_phase ^ 1, kWaitBudgetCycles) || *abort_flag) { ok = false; break; }
+                    if (!ptx::mbar_wait(&acc_empty[acc], acc_phase ^ 1, g.wait_budget) || *abort_flag) { ok = false; break; }
                     ptx::tc_fence_after();
                     const uint32_t d_tmem = tmem_base + acc * kTileCols;
                     for (int k = 0; k < g.k_iters; ++k) {
-                        if (!ready && !ptx::mbar_wait(&full[stage], phase, kWaitBudgetCycles)) { ok = false; break; }
+                        if (!ready && !ptx::mbar_wait(&full[stage], phase, g.wait_budget)) { ok = false; break; }
                         ptx::tc_fence_after();
                         const int next_stage = stage + 1 == kStages ? 0 : stage + 1;
                         const uint32_t next_phase = stage + 1 == kStages ? phase ^ 1 : phase;
@@ -312,7 +317,7 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
             }
 
             for (int nt = t.n_begin; nt < t.n_end && ok; ++nt) {
-                if (!ptx::mbar_wait(&acc_full[acc], acc_phase, kWaitBudgetCycles) || *abort_flag) { ok = false; break; }
+                if (!ptx::mbar_wait(&acc_full[acc], acc_phase, g.wait_budget) || *abort_flag) { ok = false; break; }
                 ptx::tc_fence_after();
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kTileCols;
                 const int col0 = nt * kTileCols;

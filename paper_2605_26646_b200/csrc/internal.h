@@ -13,11 +13,10 @@ namespace unity {
 constexpr int kTileM = 256;   // rows of one output tile, shared by a pair of CTAs; row groups are padded to this
 constexpr int kCtaM = 128;    // rows of A per CTA of the pair (= TMEM lanes)
 constexpr int kTileN = 256;   // columns of one output tile (TMEM columns per accumulator stage)
-constexpr int kHalfN = 128;   // rows of B loaded by each CTA of the pair
 constexpr int kBoxRows = 128; // rows of a K-major TMA box (A and B alike)
 constexpr int kTileK = 64;    // bf16 elements per shared-memory K slab (one 128-byte swizzle row)
 constexpr int kRouteBlock = 256;          // threads (= tokens) per block in the routing kernels
-constexpr long long kWaitBudgetCycles = 4000000000LL;   // ~2 s: bound of every in-kernel wait
+constexpr long long kWaitBudgetCycles = 4000000000LL;   // ~2 s: default bound of every in-kernel wait (GemmArgs::wait_budget)
 
 // Device status bits (sticky, ORed into the context's status word).
 constexpr int kStatusBadIndex = 1;
@@ -67,6 +66,9 @@ struct GemmArgs {
     int beta;                 // 0: overwrite, 1: add to C
     int l2_hints;             // L2 eviction policy (0 normal, 1 first, 2 last): bits 0-1 A loads, 2-3 B loads, 4-5 G stores
     int* status;
+    long long wait_budget;    // SM clocks after which an mbarrier wait gives up (kStatusTimeout)
+    int test_drop_slab;       // test hook: the TMA producer of every worker leaves out one K slab of its first tile
+                              // (neither the expected-bytes arrival nor the loads), so the waits behind it run out
 };
 
 // a_mn: A is MN-major (only for kEpiAccumF32, whose B operand is always MN-major).  For an MN-major operand

@@ -19,9 +19,6 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 __device__ __forceinline__ void fence_barrier_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
-__device__ __forceinline__ void fence_proxy_async() {
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.shared::cta.b64 st, [%0];\n\t}" ::"r"(smem_u32(bar))
                  : "memory");
@@ -72,15 +69,6 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long l
 __device__ __forceinline__ void prefetch_tensormap(const void* tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
 }
-// 2-D tiled load global -> shared, completion signalled on an mbarrier of this CTA.
-__device__ __forceinline__ void tma_load_2d(void* smem_dst, const void* tmap, uint64_t* bar, int32_t x, int32_t y) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(smem_u32(smem_dst)),
-        "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(x), "r"(y)
-        : "memory");
-}
-
 // ------------------------------------------------------------------------------------ epilogue arithmetic
 // 2^x with the hardware approximation (results below 2^-126 flush to zero; 2^-inf = 0).
 __device__ __forceinline__ float ex2(float x) {
@@ -199,16 +187,6 @@ __device__ __forceinline__ void cluster_sync_all() {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
-// 2-D tiled load into THIS CTA's shared memory whose completion bytes are counted on an mbarrier that may
-// belong to the peer CTA of the pair (bar_cluster_addr from mapa).  Plain load: every CTA fetches its own box.
-__device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const void* tmap, uint32_t bar_cluster_addr, int32_t x,
-                                                 int32_t y) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(smem_u32(smem_dst)),
-        "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar_cluster_addr), "r"(x), "r"(y)
-        : "memory");
-}
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_result, uint32_t ncols) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
                  "r"(ncols)
@@ -255,8 +233,8 @@ __device__ __forceinline__ void st_global_v8_hint(void* addr, unsigned r0, unsig
                  ::"l"(addr), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(r4), "r"(r5), "r"(r6), "r"(r7), "l"(policy)
                  : "memory");
 }
-// 2-D tiled load with an L2 cache hint; CTAS = 2: completion bytes go to the barrier (cluster address) of the pair's
-// leading CTA.
+// 2-D tiled load with an L2 cache hint into THIS CTA's shared memory (plain load: every CTA fetches its own box);
+// CTAS = 2: completion bytes go to the barrier (cluster address from mapa) of the pair's leading CTA.
 template <int CTAS>
 __device__ __forceinline__ void tma_load_2d_hint_on(void* smem_dst, const void* tmap, uint32_t bar_addr, int32_t x, int32_t y,
                                                     uint64_t policy) {
@@ -276,18 +254,6 @@ __device__ __forceinline__ void tma_load_2d_hint_on(void* smem_dst, const void* 
 }
 
 // Forms selected by the number of CTAs that cooperate on a tile (1, or 2 = a CTA pair).
-template <int CTAS>
-__device__ __forceinline__ void tma_load_2d_on(void* smem_dst, const void* tmap, uint32_t bar_addr, int32_t x, int32_t y) {
-    if (CTAS == 2) {
-        tma_load_2d_pair(smem_dst, tmap, bar_addr, x, y);
-    } else {
-        asm volatile(
-            "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-            ::"r"(smem_u32(smem_dst)),
-            "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar_addr), "r"(x), "r"(y)
-            : "memory");
-    }
-}
 template <int CTAS>
 __device__ __forceinline__ void mma_bf16_ss_on(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                                uint32_t accumulate) {

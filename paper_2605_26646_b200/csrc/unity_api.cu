@@ -41,6 +41,8 @@ struct unity_ctx {
     int l2_hints[UNITY_PROF_CLASSES]; // per GEMM class: GemmArgs::l2_hints
     int wide_acc;                   // 1: dHidden / dW chunk GEMMs use 512-column tiles (CTA pairs only)
     unsigned round_total;           // arrivals accumulated so far on the rendezvous counter (d_status + 16)
+    long long wait_budget;          // SM clocks after which an in-kernel wait gives up
+    int test_drop;                  // test hook: 1 + GEMM class whose producer leaves out one K slab; 0 = off
 };
 
 namespace {
@@ -93,6 +95,20 @@ struct ProfScope {
         c->ev_used += 2;
     }
 };
+
+// Fields every GEMM launch of class `cls` takes from the context: status word, L2 hints, wait bound, test hook and,
+// when `sync` is set, the round rendezvous (the counter only grows; the context keeps its running total).
+void gemm_common(unity_ctx* ctx, GemmArgs& g, int cls, GemmEpilogue epi, bool sync) {
+    g.status = ctx->d_status;
+    g.l2_hints = ctx->l2_hints[cls];
+    g.wait_budget = ctx->wait_budget;
+    g.test_drop_slab = ctx->test_drop == cls + 1;
+    if (sync) {
+        g.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
+        g.round_base = ctx->round_total;
+        ctx->round_total += gemm_round_arrivals(epi, ctx->ctas[cls], g, ctx->sm_count);
+    }
+}
 
 struct Bump {
     char* base;
@@ -302,18 +318,12 @@ int launch_forward(unity_ctx* ctx, const unity_rows* r, int slot0, int rows, flo
     g.n_splits = splits; g.tiles_per_split = tps;
     g.stats = stats; g.stats_pitch = rows;
     g.target_p = target_p; g.vocab0 = 0; g.scale = r->inv_temperature;
-    g.status = ctx->d_status;
-    g.l2_hints = ctx->l2_hints[UNITY_PROF_FWD_GEMM];
     if (z) {
         g.Z = z->Z; g.ldz = z->ldz; g.z_chunk_stride = z->chunk_stride; g.z_chunk_cols = z->chunk_cols; g.z_chunks = z->chunks;
         g.g_wide_store = (reinterpret_cast<uintptr_t>(z->Z) % 32 == 0) && (z->ldz * 2 % 32 == 0) && (z->chunk_stride * 2 % 32 == 0) &&
                          (z->chunk_cols * 2 % 32 == 0);
     }
-    if (ctx->fwd_sync) {
-        g.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
-        g.round_base = ctx->round_total;
-        ctx->round_total += gemm_round_arrivals(kEpiSoftmaxStats, ctas, g, ctx->sm_count);
-    }
+    gemm_common(ctx, g, UNITY_PROF_FWD_GEMM, kEpiSoftmaxStats, ctx->fwd_sync != 0);
     ProfScope ps(ctx, UNITY_PROF_FWD_GEMM);
     CUDA_TRY(ctx, launch_gemm(kEpiSoftmaxStats, false, ctas, tmA, tmB, g, ctx->sm_count, ctx->stream));
     return UNITY_OK;
@@ -436,6 +446,8 @@ int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace
     c->l2_hints[UNITY_PROF_DH_GEMM] = 0;
     c->l2_hints[UNITY_PROF_DW_GEMM] = 0;
     c->logit_stash = 0;
+    c->wait_budget = kWaitBudgetCycles;
+    c->test_drop = 0;
     c->ev_pool = new (std::nothrow) std::vector<cudaEvent_t>();
     c->ev_class = new (std::nothrow) std::vector<int>();
     if (cudaMalloc(&c->d_status, 256) != cudaSuccess || cudaMallocHost(&c->h_pinned, 4096) != cudaSuccess ||
@@ -469,6 +481,11 @@ size_t unity_workspace_bytes(int64_t n_tok, int32_t H, int32_t V, int32_t K, int
                  wanted_chunk_vocab(V, kDefaultChunkMult), nullptr).bytes;
 }
 
+size_t unity_workspace_hint(int64_t n_tok, int32_t H, int32_t V, int32_t K) {
+    if (n_tok < 0 || n_tok > 0x7fffff00LL) return 0;
+    return unity_workspace_bytes(n_tok, H, V, K, static_cast<int32_t>(n_tok));
+}
+
 size_t unity_workspace_bytes_stash(int64_t n_tok, int32_t H, int32_t V, int32_t K, int32_t n_inv) {
     if (n_tok < 0 || H <= 0 || V <= 0 || K <= 0 || n_inv < 0) return 0;
     int cr = wanted_chunk_rows(n_tok, K);
@@ -496,7 +513,13 @@ int unity_check_status(unity_ctx* ctx) {
     CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof(int), ctx->stream));
     CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream));
     const int bits = ctx->h_pinned[512];
-    if (bits & kStatusTimeout) return fail(ctx, UNITY_ERR_TIMEOUT, "a bounded in-kernel wait expired");
+    if (bits & kStatusTimeout) {
+        // workers that gave up did not finish their rounds: start the round rendezvous afresh (the stream is idle)
+        CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_status + 16, 0, sizeof(unsigned), ctx->stream));
+        CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream));
+        ctx->round_total = 0;
+        return fail(ctx, UNITY_ERR_TIMEOUT, "a bounded in-kernel wait expired");
+    }
     if (bits & kStatusBadIndex) return fail(ctx, UNITY_ERR_BAD_INDEX, "an index in the data was out of range (row / invocation masked)");
     return UNITY_OK;
 }
@@ -532,6 +555,17 @@ int unity_set_option(unity_ctx* ctx, int option, int value) {
         return UNITY_OK;
     }
     if (option == UNITY_OPT_WIDE_ACC && (value == 0 || value == 1)) { ctx->wide_acc = value; return UNITY_OK; }
+    if (option == UNITY_OPT_WAIT_KCYCLES && value >= 1) {
+        ctx->wait_budget = static_cast<long long>(value) * 1000;
+        if (ctx->wait_budget > 1000000) ctx->test_drop = 0;      // the test hook lives only under a short bound
+        return UNITY_OK;
+    }
+    if (option == UNITY_OPT_TEST_DROP_SLAB && value >= 0 && value <= UNITY_PROF_CLASSES) {
+        if (value != 0 && ctx->wait_budget > 1000000)
+            return fail(ctx, UNITY_ERR_INVALID_ARG, "UNITY_OPT_TEST_DROP_SLAB needs UNITY_OPT_WAIT_KCYCLES <= 1000 first");
+        ctx->test_drop = value;
+        return UNITY_OK;
+    }
     return fail(ctx, UNITY_ERR_INVALID_ARG, "unknown option %d or value %d out of range", option, value);
 }
 
@@ -971,14 +1005,9 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                             g.target_p = L.target_p; g.vocab0 = v0 + q0; g.scale = rows->inv_temperature;
                             g.coef_a = L.coef_a; g.coef_b = L.coef_b; g.row_lse = L.row_lse; g.row_ent = L.row_ent;
                             g.has_ent = params->ent_coef != 0.f;
-                            g.l2_hints = ctx->l2_hints[UNITY_PROF_GRAD_GEMM];
-                            g.G = Gc + static_cast<long long>(r0) * cv + q0; g.ldg = cv; g.status = ctx->d_status;
+                            g.G = Gc + static_cast<long long>(r0) * cv + q0; g.ldg = cv;
                             g.g_wide_store = (reinterpret_cast<uintptr_t>(g.G) % 32 == 0) && (g.ldg * 2 % 32 == 0);
-                            if (ctx->chunk_sync & 1) {
-                                g.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
-                                g.round_base = ctx->round_total;
-                                ctx->round_total += gemm_round_arrivals(kEpiLogitGrad, c_grad, g, ctx->sm_count);
-                            }
+                            gemm_common(ctx, g, UNITY_PROF_GRAD_GEMM, kEpiLogitGrad, (ctx->chunk_sync & 1) != 0);
                             ProfScope ps(ctx, UNITY_PROF_GRAD_GEMM);
                             CUDA_TRY(ctx, launch_gemm(kEpiLogitGrad, false, c_grad, tm_hp_k, tm_W_k, g, ctx->sm_count, st));
                             nl += 1;
@@ -997,13 +1026,8 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 h.k_iters = (vc + kTileK - 1) / kTileK;
                 h.group_m = ctx->chunk_group[1] / c_dh > 0 ? ctx->chunk_group[1] / c_dh : 1;
                 h.a_row0 = 0; h.a_k0 = 0; h.b_row0 = 0; h.b_k0 = v0; h.m_rows = nc; h.n_cols = H;
-                h.C = L.dHc; h.ldc = H; h.beta = v0 > 0; h.status = ctx->d_status;
-                h.l2_hints = ctx->l2_hints[UNITY_PROF_DH_GEMM];
-                if (ctx->chunk_sync & 2) {
-                    h.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
-                    h.round_base = ctx->round_total;
-                    ctx->round_total += gemm_round_arrivals(kEpiAccumF32, c_dh, h, ctx->sm_count);
-                }
+                h.C = L.dHc; h.ldc = H; h.beta = v0 > 0;
+                gemm_common(ctx, h, UNITY_PROF_DH_GEMM, kEpiAccumF32, (ctx->chunk_sync & 2) != 0);
                 {
                     ProfScope ps(ctx, UNITY_PROF_DH_GEMM);
                     CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, false, c_dh, tm_G_k, tm_W_mn, h, ctx->sm_count, st, wide_dh));
@@ -1017,13 +1041,8 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 w.group_m = ctx->chunk_group[2] / c_dw > 0 ? ctx->chunk_group[2] / c_dw : 1;
                 w.a_row0 = 0; w.a_k0 = 0; w.b_row0 = 0; w.b_k0 = slot0; w.m_rows = vc; w.n_cols = H;
                 w.C = dWk + static_cast<long long>(v0) * H; w.ldc = H;
-                w.beta = (params->accumulate_dW || c0 > 0) ? 1 : 0; w.status = ctx->d_status;
-                w.l2_hints = ctx->l2_hints[UNITY_PROF_DW_GEMM];
-                if (ctx->chunk_sync & 4) {
-                    w.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
-                    w.round_base = ctx->round_total;
-                    ctx->round_total += gemm_round_arrivals(kEpiAccumF32, c_dw, w, ctx->sm_count);
-                }
+                w.beta = (params->accumulate_dW || c0 > 0) ? 1 : 0;
+                gemm_common(ctx, w, UNITY_PROF_DW_GEMM, kEpiAccumF32, (ctx->chunk_sync & 4) != 0);
                 {
                     ProfScope ps(ctx, UNITY_PROF_DW_GEMM);
                     CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, true, c_dw, tm_G_mn, tm_hp_mn, w, ctx->sm_count, st, wide_dw));

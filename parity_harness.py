@@ -1,4 +1,6 @@
-"""Helpers shared by the GPU parity tests: run one workload through libunity and through the oracle."""
+"""Parity harness - TEST INFRASTRUCTURE, not part of the library: runs one workload through libunity (C ABI) and
+through the fp64 oracle and holds the tolerances of the parity contract.  Used by the tests, by the smoke check and by
+the benchmark's CPU-baseline leg; the product (paper_2605_26646_b200) never imports it."""
 from __future__ import annotations
 
 import numpy as np
@@ -23,6 +25,57 @@ def rel_fro(a: np.ndarray, b: np.ndarray) -> float:
     den = float(np.linalg.norm(b.astype(np.float64).ravel()))
     num = float(np.linalg.norm((a.astype(np.float64) - b.astype(np.float64)).ravel()))
     return num / den if den > 0 else num
+
+
+def worst_row_rel(a: np.ndarray, b: np.ndarray, allowance=None) -> float:
+    """Largest relative error of a row of `a` against the same row of `b` (2-norms), after taking off a per-row
+    absolute `allowance` (see dh_row_allowance); a row that is zero in `b` must be zero in `a` up to its allowance
+    (it counts as an infinite error otherwise)."""
+    a, b = a.astype(np.float64), b.astype(np.float64)
+    num = np.linalg.norm(a - b, axis=1)
+    if allowance is not None:
+        num = np.maximum(num - np.asarray(allowance, np.float64), 0.0)
+    den = np.linalg.norm(b, axis=1)
+    if np.any((den == 0) & (num > 0)):
+        return float("inf")
+    return float((num[den > 0] / den[den > 0]).max()) if np.any(den > 0) else 0.0
+
+
+def dh_row_allowance(w, o, logp_gpu, old, ref, adv, clip=None, kl_coef=None, kl_mode=None, ent_coef=None, mask=None):
+    """Per-row slack for comparing dHidden row by row.  A row's gradient is a_i * (W_y - sum_v p_v W_v) + (entropy
+    term), and a_i = dL/dlogp_i depends on the row's log-prob: the contract lets the library's log-prob differ from
+    the oracle's by up to TOL_LOGP, and for a row whose a_i nearly vanishes (zero advantage, reference log-prob
+    equal to the current one) that admissible difference moves a_i by as much as a_i itself.  The slack is that
+    effect and nothing else: |a_i evaluated at the library's log-prob - a_i of the oracle| times a bound on
+    ||tau (W_y - sum_v p_v W_v)||, namely 2 tau max_v ||W_k[v]||.  Rows are those of o["dh_index"]; `mask` is the token
+    mask the oracle was given (default: the workload's)."""
+    idx = o["dh_index"]
+    lo, hi = (w.clip_lo, w.clip_hi) if clip is None else clip
+    t = orc.ppo_token_terms(np.asarray(logp_gpu, np.float64)[idx], o["entropy"][idx], orc.to_f64(np.asarray(old))[idx],
+                            orc.to_f64(np.asarray(ref))[idx], orc.to_f64(np.asarray(adv))[idx], lo, hi,
+                            w.kl_coef if kl_coef is None else kl_coef, w.kl_mode if kl_mode is None else kl_mode,
+                            w.ent_coef if ent_coef is None else ent_coef)
+    _, tok_model = orc.token_role_model(w.cu_seqlens.numpy(), w.inv_role.numpy(), w.role_model.numpy())
+    km = tok_model[idx]
+    valid = (w.tok_mask.numpy() if mask is None else np.asarray(mask))[idx] != 0
+    a_alt = np.where(valid, t["dl_dlogp"] / o["M"][km], 0.0)
+    reach = np.array([2.0 * w.inv_temperature * float(x.float().norm(dim=1).max().item()) for x in w.W])
+    return np.abs(a_alt - o["a"][idx]) * reach[km]
+
+
+def worst_block_rel_fro(a: np.ndarray, b: np.ndarray, block: int = 256) -> float:
+    """Largest relative Frobenius error over blocks of `block` consecutive rows (the last one may be ragged)."""
+    worst = 0.0
+    for r0 in range(0, b.shape[0], block):
+        bb = b[r0:r0 + block].astype(np.float64)
+        err = np.linalg.norm(a[r0:r0 + block].astype(np.float64) - bb)
+        den = np.linalg.norm(bb)
+        if den == 0:
+            if err > 0:
+                return float("inf")
+            continue
+        worst = max(worst, err / den)
+    return worst
 
 
 def make_ctx(w: wl.Workload, extra: int = 0, stash: bool = False) -> ub.Context:
@@ -108,6 +161,14 @@ def gpu_ppo(ctx: ub.Context, w: wl.Workload, d: DeviceInputs, old, ref, adv, nor
 def oracle_ppo(w: wl.Workload, old, ref, adv, norm=None, rows=None, dW_models=None, kl_mode=None, kl_coef=None,
                ent_coef=None, clip=None, want_dW=True):
     lo, hi = (w.clip_lo, w.clip_hi) if clip is None else clip
+    out = _oracle_ppo(w, old, ref, adv, norm, rows, dW_models, kl_mode, kl_coef, ent_coef, lo, hi, want_dW)
+    # what a conditioning-aware comparison of dHidden needs later (see dh_row_allowance)
+    out["inputs"] = dict(old=np.asarray(old), ref=np.asarray(ref), adv=np.asarray(adv), clip=(lo, hi), kl_coef=kl_coef,
+                         kl_mode=kl_mode, ent_coef=ent_coef)
+    return out
+
+
+def _oracle_ppo(w, old, ref, adv, norm, rows, dW_models, kl_mode, kl_coef, ent_coef, lo, hi, want_dW):
     return orc.ppo_loss_fwd_bwd(bf16_bits(w.hidden), [bf16_bits(x) for x in w.W], w.cu_seqlens.numpy(),
                                 w.inv_role.numpy(), w.role_model.numpy(), w.target.numpy(), w.tok_mask.numpy(),
                                 np.asarray(old), np.asarray(ref), np.asarray(adv), clip_lo=lo, clip_hi=hi,

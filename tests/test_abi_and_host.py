@@ -32,6 +32,9 @@ def test_workspace_queries_and_null_context_need_no_gpu():
     full = ub.unity_workspace_bytes(1_600_000, 3584, 152064, 2, 2574)
     least = ub.unity_workspace_min_bytes(1_600_000, 3584, 152064, 2, 2574)
     assert 0 < least < full < 60 * 2 ** 30
+    hint = ub.unity_workspace_hint(1_600_000, 3584, 152064, 2)
+    assert hint == ub.unity_workspace_bytes(1_600_000, 3584, 152064, 2, 1_600_000) and full <= hint < full + 2 ** 27
+    assert ub.unity_workspace_hint(-1, 3584, 152064, 2) == 0
     assert ub.unity_workspace_bytes(-1, 3584, 152064, 2, 1) == 0
     assert lib.unity_check_status(None) == -1
     assert lib.unity_destroy(None) == -1

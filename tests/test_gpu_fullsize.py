@@ -5,12 +5,13 @@ The fp64 oracle cannot sweep 1.2 M rows x 152 k vocabulary, so the full-size run
     gradient needs only that row, W_k and the global count M_k, so the sampled values are exact at full size),
 (ii) the loss against the fp64 sum of the exported per-token losses,
 (iii) dW through properties that hold at any size: its column sums over the vocabulary vanish, and it is additive
-    over row chunks, one of which (about a thousand rows) the oracle checks in full."""
+    over row chunks; one chunk of about a thousand rows per model is checked in full by the oracle (whole tensor
+    and per block of 256 vocabulary rows), together with the dHidden rows of the chunk, row by row."""
 import numpy as np
 import pytest
 import torch
 
-import parity_util as pu
+import parity_harness as pu
 from oracle import unity_oracle as orc
 from paper_2605_26646_b200 import binding as ub
 from paper_2605_26646_b200 import workloads as wl
@@ -73,6 +74,8 @@ def test_full_size_sampled_parity(name, n_sample, chunk_rows, stash):
     assert np.abs(gl["lse"].cpu().numpy()[idx] - o["lse"][idx]).max() <= pu.TOL_LOGP
     dh = gp["dHidden"][torch.as_tensor(idx, device="cuda")].float().cpu().numpy()
     assert pu.rel_fro(dh, o["dHidden"]) <= pu.TOL_GRAD
+    slack = pu.dh_row_allowance(w, o, gp["logp"].cpu().numpy(), old.cpu().numpy(), ref.cpu().numpy(), adv.cpu().numpy())
+    assert pu.worst_row_rel(dh, o["dHidden"], slack) <= pu.TOL_GRAD
     # masked rows are zero everywhere
     off = torch.as_tensor(np.nonzero(~mask_np)[0][:4096], device="cuda")
     assert torch.all(gp["dHidden"][off] == 0) and torch.all(gp["logp"][off] == 0)
@@ -89,20 +92,32 @@ def test_full_size_sampled_parity(name, n_sample, chunk_rows, stash):
     for k in range(K):
         g = gp["dW"][k].double()
         assert g.sum(0).abs().max().item() <= 1e-2 * g.abs().sum(0).max().item()
-    k0 = K - 1
-    cand = np.nonzero(mask_np & (tok_model == k0))[0]
-    start = int(rng.integers(0, cand.size - chunk_rows))
-    chunk = cand[start:start + chunk_rows]
+    # one chunk of consecutive valid rows PER MODEL, all run in one call (a model's dW sees only its own chunk)
+    chunks = []
+    for k in range(K):
+        cand = np.nonzero(mask_np & (tok_model == k))[0]
+        start = int(rng.integers(0, cand.size - chunk_rows))
+        chunks.append(cand[start:start + chunk_rows])
+    chunk = np.concatenate(chunks)
     mask_c = np.zeros(n, np.uint8)
     mask_c[chunk] = 1
     d.tok_mask = torch.from_numpy(mask_c).cuda()
     dW_c = [torch.zeros(w.V, w.H, device="cuda") for _ in range(K)]
     gc = pu.gpu_ppo(ctx, w, d, old, ref, adv, norm=M.tolist(), dW=dW_c)
-    oc = orc.ppo_loss_fwd_bwd(*args[:-1], mask_c, old.cpu().numpy(), ref.cpu().numpy(), adv.cpu().numpy(),
-                              clip_lo=w.clip_lo, clip_hi=w.clip_hi, kl_coef=w.kl_coef, kl_mode=w.kl_mode,
-                              ent_coef=w.ent_coef, n_roles=w.n_roles, norm=M.tolist(), dW_models=[k0])
-    assert pu.rel_fro(dW_c[k0].cpu().numpy(), oc["dW"][k0]) <= pu.TOL_GRAD
-    del oc
+    for k in range(K):                       # the oracle takes one model at a time (an fp64 dW is several GB)
+        oc = orc.ppo_loss_fwd_bwd(*args, old.cpu().numpy(), ref.cpu().numpy(), adv.cpu().numpy(),
+                                  clip_lo=w.clip_lo, clip_hi=w.clip_hi, kl_coef=w.kl_coef, kl_mode=w.kl_mode,
+                                  ent_coef=w.ent_coef, n_roles=w.n_roles, norm=M.tolist(), dW_models=[k],
+                                  rows=chunks[k])
+        assert np.array_equal(oc["dh_index"], chunks[k])
+        got = dW_c[k].cpu().numpy()
+        assert pu.rel_fro(got, oc["dW"][k]) <= pu.TOL_GRAD, k
+        assert pu.worst_block_rel_fro(got, oc["dW"][k]) <= pu.TOL_GRAD, k      # per tile of 256 vocabulary rows
+        rows_k = torch.as_tensor(chunks[k], device="cuda")
+        slack = pu.dh_row_allowance(w, oc, gc["logp"].cpu().numpy(), old.cpu().numpy(), ref.cpu().numpy(),
+                                    adv.cpu().numpy())
+        assert pu.worst_row_rel(gc["dHidden"][rows_k].float().cpu().numpy(), oc["dHidden"], slack) <= pu.TOL_GRAD, k
+        del oc, got
     # the rest of the batch accumulated on top of the chunk reproduces the full-batch dW
     mask_rest = w.tok_mask.clone()
     mask_rest[torch.from_numpy(chunk)] = 0

@@ -7,7 +7,7 @@ that nothing left in the shared static scratch by one call leaks into the next. 
 import pytest
 import torch
 
-import parity_util as pu
+import parity_harness as pu
 from paper_2605_26646_b200 import binding as ub
 from paper_2605_26646_b200 import workloads as wl
 
