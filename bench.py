@@ -219,6 +219,14 @@ def measure_streaming():
 
     t_adv = timed(lambda: ctx.role_advantage(n_inv, R, G, inv_role, inv_group, inv_traj, r_node, None, None, None, 1e-6,
                                              0, cu, mask, adv_inv, adv_tok))
+    # the same batch with its invocations in a seeded random order (rollout groups interleaved, as in a buffer that
+    # fills in arrival order); token data is not moved: only the invocation-level arrays are permuted
+    perm = torch.randperm(n_inv, generator=torch.Generator().manual_seed(5)).to(dev)
+    role_s, group_s, r_s = inv_role[perm].contiguous(), inv_group[perm].contiguous(), r_node[perm].contiguous()
+    t_adv_shuf = timed(lambda: ctx.role_advantage(n_inv, R, G, role_s, group_s, inv_traj, r_s, None, None, None, 1e-6,
+                                                  0, cu, mask, adv_inv, adv_tok))
+    # reference for the write-only streams: a plain device fill of the same output
+    t_fill = timed(lambda: adv_tok.zero_())
     t_gae = timed(lambda: ctx.gae(cu, rewards, values, mask, 0.99, 0.95, a_out, r_out))
     vloss = torch.empty(R, device=dev)
     t_val = timed(lambda: ctx.value_loss_fwd_bwd(cu, inv_role, list(range(R)), R, mask, values, rewards, r_out, 0.2, None,
@@ -236,14 +244,41 @@ def measure_streaming():
     t_gat = timed(lambda: ctx.ready_batch_gather(order, cu, out_cu, totals, rewards, r_out, 0.0))
     kept_tok = int(totals[1].item())
     ctx.check_status()
+    # Host-side cost of the one synchronisation inside unity_logprob_fwd / unity_ppo_loss_fwd_bwd (the K row counts are
+    # read back to size the grouped launches): on the smallest configuration, how long the call keeps the host (it
+    # returns once everything is enqueued) and how long until the result is complete.
+    wt = wl.make("tiny", device=dev)
+    cxt = ub.Context(0, ub.unity_workspace_bytes(wt.n_tok, wt.H, wt.V, wt.K, wt.n_inv))
+    t_cu, t_role, t_tgt, t_mask = wt.cu_seqlens.to(dev), wt.inv_role.to(dev), wt.target.to(dev), wt.tok_mask.to(dev)
+    t_logp = torch.empty(wt.n_tok, device=dev)
+    ret_us, done_us = [], []
+    for i in range(23):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        cxt.logprob_fwd(wt.hidden, wt.W, t_cu, t_role, wt.role_model.tolist(), t_tgt, t_mask, 1.0, t_logp, None, None)
+        t1 = time.perf_counter()
+        torch.cuda.synchronize()
+        t2 = time.perf_counter()
+        if i >= 3:
+            ret_us.append((t1 - t0) * 1e6)
+            done_us.append((t2 - t0) * 1e6)
+    cxt.close()
+    ret_us.sort()
+    done_us.sort()
     out = {"mode": "micro", "tokens": n, "invocations": n_inv, "peak_hbm_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"],
-           "role_advantage": {"ms": t_adv, "algorithmic_bytes": 5 * n + 28 * n_inv, "gbs": (5 * n + 28 * n_inv) / t_adv / 1e6},
+           "role_advantage": {"ms": t_adv, "algorithmic_bytes": 5 * n + 28 * n_inv, "gbs": (5 * n + 28 * n_inv) / t_adv / 1e6,
+                              "ms_shuffled_invocations": t_adv_shuf},
+           "device_fill_f32": {"ms": t_fill, "algorithmic_bytes": 4 * n, "gbs": 4 * n / t_fill / 1e6,
+                               "note": "torch fill of the 256 MiB token vector: what a write-only stream reaches here"},
            "gae": {"ms": t_gae, "algorithmic_bytes": 17 * n, "gbs": 17 * n / t_gae / 1e6},
            "value_loss": {"ms": t_val, "algorithmic_bytes": 17 * n, "gbs": 17 * n / t_val / 1e6},
            "align_rewards": {"ms": t_aln, "algorithmic_bytes": 5 * n, "gbs": 5 * n / t_aln / 1e6},
            "ready_batch_gather_f32": {"ms": t_gat, "algorithmic_bytes": 8 * kept_tok, "gbs": 8 * kept_tok / t_gat / 1e6},
-           "ready_batch_plan": {"ms": t_plan, "note": "latency-bound: four small launches over the invocations"}}
-    for k in ("role_advantage", "gae", "value_loss", "align_rewards", "ready_batch_gather_f32"):
+           "ready_batch_plan": {"ms": t_plan, "note": "latency-bound: four small launches over the invocations"},
+           "logprob_fwd_tiny_host": {"call_returns_after_us": ret_us[len(ret_us) // 2], "complete_after_us": done_us[len(done_us) // 2],
+                                     "note": "median of 20 calls on the tiny configuration; the call synchronises the stream once, "
+                                             "after the routing kernels, to read K row counts"}}
+    for k in ("role_advantage", "device_fill_f32", "gae", "value_loss", "align_rewards", "ready_batch_gather_f32"):
         out[k]["frac"] = out[k]["gbs"] / peaks["hbm_gbs"]
     ctx.close()
     return out

@@ -112,6 +112,9 @@ int unity_set_profiling(unity_ctx* ctx, int enable);
 #define UNITY_OPT_L2_HINTS_FWD 16 /* 16..19: L2 eviction policy of the forward / recompute / dHidden / dW GEMM: value =
                                      A-operand loads | B-operand loads << 2 | logit-gradient stores << 4, each 0 normal,
                                      1 evict first, 2 evict last (defaults 6, 22, 0, 0: measured +0.3-0.7 % on the first two) */
+#define UNITY_OPT_SYNC_PERIOD_GRAD 22 /* 22..24: the recompute / dHidden / dW GEMM's workers meet at every n-th tile (see         */
+#define UNITY_OPT_SYNC_PERIOD_DH 23   /* UNITY_OPT_CHUNK_SYNC); 1 = every tile                                                  */
+#define UNITY_OPT_SYNC_PERIOD_DW 24
 #define UNITY_OPT_WAIT_KCYCLES 20  /* bound of every in-kernel wait in thousands of SM clocks (default 4 000 000, about 2 s); when
                                      it runs out the kernel records UNITY_ERR_TIMEOUT, frees its tensor memory and returns */
 #define UNITY_OPT_TEST_DROP_SLAB 21 /* TEST HOOK for the timeout path; accepted only while UNITY_OPT_WAIT_KCYCLES <= 1000.
@@ -143,13 +146,19 @@ int unity_get_profile(unity_ctx* ctx, double* ms, int64_t* launches);
  *   tok_mask       : u8 [n_tok] or NULL (= all 1)
  *   adv_inv        : out f32 [n_inv];  adv_tok : out f32 [n_tok] (NULL allowed when n_tok == 0)
  *   seg_mean, seg_std : out f32 [n_groups*n_roles] or NULL; index g*n_roles+v; 0 for empty segments
- * Deterministic: fixed-order reductions, no floating-point atomics.
+ * The members of a segment may sit anywhere in the batch (buffers fill in arrival order): the cost is O(n_inv)
+ * whatever the order.  Sums are taken exactly on a per-segment integer grid with integer atomics, so the result
+ * does not depend on scheduling (bitwise reproducible; no floating-point atomics), and a segment whose rewards
+ * are all equal gets exactly 0.
+ * Workspace: unity_advantage_workspace_bytes(n_inv, n_groups, n_roles) = 8 bytes per invocation + 32 bytes per
+ * (group, role) segment; n_groups*n_roles <= 2^24.
  */
 typedef struct {
     float eps; /* default 1e-6 */
     int ddof;  /* 0 (population) or 1 (sample) */
 } unity_adv_params;
 
+size_t unity_advantage_workspace_bytes(int32_t n_inv, int32_t n_groups, int32_t n_roles);
 int unity_role_advantage(unity_ctx* ctx, int32_t n_inv, int32_t n_traj, int32_t n_roles, int32_t n_groups,
                          const int32_t* inv_role, const int32_t* inv_group, const int32_t* inv_traj,
                          const float* r_node, const float* r_turn, const float* r_traj, const float* lam,
@@ -274,23 +283,29 @@ int unity_align_rewards(unity_ctx* ctx, int32_t n_inv, int64_t n_tok, const int6
  * Who needs it: hosts that may not call cudaMalloc or create a unity_ctx - a trainer whose framework
  * allocator already owns all device memory, a plug-in held to a memory budget by its host process, or a
  * caller that cannot afford the device-wide synchronisation an allocation implies.  The result is the same
- * as unity_role_advantage's; the per-invocation scratch (combined reward and segment id) sits in a fixed
- * device array inside the library instead of a workspace, so no context and no workspace are involved and
- * the call itself performs no cudaMalloc / cudaFree of any kind.
+ * as unity_role_advantage's (same kernels, same cost O(n_inv)); the scratch (combined reward and segment id per
+ * invocation, 32 bytes of accumulators per segment) sits in a fixed device array inside the library instead of a
+ * workspace, so no context and no workspace are involved and the call itself performs no cudaMalloc / cudaFree,
+ * nor any library routine that allocates.
  *
  *   device, cuda_stream : GPU to run on (made current by the call) and the stream to enqueue on
- *   n_inv               : at most UNITY_NOALLOC_MAX_INV, otherwise UNITY_ERR_SHAPE (nothing is launched)
+ *   n_inv               : at most UNITY_NOALLOC_MAX_INV, and n_groups*n_roles at most UNITY_NOALLOC_MAX_SEG,
+ *                         otherwise UNITY_ERR_SHAPE (nothing is launched)
  *   bad_index_out       : optional DEVICE int32; receives non-zero (stream-ordered, no sync) when a role,
  *                         group or trajectory id was out of range and its invocation was left out
  *   err, err_len        : optional HOST buffer that receives a one-line reason when the return is not 0
  *   every other argument: exactly as in unity_role_advantage
- * Cost: each GPU that loads the library holds the array (256 B + 8 B * UNITY_NOALLOC_MAX_INV, about 0.5 MiB)
- * until the process exits.  The first call on a device looks the array's address up once
- * (cudaGetSymbolAddress); make that first call outside any stream capture.  All calls on a device share the
- * one array and it keeps the previous call's contents - the call re-initialises what it reads, but two calls
- * whose kernels can overlap on the GPU (different streams, no ordering between them) race on it: serialise them.
+ * Cost: each GPU that loads the library holds the array (256 B + 8 B * UNITY_NOALLOC_MAX_INV + 32 B *
+ * UNITY_NOALLOC_MAX_SEG, about 2.5 MiB) until the process exits.  The first call on a device looks the array's
+ * address up (cudaGetSymbolAddress) and may make the CUDA runtime load this library's device code, which is the
+ * runtime's own one-time allocation: make that first call outside any stream capture, and count on "no
+ * allocation" from the second call on.  The address is kept for the life of the process: do not call
+ * cudaDeviceReset while the library is in use.  All calls on a device share the one array and it keeps the
+ * previous call's contents - the call clears what must start at zero, but two calls whose kernels can overlap on
+ * the GPU (different streams, no ordering between them) race on it: serialise them.
  */
 #define UNITY_NOALLOC_MAX_INV 65536
+#define UNITY_NOALLOC_MAX_SEG 65536
 int unity_role_advantage_noalloc(int device, void* cuda_stream, int32_t n_inv, int32_t n_traj, int32_t n_roles,
                                  int32_t n_groups, const int32_t* inv_role, const int32_t* inv_group,
                                  const int32_t* inv_traj, const float* r_node, const float* r_turn,

@@ -26,7 +26,7 @@ UNITY_N_METRICS = 8
 EXPORTS = ["unity_create", "unity_destroy", "unity_workspace_hint", "unity_workspace_bytes", "unity_workspace_min_bytes",
            "unity_workspace_bytes_stash",
            "unity_check_status", "unity_last_error", "unity_launch_count", "unity_set_profiling",
-           "unity_get_profile", "unity_set_option", "unity_role_advantage", "unity_reward_assembly", "unity_gae", "unity_value_loss_fwd_bwd",
+           "unity_get_profile", "unity_set_option", "unity_advantage_workspace_bytes", "unity_role_advantage", "unity_reward_assembly", "unity_gae", "unity_value_loss_fwd_bwd",
            "unity_ready_batch_plan", "unity_ready_batch_gather", "unity_align_rewards",
            "unity_role_advantage_noalloc",
            "unity_logprob_fwd", "unity_ppo_loss_fwd_bwd"]
@@ -101,6 +101,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.unity_set_option.restype = C.c_int
     lib.unity_get_profile.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
     lib.unity_get_profile.restype = C.c_int
+    lib.unity_advantage_workspace_bytes.argtypes = [i32, i32, i32]
+    lib.unity_advantage_workspace_bytes.restype = C.c_size_t
     lib.unity_role_advantage.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, f32p,
                                          C.POINTER(unity_adv_params), i64, vp, vp, vp, vp, vp, vp]
     lib.unity_role_advantage.restype = C.c_int
@@ -163,6 +165,10 @@ def unity_workspace_bytes(n_tok: int, H: int, V: int, K: int, n_inv: int) -> int
 
 def unity_workspace_min_bytes(n_tok: int, H: int, V: int, K: int, n_inv: int) -> int:
     return int(load_library().unity_workspace_min_bytes(n_tok, H, V, K, n_inv))
+
+
+def unity_advantage_workspace_bytes(n_inv: int, n_groups: int, n_roles: int) -> int:
+    return int(load_library().unity_advantage_workspace_bytes(n_inv, n_groups, n_roles))
 
 
 def unity_workspace_bytes_stash(n_tok: int, H: int, V: int, K: int, n_inv: int) -> int:
@@ -318,6 +324,7 @@ def unity_align_rewards(ctx, cu_seqlens, tok_mask, r_inv, tok_reward) -> None:
 
 
 UNITY_NOALLOC_MAX_INV = 65536
+UNITY_NOALLOC_MAX_SEG = 65536
 
 
 def unity_role_advantage_noalloc(device: int, stream_ptr: int, n_traj: int, n_roles: int, n_groups: int, inv_role,

@@ -194,39 +194,67 @@ __global__ void k_batch_parts(BatchArgs a) {
         for (int q = mine + 1; q < a.n_parts; ++q) a.part_offsets[k * a.n_parts + q] = j + 1;
 }
 
-// Gather: block (x = kept invocation, strided; y = slice) copies the invocation's contiguous bytes and fills the pad.
+// Gather: `slices` warps per kept invocation (one for per-token scalars, more for wide rows) copy the invocation's
+// contiguous bytes and fill the pad; many invocations are in flight at once, so the chain order -> offsets -> data of
+// one invocation overlaps with the copies of others.  When source and destination of an invocation are both 16-byte
+// aligned, its whole 16-byte words move as 128-bit vectors whatever the unit T is (per-token scalars are contiguous
+// across tokens); the rest, and unaligned invocations, move unit by unit.  Four accesses per lane are issued before
+// their stores.
 template <typename T>
 __global__ void k_batch_gather(const int* __restrict__ order, const int64_t* __restrict__ src_cu,
                                const int64_t* __restrict__ out_cu, const long long* __restrict__ totals,
-                               long long units_per_row, const T* __restrict__ src, T* __restrict__ dst, T pad) {
+                               long long units_per_row, const T* __restrict__ src, T* __restrict__ dst, T pad, int slices) {
     const int n_kept = static_cast<int>(totals[0]);
-    for (int j = blockIdx.x; j < n_kept; j += gridDim.x) {
-        const int s = order[j];
-        const long long n_copy = (src_cu[s + 1] - src_cu[s]) * units_per_row;
-        const long long n_slot = (out_cu[j + 1] - out_cu[j]) * units_per_row;
-        const T* from = src + src_cu[s] * units_per_row;
-        T* to = dst + out_cu[j] * units_per_row;
-        const long long stride = static_cast<long long>(gridDim.y) * blockDim.x;
-        // four units per thread and step, loads issued before the stores
-        for (long long i = static_cast<long long>(blockIdx.y) * blockDim.x + threadIdx.x; i < n_slot; i += 4 * stride) {
-            T v[4];
+    const long long warp = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+    const int j = static_cast<int>(warp / slices);
+    if (j >= n_kept) return;
+    const long long stride = static_cast<long long>(slices) * 32;
+    const long long first = (warp - static_cast<long long>(j) * slices) * 32 + (threadIdx.x & 31);
+    const int s = order[j];
+    const long long n_copy = (src_cu[s + 1] - src_cu[s]) * units_per_row;
+    const long long n_slot = (out_cu[j + 1] - out_cu[j]) * units_per_row;
+    const T* from = src + src_cu[s] * units_per_row;
+    T* to = dst + out_cu[j] * units_per_row;
+    long long done = 0;                                    // units already moved by the vector part
+    if (sizeof(T) < 16 && ((reinterpret_cast<uintptr_t>(from) | reinterpret_cast<uintptr_t>(to)) & 15) == 0) {
+        constexpr long long per = 16 / sizeof(T);
+        const long long n_vec = n_copy / per;
+        const uint4* from4 = reinterpret_cast<const uint4*>(from);
+        uint4* to4 = reinterpret_cast<uint4*>(to);
+        for (long long i = first; i < n_vec; i += 4 * stride) {
+            uint4 v[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const long long q = i + u * stride;
-                v[u] = q < n_copy ? from[q] : pad;
+                if (q < n_vec) v[u] = from4[q];
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const long long q = i + u * stride;
-                if (q < n_slot) to[q] = v[u];
+                if (q < n_vec) to4[q] = v[u];
             }
+        }
+        done = n_vec * per;
+    }
+    for (long long i = done + first; i < n_slot; i += 4 * stride) {
+        T v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const long long q = i + u * stride;
+            v[u] = q < n_copy ? from[q] : pad;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const long long q = i + u * stride;
+            if (q < n_slot) to[q] = v[u];
         }
     }
 }
 
-// Delayed rewards: one warp per invocation.  The sequence is zero-filled front to back, 16 tokens per lane and step
-// (one 128-bit mask load, four 128-bit stores) once the index is a multiple of 16; every lane remembers the last
-// unmasked token it saw, the warp takes the maximum, and after the warp's stores are ordered that token gets the reward.
+// Delayed rewards: one warp per invocation.  The sequence is zero-filled front to back; once the index is a multiple of
+// 4 the warp covers 512 tokens per step (per lane four 32-bit mask loads and four 128-bit stores, each contiguous across
+// the warp); every lane remembers the last unmasked token it saw, the warp takes the maximum, and after the warp's
+// stores are ordered that token gets the reward.
 __global__ void k_align_rewards(int n_inv, const int64_t* __restrict__ cu, const uint8_t* __restrict__ mask,
                                 const float* __restrict__ r_inv, float* __restrict__ tok_reward, int vec_ok) {
     const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -234,28 +262,31 @@ __global__ void k_align_rewards(int n_inv, const int64_t* __restrict__ cu, const
     if (s >= n_inv) return;
     const long long lo = cu[s], hi = cu[s + 1];
     long long last = -1;
-    const long long head_end = vec_ok ? min(hi, (lo + 15) & ~15LL) : hi;
+    const long long head_end = vec_ok ? min(hi, (lo + 3) & ~3LL) : hi;
     for (long long t = lo + lane; t < head_end; t += 32) {
         tok_reward[t] = 0.f;
         if (mask == nullptr || mask[t]) last = t;
     }
-    const long long n_vec = (hi - head_end) >> 4;
-    for (long long q = lane; q < n_vec; q += 32) {
-        const long long t = head_end + (q << 4);
-        float4* out = reinterpret_cast<float4*>(tok_reward + t);
+    const long long n_quad = (hi - head_end) >> 2;
+    for (long long q0 = 0; q0 < n_quad; q0 += 128) {
+        unsigned m[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) out[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (mask == nullptr) {
-            last = t + 15;
-        } else {
-            const uint4 m = *reinterpret_cast<const uint4*>(mask + t);
-            const unsigned w[4] = {m.x, m.y, m.z, m.w};
+        for (int u = 0; u < 4; ++u) {
+            const long long q = q0 + u * 32 + lane;
+            m[u] = 0u;
+            if (q < n_quad) m[u] = mask == nullptr ? 0x01010101u : *reinterpret_cast<const unsigned*>(mask + head_end + (q << 2));
+        }
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (w[j]) last = t + 4 * j + ((31 - __clz(__vcmpne4(w[j], 0u))) >> 3);   // highest non-zero byte
+        for (int u = 0; u < 4; ++u) {
+            const long long q = q0 + u * 32 + lane;
+            if (q < n_quad) {
+                const long long t = head_end + (q << 2);
+                *reinterpret_cast<float4*>(tok_reward + t) = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (m[u]) last = t + ((31 - __clz(__vcmpne4(m[u], 0u))) >> 3);   // highest non-zero byte
+            }
         }
     }
-    for (long long t = head_end + (n_vec << 4) + lane; t < hi; t += 32) {
+    for (long long t = head_end + (n_quad << 2) + lane; t < hi; t += 32) {
         tok_reward[t] = 0.f;
         if (mask == nullptr || mask[t]) last = t;
     }
@@ -273,12 +304,14 @@ cudaError_t gather_as(const GatherArgs& g, cudaStream_t stream) {
     for (int i = 0; i < 16; ++i) bytes[i] = g.pad[i % g.pad_bytes];
     memcpy(&pad, bytes, sizeof(T));
     const long long units = g.row_bytes / static_cast<long long>(sizeof(T));
-    const int gx = g.n_inv < 4096 ? (g.n_inv > 0 ? g.n_inv : 1) : 4096;
-    // slices per invocation: enough blocks for rows of many bytes, one for per-token scalars
-    long long gy = (g.row_bytes * g.avg_len + 32767) / 32768;
-    gy = gy < 1 ? 1 : (gy > 16 ? 16 : gy);
-    k_batch_gather<T><<<dim3(gx, static_cast<unsigned>(gy)), 256, 0, stream>>>(
-        g.order, g.src_cu, g.out_cu, g.totals, units, static_cast<const T*>(g.src), static_cast<T*>(g.dst), pad);
+    // warps per invocation: one per 8 KiB of an average invocation, so that per-token scalars take one warp and rows
+    // of hidden size spread over many
+    long long slices = (g.row_bytes * g.avg_len + 8191) / 8192;
+    slices = slices < 1 ? 1 : (slices > 1024 ? 1024 : slices);
+    const long long warps = static_cast<long long>(g.n_inv > 0 ? g.n_inv : 1) * slices;
+    k_batch_gather<T><<<static_cast<unsigned>((warps + 7) / 8), 256, 0, stream>>>(
+        g.order, g.src_cu, g.out_cu, g.totals, units, static_cast<const T*>(g.src), static_cast<T*>(g.dst), pad,
+        static_cast<int>(slices));
     return cudaGetLastError();
 }
 

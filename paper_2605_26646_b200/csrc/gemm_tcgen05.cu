@@ -76,11 +76,14 @@ __device__ __forceinline__ bool next_unit(const GemmArgs& g, int it, int pair, i
         const int m0 = it * gm;
         if (m0 >= g.m_tiles) return false;
         const int gm_here = min(gm, g.m_tiles - m0);
-        valid = pair < gm_here * g.n_splits;
+        const bool last = m0 >= g.last_m0;                       // the short last round: more, shorter splits
+        const int n_splits = last ? g.last_splits : g.n_splits;
+        const int tps = last ? g.last_tiles_per_split : g.tiles_per_split;
+        valid = pair < gm_here * n_splits;
         t.split = pair / gm_here;
         t.m_tile = m0 + (pair - t.split * gm_here);
-        t.n_begin = t.split * g.tiles_per_split;
-        t.n_end = min(t.n_begin + g.tiles_per_split, g.n_tiles);
+        t.n_begin = t.split * tps;
+        t.n_end = min(t.n_begin + tps, g.n_tiles);
         return true;
     } else {
         const int u = pair + it * n_pairs;
@@ -160,18 +163,26 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                 Unit t;
                 bool valid;
                 if (!next_unit<EPI>(g, it, pair, n_pairs, gm, t, valid)) break;
-                if (g.round_counter != nullptr && cta_rank == 0) {
-                    // Soft rendezvous at the start of every round: the workers that share a stream of W tiles stay in
-                    // step only while they start together, and once they drift apart by more than L2 can bridge each
-                    // of them fetches the stream from HBM again.  Purely a performance hint: after a short, bounded
-                    // wait the worker goes on regardless (some CTAs may not be resident yet).
+                if (g.round_counter != nullptr && cta_rank == 0 && (EPI == kEpiSoftmaxStats || it % g.sync_period == 0)) {
+                    // Soft rendezvous at the start of a round (softmax: every round; other epilogues, whose round is one
+                    // tile: every sync_period-th): the workers that share a stream of W tiles stay in step only while
+                    // they start together, and once they drift apart by more than L2 can bridge each of them fetches the
+                    // stream from HBM again.  Purely a performance hint: after a short, bounded wait the worker goes on
+                    // regardless (some CTAs may not be resident yet).
                     // The counter only ever grows; round_base is its value before this launch (every worker adds one
-                    // per round whether or not it waited, so the host can keep the running total).
+                    // per rendezvous whether or not it waited, so the host can keep the running total).
                     atomicAdd(g.round_counter, 1u);
-                    // arrivals expected by the end of this round: every worker (softmax), or every worker that still has
-                    // a tile (the last round of the other epilogues may be partial)
-                    unsigned expect = static_cast<unsigned>(it + 1) * static_cast<unsigned>(n_pairs);
-                    if (EPI != kEpiSoftmaxStats) expect = min(expect, static_cast<unsigned>(g.m_tiles * g.n_tiles));
+                    // arrivals expected by the end of this rendezvous: every worker (softmax), or every worker that
+                    // still has a tile (the last ones of the other epilogues may be partial)
+                    unsigned expect;
+                    if (EPI == kEpiSoftmaxStats) {
+                        expect = static_cast<unsigned>(it + 1) * static_cast<unsigned>(n_pairs);
+                    } else {
+                        const long long before = static_cast<long long>(it) * n_pairs;      // units of earlier rounds
+                        const long long left = static_cast<long long>(g.m_tiles) * g.n_tiles - before;
+                        expect = static_cast<unsigned>(it / g.sync_period) * static_cast<unsigned>(n_pairs) +
+                                 static_cast<unsigned>(left < n_pairs ? left : n_pairs);
+                    }
                     const unsigned target = g.round_base + expect;
                     const long long t0 = clock64();
                     while (static_cast<int>(*reinterpret_cast<volatile unsigned*>(g.round_counter) - target) < 0 &&
@@ -180,7 +191,10 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                 if (!valid) continue;
                 const int a_row = g.a_row0 + t.m_tile * C::kTileRows + static_cast<int>(cta_rank) * kCtaM;
                 for (int nt = t.n_begin; nt < t.n_end && ok; ++nt) {
-                    const int b_row = g.b_row0 + nt * kTileCols + static_cast<int>(cta_rank) * C::kBRows;
+                    // fp32-accumulate tiles may be narrower than 256 columns per MMA (mma_n); the B boxes keep their size, the
+                    // MMA simply leaves their last columns unread
+                    const int mma_n = EPI == kEpiAccumF32 ? g.mma_n : kTileN;
+                    const int b_row = g.b_row0 + nt * (NB * mma_n) + static_cast<int>(cta_rank) * (mma_n / CTAS);
                     for (int k = 0; k < g.k_iters; ++k) {
                         if (!ptx::mbar_wait(&empty[stage], phase ^ 1, g.wait_budget) || *abort_flag) { ok = false; break; }
                         if (g.test_drop_slab && it == 0 && nt == t.n_begin && k == (g.k_iters > 1 ? 1 : 0)) {
@@ -205,10 +219,10 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                             if (B_MN) {
 #pragma unroll
                                 for (int j = 0; j < C::kBRows / 64; ++j)
-                                    ptx::tma_load_2d_hint_on<CTAS>(sB + j * kMnBoxBytes, &tmB, bar, b_row + nb * kTileN + j * 64,
+                                    ptx::tma_load_2d_hint_on<CTAS>(sB + j * kMnBoxBytes, &tmB, bar, b_row + nb * mma_n + j * 64,
                                                                    g.b_k0 + k * kTileK, pol_b);
                             } else {
-                                ptx::tma_load_2d_hint_on<CTAS>(sB, &tmB, bar, g.b_k0 + k * kTileK, b_row + nb * kTileN, pol_b);
+                                ptx::tma_load_2d_hint_on<CTAS>(sB, &tmB, bar, g.b_k0 + k * kTileK, b_row + nb * mma_n, pol_b);
                             }
                         }
                         if (++stage == kStages) { stage = 0; phase ^= 1; }
@@ -220,7 +234,8 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (even CTA only)
         if (lane == 0 && cta_rank == 0) {
-            constexpr uint32_t idesc = ptx::idesc_bf16_f32(C::kTileRows, kTileN) | (A_MN ? (1u << 15) : 0u) | (B_MN ? (1u << 16) : 0u);
+            const uint32_t idesc = ptx::idesc_bf16_f32(C::kTileRows, EPI == kEpiAccumF32 ? g.mma_n : kTileN) |
+                                   (A_MN ? (1u << 15) : 0u) | (B_MN ? (1u << 16) : 0u);
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
@@ -320,13 +335,16 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                 if (!ptx::mbar_wait(&acc_full[acc], acc_phase, g.wait_budget) || *abort_flag) { ok = false; break; }
                 ptx::tc_fence_after();
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kTileCols;
-                const int col0 = nt * kTileCols;
+                const int mma_n = EPI == kEpiAccumF32 ? g.mma_n : kTileN;     // columns per MMA block (<= 256)
+                const int col0 = nt * (NB * mma_n);
+                const int per_block = mma_n / 32;
 #pragma unroll 1
-                for (int c = 0; c < kTileCols / 32; ++c) {
-                    const int cbase = col0 + c * 32;
+                for (int c = 0; c < NB * per_block; ++c) {
+                    const int cbase = col0 + c * 32;            // block nb of a two-block tile starts at col0 + nb * mma_n
                     if (cbase >= g.n_cols) break;               // uniform across the CTA
                     uint32_t rr[32];
-                    ptx::tmem_ld_32x32(taddr + c * 32, rr);
+                    // ... and sits at tensor-memory column nb * 256 whatever mma_n is
+                    ptx::tmem_ld_32x32(taddr + (NB == 1 ? c * 32 : (c / per_block) * kTileN + (c % per_block) * 32), rr);
                     ptx::tmem_ld_wait();
                     float v[32];
 #pragma unroll
@@ -482,7 +500,10 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                 float s0, s1, t0, t1;
                 ptx::unpack2(run_s2, s0, s1);
                 ptx::unpack2(run_t2, t0, t1);
-                g.stats[t.split * g.stats_pitch + row] = make_float4(run_m, s0 + s1, t0 + t1, z_tgt);
+                const long long at = t.m_tile >= g.last_m0
+                                         ? g.last_stats_off + t.split * g.last_pitch + (row - g.last_m0 * C::kTileRows)
+                                         : t.split * g.stats_pitch + row;
+                g.stats[at] = make_float4(run_m, s0 + s1, t0 + t1, z_tgt);
             }
         }
         if (!ok) { *abort_flag = 1; atomicOr(g.status, kStatusTimeout); }
@@ -547,7 +568,11 @@ cudaError_t gemm_set_attributes() {
 }
 
 int gemm_tile_rows(int ctas) { return kCtaM * ctas; }
-int gemm_tile_cols(bool wide) { return wide ? 2 * kTileN : kTileN; }
+int gemm_mma_n(int n_cols) {
+    const int blocks = (n_cols + kTileN - 1) / kTileN;
+    const int per = (n_cols + blocks - 1) / blocks;
+    return (per + 31) / 32 * 32;
+}
 
 namespace {
 // workers and rounds of a launch (must mirror next_unit and launch_gemm)
@@ -572,9 +597,14 @@ unsigned gemm_round_arrivals(GemmEpilogue epi, int ctas, const GemmArgs& args, i
     launch_shape(epi, ctas, args, sm_count, &workers, &rounds);
     if (workers == 0) return 0;
     if (epi == kEpiSoftmaxStats) return static_cast<unsigned>(rounds * workers);
-    // striding over units: worker p runs ceil((units - p) / workers) rounds
+    // striding over units: the workers that still have a tile in round r arrive at its rendezvous, every
+    // sync_period-th round has one
     const long long units = static_cast<long long>(args.m_tiles) * args.n_tiles;
-    return static_cast<unsigned>(units);
+    const int period = args.sync_period > 0 ? args.sync_period : 1;
+    long long total = 0;
+    for (long long before = 0; before < units; before += static_cast<long long>(period) * workers)
+        total += units - before < workers ? units - before : workers;
+    return static_cast<unsigned>(total);
 }
 
 cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, int ctas, const CUtensorMap& tmA, const CUtensorMap& tmB,
@@ -584,6 +614,7 @@ cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, int ctas, const CUtensorMap
                                 ? static_cast<long long>(args.group_m < args.m_tiles ? args.group_m : args.m_tiles) * args.n_splits
                                 : static_cast<long long>(args.m_tiles) * args.n_tiles;
     if (units <= 0 || args.m_tiles <= 0 || args.k_iters <= 0) return cudaSuccess;
+    if (epi == kEpiAccumF32 && (args.mma_n < 32 || args.mma_n > kTileN || args.mma_n % 32 != 0)) return cudaErrorInvalidValue;
     const int max_workers = sm_count / ctas;                                   // one CTA per SM
     const int workers = static_cast<int>(units < max_workers ? units : max_workers);
     const bool two = ctas == 2;

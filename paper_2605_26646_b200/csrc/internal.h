@@ -40,8 +40,14 @@ struct GemmArgs {
     int m_rows, n_cols;       // valid extent of C from (a_row0, b_row0): epilogue writes nothing beyond it
     // kEpiSoftmaxStats: a unit is (row tile, vocabulary split); a CTA keeps a unit's running statistics
     int n_splits, tiles_per_split;
+    // ... and the last round, when it holds fewer row tiles than the others, may cut the vocabulary into more splits so
+    // that it still occupies the machine: row tiles >= last_m0 use last_splits / last_tiles_per_split and write their
+    // statistics to stats[last_stats_off + split * last_pitch + (row - first row of tile last_m0)]
+    int last_m0, last_splits, last_tiles_per_split;
+    long long last_stats_off, last_pitch;
     unsigned* round_counter;  // ever-growing arrival counter (null = no rendezvous between rounds)
     unsigned round_base;      // its value before this launch
+    int sync_period;          // epilogues other than softmax: rendezvous at every sync_period-th tile of a worker (>= 1)
     float4* stats;            // [n_splits][stats_pitch], row relative to a_row0: (max acc, sum e, sum e*acc, target acc)
     long long stats_pitch;
     const int* target_p;      // [rows] packed targets (global vocabulary index), indexed from a_row0 + row
@@ -64,6 +70,8 @@ struct GemmArgs {
     float* C;
     long long ldc;
     int beta;                 // 0: overwrite, 1: add to C
+    int mma_n;                // columns per MMA block, a multiple of 32 up to 256 (a tile is 1 or 2 blocks wide); 256
+                              // unless the output's width divides better (896 columns = 4 blocks of 224)
     int l2_hints;             // L2 eviction policy (0 normal, 1 first, 2 last): bits 0-1 A loads, 2-3 B loads, 4-5 G stores
     int* status;
     long long wait_budget;    // SM clocks after which an mbarrier wait gives up (kStatusTimeout)
@@ -75,13 +83,14 @@ struct GemmArgs {
 // a_row0 / b_row0 index the contiguous dimension of its tensor map and a_k0 / b_k0 its rows.
 // ctas: 1 = one CTA per 128 x 256 tile, 2 = a CTA pair per 256 x 256 tile; args.m_tiles counts tiles of
 // gemm_tile_rows(ctas) rows.
-// wide: 512-column output tiles (kEpiAccumF32 with ctas = 2 only); args.n_tiles then counts tiles of 512 columns.
+// wide: output tiles two MMA blocks wide (kEpiAccumF32 with ctas = 2 only); args.n_tiles then counts tiles of
+// 2 * args.mma_n columns instead of args.mma_n.
 cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, int ctas, const CUtensorMap& tmA, const CUtensorMap& tmB,
                         const GemmArgs& args, int sm_count, cudaStream_t stream, bool wide = false);
 // Arrivals the launch adds to args.round_counter (rounds x workers); 0 when nothing is launched.
 unsigned gemm_round_arrivals(GemmEpilogue epi, int ctas, const GemmArgs& args, int sm_count);
 int gemm_tile_rows(int ctas);
-int gemm_tile_cols(bool wide);
+int gemm_mma_n(int n_cols);   // block width for an fp32-accumulate GEMM with n_cols output columns
 cudaError_t gemm_set_attributes();
 
 // ----------------------------------------------------------------------------------------------
@@ -99,12 +108,13 @@ struct AdvArgs {
     const int64_t* cu_seqlens;
     const uint8_t* tok_mask;
     float *adv_inv, *adv_tok, *seg_mean, *seg_std;
-    float* r_scratch;   // [n_inv]
-    int* seg_scratch;   // [n_inv]
-    int *seg_lo, *seg_hi;   // [n_groups*n_roles] first / last member index (pre-set to INT_MAX-ish / -1), or null
+    float* r_scratch;   // [n_inv] combined reward
+    int* seg_scratch;   // [n_inv] segment id g * n_roles + v, or -1 for an invocation with an id out of range
+    void* seg_table;    // advantage_table_bytes(n_groups * n_roles) bytes, 8-byte aligned; cleared by launch_advantage
     int* status;
 };
 cudaError_t launch_advantage(const AdvArgs& a, cudaStream_t stream, int* n_launches);
+size_t advantage_table_bytes(long long n_seg);   // per-segment accumulators of the statistics passes
 
 struct RouteArgs {
     long long n_tok;
@@ -135,6 +145,11 @@ struct TokenArgs {
     const float4* stats;       // per model: base stats_base[k], pitch = padded rows of the model
     long long stats_base[UNITY_MAX_MODELS];
     int model_splits[UNITY_MAX_MODELS];
+    // rows of a model from last_row0[k] on (relative to its first slot) were swept with last_splits[k] splits; their
+    // statistics start at stats_last[k] with pitch = the model's padded rows - last_row0[k]
+    int last_row0[UNITY_MAX_MODELS];
+    int last_splits[UNITY_MAX_MODELS];
+    long long stats_last[UNITY_MAX_MODELS];
     const int* slot_tok;
     const int* tok_slot;
     const int8_t* tok_model;

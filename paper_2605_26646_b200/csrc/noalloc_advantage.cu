@@ -1,8 +1,8 @@
 // unity_role_advantage_noalloc: the role-level advantage stage for callers that must not allocate.
 //
-// The regular entry point keeps two per-invocation scratch vectors (combined reward, segment id) in the
-// workspace of a context, and creating a context calls cudaMalloc / cudaMallocHost.  Some hosts of this
-// library cannot do that: a trainer that has handed every byte of device memory to its framework's caching
+// The regular entry point keeps two per-invocation scratch vectors (combined reward, segment id) and a table of
+// per-segment accumulators in the workspace of a context, and creating a context calls cudaMalloc /
+// cudaMallocHost.  Some hosts of this library cannot do that: a trainer that has handed every byte of device memory to its framework's caching
 // allocator, a plug-in running under a memory budget enforced by its host process, or code that sits on a
 // latency-critical path where the implicit device synchronisation of cudaMalloc is not acceptable.  For them
 // the scratch lives in the fixed device array below, which exists once per GPU for as long as the library
@@ -17,9 +17,11 @@ namespace {
 
 constexpr int kMaxDevices = 64;
 constexpr size_t kStatusBytes = 256;
-constexpr size_t kScratchBytes = kStatusBytes + 2 * sizeof(float) * UNITY_NOALLOC_MAX_INV;
+constexpr size_t kInvBytes = 2 * sizeof(float) * UNITY_NOALLOC_MAX_INV;
+constexpr size_t kScratchBytes = kStatusBytes + kInvBytes + 32 * static_cast<size_t>(UNITY_NOALLOC_MAX_SEG);
 
-// [0, 256): status word (bit set when an id in the data is out of range); then r[MAX_INV]; then seg[MAX_INV].
+// [0, 256): status word (bit set when an id in the data is out of range); then r[MAX_INV]; then seg[MAX_INV]; then
+// the per-segment accumulators (32 bytes each) of up to MAX_SEG segments.
 static __device__ __align__(256) unsigned char g_adv_scratch[kScratchBytes];
 
 std::mutex g_mu;
@@ -51,8 +53,8 @@ extern "C" int unity_role_advantage_noalloc(int device, void* cuda_stream, int32
         return UNITY_ERR_SHAPE;
     }
     if (n_roles < 1 || n_roles > UNITY_MAX_ROLES) { say(err, err_len, "n_roles outside [1, UNITY_MAX_ROLES]"); return UNITY_ERR_SHAPE; }
-    if (n_groups < 1 || static_cast<long long>(n_groups) * n_roles > (1 << 24)) {
-        say(err, err_len, "n_groups*n_roles outside [1, 2^24]");
+    if (n_groups < 1 || static_cast<long long>(n_groups) * n_roles > UNITY_NOALLOC_MAX_SEG) {
+        say(err, err_len, "n_groups*n_roles outside [1, UNITY_NOALLOC_MAX_SEG]: use unity_role_advantage with a workspace");
         return UNITY_ERR_SHAPE;
     }
     if (n_inv > 0 && (!inv_role || !inv_group || !adv_inv)) { say(err, err_len, "inv_role / inv_group / adv_inv is NULL"); return UNITY_ERR_INVALID_ARG; }
@@ -87,6 +89,7 @@ extern "C" int unity_role_advantage_noalloc(int device, void* cuda_stream, int32
     a.status = reinterpret_cast<int*>(base);
     a.r_scratch = reinterpret_cast<float*>(base + kStatusBytes);
     a.seg_scratch = reinterpret_cast<int*>(base + kStatusBytes + sizeof(float) * UNITY_NOALLOC_MAX_INV);
+    a.seg_table = base + kStatusBytes + kInvBytes;
     a.n_inv = n_inv; a.n_traj = n_traj; a.n_roles = n_roles; a.n_groups = n_groups;
     a.inv_role = inv_role; a.inv_group = inv_group; a.inv_traj = inv_traj;
     a.r_node = r_node; a.r_turn = r_turn; a.r_traj = r_traj;
@@ -95,7 +98,8 @@ extern "C" int unity_role_advantage_noalloc(int device, void* cuda_stream, int32
     a.eps = eps; a.ddof = ddof; a.n_tok = n_tok; a.cu_seqlens = cu_seqlens; a.tok_mask = tok_mask;
     a.adv_inv = adv_inv; a.adv_tok = adv_tok; a.seg_mean = seg_mean; a.seg_std = seg_std;
 
-    // The array keeps whatever the previous call left.  Only the status word must start at zero; the reward and
+    // The array keeps whatever the previous call left.  The status word must start at zero, and so must the
+    // accumulators of the n_groups*n_roles segments (launch_advantage clears those on the stream); the reward and
     // segment vectors are fully rewritten for [0, n_inv) before anything reads them.
     if (cudaMemsetAsync(a.status, 0, sizeof(int), st) != cudaSuccess) { cudaGetLastError(); say(err, err_len, "cudaMemsetAsync failed"); return UNITY_ERR_CUDA; }
     int nl = 0;

@@ -34,6 +34,44 @@ __device__ __forceinline__ int find_invocation(const int64_t* __restrict__ cu, i
 // ------------------------------------------------------------------------------------------------
 // Stage 1: advantage
 // ------------------------------------------------------------------------------------------------
+// Segment statistics without any ordering assumption.  Invocations of a (group, role) segment may sit anywhere in the
+// batch (buffers fill in arrival order), so nothing here sweeps index ranges: every pass is one thread per invocation
+// plus integer atomics on a per-segment table.  Integer addition is associative, so the result does not depend on the
+// order in which the atomics land: the statistics are exact on the segment's grid and bitwise reproducible.
+//   pass 1 (k_adv_combine): r_s, segment id; per segment the member count and max |r|
+//   pass 2 (k_adv_sum)    : q_s = r_s on the segment's integer grid; per segment sum q
+//   pass 3 (k_adv_m2)     : e_s = n q_s - sum q (n times the deviation from the mean, an exact integer; zero for every
+//                           member of a segment whose rewards are all equal); per segment sum e^2 in 128 bits
+//   pass 4 (k_adv_finish) : mean, sigma, advantages
+// Grid of a segment with n <= 2^L members and max |r| < 2^(E+1): multiples of 2^-shift, shift = B - (E + 1), with
+// B = min(61 - L, (125 - 3 L) / 2) bits per value, so that sum q stays below 2^62 and sum e^2 below 2^127.  For
+// segments of up to 64 members that is 53 or more bits (every fp32 reward within 2^29 of the largest is exact).
+struct SegTable {
+    int* cnt;
+    unsigned* maxbits;
+    long long* sum;
+    unsigned long long *m2lo, *m2hi;
+};
+__device__ __forceinline__ SegTable seg_table(const AdvArgs& a) {
+    const size_t n = static_cast<size_t>(a.n_groups) * a.n_roles;
+    SegTable t;
+    t.cnt = reinterpret_cast<int*>(a.seg_table);
+    t.maxbits = reinterpret_cast<unsigned*>(t.cnt + n);
+    t.sum = reinterpret_cast<long long*>(t.maxbits + n);
+    t.m2lo = reinterpret_cast<unsigned long long*>(t.sum + n);
+    t.m2hi = t.m2lo + n;
+    return t;
+}
+__device__ __forceinline__ int seg_shift(unsigned maxbits, int cnt) {
+    const int E = ilogbf(__uint_as_float(maxbits));              // max |r| > 0 (subnormals included)
+    const int L = cnt > 1 ? 32 - __clz(cnt - 1) : 0;             // cnt <= 2^L
+    const int B = min(61 - L, (125 - 3 * L) / 2);
+    return B - (E + 1);
+}
+__device__ __forceinline__ long long seg_quantise(float r, int shift) {
+    return __double2ll_rn(ldexp(static_cast<double>(r), shift));
+}
+
 __global__ void k_adv_combine(AdvArgs a) {
     const int s = blockIdx.x * blockDim.x + threadIdx.x;
     if (s >= a.n_inv) return;
@@ -54,102 +92,88 @@ __global__ void k_adv_combine(AdvArgs a) {
         const float rt = a.r_turn ? a.r_turn[s] : 0.f;
         r = __fadd_rn(__fadd_rn(__fmul_rn(ln, rn), __fmul_rn(lt, rt)), __fmul_rn(lj, rj));
         seg = g * a.n_roles + v;
-        if (a.seg_lo) { atomicMin(&a.seg_lo[seg], s); atomicMax(&a.seg_hi[seg], s); }
+        const SegTable t = seg_table(a);
+        atomicAdd(&t.cnt[seg], 1);
+        atomicMax(&t.maxbits[seg], __float_as_uint(fabsf(r)));   // bit patterns of non-negative floats order like the floats
     } else {
         atomicOr(a.status, kStatusBadIndex);
     }
     a.r_scratch[s] = r;
     a.seg_scratch[s] = seg;
-    a.adv_inv[s] = 0.f;
 }
 
-// One warp per (group, role) segment.  Three sweeps with 128-bit loads over the span of invocation indices that
-// contains the segment's members (recorded by k_adv_combine; rollout groups are normally contiguous, so spans are
-// short and the whole stage is O(n_inv)): count + sum -> mean; sum of squared deviations -> sigma; advantages.
-__global__ void k_adv_segment(AdvArgs a) {
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
+__global__ void k_adv_sum(AdvArgs a) {
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= a.n_inv) return;
+    const int seg = a.seg_scratch[s];
+    if (seg < 0) return;
+    const SegTable t = seg_table(a);
+    const unsigned mb = t.maxbits[seg];
+    if (mb == 0u) return;                                        // every reward of the segment is zero
+    const long long q = seg_quantise(a.r_scratch[s], seg_shift(mb, t.cnt[seg]));
+    atomicAdd(reinterpret_cast<unsigned long long*>(&t.sum[seg]), static_cast<unsigned long long>(q));
+}
+
+__global__ void k_adv_m2(AdvArgs a) {
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= a.n_inv) return;
+    const int seg = a.seg_scratch[s];
+    if (seg < 0) return;
+    const SegTable t = seg_table(a);
+    const unsigned mb = t.maxbits[seg];
+    if (mb == 0u) return;
+    const int cnt = t.cnt[seg];
+    const long long q = seg_quantise(a.r_scratch[s], seg_shift(mb, cnt));
+    const long long e = static_cast<long long>(cnt) * q - t.sum[seg];
+    if (e == 0) return;
+    const unsigned long long m = static_cast<unsigned long long>(e < 0 ? -e : e);
+    const unsigned long long lo = m * m, hi = __umul64hi(m, m);
+    // 128-bit accumulation with two 64-bit atomics: the low word's wrap-arounds are carried into the high word by
+    // whoever caused them, so the final pair is the exact sum whatever the order
+    const unsigned long long old = atomicAdd(&t.m2lo[seg], lo);
+    const unsigned long long carry = (old + lo < old) ? 1ull : 0ull;
+    if (hi + carry != 0ull) atomicAdd(&t.m2hi[seg], hi + carry);
+}
+
+// Thread i finishes invocation i (advantage) and segment i (mean and sigma for the caller).
+__global__ void k_adv_finish(AdvArgs a) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
     const int n_seg = a.n_groups * a.n_roles;
-    if (warp >= n_seg) return;
-    const int q = warp;
-    int lo = 0, hi = a.n_inv;                       // [lo, hi): invocation indices to look at
-    if (a.seg_lo) { lo = a.seg_lo[q]; hi = a.seg_hi[q] + 1; }
-    if (lo >= hi) {                                 // empty segment
-        if (lane == 0) { if (a.seg_mean) a.seg_mean[q] = 0.f; if (a.seg_std) a.seg_std[q] = 0.f; }
-        return;
-    }
-    const int q0 = lo >> 2, q1 = hi >> 2;           // whole quads [q0, q1); head and tail handled per element
-    const int head_end = min(hi, (q0 << 2) == lo ? lo : (q0 + 1) << 2);
-    const int quad_lo = (q0 << 2) == lo ? q0 : q0 + 1;
-    const int tail_begin = max(head_end, q1 << 2);
-    const int4* seg4 = reinterpret_cast<const int4*>(a.seg_scratch);
-    const float4* r4 = reinterpret_cast<const float4*>(a.r_scratch);
-
-    // Pivot = reward of the segment's first member.  All sums run over r - pivot, so a segment whose rewards are all
-    // equal gives exactly zero deviations (and zero advantages) whatever the order of the floating-point sums.
-    int first = lo;
-    if (!a.seg_lo) {
-        first = a.n_inv;
-        for (int s = lane; s < a.n_inv; s += 32)
-            if (a.seg_scratch[s] == q) { first = s; break; }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) first = min(first, __shfl_xor_sync(kFull, first, o));
-        if (first >= a.n_inv) {                     // empty segment
-            if (lane == 0) { if (a.seg_mean) a.seg_mean[q] = 0.f; if (a.seg_std) a.seg_std[q] = 0.f; }
-            return;
+    const SegTable t = seg_table(a);
+    auto stats = [&](int seg, double& mean, double& sigma, double& unit, int& cnt, int& shift) {
+        cnt = t.cnt[seg];
+        const unsigned mb = t.maxbits[seg];
+        mean = 0.0; sigma = 0.0; unit = 0.0; shift = 0;
+        if (cnt == 0 || mb == 0u) return;
+        shift = seg_shift(mb, cnt);
+        unit = ldexp(1.0 / static_cast<double>(cnt), -shift);            // value of one step of e = n q - sum q
+        mean = static_cast<double>(t.sum[seg]) * unit;
+        const int dof = cnt - a.ddof;
+        if (dof > 0) {
+            const double m2 = (ldexp(static_cast<double>(t.m2hi[seg]), 64) + static_cast<double>(t.m2lo[seg])) * unit * unit;
+            sigma = sqrt(m2 / static_cast<double>(dof));
         }
+    };
+    double mean, sigma, unit;
+    int cnt, shift;
+    if (i < n_seg && (a.seg_mean != nullptr || a.seg_std != nullptr)) {
+        stats(i, mean, sigma, unit, cnt, shift);
+        if (a.seg_mean) a.seg_mean[i] = static_cast<float>(mean);
+        if (a.seg_std) a.seg_std[i] = static_cast<float>(sigma);
     }
-    const float pivot = a.r_scratch[first];
-
-    int cnt = 0;
-    float sum = 0.f;
-    for (int s = lo + lane; s < head_end; s += 32)
-        if (a.seg_scratch[s] == q) { cnt++; sum += a.r_scratch[s] - pivot; }
-    for (int i = quad_lo + lane; i < q1; i += 32) {
-        const int4 sg = seg4[i];
-        if (sg.x == q || sg.y == q || sg.z == q || sg.w == q) {
-            const float4 r = r4[i];
-            if (sg.x == q) { cnt++; sum += r.x - pivot; }
-            if (sg.y == q) { cnt++; sum += r.y - pivot; }
-            if (sg.z == q) { cnt++; sum += r.z - pivot; }
-            if (sg.w == q) { cnt++; sum += r.w - pivot; }
+    if (i < a.n_inv) {
+        const int seg = a.seg_scratch[i];
+        float adv = 0.f;
+        if (seg >= 0) {
+            stats(seg, mean, sigma, unit, cnt, shift);
+            const double denom = sigma + static_cast<double>(a.eps);
+            if (cnt - a.ddof > 0 && denom != 0.0 && unit != 0.0) {
+                const long long e = static_cast<long long>(cnt) * seg_quantise(a.r_scratch[i], shift) - t.sum[seg];
+                adv = static_cast<float>(static_cast<double>(e) * unit / denom);
+            }
         }
+        a.adv_inv[i] = adv;
     }
-    for (int s = tail_begin + lane; s < hi; s += 32)
-        if (a.seg_scratch[s] == q) { cnt++; sum += a.r_scratch[s] - pivot; }
-    cnt = warp_sum_int(cnt);
-    sum = warp_sum(sum);
-    const float dmu = cnt > 0 ? sum / static_cast<float>(cnt) : 0.f;     // mean of r - pivot
-    const float mu = pivot + dmu;
-
-    float m2 = 0.f;
-    for (int s = lo + lane; s < head_end; s += 32)
-        if (a.seg_scratch[s] == q) { const float d = (a.r_scratch[s] - pivot) - dmu; m2 += d * d; }
-    for (int i = quad_lo + lane; i < q1; i += 32) {
-        const int4 sg = seg4[i];
-        if (sg.x == q || sg.y == q || sg.z == q || sg.w == q) {
-            const float4 r = r4[i];
-            if (sg.x == q) { const float d = (r.x - pivot) - dmu; m2 += d * d; }
-            if (sg.y == q) { const float d = (r.y - pivot) - dmu; m2 += d * d; }
-            if (sg.z == q) { const float d = (r.z - pivot) - dmu; m2 += d * d; }
-            if (sg.w == q) { const float d = (r.w - pivot) - dmu; m2 += d * d; }
-        }
-    }
-    for (int s = tail_begin + lane; s < hi; s += 32)
-        if (a.seg_scratch[s] == q) { const float d = (a.r_scratch[s] - pivot) - dmu; m2 += d * d; }
-    m2 = warp_sum(m2);
-
-    const int dof = cnt - a.ddof;
-    const float sigma = dof > 0 ? sqrtf(m2 / static_cast<float>(dof)) : 0.f;
-    const float denom = sigma + a.eps;
-    if (lane == 0) {
-        if (a.seg_mean) a.seg_mean[q] = mu;
-        if (a.seg_std) a.seg_std[q] = sigma;
-    }
-    if (cnt == 0) return;
-    for (int s = lo + lane; s < hi; s += 32)
-        if (a.seg_scratch[s] == q)
-            a.adv_inv[s] = (dof > 0 && denom != 0.f) ? ((a.r_scratch[s] - pivot) - dmu) / denom : 0.f;
 }
 
 // A block broadcasts rounds x 1024 tokens; in a round each thread handles four consecutive tokens (one 32-bit mask
@@ -192,28 +216,36 @@ __global__ void k_adv_broadcast(AdvArgs a, int rounds) {
 }
 
 // The same broadcast with one warp per invocation, for batches of long invocations: no search; after the tokens up to
-// the next multiple of 16, every lane handles 16 tokens per step (one 128-bit mask load, four 128-bit stores).
+// the next multiple of 4, the warp walks the invocation 512 tokens per step: four times, every lane loads the four
+// mask bytes of its quad of tokens (128 B contiguous per warp) and stores one 128-bit vector (512 B contiguous per
+// warp), all four loads issued before the first store.
 __global__ void k_adv_broadcast_inv(AdvArgs a) {
     const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (s >= a.n_inv) return;
     const long long lo = a.cu_seqlens[s], hi = a.cu_seqlens[s + 1];
     const float adv = a.adv_inv[s];
-    const long long head_end = min(hi, (lo + 15) & ~15LL);
+    const long long head_end = min(hi, (lo + 3) & ~3LL);
     for (long long i = lo + lane; i < head_end; i += 32) a.adv_tok[i] = (a.tok_mask == nullptr || a.tok_mask[i]) ? adv : 0.f;
-    const long long n_vec = (hi - head_end) >> 4;
-    for (long long q = lane; q < n_vec; q += 32) {
-        const long long i = head_end + (q << 4);
-        uint4 m = make_uint4(0x01010101u, 0x01010101u, 0x01010101u, 0x01010101u);
-        if (a.tok_mask) m = *reinterpret_cast<const uint4*>(a.tok_mask + i);
-        const unsigned w[4] = {m.x, m.y, m.z, m.w};
-        float4* out = reinterpret_cast<float4*>(a.adv_tok + i);
+    const long long n_quad = (hi - head_end) >> 2;
+    for (long long q0 = 0; q0 < n_quad; q0 += 128) {
+        unsigned m[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-            out[j] = make_float4((w[j] & 0xffu) ? adv : 0.f, (w[j] & 0xff00u) ? adv : 0.f, (w[j] & 0xff0000u) ? adv : 0.f,
-                                 (w[j] & 0xff000000u) ? adv : 0.f);
+        for (int u = 0; u < 4; ++u) {
+            const long long q = q0 + u * 32 + lane;
+            m[u] = 0x01010101u;
+            if (a.tok_mask != nullptr && q < n_quad) m[u] = *reinterpret_cast<const unsigned*>(a.tok_mask + head_end + (q << 2));
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const long long q = q0 + u * 32 + lane;
+            if (q < n_quad)
+                *reinterpret_cast<float4*>(a.adv_tok + head_end + (q << 2)) =
+                    make_float4((m[u] & 0xffu) ? adv : 0.f, (m[u] & 0xff00u) ? adv : 0.f, (m[u] & 0xff0000u) ? adv : 0.f,
+                                (m[u] & 0xff000000u) ? adv : 0.f);
+        }
     }
-    for (long long i = head_end + (n_vec << 4) + lane; i < hi; i += 32)
+    for (long long i = head_end + (n_quad << 2) + lane; i < hi; i += 32)
         a.adv_tok[i] = (a.tok_mask == nullptr || a.tok_mask[i]) ? adv : 0.f;
 }
 
@@ -361,9 +393,15 @@ __global__ void k_finish_rows(TokenArgs a, int with_loss) {
         // the caller already evaluated this policy on these rows (unity_logprob_fwd): no forward sweep was run
         lse = a.lse_in[tok]; ent = a.entropy_in[tok]; logp = a.logp_in[tok];
     } else {
-        const long long pitch = a.offsets[k + 1] - a.offsets[k];
-        const float4* st = a.stats + a.stats_base[k] + (slot - a.offsets[k]);
-        const int n_splits = a.model_splits[k];
+        long long pitch = a.offsets[k + 1] - a.offsets[k];
+        const int r = slot - a.offsets[k];
+        const float4* st = a.stats + a.stats_base[k] + r;
+        int n_splits = a.model_splits[k];
+        if (r >= a.last_row0[k]) {                            // swept in the launch's short last round
+            pitch -= a.last_row0[k];
+            st = a.stats + a.stats_last[k] + (r - a.last_row0[k]);
+            n_splits = a.last_splits[k];
+        }
         const float c = a.scale * 1.4426950408889634f;    // exp(scale*x) = exp2(c*x)
         float m = -3.0e38f;
         for (int j = 0; j < n_splits; ++j) m = fmaxf(m, st[j * pitch].x);
@@ -828,12 +866,23 @@ __global__ void k_value_class(ValueArgs a) {
 // ------------------------------------------------------------------------------------------------
 // launchers
 // ------------------------------------------------------------------------------------------------
+size_t advantage_table_bytes(long long n_seg) { return static_cast<size_t>(n_seg) * 32; }
+
 cudaError_t launch_advantage(const AdvArgs& a, cudaStream_t stream, int* n_launches) {
-    if (a.n_inv > 0) {
-        k_adv_combine<<<(a.n_inv + 255) / 256, 256, 0, stream>>>(a);
-        const int n_seg = a.n_groups * a.n_roles;
-        k_adv_segment<<<(n_seg + 7) / 8, 256, 0, stream>>>(a);
-        *n_launches += 2;
+    const int n_seg = a.n_groups * a.n_roles;
+    if (a.n_inv > 0 || a.seg_mean || a.seg_std) {
+        cudaError_t e = cudaMemsetAsync(a.seg_table, 0, advantage_table_bytes(n_seg), stream);
+        if (e != cudaSuccess) return e;
+        const int blocks = (a.n_inv + 255) / 256;
+        if (blocks > 0) {
+            k_adv_combine<<<blocks, 256, 0, stream>>>(a);
+            k_adv_sum<<<blocks, 256, 0, stream>>>(a);
+            k_adv_m2<<<blocks, 256, 0, stream>>>(a);
+            *n_launches += 3;
+        }
+        const int n_fin = a.n_inv > n_seg ? a.n_inv : n_seg;
+        k_adv_finish<<<(n_fin + 255) / 256, 256, 0, stream>>>(a);
+        *n_launches += 1;
     }
     const bool aligned = (reinterpret_cast<uintptr_t>(a.tok_mask) & 15) == 0 && (reinterpret_cast<uintptr_t>(a.adv_tok) & 15) == 0;
     if (a.n_tok > 0 && aligned && a.n_tok / a.n_inv >= 128 && a.n_inv >= 1024) {

@@ -41,6 +41,7 @@ struct unity_ctx {
     int l2_hints[UNITY_PROF_CLASSES]; // per GEMM class: GemmArgs::l2_hints
     int wide_acc;                   // 1: dHidden / dW chunk GEMMs use 512-column tiles (CTA pairs only)
     unsigned round_total;           // arrivals accumulated so far on the rendezvous counter (d_status + 16)
+    int chunk_sync_period[3];       // recompute / dHidden / dW GEMM: rendezvous at every n-th tile of a worker
     long long wait_budget;          // SM clocks after which an in-kernel wait gives up
     int test_drop;                  // test hook: 1 + GEMM class whose producer leaves out one K slab; 0 = off
 };
@@ -103,6 +104,7 @@ void gemm_common(unity_ctx* ctx, GemmArgs& g, int cls, GemmEpilogue epi, bool sy
     g.l2_hints = ctx->l2_hints[cls];
     g.wait_budget = ctx->wait_budget;
     g.test_drop_slab = ctx->test_drop == cls + 1;
+    g.sync_period = cls == UNITY_PROF_FWD_GEMM ? 1 : ctx->chunk_sync_period[cls - 1];
     if (sync) {
         g.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
         g.round_base = ctx->round_total;
@@ -246,11 +248,17 @@ int validate_rows(unity_ctx* ctx, const unity_rows* r) {
     return UNITY_OK;
 }
 
+struct FwdShape {
+    int gm, splits, tps;                  // row tiles per round; vocabulary splits and tiles per split of a full round
+    int last_m0, last_splits, last_tps;   // first row tile, splits and tiles per split of a short last round
+                                          // (last_m0 = number of row tiles when the last round is like the others)
+    long long stats_rows;                 // float4 entries the launch writes: splits x rows + last_splits x last rows
+};
 struct RowPlan {
     Layout L;
     int counts[UNITY_MAX_MODELS];
     int offsets[UNITY_MAX_MODELS + 1];
-    int splits[UNITY_MAX_MODELS];
+    FwdShape shape[UNITY_MAX_MODELS];     // split layout of each model's forward launch
     long long stats_base[UNITY_MAX_MODELS];
     int n_slots;
 };
@@ -259,39 +267,49 @@ struct RowPlan {
 // vocabulary splits.  One round of the persistent kernel = gm row tiles x splits vocabulary splits <= number of
 // workers (CTAs or CTA pairs): gm bounds the hidden rows that must stay L2 resident (48 tiles of 128 rows by default:
 // 6 k rows, 44 MB at H = 3584, loaded with an evict-last hint), splits fill the machine.
-void forward_shape(const unity_ctx* ctx, int V, int rows, int* gm_out, int* splits_out, int* tps_out) {
+FwdShape forward_shape(const unity_ctx* ctx, int V, int rows) {
     const int ctas = ctx->ctas[UNITY_PROF_FWD_GEMM];
-    const int m_tiles = rows / gemm_tile_rows(ctas);
+    const int tile_rows = gemm_tile_rows(ctas);
+    const int m_tiles = rows / tile_rows;
     const int n_tiles = (V + kTileN - 1) / kTileN;
     const int n_pairs = ctx->sm_count / ctas;
     int gmax = ctx->fwd_group > 0 ? ctx->fwd_group / ctas : n_pairs / 4;
     if (gmax < 1) gmax = 1;
     if (gmax > n_pairs) gmax = n_pairs;
-    // Among round sizes from two thirds of gmax up to gmax, take the one with the least work per worker: rounds x
-    // vocabulary tiles per split (a batch whose row tiles do not divide well would otherwise idle part of the machine
-    // or run a nearly empty last round); ties go to the larger round, which streams W less often.
-    int gm = 1, splits = 1;
-    long long best = -1;
+    auto splits_for = [&](int tiles) {
+        int sp = n_pairs / (tiles > 0 ? tiles : 1);
+        if (sp > 32) sp = 32;
+        if (sp > n_tiles) sp = n_tiles;
+        return sp < 1 ? 1 : sp;
+    };
+    auto ceil_div = [](int a, int b) { return (a + b - 1) / b; };
+    // Among round sizes from two thirds of gmax up to gmax, take the one with the least work per worker: vocabulary
+    // tiles per split, summed over the rounds, the last of which may hold fewer row tiles and then cuts the vocabulary
+    // into more splits (a batch whose row tiles do not divide well would otherwise idle part of the machine in its
+    // last round); ties go to the larger round, which streams W less often.
+    FwdShape best;
+    long long best_cost = -1;
     const int cand_min = m_tiles <= gmax ? 1 : (2 * gmax + 2) / 3;      // few row tiles: any round size is L2-safe
     for (int cand = gmax; cand >= cand_min; --cand) {
         const int c = cand < m_tiles ? cand : (m_tiles > 0 ? m_tiles : 1);
-        int sp = n_pairs / c;
-        if (sp > 32) sp = 32;
-        if (sp > n_tiles) sp = n_tiles;
-        if (sp < 1) sp = 1;
-        const long long rounds = (m_tiles + c - 1) / c;
-        const long long cost = rounds * ((n_tiles + sp - 1) / sp);
-        if (best < 0 || cost < best) { best = cost; gm = c; splits = sp; }
+        const int sp = splits_for(c);
+        const int full_rounds = m_tiles / c, rest = m_tiles - full_rounds * c;
+        const int sp_last = rest > 0 ? splits_for(rest) : sp;
+        const long long cost = static_cast<long long>(full_rounds) * ceil_div(n_tiles, sp) + (rest > 0 ? ceil_div(n_tiles, sp_last) : 0);
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost;
+            best.gm = c;
+            best.tps = ceil_div(n_tiles, sp);
+            best.splits = ceil_div(n_tiles, best.tps);
+            best.last_m0 = rest > 0 && sp_last != sp ? full_rounds * c : m_tiles;
+            best.last_tps = ceil_div(n_tiles, sp_last);
+            best.last_splits = ceil_div(n_tiles, best.last_tps);
+        }
     }
-    const int tps = (n_tiles + splits - 1) / splits;
-    *gm_out = gm > 0 ? gm : 1;
-    *splits_out = (n_tiles + tps - 1) / tps;
-    *tps_out = tps;
-}
-int forward_splits(const unity_ctx* ctx, int V, int rows) {
-    int gm, splits, tps;
-    forward_shape(ctx, V, rows, &gm, &splits, &tps);
-    return splits;
+    if (best_cost < 0) { best.gm = 1; best.splits = 1; best.tps = n_tiles; best.last_m0 = m_tiles; best.last_splits = 1; best.last_tps = n_tiles; }
+    const long long last_rows = static_cast<long long>(m_tiles - best.last_m0) * tile_rows;
+    best.stats_rows = static_cast<long long>(best.splits) * rows + best.last_splits * last_rows;
+    return best;
 }
 
 // Optional stash of the scaled logits written by the forward kernel (see GemmArgs::Z).
@@ -304,18 +322,20 @@ struct ZStash {
 // LM-head GEMM + online softmax statistics for packed rows [slot0, slot0 + rows) of one model; statistics go to
 // stats[split * rows + (slot - slot0)].
 int launch_forward(unity_ctx* ctx, const unity_rows* r, int slot0, int rows, float4* stats, const int* target_p,
-                   const CUtensorMap& tmA, const CUtensorMap& tmB, const ZStash* z, int* splits_out) {
+                   const CUtensorMap& tmA, const CUtensorMap& tmB, const ZStash* z, FwdShape* shape_out) {
     const int ctas = ctx->ctas[UNITY_PROF_FWD_GEMM];
-    int gm, splits, tps;
-    forward_shape(ctx, r->V, rows, &gm, &splits, &tps);
-    *splits_out = splits;
+    const FwdShape fs = forward_shape(ctx, r->V, rows);
+    *shape_out = fs;
     GemmArgs g;
     memset(&g, 0, sizeof(g));
     g.m_tiles = rows / gemm_tile_rows(ctas); g.n_tiles = (r->V + kTileN - 1) / kTileN; g.k_iters = r->H / kTileK;
-    g.group_m = gm;
+    g.group_m = fs.gm;
     g.a_row0 = slot0; g.b_row0 = 0; g.a_k0 = 0; g.b_k0 = 0;
     g.m_rows = rows; g.n_cols = r->V;
-    g.n_splits = splits; g.tiles_per_split = tps;
+    g.n_splits = fs.splits; g.tiles_per_split = fs.tps;
+    g.last_m0 = fs.last_m0; g.last_splits = fs.last_splits; g.last_tiles_per_split = fs.last_tps;
+    g.last_stats_off = static_cast<long long>(fs.splits) * rows;
+    g.last_pitch = rows - static_cast<long long>(fs.last_m0) * gemm_tile_rows(ctas);
     g.stats = stats; g.stats_pitch = rows;
     g.target_p = target_p; g.vocab0 = 0; g.scale = r->inv_temperature;
     if (z) {
@@ -365,30 +385,43 @@ int forward_sweep(unity_ctx* ctx, const unity_rows* r, RowPlan& P, bool run_gemm
     }
     long long sbase = 0;
     for (int k = 0; k < r->K; ++k) {
-        P.splits[k] = 1;
+        memset(&P.shape[k], 0, sizeof(FwdShape));
+        P.shape[k].splits = P.shape[k].last_splits = 1;
+        P.shape[k].last_m0 = 0x3fffffff;
         P.stats_base[k] = sbase;
         const int rows_k = P.offsets[k + 1] - P.offsets[k];
         if (rows_k == 0 || !run_gemm) continue;
         CUtensorMap tmB;
         int rc = make_tmap(ctx, &tmB, r->W[k], r->H, r->V, static_cast<uint64_t>(r->H) * 2, kTileN / ctx->ctas[UNITY_PROF_FWD_GEMM]);
         if (rc) return rc;
-        if (sbase + static_cast<long long>(forward_splits(ctx, r->V, rows_k)) * rows_k > L.stats_cap)
+        if (sbase + forward_shape(ctx, r->V, rows_k).stats_rows > L.stats_cap)
             return fail(ctx, UNITY_ERR_WORKSPACE, "internal: statistics scratch too small");
-        rc = launch_forward(ctx, r, P.offsets[k], rows_k, L.stats + sbase, L.target_p, tmA, tmB, nullptr, &P.splits[k]);
+        rc = launch_forward(ctx, r, P.offsets[k], rows_k, L.stats + sbase, L.target_p, tmA, tmB, nullptr, &P.shape[k]);
         if (rc) return rc;
-        sbase += static_cast<long long>(P.splits[k]) * rows_k;
+        sbase += P.shape[k].stats_rows;
         nl += 1;
     }
     ctx->launches += nl;
     return UNITY_OK;
 }
 
-void fill_token_args(TokenArgs& t, const unity_rows* r, const RowPlan& P) {
+// Where k_finish_rows finds the per-split statistics of model k's rows (see launch_forward).
+void set_token_stats(TokenArgs& t, int k, long long base, const FwdShape& fs, int rows, int tile_rows) {
+    t.stats_base[k] = base;
+    t.model_splits[k] = fs.splits;
+    const long long last_row0 = static_cast<long long>(fs.last_m0) * tile_rows;
+    t.last_row0[k] = last_row0 < rows ? static_cast<int>(last_row0) : 0x7fffffff;
+    t.last_splits[k] = fs.last_splits;
+    t.stats_last[k] = base + static_cast<long long>(fs.splits) * rows;
+}
+
+void fill_token_args(TokenArgs& t, const unity_ctx* ctx, const unity_rows* r, const RowPlan& P) {
     memset(&t, 0, sizeof(t));
     const Layout& L = P.L;
     t.n_slots = P.n_slots; t.K = r->K; t.n_roles = r->n_roles; t.n_inv = r->n_inv; t.n_tok = r->n_tok;
     t.stats = L.stats;
-    for (int k = 0; k < r->K; ++k) { t.stats_base[k] = P.stats_base[k]; t.model_splits[k] = P.splits[k]; }
+    const int tile_rows = gemm_tile_rows(ctx->ctas[UNITY_PROF_FWD_GEMM]);
+    for (int k = 0; k < r->K; ++k) set_token_stats(t, k, P.stats_base[k], P.shape[k], P.offsets[k + 1] - P.offsets[k], tile_rows);
     for (int k = 0; k <= r->K; ++k) t.offsets[k] = P.offsets[k];
     t.slot_tok = L.slot_tok; t.tok_slot = L.tok_slot; t.tok_model = L.tok_model;
     t.scale = r->inv_temperature;
@@ -446,6 +479,7 @@ int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace
     c->l2_hints[UNITY_PROF_DH_GEMM] = 0;
     c->l2_hints[UNITY_PROF_DW_GEMM] = 0;
     c->logit_stash = 0;
+    c->chunk_sync_period[0] = c->chunk_sync_period[1] = c->chunk_sync_period[2] = 1;
     c->wait_budget = kWaitBudgetCycles;
     c->test_drop = 0;
     c->ev_pool = new (std::nothrow) std::vector<cudaEvent_t>();
@@ -479,6 +513,15 @@ size_t unity_workspace_bytes(int64_t n_tok, int32_t H, int32_t V, int32_t K, int
     if (n_tok < 0 || H <= 0 || V <= 0 || K <= 0 || n_inv < 0) return 0;
     return carve(nullptr, ~size_t(0), n_tok, H, V, K, n_inv, wanted_chunk_rows(n_tok, K, kDefaultChunkMult),
                  wanted_chunk_vocab(V, kDefaultChunkMult), nullptr).bytes;
+}
+
+size_t unity_advantage_workspace_bytes(int32_t n_inv, int32_t n_groups, int32_t n_roles) {
+    if (n_inv < 0 || n_groups < 1 || n_roles < 1) return 0;
+    Bump b{nullptr, 0, ~size_t(0), true};
+    b.take<float>(static_cast<size_t>(n_inv) + 4);
+    b.take<int>(static_cast<size_t>(n_inv) + 4);
+    b.take<char>(advantage_table_bytes(static_cast<long long>(n_groups) * n_roles));
+    return up(b.off, kAlign);
 }
 
 size_t unity_workspace_hint(int64_t n_tok, int32_t H, int32_t V, int32_t K) {
@@ -555,6 +598,10 @@ int unity_set_option(unity_ctx* ctx, int option, int value) {
         return UNITY_OK;
     }
     if (option == UNITY_OPT_WIDE_ACC && (value == 0 || value == 1)) { ctx->wide_acc = value; return UNITY_OK; }
+    if (option >= UNITY_OPT_SYNC_PERIOD_GRAD && option <= UNITY_OPT_SYNC_PERIOD_DW && value >= 1 && value <= 1024) {
+        ctx->chunk_sync_period[option - UNITY_OPT_SYNC_PERIOD_GRAD] = value;
+        return UNITY_OK;
+    }
     if (option == UNITY_OPT_WAIT_KCYCLES && value >= 1) {
         ctx->wait_budget = static_cast<long long>(value) * 1000;
         if (ctx->wait_budget > 1000000) ctx->test_drop = 0;      // the test hook lives only under a short bound
@@ -617,12 +664,9 @@ int unity_role_advantage(unity_ctx* ctx, int32_t n_inv, int32_t n_traj, int32_t 
     memset(&a, 0, sizeof(a));
     a.r_scratch = b.take<float>(n_inv + 4);
     a.seg_scratch = b.take<int>(n_inv + 4);
-    const size_t n_seg = static_cast<size_t>(n_groups) * n_roles;
-    a.seg_lo = b.take<int>(n_seg);
-    a.seg_hi = b.take<int>(n_seg);
-    if (!b.ok) return fail(ctx, UNITY_ERR_WORKSPACE, "workspace too small: need %zu bytes", b.off);
-    CUDA_TRY(ctx, cudaMemsetAsync(a.seg_lo, 0x7f, sizeof(int) * n_seg, ctx->stream));   // 0x7f7f7f7f: above any index
-    CUDA_TRY(ctx, cudaMemsetAsync(a.seg_hi, 0xff, sizeof(int) * n_seg, ctx->stream));   // -1
+    a.seg_table = b.take<char>(advantage_table_bytes(static_cast<long long>(n_groups) * n_roles));
+    if (!b.ok)
+        return fail(ctx, UNITY_ERR_WORKSPACE, "workspace too small: stage 1 needs %zu bytes (unity_advantage_workspace_bytes)", b.off);
     a.n_inv = n_inv; a.n_traj = n_traj; a.n_roles = n_roles; a.n_groups = n_groups;
     a.inv_role = inv_role; a.inv_group = inv_group; a.inv_traj = inv_traj;
     a.r_node = r_node; a.r_turn = r_turn; a.r_traj = r_traj;
@@ -828,7 +872,7 @@ int unity_logprob_fwd(unity_ctx* ctx, const unity_rows* rows, float* logp, float
     rc = forward_sweep(ctx, rows, P);
     if (rc) return rc;
     TokenArgs t;
-    fill_token_args(t, rows, P);
+    fill_token_args(t, ctx, rows, P);
     t.logp = logp; t.entropy = entropy; t.lse = lse;
     int nl = 0;
     CUDA_TRY(ctx, launch_finish_forward(t, false, st, &nl));
@@ -905,7 +949,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
     int nl = 0;
 
     TokenArgs t;
-    fill_token_args(t, rows, P);
+    fill_token_args(t, ctx, rows, P);
     t.logp = logp; t.entropy = entropy; t.lse = nullptr;
     if (have_fwd) { t.logp_in = params->logp_in; t.entropy_in = params->entropy_in; t.lse_in = params->lse_in; }
     t.old_logp = old_logp; t.ref_logp = ref_logp; t.adv_tok = adv_tok;
@@ -933,12 +977,14 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
     const int n_workers = ctx->sm_count / 2;
     auto pick_wide = [&](int cls, int m_tiles) {
         if (!ctx->wide_acc || ctx->ctas[cls] != 2) return false;
-        auto useful = [&](int cols) {
+        const int mma_n = gemm_mma_n(H);
+        auto useful = [&](int blocks) {
+            const int cols = blocks * mma_n;
             const long long nt = (H + cols - 1) / cols, tiles = nt * m_tiles;
             const long long waves = (tiles + n_workers - 1) / n_workers;
             return (static_cast<double>(H) / (nt * cols)) * (static_cast<double>(tiles) / (waves * n_workers));
         };
-        return m_tiles <= 0 || 1.04 * useful(2 * kTileN) >= useful(kTileN);
+        return m_tiles <= 0 || 1.04 * useful(2) >= useful(1);
     };
     const int c_grad = ctx->ctas[UNITY_PROF_GRAD_GEMM], c_dh = ctx->ctas[UNITY_PROF_DH_GEMM],
               c_dw = ctx->ctas[UNITY_PROF_DW_GEMM];
@@ -962,12 +1008,12 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
             if (stash) {
                 // forward over this block of rows, keeping its logits; then the per-row loss terms of the block
                 const ZStash z{L.G, cv, static_cast<long long>(cr) * cv, z_base, z_chunks};
-                int splits = 1;
-                if ((rc = launch_forward(ctx, rows, slot0, nc, L.stats, L.target_p, tm_hp_k, tm_W_f, &z, &splits))) return rc;
+                FwdShape fs;
+                if ((rc = launch_forward(ctx, rows, slot0, nc, L.stats, L.target_p, tm_hp_k, tm_W_f, &z, &fs))) return rc;
                 TokenArgs tc = t;
                 tc.slot_begin = slot0; tc.n_slots = slot0 + nc;
                 tc.offsets[k] = slot0; tc.offsets[k + 1] = slot0 + nc;
-                tc.stats_base[k] = 0; tc.model_splits[k] = splits;
+                set_token_stats(tc, k, 0, fs, nc, gemm_tile_rows(ctx->ctas[UNITY_PROF_FWD_GEMM]));
                 CUDA_TRY(ctx, launch_finish_rows(tc, true, st, &nl));
                 nl += 1;
             }
@@ -1022,7 +1068,10 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 GemmArgs h;
                 memset(&h, 0, sizeof(h));
                 const bool wide_dh = pick_wide(UNITY_PROF_DH_GEMM, nc / gemm_tile_rows(c_dh));
-                h.m_tiles = nc / gemm_tile_rows(c_dh); h.n_tiles = (H + gemm_tile_cols(wide_dh) - 1) / gemm_tile_cols(wide_dh);
+                const int mma_n = gemm_mma_n(H);                       // dHidden and dW both have H output columns
+                const int cols_dh = (wide_dh ? 2 : 1) * mma_n;
+                h.mma_n = mma_n;
+                h.m_tiles = nc / gemm_tile_rows(c_dh); h.n_tiles = (H + cols_dh - 1) / cols_dh;
                 h.k_iters = (vc + kTileK - 1) / kTileK;
                 h.group_m = ctx->chunk_group[1] / c_dh > 0 ? ctx->chunk_group[1] / c_dh : 1;
                 h.a_row0 = 0; h.a_k0 = 0; h.b_row0 = 0; h.b_k0 = v0; h.m_rows = nc; h.n_cols = H;
@@ -1037,7 +1086,9 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 memset(&w, 0, sizeof(w));
                 w.m_tiles = (vc + gemm_tile_rows(c_dw) - 1) / gemm_tile_rows(c_dw);
                 const bool wide_dw = pick_wide(UNITY_PROF_DW_GEMM, w.m_tiles);
-                w.n_tiles = (H + gemm_tile_cols(wide_dw) - 1) / gemm_tile_cols(wide_dw); w.k_iters = nc / kTileK;
+                const int cols_dw = (wide_dw ? 2 : 1) * mma_n;
+                w.mma_n = mma_n;
+                w.n_tiles = (H + cols_dw - 1) / cols_dw; w.k_iters = nc / kTileK;
                 w.group_m = ctx->chunk_group[2] / c_dw > 0 ? ctx->chunk_group[2] / c_dw : 1;
                 w.a_row0 = 0; w.a_k0 = 0; w.b_row0 = 0; w.b_k0 = slot0; w.m_rows = vc; w.n_cols = H;
                 w.C = dWk + static_cast<long long>(v0) * H; w.ldc = H;

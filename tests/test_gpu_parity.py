@@ -111,6 +111,85 @@ def test_advantage_variants(ddof, eps, one_group):
     ctx.close()
 
 
+def shuffled_structure(name, seed=11, **kw):
+    """A configuration's invocations in a seeded random order (rollout groups interleaved, as a buffer filled in
+    arrival order holds them); token data follows its invocation."""
+    w = wl.make_structure(name, **kw)
+    perm = torch.from_numpy(np.random.default_rng(seed).permutation(w.n_inv))
+    lens = (w.cu_seqlens[1:] - w.cu_seqlens[:-1])[perm]
+    starts = w.cu_seqlens[:-1][perm]
+    tok_src = torch.cat([torch.arange(int(a), int(a) + int(n)) for a, n in zip(starts, lens)]) if w.n_tok else None
+    for key in ("inv_role", "inv_group", "inv_traj", "r_node", "r_turn"):
+        setattr(w, key, getattr(w, key)[perm].contiguous())
+    w.cu_seqlens = torch.cat([torch.zeros(1, dtype=torch.int64), torch.cumsum(lens, 0)])
+    if tok_src is not None:
+        w.tok_mask = w.tok_mask[tok_src].contiguous()
+    return w
+
+
+@pytest.mark.parametrize("name", ["search", "stress"])
+def test_advantage_with_invocations_in_shuffled_order(name):
+    w = shuffled_structure(name)
+    assert (w.inv_group[1:] < w.inv_group[:-1]).any()              # groups really are interleaved
+    d = pu.DeviceInputs(w)
+    ctx = ub.Context(0, 1 << 22)
+    g, o = pu.gpu_advantage(ctx, w, d), pu.oracle_advantage(w)
+    for key in ("adv_inv", "adv_tok", "seg_mean", "seg_std"):
+        assert np.abs(g[key].cpu().numpy() - o[key]).max() <= pu.TOL_ADV, key
+    again = pu.gpu_advantage(ctx, w, d)                              # order-free integer sums: bitwise reproducible
+    assert all(torch.equal(g[k], again[k]) for k in g)
+    ctx.close()
+
+
+@pytest.mark.parametrize("case", ["offset", "tiny", "huge", "one_segment", "pairs"])
+def test_advantage_statistics_on_awkward_rewards(case):
+    """Rewards with a large common offset, very small and very large magnitudes, one segment holding the whole batch
+    (16384 members per role) and segments of two: the per-segment integer grid must keep the oracle's result."""
+    n_inv, R = 65536, 4
+    G = {"one_segment": 1, "pairs": n_inv // (2 * R)}.get(case, 2048)
+    rng = np.random.default_rng(3)
+    w = wl.make_structure("tiny")
+    w.n_inv, w.n_roles, w.n_groups, w.n_traj = n_inv, R, G, n_inv
+    w.inv_role = torch.from_numpy(rng.integers(0, R, n_inv).astype(np.int32))
+    w.inv_group = torch.from_numpy(rng.integers(0, G, n_inv).astype(np.int32))
+    w.inv_traj = torch.arange(n_inv, dtype=torch.int32)
+    base = rng.normal(size=n_inv).astype(np.float32)
+    r = {"offset": 1000.0 + 0.01 * base, "tiny": 1e-30 * base, "huge": 1e30 * base}.get(case, base)
+    w.r_node = torch.from_numpy(np.asarray(r, np.float32))
+    w.r_turn = torch.zeros(n_inv)
+    w.r_traj = torch.zeros(n_inv)
+    w.lam = torch.ones(R, 3)
+    w.cu_seqlens = torch.arange(n_inv + 1, dtype=torch.int64) * 2
+    w.n_tok = 2 * n_inv
+    w.tok_mask = torch.ones(w.n_tok, dtype=torch.uint8)
+    d = pu.DeviceInputs(w)
+    ctx = ub.Context(0, ub.unity_advantage_workspace_bytes(n_inv, G, R))
+    eps = 0.0 if case in ("tiny", "huge") else 1e-6          # eps = 1e-6 would swamp a sigma of 1e-30
+    g, o = pu.gpu_advantage(ctx, w, d, eps=eps), pu.oracle_advantage(w, eps=eps)
+    assert np.abs(g["adv_inv"].cpu().numpy() - o["adv_inv"]).max() <= pu.TOL_ADV
+    assert np.abs(g["adv_tok"].cpu().numpy() - o["adv_tok"]).max() <= pu.TOL_ADV
+    scale = max(1.0, float(np.abs(o["seg_mean"]).max()))
+    assert np.abs(g["seg_mean"].cpu().numpy() - o["seg_mean"]).max() <= 1e-6 * scale
+    assert np.abs(g["seg_std"].cpu().numpy() - o["seg_std"]).max() <= 1e-6 * max(1e-30, float(o["seg_std"].max()))
+    ctx.close()
+
+
+def test_advantage_workspace_query_and_too_small_workspace():
+    w = wl.make_structure("stress")
+    d = pu.DeviceInputs(w)
+    need = ub.unity_advantage_workspace_bytes(w.n_inv, w.n_groups, w.n_roles)
+    assert 8 * w.n_inv + 32 * w.n_groups * w.n_roles <= need <= 8 * w.n_inv + 32 * w.n_groups * w.n_roles + 1024
+    ctx = ub.Context(0, need)
+    g, o = pu.gpu_advantage(ctx, w, d), pu.oracle_advantage(w)
+    assert np.abs(g["adv_tok"].cpu().numpy() - o["adv_tok"]).max() <= pu.TOL_ADV
+    ctx.close()
+    ctx = ub.Context(0, need - 512)
+    with pytest.raises(ub.UnityError) as e:
+        pu.gpu_advantage(ctx, w, d)
+    assert e.value.code == -4 and "unity_advantage_workspace_bytes" in str(e.value)
+    ctx.close()
+
+
 def test_advantage_null_inputs_unaligned_views_and_empty_batch():
     import oracle.unity_oracle as orc
     w = wl.make_structure("rag_qa")
