@@ -225,6 +225,11 @@ def measure_streaming():
     role_s, group_s, r_s = inv_role[perm].contiguous(), inv_group[perm].contiguous(), r_node[perm].contiguous()
     t_adv_shuf = timed(lambda: ctx.role_advantage(n_inv, R, G, role_s, group_s, inv_traj, r_s, None, None, None, 1e-6,
                                                   0, cu, mask, adv_inv, adv_tok))
+    # the statistics passes alone (same invocations, no tokens): what remains of the call is the token broadcast
+    cu0 = torch.zeros(n_inv + 1, dtype=torch.int64, device=dev)
+    none_tok = torch.empty(0, device=dev)
+    t_adv_stats = timed(lambda: ctx.role_advantage(n_inv, R, G, inv_role, inv_group, inv_traj, r_node, None, None, None,
+                                                   1e-6, 0, cu0, None, adv_inv, none_tok))
     # reference for the write-only streams: a plain device fill of the same output
     t_fill = timed(lambda: adv_tok.zero_())
     t_gae = timed(lambda: ctx.gae(cu, rewards, values, mask, 0.99, 0.95, a_out, r_out))
@@ -267,7 +272,9 @@ def measure_streaming():
     done_us.sort()
     out = {"mode": "micro", "tokens": n, "invocations": n_inv, "peak_hbm_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"],
            "role_advantage": {"ms": t_adv, "algorithmic_bytes": 5 * n + 28 * n_inv, "gbs": (5 * n + 28 * n_inv) / t_adv / 1e6,
-                              "ms_shuffled_invocations": t_adv_shuf},
+                              "ms_shuffled_invocations": t_adv_shuf, "ms_statistics_passes_alone": t_adv_stats,
+                              "broadcast_gbs": 5 * n / max(t_adv - t_adv_stats, 1e-6) / 1e6,
+                              "broadcast_frac": 5 * n / max(t_adv - t_adv_stats, 1e-6) / 1e6 / peaks["hbm_gbs"]},
            "device_fill_f32": {"ms": t_fill, "algorithmic_bytes": 4 * n, "gbs": 4 * n / t_fill / 1e6,
                                "note": "torch fill of the 256 MiB token vector: what a write-only stream reaches here"},
            "gae": {"ms": t_gae, "algorithmic_bytes": 17 * n, "gbs": 17 * n / t_gae / 1e6},

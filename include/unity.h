@@ -93,7 +93,7 @@ int unity_set_profiling(unity_ctx* ctx, int enable);
 #define UNITY_OPT_CTAS_DH 2
 #define UNITY_OPT_CTAS_DW 3
 #define UNITY_OPT_L2_PROMOTION 4  /* TMA tensor-map L2 promotion: 0 none, 1 64 B, 2 128 B, 3 256 B (default)          */
-#define UNITY_OPT_CHUNK_GROUP 5   /* raster group of all three gradient-chunk GEMMs in 128-row tiles (default 32)       */
+#define UNITY_OPT_CHUNK_GROUP 5   /* raster group of all three gradient-chunk GEMMs in 128-row tiles (defaults 40, 32, 32)       */
 #define UNITY_OPT_CHUNK_ROWS 6    /* gradient chunk rows = value x 18944 (default 2; larger needs a larger workspace)   */
 #define UNITY_OPT_CHUNK_VOCAB 7   /* gradient chunk vocabulary entries = value x 18944 (default 2)                      */
 #define UNITY_OPT_FWD_GROUP 8     /* 128-row tiles per round of the forward kernel (default 48; 0 = a quarter of the SMs) */
@@ -150,7 +150,7 @@ int unity_get_profile(unity_ctx* ctx, double* ms, int64_t* launches);
  * whatever the order.  Sums are taken exactly on a per-segment integer grid with integer atomics, so the result
  * does not depend on scheduling (bitwise reproducible; no floating-point atomics), and a segment whose rewards
  * are all equal gets exactly 0.
- * Workspace: unity_advantage_workspace_bytes(n_inv, n_groups, n_roles) = 8 bytes per invocation + 32 bytes per
+ * Workspace: unity_advantage_workspace_bytes(n_inv, n_groups, n_roles), about 8 bytes per invocation + 32 bytes per
  * (group, role) segment; n_groups*n_roles <= 2^24.
  */
 typedef struct {
@@ -295,7 +295,7 @@ int unity_align_rewards(unity_ctx* ctx, int32_t n_inv, int64_t n_tok, const int6
  *                         group or trajectory id was out of range and its invocation was left out
  *   err, err_len        : optional HOST buffer that receives a one-line reason when the return is not 0
  *   every other argument: exactly as in unity_role_advantage
- * Cost: each GPU that loads the library holds the array (256 B + 8 B * UNITY_NOALLOC_MAX_INV + 32 B *
+ * Cost: each GPU that loads the library holds the array (512 B + 8 B * UNITY_NOALLOC_MAX_INV + 32 B *
  * UNITY_NOALLOC_MAX_SEG, about 2.5 MiB) until the process exits.  The first call on a device looks the array's
  * address up (cudaGetSymbolAddress) and may make the CUDA runtime load this library's device code, which is the
  * runtime's own one-time allocation: make that first call outside any stream capture, and count on "no

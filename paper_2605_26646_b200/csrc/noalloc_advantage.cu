@@ -18,10 +18,11 @@ namespace {
 constexpr int kMaxDevices = 64;
 constexpr size_t kStatusBytes = 256;
 constexpr size_t kInvBytes = 2 * sizeof(float) * UNITY_NOALLOC_MAX_INV;
-constexpr size_t kScratchBytes = kStatusBytes + kInvBytes + 32 * static_cast<size_t>(UNITY_NOALLOC_MAX_SEG);
+constexpr size_t kTableBytes = 256 + 32 * static_cast<size_t>(UNITY_NOALLOC_MAX_SEG);   // advantage_table_bytes(MAX_SEG)
+constexpr size_t kScratchBytes = kStatusBytes + kInvBytes + kTableBytes;
 
 // [0, 256): status word (bit set when an id in the data is out of range); then r[MAX_INV]; then seg[MAX_INV]; then
-// the per-segment accumulators (32 bytes each) of up to MAX_SEG segments.
+// the table of the statistics passes (a 256-byte header and 32 bytes of accumulators per segment, up to MAX_SEG).
 static __device__ __align__(256) unsigned char g_adv_scratch[kScratchBytes];
 
 std::mutex g_mu;
@@ -90,6 +91,7 @@ extern "C" int unity_role_advantage_noalloc(int device, void* cuda_stream, int32
     a.r_scratch = reinterpret_cast<float*>(base + kStatusBytes);
     a.seg_scratch = reinterpret_cast<int*>(base + kStatusBytes + sizeof(float) * UNITY_NOALLOC_MAX_INV);
     a.seg_table = base + kStatusBytes + kInvBytes;
+    if (advantage_table_bytes(UNITY_NOALLOC_MAX_SEG) > kTableBytes) { say(err, err_len, "internal: static table too small"); return UNITY_ERR_CUDA; }
     a.n_inv = n_inv; a.n_traj = n_traj; a.n_roles = n_roles; a.n_groups = n_groups;
     a.inv_role = inv_role; a.inv_group = inv_group; a.inv_traj = inv_traj;
     a.r_node = r_node; a.r_turn = r_turn; a.r_traj = r_traj;

@@ -38,28 +38,31 @@ __device__ __forceinline__ int find_invocation(const int64_t* __restrict__ cu, i
 // batch (buffers fill in arrival order), so nothing here sweeps index ranges: every pass is one thread per invocation
 // plus integer atomics on a per-segment table.  Integer addition is associative, so the result does not depend on the
 // order in which the atomics land: the statistics are exact on the segment's grid and bitwise reproducible.
-//   pass 1 (k_adv_combine): r_s, segment id; per segment the member count and max |r|
-//   pass 2 (k_adv_sum)    : q_s = r_s on the segment's integer grid; per segment sum q
-//   pass 3 (k_adv_m2)     : e_s = n q_s - sum q (n times the deviation from the mean, an exact integer; zero for every
-//                           member of a segment whose rewards are all equal); per segment sum e^2 in 128 bits
-//   pass 4 (k_adv_finish) : mean, sigma, advantages
+//   pass 1 : r_s, segment id; per segment the member count n and max |r|
+//   pass 2 : q_s = r_s on the segment's integer grid; per segment S = sum q (64 bits) and Q = sum q^2 (128 bits)
+//   pass 3 : n Q - S^2 = n * sum (q - S/n)^2 exactly, in 128-bit integers (no rounding, hence none of the cancellation
+//            that makes E[r^2] - mean^2 unusable in floating point; 0 for a segment whose rewards are all equal);
+//            mean, sigma and the advantages (n q_s - S) / (n (sigma + eps)) follow in fp64 and are rounded to fp32
 // Grid of a segment with n <= 2^L members and max |r| < 2^(E+1): multiples of 2^-shift, shift = B - (E + 1), with
-// B = min(61 - L, (125 - 3 L) / 2) bits per value, so that sum q stays below 2^62 and sum e^2 below 2^127.  For
-// segments of up to 64 members that is 53 or more bits (every fp32 reward within 2^29 of the largest is exact).
+// B = min(61 - L, (125 - 3 L) / 2) bits per value, so that S stays below 2^62 and n Q below 2^127.  For segments of
+// up to 64 members that is 53 or more bits (every fp32 reward within 2^29 of the largest is exact).
+// The three passes run as ONE cooperative launch with a bounded grid barrier between them (all blocks are resident by
+// construction of the launch); a device without cooperative launch gets three launches of the same code.
 struct SegTable {
     int* cnt;
     unsigned* maxbits;
     long long* sum;
-    unsigned long long *m2lo, *m2hi;
+    unsigned long long *sqlo, *sqhi;
 };
+constexpr size_t kSegHeaderBytes = 256;     // the table starts with the barrier counter of the fused launch
 __device__ __forceinline__ SegTable seg_table(const AdvArgs& a) {
     const size_t n = static_cast<size_t>(a.n_groups) * a.n_roles;
     SegTable t;
-    t.cnt = reinterpret_cast<int*>(a.seg_table);
+    t.cnt = reinterpret_cast<int*>(static_cast<char*>(a.seg_table) + kSegHeaderBytes);
     t.maxbits = reinterpret_cast<unsigned*>(t.cnt + n);
     t.sum = reinterpret_cast<long long*>(t.maxbits + n);
-    t.m2lo = reinterpret_cast<unsigned long long*>(t.sum + n);
-    t.m2hi = t.m2lo + n;
+    t.sqlo = reinterpret_cast<unsigned long long*>(t.sum + n);
+    t.sqhi = t.sqlo + n;
     return t;
 }
 __device__ __forceinline__ int seg_shift(unsigned maxbits, int cnt) {
@@ -72,9 +75,7 @@ __device__ __forceinline__ long long seg_quantise(float r, int shift) {
     return __double2ll_rn(ldexp(static_cast<double>(r), shift));
 }
 
-__global__ void k_adv_combine(AdvArgs a) {
-    const int s = blockIdx.x * blockDim.x + threadIdx.x;
-    if (s >= a.n_inv) return;
+__device__ __forceinline__ void adv_pass_combine(const AdvArgs& a, int s) {
     const int v = a.inv_role[s], g = a.inv_group[s];
     bool ok = (v >= 0 && v < a.n_roles && g >= 0 && g < a.n_groups);
     float rj = 0.f;
@@ -102,42 +103,26 @@ __global__ void k_adv_combine(AdvArgs a) {
     a.seg_scratch[s] = seg;
 }
 
-__global__ void k_adv_sum(AdvArgs a) {
-    const int s = blockIdx.x * blockDim.x + threadIdx.x;
-    if (s >= a.n_inv) return;
+__device__ __forceinline__ void adv_pass_sums(const AdvArgs& a, int s) {
     const int seg = a.seg_scratch[s];
     if (seg < 0) return;
     const SegTable t = seg_table(a);
     const unsigned mb = t.maxbits[seg];
     if (mb == 0u) return;                                        // every reward of the segment is zero
     const long long q = seg_quantise(a.r_scratch[s], seg_shift(mb, t.cnt[seg]));
+    if (q == 0) return;
     atomicAdd(reinterpret_cast<unsigned long long*>(&t.sum[seg]), static_cast<unsigned long long>(q));
-}
-
-__global__ void k_adv_m2(AdvArgs a) {
-    const int s = blockIdx.x * blockDim.x + threadIdx.x;
-    if (s >= a.n_inv) return;
-    const int seg = a.seg_scratch[s];
-    if (seg < 0) return;
-    const SegTable t = seg_table(a);
-    const unsigned mb = t.maxbits[seg];
-    if (mb == 0u) return;
-    const int cnt = t.cnt[seg];
-    const long long q = seg_quantise(a.r_scratch[s], seg_shift(mb, cnt));
-    const long long e = static_cast<long long>(cnt) * q - t.sum[seg];
-    if (e == 0) return;
-    const unsigned long long m = static_cast<unsigned long long>(e < 0 ? -e : e);
+    const unsigned long long m = static_cast<unsigned long long>(q < 0 ? -q : q);
     const unsigned long long lo = m * m, hi = __umul64hi(m, m);
     // 128-bit accumulation with two 64-bit atomics: the low word's wrap-arounds are carried into the high word by
     // whoever caused them, so the final pair is the exact sum whatever the order
-    const unsigned long long old = atomicAdd(&t.m2lo[seg], lo);
+    const unsigned long long old = atomicAdd(&t.sqlo[seg], lo);
     const unsigned long long carry = (old + lo < old) ? 1ull : 0ull;
-    if (hi + carry != 0ull) atomicAdd(&t.m2hi[seg], hi + carry);
+    if (hi + carry != 0ull) atomicAdd(&t.sqhi[seg], hi + carry);
 }
 
-// Thread i finishes invocation i (advantage) and segment i (mean and sigma for the caller).
-__global__ void k_adv_finish(AdvArgs a) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+// Index i finishes invocation i (advantage) and segment i (mean and sigma for the caller).
+__device__ __forceinline__ void adv_pass_finish(const AdvArgs& a, int i) {
     const int n_seg = a.n_groups * a.n_roles;
     const SegTable t = seg_table(a);
     auto stats = [&](int seg, double& mean, double& sigma, double& unit, int& cnt, int& shift) {
@@ -146,12 +131,18 @@ __global__ void k_adv_finish(AdvArgs a) {
         mean = 0.0; sigma = 0.0; unit = 0.0; shift = 0;
         if (cnt == 0 || mb == 0u) return;
         shift = seg_shift(mb, cnt);
-        unit = ldexp(1.0 / static_cast<double>(cnt), -shift);            // value of one step of e = n q - sum q
-        mean = static_cast<double>(t.sum[seg]) * unit;
+        unit = ldexp(1.0 / static_cast<double>(cnt), -shift);            // value of one step of n q - S
+        const long long S = t.sum[seg];
+        mean = static_cast<double>(S) * unit;
         const int dof = cnt - a.ddof;
         if (dof > 0) {
-            const double m2 = (ldexp(static_cast<double>(t.m2hi[seg]), 64) + static_cast<double>(t.m2lo[seg])) * unit * unit;
-            sigma = sqrt(m2 / static_cast<double>(dof));
+            const unsigned __int128 Q = (static_cast<unsigned __int128>(t.sqhi[seg]) << 64) | t.sqlo[seg];
+            const unsigned long long absS = static_cast<unsigned long long>(S < 0 ? -S : S);
+            const unsigned __int128 d = Q * static_cast<unsigned>(cnt) - static_cast<unsigned __int128>(absS) * absS;   // n Q - S^2 >= 0
+            const double dd = ldexp(static_cast<double>(static_cast<unsigned long long>(d >> 64)), 64) +
+                              static_cast<double>(static_cast<unsigned long long>(d));
+            // sum (r - mean)^2 = (n Q - S^2) / n in grid units^2 = (n Q - S^2) * n * unit^2
+            sigma = sqrt(dd * static_cast<double>(cnt) * unit * unit / static_cast<double>(dof));
         }
     };
     double mean, sigma, unit;
@@ -174,6 +165,39 @@ __global__ void k_adv_finish(AdvArgs a) {
         }
         a.adv_inv[i] = adv;
     }
+}
+
+// All blocks of a cooperative launch meet: counter reaches `target`.  Bounded: on expiry the timeout status is set and
+// the block goes on (the call's results are then undefined, the host sees UNITY_ERR_TIMEOUT).
+__device__ __forceinline__ void adv_grid_barrier(const AdvArgs& a, unsigned target) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned* counter = reinterpret_cast<unsigned*>(a.seg_table);
+        __threadfence();
+        atomicAdd(counter, 1u);
+        const long long t0 = clock64();
+        bool ok = true;
+        while (*reinterpret_cast<volatile unsigned*>(counter) < target) {
+            if (clock64() - t0 > 2000000000LL) { ok = false; break; }
+        }
+        if (!ok) atomicOr(a.status, kStatusTimeout);
+        __threadfence();
+    }
+    __syncthreads();
+}
+
+// phase 0: all three passes with grid barriers (cooperative launch); 1, 2, 3: one pass (plain launches)
+__global__ void k_adv_stats(AdvArgs a, int phase) {
+    const int n_fin = max(a.n_inv, a.n_groups * a.n_roles);
+    const int stride = gridDim.x * blockDim.x, first = blockIdx.x * blockDim.x + threadIdx.x;
+    if (phase == 0 || phase == 1)
+        for (int s = first; s < a.n_inv; s += stride) adv_pass_combine(a, s);
+    if (phase == 0) adv_grid_barrier(a, gridDim.x);
+    if (phase == 0 || phase == 2)
+        for (int s = first; s < a.n_inv; s += stride) adv_pass_sums(a, s);
+    if (phase == 0) adv_grid_barrier(a, 2u * gridDim.x);
+    if (phase == 0 || phase == 3)
+        for (int i = first; i < n_fin; i += stride) adv_pass_finish(a, i);
 }
 
 // A block broadcasts rounds x 1024 tokens; in a round each thread handles four consecutive tokens (one 32-bit mask
@@ -866,23 +890,46 @@ __global__ void k_value_class(ValueArgs a) {
 // ------------------------------------------------------------------------------------------------
 // launchers
 // ------------------------------------------------------------------------------------------------
-size_t advantage_table_bytes(long long n_seg) { return static_cast<size_t>(n_seg) * 32; }
+size_t advantage_table_bytes(long long n_seg) { return kSegHeaderBytes + static_cast<size_t>(n_seg) * 32; }
 
 cudaError_t launch_advantage(const AdvArgs& a, cudaStream_t stream, int* n_launches) {
     const int n_seg = a.n_groups * a.n_roles;
     if (a.n_inv > 0 || a.seg_mean || a.seg_std) {
         cudaError_t e = cudaMemsetAsync(a.seg_table, 0, advantage_table_bytes(n_seg), stream);
         if (e != cudaSuccess) return e;
-        const int blocks = (a.n_inv + 255) / 256;
-        if (blocks > 0) {
-            k_adv_combine<<<blocks, 256, 0, stream>>>(a);
-            k_adv_sum<<<blocks, 256, 0, stream>>>(a);
-            k_adv_m2<<<blocks, 256, 0, stream>>>(a);
+        const int n_fin = a.n_inv > n_seg ? a.n_inv : n_seg;
+        const int want = (n_fin + 255) / 256;
+        // blocks of k_adv_stats that fit the current device at once (0: no cooperative launch), looked up once per device
+        static int resident_cache[64];
+        static bool resident_known[64];
+        int dev = 0;
+        if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+        int resident = 0;
+        if (dev >= 0 && dev < 64 && resident_known[dev]) {
+            resident = resident_cache[dev];
+        } else {
+            int coop = 0, sms = 0, per_sm = 0;
+            cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+            if (coop && cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_adv_stats, 256, 0) == cudaSuccess)
+                resident = sms * per_sm;
+            cudaGetLastError();
+            if (dev >= 0 && dev < 64) { resident_cache[dev] = resident; resident_known[dev] = true; }
+        }
+        if (resident > 0) {
+            // one cooperative launch: every block resident, so the grid barriers between the passes cannot starve
+            int phase = 0;
+            AdvArgs args = a;
+            void* params[2] = {&args, &phase};
+            e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(k_adv_stats), dim3(want < resident ? want : resident), dim3(256),
+                                            params, 0, stream);
+            if (e != cudaSuccess) return e;
+            *n_launches += 1;
+        } else {
+            cudaGetLastError();
+            for (int phase = 1; phase <= 3; ++phase) k_adv_stats<<<want, 256, 0, stream>>>(a, phase);
             *n_launches += 3;
         }
-        const int n_fin = a.n_inv > n_seg ? a.n_inv : n_seg;
-        k_adv_finish<<<(n_fin + 255) / 256, 256, 0, stream>>>(a);
-        *n_launches += 1;
     }
     const bool aligned = (reinterpret_cast<uintptr_t>(a.tok_mask) & 15) == 0 && (reinterpret_cast<uintptr_t>(a.adv_tok) & 15) == 0;
     if (a.n_tok > 0 && aligned && a.n_tok / a.n_inv >= 128 && a.n_inv >= 1024) {

@@ -178,7 +178,7 @@ def test_advantage_workspace_query_and_too_small_workspace():
     w = wl.make_structure("stress")
     d = pu.DeviceInputs(w)
     need = ub.unity_advantage_workspace_bytes(w.n_inv, w.n_groups, w.n_roles)
-    assert 8 * w.n_inv + 32 * w.n_groups * w.n_roles <= need <= 8 * w.n_inv + 32 * w.n_groups * w.n_roles + 1024
+    assert 8 * w.n_inv + 32 * w.n_groups * w.n_roles <= need <= 8 * w.n_inv + 32 * w.n_groups * w.n_roles + 2048
     ctx = ub.Context(0, need)
     g, o = pu.gpu_advantage(ctx, w, d), pu.oracle_advantage(w)
     assert np.abs(g["adv_tok"].cpu().numpy() - o["adv_tok"]).max() <= pu.TOL_ADV
