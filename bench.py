@@ -32,8 +32,8 @@ UNIT = "tokens/s"
 # (valid rows x vocabulary columns).  Traffic grows in proportion to the logits covered (same chunk and group sizes),
 # so a full-size launch is estimated as bytes_per_logit x its logits.  Valid only for the kernel source it was taken
 # from: when the hash of gemm_tcgen05.cu differs, the benchmark reports null.
-NCU_TRAFFIC = {"source_sha256_16": "058d184633b06d97",
-               "bytes_per_logit": {"fwd_gemm": 1.802, "grad_gemm": 6.540, "dh_gemm": 6.351, "dw_gemm": 6.344}}
+NCU_TRAFFIC = {"source_sha256_16": "15538ac9efb39bde",
+               "bytes_per_logit": {"fwd_gemm": 1.959, "grad_gemm": 3.942, "dh_gemm": 6.354, "dw_gemm": 6.352}}
 
 
 def ncu_traffic_per_launch(cls: str, logits_per_launch: float):

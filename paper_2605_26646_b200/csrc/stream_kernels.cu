@@ -804,10 +804,14 @@ __global__ void k_value_norm(ValueArgs a) {
     __shared__ float sh[32];
     const int k = blockIdx.x;
     float cnt = 0.f;
+    // branch-free body, eight invocations per step: the loads of a step are independent and issue together (a thread
+    // still adds its values in index order)
+#pragma unroll 8
     for (int s = threadIdx.x; s < a.n_inv; s += 1024) {
         const int role = a.inv_role[s];
-        if (role < 0 || role >= a.n_roles || a.role_model[role] != k) continue;
-        cnt += a.inv_sums[s * 3 + 0];
+        const float c = a.inv_sums[s * 3 + 0];
+        const bool mine = role >= 0 && role < a.n_roles && a.role_model[role] == k;
+        cnt += mine ? c : 0.f;
     }
     cnt = block_sum_1024(cnt, sh);
     if (threadIdx.x == 0) {
@@ -873,10 +877,13 @@ __global__ void k_value_class(ValueArgs a) {
     __shared__ float sh[32];
     const int k = blockIdx.x;
     float sum = 0.f, clp = 0.f;
+#pragma unroll 8
     for (int s = threadIdx.x; s < a.n_inv; s += 1024) {
         const int role = a.inv_role[s];
-        if (role < 0 || role >= a.n_roles || a.role_model[role] != k) continue;
-        sum += a.inv_sums[s * 3 + 1]; clp += a.inv_sums[s * 3 + 2];
+        const float l = a.inv_sums[s * 3 + 1], c = a.inv_sums[s * 3 + 2];
+        const bool mine = role >= 0 && role < a.n_roles && a.role_model[role] == k;
+        sum += mine ? l : 0.f;
+        clp += mine ? c : 0.f;
     }
     sum = block_sum_1024(sum, sh);
     clp = block_sum_1024(clp, sh);
