@@ -391,6 +391,40 @@ def test_single_cta_and_cta_pair_kernels(ctas):
     run_all_stages(wl.make("tiny", device="cuda"), ctas=ctas)
 
 
+def test_scheduling_options_do_not_change_results():
+    """Raster groups, rendezvous switches and periods, L2 hints and tensor-map promotion only move work in time or
+    space: every output must be bitwise what the defaults give.  The forward round size changes the number of
+    vocabulary splits and with it the order of a four-term merge: equal within rounding."""
+    w = small_workload(320, 4096 + 264, 900)
+    d = pu.DeviceInputs(w)
+    ol = pu.oracle_logprob(w)
+    cur = torch.from_numpy(ol["logp"].astype(np.float32))
+    old, ref = (cur + w.noise_old).cuda(), (cur + w.noise_ref).cuda()
+    adv = wl.normal(3, 97, w.n_tok).cuda()
+
+    def run(options):
+        ctx = pu.make_ctx(w)
+        for option, value in options:
+            ctx.set_option(option, value)
+        out = pu.gpu_ppo(ctx, w, d, old, ref, adv, ent_coef=0.01)
+        ctx.close()
+        return out
+
+    base = run([])
+    same = [[(4, 0)], [(5, 8)], [(9, 0)], [(10, 0)], [(10, 5)], [(12, 4), (13, 6), (14, 2)], [(16, 0), (17, 0)],
+            [(17, 41), (18, 9), (19, 38)], [(22, 3), (23, 2), (24, 5)]]
+    for options in same:
+        out = run(options)
+        for key in ("loss", "logp", "entropy", "tok_loss", "dHidden", "metrics"):
+            assert torch.equal(out[key], base[key]), (options, key)
+        assert all(torch.equal(a, b) for a, b in zip(out["dW"], base["dW"])), options
+    out = run([(8, 16)])
+    assert (out["logp"] - base["logp"]).abs().max().item() <= 1e-5
+    assert pu.rel_fro(out["dHidden"].float().cpu().numpy(), base["dHidden"].float().cpu().numpy()) <= 1e-3
+    for a, b in zip(out["dW"], base["dW"]):
+        assert pu.rel_fro(a.cpu().numpy(), b.cpu().numpy()) <= 1e-4
+
+
 @pytest.mark.parametrize("wide", [0, 1])
 def test_accumulate_gemms_with_256_and_512_column_tiles(wide):
     # the dHidden / dW chunk GEMMs of CTA pairs exist with 256 x 256 tiles (two accumulator stages) and with
