@@ -15,11 +15,13 @@
 //   warps 2..5  : epilogue      - each thread owns one accumulator row (one TMEM lane), drains it 32 columns at a
 //                                 time with tcgen05.ld while the MMAs already fill the other stage
 //
-// The fp32-accumulate epilogue also exists with 512-column tiles (template parameter NB = 2, CTA pairs only): two
-// N = 256 MMAs per K step fill all of tensor memory as ONE accumulator stage, so a K slab of A is loaded once for
+// The fp32-accumulate epilogue also exists with tiles two MMA blocks wide (template parameter NB = 2, CTA pairs
+// only): two MMAs per K step fill all of tensor memory as ONE accumulator stage, so a K slab of A is loaded once for
 // twice the columns (a quarter less operand traffic from L2 and DRAM).  The epilogue then does not overlap the next
 // tile's MMAs, which is affordable only because these GEMMs contract over a whole gradient chunk (hundreds of K
-// slabs per tile); it adds into C with fire-and-forget vector reductions instead of load-add-store.
+// slabs per tile); it adds into C with fire-and-forget vector reductions instead of load-add-store.  The block width of
+// this epilogue is a run-time value (GemmArgs::mma_n, a multiple of 32 up to 256): an output of 896 columns runs as
+// blocks of 224 instead of padding a fourth block of 256 with zeros.
 //
 // Three epilogues share the main loop:
 //   softmax statistics : running (max, sum exp, sum exp*z, target logit) per row across a sweep of vocabulary
@@ -115,7 +117,7 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
     using C = Cfg<CTAS, NB>;
     constexpr int kStages = C::kStages, kStageBytes = C::kStageBytes, kABytes = C::kABytes, kBBytes = C::kBBytes;
     constexpr int kAccStages = C::kAccStages, kTileCols = C::kTileCols;
-    static_assert(NB == 1 || (EPI == kEpiAccumF32 && CTAS == 2), "512-column tiles: fp32-accumulate epilogue, CTA pairs");
+    static_assert(NB == 1 || (EPI == kEpiAccumF32 && CTAS == 2), "two-block tiles: fp32-accumulate epilogue, CTA pairs");
     extern __shared__ uint8_t smem_raw[];
     // the dynamic shared-memory window starts at the same offset in both CTAs of a pair, so all offsets below match
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));

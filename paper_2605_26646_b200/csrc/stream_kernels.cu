@@ -107,9 +107,10 @@ __device__ __forceinline__ void adv_pass_sums(const AdvArgs& a, int s) {
     const int seg = a.seg_scratch[s];
     if (seg < 0) return;
     const SegTable t = seg_table(a);
-    const unsigned mb = t.maxbits[seg];
+    // (the table is written by atomics of other blocks in the pass before: read it from L2, not through L1)
+    const unsigned mb = __ldcg(&t.maxbits[seg]);
     if (mb == 0u) return;                                        // every reward of the segment is zero
-    const long long q = seg_quantise(a.r_scratch[s], seg_shift(mb, t.cnt[seg]));
+    const long long q = seg_quantise(a.r_scratch[s], seg_shift(mb, __ldcg(&t.cnt[seg])));
     if (q == 0) return;
     atomicAdd(reinterpret_cast<unsigned long long*>(&t.sum[seg]), static_cast<unsigned long long>(q));
     const unsigned long long m = static_cast<unsigned long long>(q < 0 ? -q : q);
@@ -126,17 +127,17 @@ __device__ __forceinline__ void adv_pass_finish(const AdvArgs& a, int i) {
     const int n_seg = a.n_groups * a.n_roles;
     const SegTable t = seg_table(a);
     auto stats = [&](int seg, double& mean, double& sigma, double& unit, int& cnt, int& shift) {
-        cnt = t.cnt[seg];
-        const unsigned mb = t.maxbits[seg];
+        cnt = __ldcg(&t.cnt[seg]);
+        const unsigned mb = __ldcg(&t.maxbits[seg]);
         mean = 0.0; sigma = 0.0; unit = 0.0; shift = 0;
         if (cnt == 0 || mb == 0u) return;
         shift = seg_shift(mb, cnt);
         unit = ldexp(1.0 / static_cast<double>(cnt), -shift);            // value of one step of n q - S
-        const long long S = t.sum[seg];
+        const long long S = __ldcg(&t.sum[seg]);
         mean = static_cast<double>(S) * unit;
         const int dof = cnt - a.ddof;
         if (dof > 0) {
-            const unsigned __int128 Q = (static_cast<unsigned __int128>(t.sqhi[seg]) << 64) | t.sqlo[seg];
+            const unsigned __int128 Q = (static_cast<unsigned __int128>(__ldcg(&t.sqhi[seg])) << 64) | __ldcg(&t.sqlo[seg]);
             const unsigned long long absS = static_cast<unsigned long long>(S < 0 ? -S : S);
             const unsigned __int128 d = Q * static_cast<unsigned>(cnt) - static_cast<unsigned __int128>(absS) * absS;   // n Q - S^2 >= 0
             const double dd = ldexp(static_cast<double>(static_cast<unsigned long long>(d >> 64)), 64) +
@@ -159,7 +160,7 @@ __device__ __forceinline__ void adv_pass_finish(const AdvArgs& a, int i) {
             stats(seg, mean, sigma, unit, cnt, shift);
             const double denom = sigma + static_cast<double>(a.eps);
             if (cnt - a.ddof > 0 && denom != 0.0 && unit != 0.0) {
-                const long long e = static_cast<long long>(cnt) * seg_quantise(a.r_scratch[i], shift) - t.sum[seg];
+                const long long e = static_cast<long long>(cnt) * seg_quantise(a.r_scratch[i], shift) - __ldcg(&t.sum[seg]);
                 adv = static_cast<float>(static_cast<double>(e) * unit / denom);
             }
         }

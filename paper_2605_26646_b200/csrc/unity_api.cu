@@ -39,7 +39,7 @@ struct unity_ctx {
     int chunk_sync;                 // bit 0: same for the recompute GEMM, bit 1: dHidden GEMM, bit 2: dW GEMM
     int logit_stash;                // 1: the loss call keeps the logits of one row block instead of recomputing them
     int l2_hints[UNITY_PROF_CLASSES]; // per GEMM class: GemmArgs::l2_hints
-    int wide_acc;                   // 1: dHidden / dW chunk GEMMs use 512-column tiles (CTA pairs only)
+    int wide_acc;                   // 1: dHidden / dW chunk GEMMs may use tiles two MMA blocks wide (CTA pairs only)
     unsigned round_total;           // arrivals accumulated so far on the rendezvous counter (d_status + 16)
     int chunk_sync_period[3];       // recompute / dHidden / dW GEMM: rendezvous at every n-th tile of a worker
     long long wait_budget;          // SM clocks after which an in-kernel wait gives up
@@ -972,7 +972,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
         if ((rc = make_tmap(ctx, &tm_hp_k, L.hp, H, P.n_slots, static_cast<uint64_t>(H) * 2, kBoxRows))) return rc;
         if ((rc = make_tmap(ctx, &tm_hp_mn, L.hp, H, P.n_slots, static_cast<uint64_t>(H) * 2, kTileK))) return rc;
     }
-    // 512-column tiles unless 256-column tiles waste clearly less of this launch: the share of executed MMA work that
+    // Tiles two blocks wide unless one-block tiles waste clearly less of this launch: the share of executed MMA work that
     // is useful = (H / padded columns) x (tiles / tiles rounded up to whole waves of CTA pairs); the wide form gets a
     // 15 % bonus for its lower operand traffic (at H = 896 the narrow form is bound by the stream of G, not by MMA time:
     // dHidden +13 %, dW +7 % with the wide form although it wastes an eighth more of its last wave).

@@ -384,6 +384,16 @@ def test_small_shapes_and_ragged_tails(H, V, rows):
     run_all_stages(small_workload(H, V, rows))
 
 
+@pytest.mark.parametrize("rows,valid,ctas", [(7700, 6289, 2), (7700, 6289, 1), (15400, 12326, 2)])
+def test_forward_rounds_with_a_short_last_round(rows, valid, ctas):
+    # 6289 valid rows = 25 row tiles of 256 (or 50 of 128): one full round of 24 (48) row tiles x 3 splits and a last
+    # round of ONE row tile (two), which the planner cuts into 32 vocabulary splits; 12326 valid rows = 49 row tiles:
+    # two full rounds and a last one of one tile
+    w = small_workload(128, 8192 + 264, rows, max_len=200, role_model=[0, 0, 0], K=1)
+    assert (w.tok_mask != 0).sum().item() == valid
+    run_all_stages(w, ctas=(ctas,) * 4)
+
+
 @pytest.mark.parametrize("ctas", [(1, 1, 1, 1), (2, 2, 2, 2), (2, 1, 1, 2)])
 def test_single_cta_and_cta_pair_kernels(ctas):
     # every GEMM class exists as a one-CTA kernel (128-row tiles) and as a CTA-pair kernel (256-row tiles)
