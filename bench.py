@@ -283,8 +283,8 @@ def measure_streaming():
            "ready_batch_gather_f32": {"ms": t_gat, "algorithmic_bytes": 8 * kept_tok, "gbs": 8 * kept_tok / t_gat / 1e6},
            "ready_batch_plan": {"ms": t_plan, "note": "latency-bound: four small launches over the invocations"},
            "logprob_fwd_tiny_host": {"call_returns_after_us": ret_us[len(ret_us) // 2], "complete_after_us": done_us[len(done_us) // 2],
-                                     "note": "median of 20 calls on the tiny configuration; the call synchronises the stream once, "
-                                             "after the routing kernels, to read K row counts"}}
+                                     "note": "median of 20 calls on the tiny configuration; by default the call synchronises the stream "
+                                             "once, after the routing kernels, to read K row counts (UNITY_OPT_HOST_COUNTS)"}}
     for k in ("role_advantage", "device_fill_f32", "gae", "value_loss", "align_rewards", "ready_batch_gather_f32"):
         out[k]["frac"] = out[k]["gbs"] / peaks["hbm_gbs"]
     ctx.close()

@@ -177,6 +177,7 @@ def unity_workspace_bytes_stash(n_tok: int, H: int, V: int, K: int, n_inv: int) 
 
 OPT_LOGIT_STASH = 15
 OPT_WAIT_KCYCLES = 20
+OPT_HOST_COUNTS = 25
 OPT_TEST_DROP_SLAB = 21
 
 

@@ -111,10 +111,46 @@ __device__ __forceinline__ unsigned pack_bf16(float lo, float hi) {
     return *reinterpret_cast<unsigned*>(&v);
 }
 
+// The launch's arguments with everything that depends on the number of rows filled in from the device plan.
+template <int TILE_ROWS>
+__device__ __noinline__ GemmArgs resolve_span(const GemmArgs& in) {
+    GemmArgs g = in;
+    if (in.span.plan == nullptr) return g;
+    int slot0, n_rows;
+    span_resolve(in.span, slot0, n_rows);
+    if (in.span_mode == kSpanForward) {
+        const FwdShape fs = forward_shape(in.fwd, n_rows);
+        g.a_row0 = slot0;
+        g.m_rows = n_rows;
+        g.m_tiles = n_rows / TILE_ROWS;
+        g.group_m = fs.gm; g.n_splits = fs.splits; g.tiles_per_split = fs.tps;
+        g.last_m0 = fs.last_m0; g.last_splits = fs.last_splits; g.last_tiles_per_split = fs.last_tps;
+        g.last_stats_off = static_cast<long long>(fs.splits) * n_rows;
+        g.last_pitch = n_rows - static_cast<long long>(fs.last_m0) * TILE_ROWS;
+        g.stats_pitch = n_rows;
+        if (in.stats_from_plan) g.stats = in.stats + in.span.plan->stats_base[in.span.model];
+    } else if (in.span_mode == kSpanRowsA) {
+        g.a_row0 = in.a_row0 + slot0;
+        g.m_rows = n_rows;
+        g.m_tiles = n_rows / TILE_ROWS;
+    } else if (in.span_mode == kSpanRowsM) {
+        g.m_rows = n_rows;
+        g.m_tiles = n_rows / TILE_ROWS;
+    } else if (in.span_mode == kSpanRowsK) {
+        g.k_iters = n_rows / kTileK;
+        g.b_k0 = in.b_k0 + slot0;
+    }
+    return g;
+}
+
 template <int EPI, bool A_MN, bool B_MN, int CTAS, int NB = 1>
 __global__ void __launch_bounds__(kThreads, 1)
-k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs g) {
+k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs g_in) {
     using C = Cfg<CTAS, NB>;
+    // The row extent of a launch may be known on the device only: derive it from the plan before anything else.  Every
+    // thread of both CTAs reads the same plan, so a launch whose span is empty is left by all of them, here.
+    const GemmArgs g = resolve_span<C::kTileRows>(g_in);
+    if (g.m_tiles <= 0 || g.n_tiles <= 0 || g.k_iters <= 0) return;
     constexpr int kStages = C::kStages, kStageBytes = C::kStageBytes, kABytes = C::kABytes, kBBytes = C::kBBytes;
     constexpr int kAccStages = C::kAccStages, kTileCols = C::kTileCols;
     static_assert(NB == 1 || (EPI == kEpiAccumF32 && CTAS == 2), "two-block tiles: fp32-accumulate epilogue, CTA pairs");
@@ -171,8 +207,7 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                     // they start together, and once they drift apart by more than L2 can bridge each of them fetches the
                     // stream from HBM again.  Purely a performance hint: after a short, bounded wait the worker goes on
                     // regardless (some CTAs may not be resident yet).
-                    // The counter only ever grows; round_base is its value before this launch (every worker adds one
-                    // per rendezvous whether or not it waited, so the host can keep the running total).
+                    // The counter belongs to this launch and starts at zero.
                     atomicAdd(g.round_counter, 1u);
                     // arrivals expected by the end of this rendezvous: every worker (softmax), or every worker that
                     // still has a tile (the last ones of the other epilogues may be partial)
@@ -185,7 +220,7 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                         expect = static_cast<unsigned>(it / g.sync_period) * static_cast<unsigned>(n_pairs) +
                                  static_cast<unsigned>(left < n_pairs ? left : n_pairs);
                     }
-                    const unsigned target = g.round_base + expect;
+                    const unsigned target = expect;
                     const long long t0 = clock64();
                     while (static_cast<int>(*reinterpret_cast<volatile unsigned*>(g.round_counter) - target) < 0 &&
                            clock64() - t0 < 400000) { }
@@ -576,49 +611,20 @@ int gemm_mma_n(int n_cols) {
     return (per + 31) / 32 * 32;
 }
 
-namespace {
-// workers and rounds of a launch (must mirror next_unit and launch_gemm)
-void launch_shape(GemmEpilogue epi, int ctas, const GemmArgs& args, int sm_count, int* workers, long long* rounds) {
-    const long long gm = args.group_m < args.m_tiles ? args.group_m : args.m_tiles;
-    const long long units = epi == kEpiSoftmaxStats ? (gm < 1 ? 1 : gm) * args.n_splits
-                                                    : static_cast<long long>(args.m_tiles) * args.n_tiles;
-    const int max_workers = sm_count / ctas;
-    *workers = static_cast<int>(units < max_workers ? units : max_workers);
-    if (units <= 0 || args.m_tiles <= 0 || args.k_iters <= 0) { *workers = 0; *rounds = 0; return; }
-    if (epi == kEpiSoftmaxStats) {
-        const long long g1 = args.group_m < 1 ? 1 : args.group_m;
-        *rounds = (args.m_tiles + g1 - 1) / g1;
-    } else {
-        *rounds = (units + *workers - 1) / *workers;   // workers with a shorter loop stop arriving: see below
-    }
-}
-}  // namespace
-
-unsigned gemm_round_arrivals(GemmEpilogue epi, int ctas, const GemmArgs& args, int sm_count) {
-    int workers; long long rounds;
-    launch_shape(epi, ctas, args, sm_count, &workers, &rounds);
-    if (workers == 0) return 0;
-    if (epi == kEpiSoftmaxStats) return static_cast<unsigned>(rounds * workers);
-    // striding over units: the workers that still have a tile in round r arrive at its rendezvous, every
-    // sync_period-th round has one
-    const long long units = static_cast<long long>(args.m_tiles) * args.n_tiles;
-    const int period = args.sync_period > 0 ? args.sync_period : 1;
-    long long total = 0;
-    for (long long before = 0; before < units; before += static_cast<long long>(period) * workers)
-        total += units - before < workers ? units - before : workers;
-    return static_cast<unsigned>(total);
-}
-
 cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, int ctas, const CUtensorMap& tmA, const CUtensorMap& tmB,
                         const GemmArgs& args, int sm_count, cudaStream_t stream, bool wide) {
-    // softmax: one round handles group_m row tiles x n_splits; other epilogues: plain striding over all tiles
-    const long long units = epi == kEpiSoftmaxStats
-                                ? static_cast<long long>(args.group_m < args.m_tiles ? args.group_m : args.m_tiles) * args.n_splits
-                                : static_cast<long long>(args.m_tiles) * args.n_tiles;
-    if (units <= 0 || args.m_tiles <= 0 || args.k_iters <= 0) return cudaSuccess;
-    if (epi == kEpiAccumF32 && (args.mma_n < 32 || args.mma_n > kTileN || args.mma_n % 32 != 0)) return cudaErrorInvalidValue;
+    // softmax: one round handles group_m row tiles x n_splits; other epilogues: plain striding over all tiles.  With the
+    // row extent known on the device only, the launch takes the whole machine; workers without a unit leave at once.
     const int max_workers = sm_count / ctas;                                   // one CTA per SM
-    const int workers = static_cast<int>(units < max_workers ? units : max_workers);
+    int workers = max_workers;
+    if (args.span.plan == nullptr) {
+        const long long units = epi == kEpiSoftmaxStats
+                                    ? static_cast<long long>(args.group_m < args.m_tiles ? args.group_m : args.m_tiles) * args.n_splits
+                                    : static_cast<long long>(args.m_tiles) * args.n_tiles;
+        if (units <= 0 || args.m_tiles <= 0 || args.k_iters <= 0) return cudaSuccess;
+        workers = static_cast<int>(units < max_workers ? units : max_workers);
+    }
+    if (epi == kEpiAccumF32 && (args.mma_n < 32 || args.mma_n > kTileN || args.mma_n % 32 != 0)) return cudaErrorInvalidValue;
     const bool two = ctas == 2;
     switch (epi) {
         case kEpiSoftmaxStats:

@@ -23,8 +23,90 @@ constexpr int kStatusBadIndex = 1;
 constexpr int kStatusTimeout = 2;
 
 // ----------------------------------------------------------------------------------------------
+// Row layout on the device.  The number of valid rows per model is known only after the routing kernels have run, and
+// the host never reads it back (the calls stay asynchronous): every kernel whose extent depends on it takes the plan
+// and a span of rows and works out its own extent; a launch whose span turns out empty returns at once.
+// ----------------------------------------------------------------------------------------------
+struct DevPlan {
+    int counts[UNITY_MAX_MODELS];             // valid rows per model
+    int off[UNITY_MAX_MODELS + 1];            // first packed slot per model (multiples of kTileM); off[K] = slots in use
+    long long stats_base[UNITY_MAX_MODELS];   // first float4 of model k's forward statistics
+};
+// Rows [row_begin, row_begin + row_cap) of `model`'s packed range, cut to the rows the model has.
+struct RowSpan {
+    const DevPlan* plan;
+    int model, row_begin, row_cap;
+};
+__device__ __forceinline__ void span_resolve(const RowSpan& s, int& slot0, int& n_rows) {
+    const int first = s.plan->off[s.model];
+    const int rows = s.plan->off[s.model + 1] - first;
+    const int left = rows - s.row_begin;
+    n_rows = left < 0 ? 0 : (left < s.row_cap ? left : s.row_cap);
+    slot0 = first + s.row_begin;
+}
+
+// Shape of one forward launch over `rows` packed rows (a multiple of the row tile): row tiles per round and
+// vocabulary splits.  One round of the persistent kernel = gm row tiles x splits vocabulary splits <= number of
+// workers (CTAs or CTA pairs): gm bounds the hidden rows that must stay L2 resident (48 tiles of 128 rows by default:
+// 6 k rows, 44 MB at H = 3584, loaded with an evict-last hint), splits fill the machine.  Computed identically
+// wherever it is needed (the forward kernel, the kernel that merges its splits, the host's size bounds).
+struct FwdShape {
+    int gm, splits, tps;                  // row tiles per round; vocabulary splits and tiles per split of a full round
+    int last_m0, last_splits, last_tps;   // first row tile, splits and tiles per split of a short last round
+                                          // (last_m0 = number of row tiles when the last round is like the others)
+    long long stats_rows;                 // float4 entries the launch writes: splits x rows + last_splits x last rows
+};
+struct FwdPlanParams {
+    int n_pairs;     // workers (CTAs or CTA pairs) of the forward kernel
+    int gmax;        // largest round, in row tiles
+    int tile_rows;   // rows of a row tile (128 or 256)
+    int n_tiles;     // vocabulary tiles of 256
+};
+__host__ __device__ inline FwdShape forward_shape(const FwdPlanParams& p, int rows) {
+    const int m_tiles = rows / p.tile_rows;
+    // Among round sizes from two thirds of gmax up to gmax, take the one with the least work per worker: vocabulary
+    // tiles per split, summed over the rounds, the last of which may hold fewer row tiles and then cuts the vocabulary
+    // into more splits (a batch whose row tiles do not divide well would otherwise idle part of the machine in its
+    // last round); ties go to the larger round, which streams W less often.
+    FwdShape best;
+    best.gm = 1; best.splits = 1; best.tps = p.n_tiles; best.last_m0 = m_tiles; best.last_splits = 1; best.last_tps = p.n_tiles;
+    long long best_cost = -1;
+    const int cand_min = m_tiles <= p.gmax ? 1 : (2 * p.gmax + 2) / 3;      // few row tiles: any round size is L2-safe
+    for (int cand = p.gmax; cand >= cand_min; --cand) {
+        const int c = cand < m_tiles ? cand : (m_tiles > 0 ? m_tiles : 1);
+        int sp = p.n_pairs / c;
+        sp = sp > 32 ? 32 : sp;
+        sp = sp > p.n_tiles ? p.n_tiles : sp;
+        sp = sp < 1 ? 1 : sp;
+        const int full_rounds = m_tiles / c, rest = m_tiles - full_rounds * c;
+        int sp_last = sp;
+        if (rest > 0) {
+            sp_last = p.n_pairs / rest;
+            sp_last = sp_last > 32 ? 32 : sp_last;
+            sp_last = sp_last > p.n_tiles ? p.n_tiles : sp_last;
+            sp_last = sp_last < 1 ? 1 : sp_last;
+        }
+        const long long cost = static_cast<long long>(full_rounds) * ((p.n_tiles + sp - 1) / sp) +
+                               (rest > 0 ? (p.n_tiles + sp_last - 1) / sp_last : 0);
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost;
+            best.gm = c;
+            best.tps = (p.n_tiles + sp - 1) / sp;
+            best.splits = (p.n_tiles + best.tps - 1) / best.tps;
+            best.last_m0 = rest > 0 && sp_last != sp ? full_rounds * c : m_tiles;
+            best.last_tps = (p.n_tiles + sp_last - 1) / sp_last;
+            best.last_splits = (p.n_tiles + best.last_tps - 1) / best.last_tps;
+        }
+    }
+    const long long last_rows = static_cast<long long>(m_tiles - best.last_m0) * p.tile_rows;
+    best.stats_rows = static_cast<long long>(best.splits) * rows + best.last_splits * last_rows;
+    return best;
+}
+
+// ----------------------------------------------------------------------------------------------
 // GEMM  C[m, n] = sum_k A[m, k] * B[n, k]   (bf16 operands, K-major or MN-major, fp32 accumulation in TMEM)
 // ----------------------------------------------------------------------------------------------
+enum : int { kSpanNone = 0, kSpanForward = 1, kSpanRowsA = 2, kSpanRowsM = 3, kSpanRowsK = 4 };
 enum GemmEpilogue : int {
     kEpiSoftmaxStats = 0,   // online (max, sum exp, sum exp*z, target logit) per row; nothing of size M x N stored
     kEpiLogitGrad = 1,      // dL/dz in bf16 for a bounded (rows x vocab) chunk
@@ -45,8 +127,7 @@ struct GemmArgs {
     // statistics to stats[last_stats_off + split * last_pitch + (row - first row of tile last_m0)]
     int last_m0, last_splits, last_tiles_per_split;
     long long last_stats_off, last_pitch;
-    unsigned* round_counter;  // ever-growing arrival counter (null = no rendezvous between rounds)
-    unsigned round_base;      // its value before this launch
+    unsigned* round_counter;  // this launch's arrival counter, zero before the launch (null = no rendezvous between rounds)
     int sync_period;          // epilogues other than softmax: rendezvous at every sync_period-th tile of a worker (>= 1)
     float4* stats;            // [n_splits][stats_pitch], row relative to a_row0: (max acc, sum e, sum e*acc, target acc)
     long long stats_pitch;
@@ -74,6 +155,16 @@ struct GemmArgs {
                               // unless the output's width divides better (896 columns = 4 blocks of 224)
     int l2_hints;             // L2 eviction policy (0 normal, 1 first, 2 last): bits 0-1 A loads, 2-3 B loads, 4-5 G stores
     int* status;
+    // Rows known on the device only (span.plan != null): the kernel derives the row extent of the launch from the plan
+    //   kSpanForward : A rows = the span; m_tiles, the round / split shape (forward_shape) and, with stats_from_plan,
+    //                  the base of the statistics follow from it
+    //   kSpanRowsA   : A rows = the span inside the hidden rows (recompute): a_row0 += first slot, m_rows, m_tiles
+    //   kSpanRowsM   : M extent = the span's length (dHidden: A is the chunk-local G): m_rows, m_tiles
+    //   kSpanRowsK   : K extent = the span's length (dW): k_iters, b_k0 += first slot
+    RowSpan span;
+    int span_mode;
+    int stats_from_plan;
+    FwdPlanParams fwd;
     long long wait_budget;    // SM clocks after which an mbarrier wait gives up (kStatusTimeout)
     int test_drop_slab;       // test hook: the TMA producer of every worker leaves out one K slab of its first tile
                               // (neither the expected-bytes arrival nor the loads), so the waits behind it run out
@@ -87,8 +178,6 @@ struct GemmArgs {
 // 2 * args.mma_n columns instead of args.mma_n.
 cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, int ctas, const CUtensorMap& tmA, const CUtensorMap& tmB,
                         const GemmArgs& args, int sm_count, cudaStream_t stream, bool wide = false);
-// Arrivals the launch adds to args.round_counter (rounds x workers); 0 when nothing is launched.
-unsigned gemm_round_arrivals(GemmEpilogue epi, int ctas, const GemmArgs& args, int sm_count);
 int gemm_tile_rows(int ctas);
 int gemm_mma_n(int n_cols);   // block width for an fp32-accumulate GEMM with n_cols output columns
 cudaError_t gemm_set_attributes();
@@ -126,8 +215,8 @@ struct RouteArgs {
     const uint8_t* tok_mask;
     int n_blocks;                // ceil(n_tok / kRouteBlock)
     int* blk_cnt;                // [n_blocks * K] -> exclusive prefix per model after the scan
-    int* counts;                 // [K] valid rows per model
-    int* offsets;                // [K+1] first slot of each model (multiples of kTileM), offsets[K] = total slots
+    DevPlan* plan;               // out: valid rows, first slot (multiples of kTileM) and statistics base of each model
+    FwdPlanParams fwd;           // inputs of the forward planner (for the statistics bases)
     int* tok_slot;               // [n_tok] slot of a token or -1
     int* slot_tok;               // [max_slots] token of a slot or -1 (pre-filled with -1)
     int8_t* tok_model;           // [n_tok] model id or -1
@@ -135,36 +224,36 @@ struct RouteArgs {
 };
 cudaError_t launch_route(const RouteArgs& a, cudaStream_t stream, int* n_launches);
 
-cudaError_t launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* target, const int* slot_tok, int n_slots,
-                               int H, __nv_bfloat16* hp, int* target_p, cudaStream_t stream);
+// packs the rows of slots [0, plan->off[K]); max_slots bounds the grid
+cudaError_t launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* target, const int* slot_tok,
+                               const DevPlan* plan, int K, long long max_slots, int H, __nv_bfloat16* hp, int* target_p,
+                               cudaStream_t stream);
 
 struct TokenArgs {
-    int slot_begin;            // k_finish_rows works on slots [slot_begin, n_slots)
-    int n_slots, n_splits, K, n_roles, n_inv;
+    // k_finish_rows works on the rows of `block` (block.model >= 0: one block of one model's rows, whose forward ran as
+    // a launch of its own with its statistics at stats[0..]), or on every packed row (block.model < 0)
+    RowSpan block;
+    const DevPlan* plan;
+    FwdPlanParams fwd;         // the forward planner's inputs: the split layout of the statistics follows from the rows
+    long long max_slots;       // bound of the packed rows (sizes the grid)
+    int K, n_roles, n_inv;
     long long n_tok;
-    const float4* stats;       // per model: base stats_base[k], pitch = padded rows of the model
-    long long stats_base[UNITY_MAX_MODELS];
-    int model_splits[UNITY_MAX_MODELS];
-    // rows of a model from last_row0[k] on (relative to its first slot) were swept with last_splits[k] splits; their
-    // statistics start at stats_last[k] with pitch = the model's padded rows - last_row0[k]
-    int last_row0[UNITY_MAX_MODELS];
-    int last_splits[UNITY_MAX_MODELS];
-    long long stats_last[UNITY_MAX_MODELS];
+    const float4* stats;       // per model: base plan->stats_base[k], pitch = padded rows of the model
     const int* slot_tok;
     const int* tok_slot;
     const int8_t* tok_model;
-    int offsets[UNITY_MAX_MODELS + 1];
     float scale;               // inv_temperature
     // forward outputs (packed and caller order)
-    float *row_lse, *row_ent, *row_logp;      // packed [n_slots]
+    float *row_lse, *row_ent, *row_logp;      // packed [slots]
     float *logp, *entropy, *lse;              // caller order [n_tok], nullable
     const float *logp_in, *entropy_in, *lse_in;   // caller order [n_tok]: results of an earlier forward (or all null)
     // loss part (null for logprob_fwd)
     const float *old_logp, *ref_logp, *adv_tok;
     float clip_lo, clip_hi, kl_coef, ent_coef;
     int kl_mode;
-    float norm[UNITY_MAX_MODELS];   // M_k
-    float *coef_a, *coef_b;    // packed [n_slots], already multiplied by scale
+    int has_norm;                   // 1: M_k = norm[k]; 0: M_k = max(valid rows of model k, 1) from the plan
+    float norm[UNITY_MAX_MODELS];
+    float *coef_a, *coef_b;    // packed [slots], already multiplied by scale
     float* tok_loss;           // caller order, nullable
     const int64_t* cu_seqlens;
     const int32_t* inv_role;
@@ -174,16 +263,17 @@ struct TokenArgs {
     float* metrics;            // [(K + n_roles) * 8] nullable
 };
 cudaError_t launch_finish_forward(const TokenArgs& a, bool with_loss, cudaStream_t stream, int* n_launches);
-// the two halves of the above: per-row terms for slots [a.slot_begin, a.n_slots), and the loss / metric reductions
+// the two halves of the above: per-row terms for the rows of a.block (or all packed rows), and the loss / metric reductions
 cudaError_t launch_finish_rows(const TokenArgs& a, bool with_loss, cudaStream_t stream, int* n_launches);
 cudaError_t launch_loss_reduce(const TokenArgs& a, cudaStream_t stream, int* n_launches);
 
 // In place, for a block of rows x cols (row pitch ld) of stashed scaled logits z: z <- dL/dz =
-// -p*(a + b*(z - lse + H)) (+ a at the target), p = exp(z - lse); per-row vectors are indexed from `row0`.
+// -p*(a + b*(z - lse + H)) (+ a at the target), p = exp(z - lse).
 struct LogitGradArgs {
     __nv_bfloat16* Z;
     long long ld;
-    int rows, cols, row0, vocab0;
+    RowSpan span;              // the rows of the block; per-row vectors are indexed from its first slot
+    int cols, vocab0;
     const int* target_p;
     const float *coef_a, *coef_b, *row_lse, *row_ent;
 };
@@ -191,9 +281,11 @@ cudaError_t launch_logit_grad_inplace(const LogitGradArgs& a, cudaStream_t strea
 
 cudaError_t launch_zero_masked_rows(const int* tok_slot, long long n_tok, int H, __nv_bfloat16* dHidden,
                                     cudaStream_t stream);
-// dHidden[slot_tok[slot0 + r], :] = bf16(dHc[r, :]) for r < n_rows with a token
-cudaError_t launch_store_dhidden(const float* dHc, const int* slot_tok, int slot0, int n_rows, int H,
+// dHidden[slot_tok[first slot of the span + r], :] = bf16(dHc[r, :]) for the rows r of the span that hold a token
+cudaError_t launch_store_dhidden(const float* dHc, const int* slot_tok, const RowSpan& span, int H,
                                  __nv_bfloat16* dHidden, cudaStream_t stream);
+// dst[0, n) = 0 when model k has no valid row (its dW when nothing accumulates into it)
+cudaError_t launch_zero_if_empty(float* dst, long long n, const DevPlan* plan, int k, cudaStream_t stream);
 
 cudaError_t launch_gae(int n_inv, const int64_t* cu_seqlens, const float* rewards, const float* values,
                        const uint8_t* tok_mask, float gamma, float lam, float* adv, float* ret, cudaStream_t stream);

@@ -327,12 +327,16 @@ __global__ void k_route_scan(RouteArgs a) {
     }
     if (tid == 0) {
         int off = 0;
+        long long sbase = 0;
         for (int k = 0; k < a.K; ++k) {
-            a.counts[k] = total[k];
-            a.offsets[k] = off;
-            off += (total[k] + kTileM - 1) / kTileM * kTileM;
+            const int rows = (total[k] + kTileM - 1) / kTileM * kTileM;
+            a.plan->counts[k] = total[k];
+            a.plan->off[k] = off;
+            a.plan->stats_base[k] = sbase;
+            off += rows;
+            sbase += rows > 0 ? forward_shape(a.fwd, rows).stats_rows : 0;
         }
-        a.offsets[a.K] = off;
+        a.plan->off[a.K] = off;
     }
 }
 
@@ -352,18 +356,18 @@ __global__ void k_route_assign(RouteArgs a) {
     if (model < 0) { a.tok_slot[i] = -1; return; }
     int before = 0;
     for (int w = 0; w < warp; ++w) before += warp_cnt[w][model];
-    const int slot = a.offsets[model] + a.blk_cnt[blockIdx.x * a.K + model] + before + rank;
+    const int slot = a.plan->off[model] + a.blk_cnt[blockIdx.x * a.K + model] + before + rank;
     a.tok_slot[i] = slot;
     a.slot_tok[slot] = static_cast<int>(i);
 }
 
 // One warp per packed row: 128-bit copies of the hidden row (zeros for padding slots).
 __global__ void k_gather_rows(const __nv_bfloat16* __restrict__ hidden, const int32_t* __restrict__ target,
-                              const int* __restrict__ slot_tok, int n_slots, int H, __nv_bfloat16* __restrict__ hp,
-                              int* __restrict__ target_p) {
-    const int slot = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+                              const int* __restrict__ slot_tok, const DevPlan* __restrict__ plan, int K, int H,
+                              __nv_bfloat16* __restrict__ hp, int* __restrict__ target_p) {
+    const long long slot = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
-    if (slot >= n_slots) return;
+    if (slot >= plan->off[K]) return;
     const int tok = slot_tok[slot];
     const int n16 = H >> 3;
     uint4* dst = reinterpret_cast<uint4*>(hp + static_cast<long long>(slot) * H);
@@ -404,8 +408,36 @@ __device__ __forceinline__ PpoTerms ppo_terms(float logp, float ent, float old_l
 
 // One thread per packed row: merge the vocabulary splits, form lse / entropy / logp, then the loss terms.
 __global__ void k_finish_rows(TokenArgs a, int with_loss) {
-    const int slot = a.slot_begin + blockIdx.x * blockDim.x + threadIdx.x;
-    if (slot >= a.n_slots) return;
+    // Where the statistics of a row lie follows from the shape of the forward launch that wrote them, and that from the
+    // rows the launch covered: one block of one model's rows, or each model's whole range.
+    __shared__ FwdShape sh_shape[UNITY_MAX_MODELS];
+    __shared__ int sh_first[UNITY_MAX_MODELS], sh_rows[UNITY_MAX_MODELS];
+    __shared__ long long sh_base[UNITY_MAX_MODELS];
+    __shared__ int sh_lo, sh_hi;
+    if (threadIdx.x < UNITY_MAX_MODELS) {
+        const int k = threadIdx.x;
+        int first = 0, rows = 0;
+        long long base = 0;
+        if (k < a.K) {
+            if (a.block.model >= 0) {
+                if (k == a.block.model) span_resolve(a.block, first, rows);
+            } else {
+                first = a.plan->off[k];
+                rows = a.plan->off[k + 1] - first;
+                base = a.plan->stats_base[k];
+            }
+        }
+        sh_first[k] = first; sh_rows[k] = rows; sh_base[k] = base;
+        if (rows > 0 && a.lse_in == nullptr) sh_shape[k] = forward_shape(a.fwd, rows);
+        if (k == 0) {
+            if (a.block.model >= 0) { int f, r; span_resolve(a.block, f, r); sh_lo = f; sh_hi = f + r; }
+            else { sh_lo = 0; sh_hi = a.plan->off[a.K]; }
+        }
+    }
+    __syncthreads();
+    const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (idx >= sh_hi - sh_lo) return;
+    const int slot = sh_lo + static_cast<int>(idx);
     const int tok = a.slot_tok[slot];
     if (tok < 0) {
         a.row_lse[slot] = 0.f; a.row_ent[slot] = 0.f; a.row_logp[slot] = 0.f;
@@ -418,14 +450,16 @@ __global__ void k_finish_rows(TokenArgs a, int with_loss) {
         // the caller already evaluated this policy on these rows (unity_logprob_fwd): no forward sweep was run
         lse = a.lse_in[tok]; ent = a.entropy_in[tok]; logp = a.logp_in[tok];
     } else {
-        long long pitch = a.offsets[k + 1] - a.offsets[k];
-        const int r = slot - a.offsets[k];
-        const float4* st = a.stats + a.stats_base[k] + r;
-        int n_splits = a.model_splits[k];
-        if (r >= a.last_row0[k]) {                            // swept in the launch's short last round
-            pitch -= a.last_row0[k];
-            st = a.stats + a.stats_last[k] + (r - a.last_row0[k]);
-            n_splits = a.last_splits[k];
+        const FwdShape& fs = sh_shape[k];
+        long long pitch = sh_rows[k];
+        const int r = slot - sh_first[k];
+        const float4* st = a.stats + sh_base[k] + r;
+        int n_splits = fs.splits;
+        const long long last_row0 = static_cast<long long>(fs.last_m0) * a.fwd.tile_rows;
+        if (r >= last_row0) {                                 // swept in the launch's short last round
+            st = a.stats + sh_base[k] + static_cast<long long>(fs.splits) * pitch + (r - last_row0);
+            pitch -= last_row0;
+            n_splits = fs.last_splits;
         }
         const float c = a.scale * 1.4426950408889634f;    // exp(scale*x) = exp2(c*x)
         float m = -3.0e38f;
@@ -447,7 +481,7 @@ __global__ void k_finish_rows(TokenArgs a, int with_loss) {
     if (a.entropy) a.entropy[tok] = ent;
     if (a.lse) a.lse[tok] = lse;
     if (!with_loss) return;
-    const float Mk = a.norm[k];
+    const float Mk = a.has_norm ? a.norm[k] : fmaxf(static_cast<float>(a.plan->counts[k]), 1.f);
     const PpoTerms p = ppo_terms(logp, ent, a.old_logp[tok], a.ref_logp[tok], a.adv_tok[tok], a.clip_lo, a.clip_hi,
                                  a.kl_coef, a.kl_mode, a.ent_coef);
     a.coef_a[slot] = a.scale * (p.dl_dlogp / Mk);
@@ -504,7 +538,7 @@ __global__ void k_class_reduce(TokenArgs a) {
         m[0] = acc[0];
         for (int j = 1; j < 8; ++j) m[j] = acc[j] / dn;
     }
-    if (c < a.K) a.loss[c] = acc[8] / a.norm[c];
+    if (c < a.K) a.loss[c] = acc[8] / (a.has_norm ? a.norm[c] : fmaxf(static_cast<float>(a.plan->counts[c]), 1.f));
 }
 
 // Stashed logits -> logit gradients, in place.  A block converts 8192 consecutive columns of one row: every thread
@@ -513,8 +547,10 @@ __global__ void k_class_reduce(TokenArgs a) {
 constexpr int kGradVecs = 4;
 __global__ void __launch_bounds__(256) k_logit_grad_inplace(LogitGradArgs a) {
     const int c_first = blockIdx.x * (256 * 8 * kGradVecs) + threadIdx.x * 8;
-    for (int r = blockIdx.y; r < a.rows; r += gridDim.y) {
-        const int slot = a.row0 + r;
+    int row0, rows;
+    span_resolve(a.span, row0, rows);
+    for (int r = blockIdx.y; r < rows; r += gridDim.y) {
+        const int slot = row0 + r;
         uint4* row = reinterpret_cast<uint4*>(a.Z + static_cast<long long>(r) * a.ld);
         uint4 raw[kGradVecs];
 #pragma unroll
@@ -555,10 +591,20 @@ __global__ void k_zero_masked_rows(const int* __restrict__ tok_slot, long long n
     for (int j = lane; j < (H >> 3); j += 32) dst[j] = make_uint4(0, 0, 0, 0);
 }
 
-__global__ void k_store_dhidden(const float* __restrict__ dHc, const int* __restrict__ slot_tok, int slot0, int n_rows,
+// dst[0, n4) = 0 (128-bit stores, grid-stride) when model k has no valid row; returns at once otherwise.
+__global__ void k_zero_if_empty(float4* __restrict__ dst, long long n4, const DevPlan* __restrict__ plan, int k) {
+    if (plan->counts[k] != 0) return;
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n4; i += stride)
+        dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
+__global__ void k_store_dhidden(const float* __restrict__ dHc, const int* __restrict__ slot_tok, RowSpan span,
                                 int H, __nv_bfloat16* __restrict__ dHidden) {
     const int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
+    int slot0, n_rows;
+    span_resolve(span, slot0, n_rows);
     if (r >= n_rows) return;
     const int tok = slot_tok[slot0 + r];
     if (tok < 0) return;
@@ -964,15 +1010,17 @@ cudaError_t launch_route(const RouteArgs& a, cudaStream_t stream, int* n_launche
     return cudaGetLastError();
 }
 
-cudaError_t launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* target, const int* slot_tok, int n_slots,
-                               int H, __nv_bfloat16* hp, int* target_p, cudaStream_t stream) {
-    if (n_slots == 0) return cudaSuccess;
-    k_gather_rows<<<(n_slots + 7) / 8, 256, 0, stream>>>(hidden, target, slot_tok, n_slots, H, hp, target_p);
+cudaError_t launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* target, const int* slot_tok,
+                               const DevPlan* plan, int K, long long max_slots, int H, __nv_bfloat16* hp, int* target_p,
+                               cudaStream_t stream) {
+    if (max_slots == 0) return cudaSuccess;
+    k_gather_rows<<<static_cast<unsigned>((max_slots + 7) / 8), 256, 0, stream>>>(hidden, target, slot_tok, plan, K, H, hp,
+                                                                                  target_p);
     return cudaGetLastError();
 }
 
 cudaError_t launch_finish_rows(const TokenArgs& a, bool with_loss, cudaStream_t stream, int* n_launches) {
-    const int n = a.n_slots - a.slot_begin;
+    const long long n = a.block.model >= 0 ? a.block.row_cap : a.max_slots;      // bound of the rows; the kernel knows the extent
     if (n > 0) {
         k_finish_rows<<<(n + 255) / 256, 256, 0, stream>>>(a, with_loss ? 1 : 0);
         *n_launches += 1;
@@ -997,10 +1045,10 @@ cudaError_t launch_finish_forward(const TokenArgs& a, bool with_loss, cudaStream
 }
 
 cudaError_t launch_logit_grad_inplace(const LogitGradArgs& a, cudaStream_t stream) {
-    if (a.rows <= 0 || a.cols <= 0) return cudaSuccess;
+    if (a.span.row_cap <= 0 || a.cols <= 0) return cudaSuccess;
     // a block covers 8192 columns of one row; y walks the rows (grid-stride, the y extent is limited to 65535)
     const unsigned gx = static_cast<unsigned>((a.cols + 8191) / 8192);
-    const unsigned gy = static_cast<unsigned>(a.rows < 32768 ? a.rows : 32768);
+    const unsigned gy = static_cast<unsigned>(a.span.row_cap < 32768 ? a.span.row_cap : 32768);
     k_logit_grad_inplace<<<dim3(gx, gy), 256, 0, stream>>>(a);
     return cudaGetLastError();
 }
@@ -1012,10 +1060,16 @@ cudaError_t launch_zero_masked_rows(const int* tok_slot, long long n_tok, int H,
     return cudaGetLastError();
 }
 
-cudaError_t launch_store_dhidden(const float* dHc, const int* slot_tok, int slot0, int n_rows, int H,
+cudaError_t launch_store_dhidden(const float* dHc, const int* slot_tok, const RowSpan& span, int H,
                                  __nv_bfloat16* dHidden, cudaStream_t stream) {
-    if (n_rows == 0) return cudaSuccess;
-    k_store_dhidden<<<(n_rows + 7) / 8, 256, 0, stream>>>(dHc, slot_tok, slot0, n_rows, H, dHidden);
+    if (span.row_cap == 0) return cudaSuccess;
+    k_store_dhidden<<<(span.row_cap + 7) / 8, 256, 0, stream>>>(dHc, slot_tok, span, H, dHidden);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_zero_if_empty(float* dst, long long n, const DevPlan* plan, int k, cudaStream_t stream) {
+    if (n == 0) return cudaSuccess;
+    k_zero_if_empty<<<1184, 256, 0, stream>>>(reinterpret_cast<float4*>(dst), n >> 2, plan, k);
     return cudaGetLastError();
 }
 

@@ -40,7 +40,8 @@ struct unity_ctx {
     int logit_stash;                // 1: the loss call keeps the logits of one row block instead of recomputing them
     int l2_hints[UNITY_PROF_CLASSES]; // per GEMM class: GemmArgs::l2_hints
     int wide_acc;                   // 1: dHidden / dW chunk GEMMs may use tiles two MMA blocks wide (CTA pairs only)
-    unsigned round_total;           // arrivals accumulated so far on the rendezvous counter (d_status + 16)
+    int host_counts;                // 1 (default): stages 2 and 3 read the K row counts back (one stream synchronisation)
+                                    // and skip the launches that would be empty; 0: fully asynchronous
     int chunk_sync_period[3];       // recompute / dHidden / dW GEMM: rendezvous at every n-th tile of a worker
     long long wait_budget;          // SM clocks after which an in-kernel wait gives up
     int test_drop;                  // test hook: 1 + GEMM class whose producer leaves out one K slab; 0 = off
@@ -56,6 +57,7 @@ constexpr int kChunkVocab = 74 * kTileN;     // 18944 vocabulary entries
 // A gradient chunk spans kDefaultChunkMult x kDefaultChunkMult such blocks by default: the dHidden / dW GEMMs then
 // contract over twice as many vocabulary entries / rows per output tile and read-modify-write their outputs half as often.
 constexpr int kDefaultChunkMult = 2;
+constexpr int kSyncCounters = 16384;       // rendezvous counters per call (4 bytes each)
 constexpr int kMinChunkRows = 1024;
 constexpr int kMinChunkVocab = 1024;
 
@@ -97,19 +99,22 @@ struct ProfScope {
     }
 };
 
+// Arrival counters of the round rendezvous: one per launch, all cleared at the start of a call.
+struct SyncCounters {
+    unsigned* base;
+    int used, cap;
+    unsigned* next() { return used < cap ? base + used++ : nullptr; }   // beyond the array: that launch runs without
+};
+
 // Fields every GEMM launch of class `cls` takes from the context: status word, L2 hints, wait bound, test hook and,
-// when `sync` is set, the round rendezvous (the counter only grows; the context keeps its running total).
-void gemm_common(unity_ctx* ctx, GemmArgs& g, int cls, GemmEpilogue epi, bool sync) {
+// when `sync` is set, a fresh counter for the round rendezvous.
+void gemm_common(unity_ctx* ctx, GemmArgs& g, int cls, SyncCounters* counters, bool sync) {
     g.status = ctx->d_status;
     g.l2_hints = ctx->l2_hints[cls];
     g.wait_budget = ctx->wait_budget;
     g.test_drop_slab = ctx->test_drop == cls + 1;
     g.sync_period = cls == UNITY_PROF_FWD_GEMM ? 1 : ctx->chunk_sync_period[cls - 1];
-    if (sync) {
-        g.round_counter = reinterpret_cast<unsigned*>(ctx->d_status + 16);
-        g.round_base = ctx->round_total;
-        ctx->round_total += gemm_round_arrivals(epi, ctx->ctas[cls], g, ctx->sm_count);
-    }
+    if (sync && counters) g.round_counter = counters->next();
 }
 
 struct Bump {
@@ -127,7 +132,7 @@ struct Bump {
 
 struct Layout {
     // routing + forward
-    int* tok_slot; int* slot_tok; int8_t* tok_model; int* blk_cnt; int* counts; int* offsets;
+    int* tok_slot; int* slot_tok; int8_t* tok_model; int* blk_cnt; DevPlan* plan; unsigned* sync_counters;
     __nv_bfloat16* hp; int* target_p; float4* stats; float *row_lse, *row_ent, *row_logp;
     // loss + backward
     float *coef_a, *coef_b, *inv_sums;
@@ -153,8 +158,8 @@ Layout carve(char* base, size_t cap, long long n_tok, int H, int V, int K, int n
     L.slot_tok = b.take<int>(L.max_slots);
     L.tok_model = b.take<int8_t>(n_tok);
     L.blk_cnt = b.take<int>(static_cast<size_t>(L.n_blocks) * K + 1);
-    L.counts = b.take<int>(UNITY_MAX_MODELS);
-    L.offsets = b.take<int>(UNITY_MAX_MODELS + 1);
+    L.plan = b.take<DevPlan>(1);
+    L.sync_counters = b.take<unsigned>(kSyncCounters);
     L.hp = b.take<__nv_bfloat16>(static_cast<size_t>(L.max_slots) * H);
     L.target_p = b.take<int>(L.max_slots);
     L.stats = b.take<float4>(L.stats_cap);
@@ -248,68 +253,28 @@ int validate_rows(unity_ctx* ctx, const unity_rows* r) {
     return UNITY_OK;
 }
 
-struct FwdShape {
-    int gm, splits, tps;                  // row tiles per round; vocabulary splits and tiles per split of a full round
-    int last_m0, last_splits, last_tps;   // first row tile, splits and tiles per split of a short last round
-                                          // (last_m0 = number of row tiles when the last round is like the others)
-    long long stats_rows;                 // float4 entries the launch writes: splits x rows + last_splits x last rows
-};
+// Everything the launches of one call share: the carved workspace, the rendezvous counters, and, only when the host was
+// asked to read the row counts back, the padded rows of each model (otherwise -1: not known here).
 struct RowPlan {
     Layout L;
-    int counts[UNITY_MAX_MODELS];
-    int offsets[UNITY_MAX_MODELS + 1];
-    FwdShape shape[UNITY_MAX_MODELS];     // split layout of each model's forward launch
-    long long stats_base[UNITY_MAX_MODELS];
-    int n_slots;
+    SyncCounters counters;
+    FwdPlanParams fwd;
+    int rows_known[UNITY_MAX_MODELS];
+    long long rows_bound;                 // padded rows a model can have at most: every row of the batch
 };
 
-// Shape of one forward launch over `rows` packed rows (a multiple of the row tile): row tiles per round and
-// vocabulary splits.  One round of the persistent kernel = gm row tiles x splits vocabulary splits <= number of
-// workers (CTAs or CTA pairs): gm bounds the hidden rows that must stay L2 resident (48 tiles of 128 rows by default:
-// 6 k rows, 44 MB at H = 3584, loaded with an evict-last hint), splits fill the machine.
-FwdShape forward_shape(const unity_ctx* ctx, int V, int rows) {
+// Inputs of the forward planner that the host knows.
+FwdPlanParams fwd_params(const unity_ctx* ctx, int V) {
     const int ctas = ctx->ctas[UNITY_PROF_FWD_GEMM];
-    const int tile_rows = gemm_tile_rows(ctas);
-    const int m_tiles = rows / tile_rows;
-    const int n_tiles = (V + kTileN - 1) / kTileN;
-    const int n_pairs = ctx->sm_count / ctas;
-    int gmax = ctx->fwd_group > 0 ? ctx->fwd_group / ctas : n_pairs / 4;
+    FwdPlanParams p;
+    p.n_pairs = ctx->sm_count / ctas;
+    p.tile_rows = gemm_tile_rows(ctas);
+    p.n_tiles = (V + kTileN - 1) / kTileN;
+    int gmax = ctx->fwd_group > 0 ? ctx->fwd_group / ctas : p.n_pairs / 4;
     if (gmax < 1) gmax = 1;
-    if (gmax > n_pairs) gmax = n_pairs;
-    auto splits_for = [&](int tiles) {
-        int sp = n_pairs / (tiles > 0 ? tiles : 1);
-        if (sp > 32) sp = 32;
-        if (sp > n_tiles) sp = n_tiles;
-        return sp < 1 ? 1 : sp;
-    };
-    auto ceil_div = [](int a, int b) { return (a + b - 1) / b; };
-    // Among round sizes from two thirds of gmax up to gmax, take the one with the least work per worker: vocabulary
-    // tiles per split, summed over the rounds, the last of which may hold fewer row tiles and then cuts the vocabulary
-    // into more splits (a batch whose row tiles do not divide well would otherwise idle part of the machine in its
-    // last round); ties go to the larger round, which streams W less often.
-    FwdShape best;
-    long long best_cost = -1;
-    const int cand_min = m_tiles <= gmax ? 1 : (2 * gmax + 2) / 3;      // few row tiles: any round size is L2-safe
-    for (int cand = gmax; cand >= cand_min; --cand) {
-        const int c = cand < m_tiles ? cand : (m_tiles > 0 ? m_tiles : 1);
-        const int sp = splits_for(c);
-        const int full_rounds = m_tiles / c, rest = m_tiles - full_rounds * c;
-        const int sp_last = rest > 0 ? splits_for(rest) : sp;
-        const long long cost = static_cast<long long>(full_rounds) * ceil_div(n_tiles, sp) + (rest > 0 ? ceil_div(n_tiles, sp_last) : 0);
-        if (best_cost < 0 || cost < best_cost) {
-            best_cost = cost;
-            best.gm = c;
-            best.tps = ceil_div(n_tiles, sp);
-            best.splits = ceil_div(n_tiles, best.tps);
-            best.last_m0 = rest > 0 && sp_last != sp ? full_rounds * c : m_tiles;
-            best.last_tps = ceil_div(n_tiles, sp_last);
-            best.last_splits = ceil_div(n_tiles, best.last_tps);
-        }
-    }
-    if (best_cost < 0) { best.gm = 1; best.splits = 1; best.tps = n_tiles; best.last_m0 = m_tiles; best.last_splits = 1; best.last_tps = n_tiles; }
-    const long long last_rows = static_cast<long long>(m_tiles - best.last_m0) * tile_rows;
-    best.stats_rows = static_cast<long long>(best.splits) * rows + best.last_splits * last_rows;
-    return best;
+    if (gmax > p.n_pairs) gmax = p.n_pairs;
+    p.gmax = gmax;
+    return p;
 }
 
 // Optional stash of the scaled logits written by the forward kernel (see GemmArgs::Z).
@@ -319,110 +284,88 @@ struct ZStash {
     int chunk_cols, chunks;
 };
 
-// LM-head GEMM + online softmax statistics for packed rows [slot0, slot0 + rows) of one model; statistics go to
-// stats[split * rows + (slot - slot0)].
-int launch_forward(unity_ctx* ctx, const unity_rows* r, int slot0, int rows, float4* stats, const int* target_p,
-                   const CUtensorMap& tmA, const CUtensorMap& tmB, const ZStash* z, FwdShape* shape_out) {
+// LM-head GEMM + online softmax statistics for the rows of `span` (a whole model, or one block of its rows).  The
+// kernel derives rows, rounds and splits from the device plan; statistics go to stats (+ the model's base with
+// `stats_from_plan`) as [split][row - first row of the span].
+int launch_forward(unity_ctx* ctx, const unity_rows* r, RowPlan& P, const RowSpan& span, bool stats_from_plan,
+                   const CUtensorMap& tmA, const CUtensorMap& tmB, const ZStash* z) {
     const int ctas = ctx->ctas[UNITY_PROF_FWD_GEMM];
-    const FwdShape fs = forward_shape(ctx, r->V, rows);
-    *shape_out = fs;
     GemmArgs g;
     memset(&g, 0, sizeof(g));
-    g.m_tiles = rows / gemm_tile_rows(ctas); g.n_tiles = (r->V + kTileN - 1) / kTileN; g.k_iters = r->H / kTileK;
-    g.group_m = fs.gm;
-    g.a_row0 = slot0; g.b_row0 = 0; g.a_k0 = 0; g.b_k0 = 0;
-    g.m_rows = rows; g.n_cols = r->V;
-    g.n_splits = fs.splits; g.tiles_per_split = fs.tps;
-    g.last_m0 = fs.last_m0; g.last_splits = fs.last_splits; g.last_tiles_per_split = fs.last_tps;
-    g.last_stats_off = static_cast<long long>(fs.splits) * rows;
-    g.last_pitch = rows - static_cast<long long>(fs.last_m0) * gemm_tile_rows(ctas);
-    g.stats = stats; g.stats_pitch = rows;
-    g.target_p = target_p; g.vocab0 = 0; g.scale = r->inv_temperature;
+    g.span = span; g.span_mode = kSpanForward; g.stats_from_plan = stats_from_plan ? 1 : 0; g.fwd = P.fwd;
+    g.m_tiles = 1;                                   // set by the kernel
+    g.n_tiles = (r->V + kTileN - 1) / kTileN; g.k_iters = r->H / kTileK;
+    g.b_row0 = 0; g.a_k0 = 0; g.b_k0 = 0;
+    g.n_cols = r->V;
+    g.stats = P.L.stats;
+    g.target_p = P.L.target_p; g.vocab0 = 0; g.scale = r->inv_temperature;
     if (z) {
         g.Z = z->Z; g.ldz = z->ldz; g.z_chunk_stride = z->chunk_stride; g.z_chunk_cols = z->chunk_cols; g.z_chunks = z->chunks;
         g.g_wide_store = (reinterpret_cast<uintptr_t>(z->Z) % 32 == 0) && (z->ldz * 2 % 32 == 0) && (z->chunk_stride * 2 % 32 == 0) &&
                          (z->chunk_cols * 2 % 32 == 0);
     }
-    gemm_common(ctx, g, UNITY_PROF_FWD_GEMM, kEpiSoftmaxStats, ctx->fwd_sync != 0);
+    gemm_common(ctx, g, UNITY_PROF_FWD_GEMM, &P.counters, ctx->fwd_sync != 0);
     ProfScope ps(ctx, UNITY_PROF_FWD_GEMM);
     CUDA_TRY(ctx, launch_gemm(kEpiSoftmaxStats, false, ctas, tmA, tmB, g, ctx->sm_count, ctx->stream));
     return UNITY_OK;
 }
+
+// Padded rows of model k as far as the host knows: the exact number when it read the counts back, else the bound.
+long long rows_of(const RowPlan& P, int k) { return P.rows_known[k] >= 0 ? P.rows_known[k] : P.rows_bound; }
 
 // Routing, packing and the forward sweep: fills per-split softmax statistics for every packed row.
 int forward_sweep(unity_ctx* ctx, const unity_rows* r, RowPlan& P, bool run_gemm = true) {
     const Layout& L = P.L;
     cudaStream_t st = ctx->stream;
     int nl = 0;
+    P.fwd = fwd_params(ctx, r->V);
+    P.counters = SyncCounters{L.sync_counters, 0, kSyncCounters};
+    P.rows_bound = static_cast<long long>(up(r->n_tok, kTileM));
+    for (int k = 0; k < UNITY_MAX_MODELS; ++k) P.rows_known[k] = -1;
     CUDA_TRY(ctx, cudaMemsetAsync(L.slot_tok, 0xff, sizeof(int) * L.max_slots, st));
+    CUDA_TRY(ctx, cudaMemsetAsync(L.sync_counters, 0, sizeof(unsigned) * kSyncCounters, st));
     RouteArgs ra;
     memset(&ra, 0, sizeof(ra));
     ra.n_tok = r->n_tok; ra.n_inv = r->n_inv; ra.n_roles = r->n_roles; ra.K = r->K; ra.V = r->V;
     ra.cu_seqlens = r->cu_seqlens; ra.inv_role = r->inv_role; ra.target = r->target; ra.tok_mask = r->tok_mask;
     for (int v = 0; v < r->n_roles; ++v) ra.role_model[v] = r->role_model[v];
-    ra.n_blocks = L.n_blocks; ra.blk_cnt = L.blk_cnt; ra.counts = L.counts; ra.offsets = L.offsets;
+    ra.n_blocks = L.n_blocks; ra.blk_cnt = L.blk_cnt; ra.plan = L.plan; ra.fwd = P.fwd;
     ra.tok_slot = L.tok_slot; ra.slot_tok = L.slot_tok; ra.tok_model = L.tok_model; ra.status = ctx->d_status;
     CUDA_TRY(ctx, launch_route(ra, st, &nl));
-    CUDA_TRY(ctx, cudaMemcpyAsync(ctx->h_pinned, L.counts, sizeof(int) * UNITY_MAX_MODELS, cudaMemcpyDeviceToHost, st));
-    CUDA_TRY(ctx, cudaStreamSynchronize(st));
-    int off = 0;
-    for (int k = 0; k < r->K; ++k) {
-        P.counts[k] = ctx->h_pinned[k];
-        P.offsets[k] = off;
-        off += static_cast<int>(up(P.counts[k], kTileM));
+    if (ctx->host_counts) {
+        // optional: the host learns the K row counts (a few bytes, one synchronisation) and skips empty launches
+        CUDA_TRY(ctx, cudaMemcpyAsync(ctx->h_pinned, L.plan, sizeof(int) * UNITY_MAX_MODELS, cudaMemcpyDeviceToHost, st));
+        CUDA_TRY(ctx, cudaStreamSynchronize(st));
+        for (int k = 0; k < r->K; ++k) P.rows_known[k] = static_cast<int>(up(ctx->h_pinned[k], kTileM));
     }
-    P.offsets[r->K] = off;
-    P.n_slots = off;
-
-    CUDA_TRY(ctx, launch_gather_rows(static_cast<const __nv_bfloat16*>(r->hidden), r->target, L.slot_tok, P.n_slots,
-                                     r->H, L.hp, L.target_p, st));
-    nl += P.n_slots > 0;
+    CUDA_TRY(ctx, launch_gather_rows(static_cast<const __nv_bfloat16*>(r->hidden), r->target, L.slot_tok, L.plan, r->K,
+                                     L.max_slots, r->H, L.hp, L.target_p, st));
+    nl += 1;
 
     CUtensorMap tmA;
-    if (P.n_slots > 0) {
-        int rc = make_tmap(ctx, &tmA, L.hp, r->H, P.n_slots, static_cast<uint64_t>(r->H) * 2, kBoxRows);
-        if (rc) return rc;
-    }
-    long long sbase = 0;
-    for (int k = 0; k < r->K; ++k) {
-        memset(&P.shape[k], 0, sizeof(FwdShape));
-        P.shape[k].splits = P.shape[k].last_splits = 1;
-        P.shape[k].last_m0 = 0x3fffffff;
-        P.stats_base[k] = sbase;
-        const int rows_k = P.offsets[k + 1] - P.offsets[k];
-        if (rows_k == 0 || !run_gemm) continue;
+    int rc = make_tmap(ctx, &tmA, L.hp, r->H, L.max_slots, static_cast<uint64_t>(r->H) * 2, kBoxRows);
+    if (rc) return rc;
+    for (int k = 0; k < r->K && run_gemm; ++k) {
+        if (rows_of(P, k) == 0) continue;
         CUtensorMap tmB;
-        int rc = make_tmap(ctx, &tmB, r->W[k], r->H, r->V, static_cast<uint64_t>(r->H) * 2, kTileN / ctx->ctas[UNITY_PROF_FWD_GEMM]);
+        rc = make_tmap(ctx, &tmB, r->W[k], r->H, r->V, static_cast<uint64_t>(r->H) * 2, kTileN / ctx->ctas[UNITY_PROF_FWD_GEMM]);
         if (rc) return rc;
-        if (sbase + forward_shape(ctx, r->V, rows_k).stats_rows > L.stats_cap)
-            return fail(ctx, UNITY_ERR_WORKSPACE, "internal: statistics scratch too small");
-        rc = launch_forward(ctx, r, P.offsets[k], rows_k, L.stats + sbase, L.target_p, tmA, tmB, nullptr, &P.shape[k]);
+        const RowSpan whole{L.plan, k, 0, 0x7fffff00};
+        rc = launch_forward(ctx, r, P, whole, true, tmA, tmB, nullptr);
         if (rc) return rc;
-        sbase += P.shape[k].stats_rows;
         nl += 1;
     }
     ctx->launches += nl;
     return UNITY_OK;
 }
 
-// Where k_finish_rows finds the per-split statistics of model k's rows (see launch_forward).
-void set_token_stats(TokenArgs& t, int k, long long base, const FwdShape& fs, int rows, int tile_rows) {
-    t.stats_base[k] = base;
-    t.model_splits[k] = fs.splits;
-    const long long last_row0 = static_cast<long long>(fs.last_m0) * tile_rows;
-    t.last_row0[k] = last_row0 < rows ? static_cast<int>(last_row0) : 0x7fffffff;
-    t.last_splits[k] = fs.last_splits;
-    t.stats_last[k] = base + static_cast<long long>(fs.splits) * rows;
-}
-
-void fill_token_args(TokenArgs& t, const unity_ctx* ctx, const unity_rows* r, const RowPlan& P) {
+void fill_token_args(TokenArgs& t, const unity_rows* r, const RowPlan& P) {
     memset(&t, 0, sizeof(t));
     const Layout& L = P.L;
-    t.n_slots = P.n_slots; t.K = r->K; t.n_roles = r->n_roles; t.n_inv = r->n_inv; t.n_tok = r->n_tok;
+    t.block = RowSpan{L.plan, -1, 0, 0};
+    t.plan = L.plan; t.fwd = P.fwd; t.max_slots = L.max_slots;
+    t.K = r->K; t.n_roles = r->n_roles; t.n_inv = r->n_inv; t.n_tok = r->n_tok;
     t.stats = L.stats;
-    const int tile_rows = gemm_tile_rows(ctx->ctas[UNITY_PROF_FWD_GEMM]);
-    for (int k = 0; k < r->K; ++k) set_token_stats(t, k, P.stats_base[k], P.shape[k], P.offsets[k + 1] - P.offsets[k], tile_rows);
-    for (int k = 0; k <= r->K; ++k) t.offsets[k] = P.offsets[k];
     t.slot_tok = L.slot_tok; t.tok_slot = L.tok_slot; t.tok_model = L.tok_model;
     t.scale = r->inv_temperature;
     t.row_lse = L.row_lse; t.row_ent = L.row_ent; t.row_logp = L.row_logp;
@@ -481,6 +424,7 @@ int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace
     c->l2_hints[UNITY_PROF_DW_GEMM] = 0;
     c->logit_stash = 0;
     c->chunk_sync_period[0] = c->chunk_sync_period[1] = c->chunk_sync_period[2] = 1;
+    c->host_counts = 1;
     c->wait_budget = kWaitBudgetCycles;
     c->test_drop = 0;
     c->ev_pool = new (std::nothrow) std::vector<cudaEvent_t>();
@@ -557,13 +501,7 @@ int unity_check_status(unity_ctx* ctx) {
     CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof(int), ctx->stream));
     CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream));
     const int bits = ctx->h_pinned[512];
-    if (bits & kStatusTimeout) {
-        // workers that gave up did not finish their rounds: start the round rendezvous afresh (the stream is idle)
-        CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_status + 16, 0, sizeof(unsigned), ctx->stream));
-        CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream));
-        ctx->round_total = 0;
-        return fail(ctx, UNITY_ERR_TIMEOUT, "a bounded in-kernel wait expired");
-    }
+    if (bits & kStatusTimeout) return fail(ctx, UNITY_ERR_TIMEOUT, "a bounded in-kernel wait expired");
     if (bits & kStatusBadIndex) return fail(ctx, UNITY_ERR_BAD_INDEX, "an index in the data was out of range (row / invocation masked)");
     return UNITY_OK;
 }
@@ -603,6 +541,7 @@ int unity_set_option(unity_ctx* ctx, int option, int value) {
         ctx->chunk_sync_period[option - UNITY_OPT_SYNC_PERIOD_GRAD] = value;
         return UNITY_OK;
     }
+    if (option == UNITY_OPT_HOST_COUNTS && (value == 0 || value == 1)) { ctx->host_counts = value; return UNITY_OK; }
     if (option == UNITY_OPT_WAIT_KCYCLES && value >= 1) {
         ctx->wait_budget = static_cast<long long>(value) * 1000;
         if (ctx->wait_budget > 1000000) ctx->test_drop = 0;      // the test hook lives only under a short bound
@@ -873,7 +812,7 @@ int unity_logprob_fwd(unity_ctx* ctx, const unity_rows* rows, float* logp, float
     rc = forward_sweep(ctx, rows, P);
     if (rc) return rc;
     TokenArgs t;
-    fill_token_args(t, ctx, rows, P);
+    fill_token_args(t, rows, P);
     t.logp = logp; t.entropy = entropy; t.lse = lse;
     int nl = 0;
     CUDA_TRY(ctx, launch_finish_forward(t, false, st, &nl));
@@ -950,14 +889,14 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
     int nl = 0;
 
     TokenArgs t;
-    fill_token_args(t, ctx, rows, P);
+    fill_token_args(t, rows, P);
     t.logp = logp; t.entropy = entropy; t.lse = nullptr;
     if (have_fwd) { t.logp_in = params->logp_in; t.entropy_in = params->entropy_in; t.lse_in = params->lse_in; }
     t.old_logp = old_logp; t.ref_logp = ref_logp; t.adv_tok = adv_tok;
     t.clip_lo = params->clip_lo; t.clip_hi = params->clip_hi; t.kl_coef = params->kl_coef;
     t.ent_coef = params->ent_coef; t.kl_mode = params->kl_mode;
-    for (int k = 0; k < K; ++k)
-        t.norm[k] = params->norm ? params->norm[k] : static_cast<float>(P.counts[k] > 0 ? P.counts[k] : 1);
+    t.has_norm = params->norm != nullptr;
+    for (int k = 0; k < K && params->norm; ++k) t.norm[k] = params->norm[k];
     t.coef_a = L.coef_a; t.coef_b = L.coef_b; t.tok_loss = tok_loss;
     t.inv_sums = L.inv_sums; t.loss = loss; t.metrics = metrics;
     if (!stash) CUDA_TRY(ctx, launch_finish_forward(t, true, st, &nl));
@@ -968,10 +907,8 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
     // Operands are read in place: hidden rows and W serve as K-major operands (contraction over H) and as
     // MN-major operands (contraction over tokens / vocabulary); nothing is transposed in memory.
     CUtensorMap tm_hp_k, tm_hp_mn;
-    if (P.n_slots > 0) {
-        if ((rc = make_tmap(ctx, &tm_hp_k, L.hp, H, P.n_slots, static_cast<uint64_t>(H) * 2, kBoxRows))) return rc;
-        if ((rc = make_tmap(ctx, &tm_hp_mn, L.hp, H, P.n_slots, static_cast<uint64_t>(H) * 2, kTileK))) return rc;
-    }
+    if ((rc = make_tmap(ctx, &tm_hp_k, L.hp, H, L.max_slots, static_cast<uint64_t>(H) * 2, kBoxRows))) return rc;
+    if ((rc = make_tmap(ctx, &tm_hp_mn, L.hp, H, L.max_slots, static_cast<uint64_t>(H) * 2, kTileK))) return rc;
     // Tiles two blocks wide unless one-block tiles waste clearly less of this launch: the share of executed MMA work that
     // is useful = (H / padded columns) x (tiles / tiles rounded up to whole waves of CTA pairs); the wide form gets a
     // 15 % bonus for its lower operand traffic (at H = 896 the narrow form is bound by the stream of G, not by MMA time:
@@ -991,31 +928,32 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
     const int c_grad = ctx->ctas[UNITY_PROF_GRAD_GEMM], c_dh = ctx->ctas[UNITY_PROF_DH_GEMM],
               c_dw = ctx->ctas[UNITY_PROF_DW_GEMM];
 
+    // The host does not know how many rows a model has (unless it was asked to read the counts back): it walks every
+    // chunk a model could have, each kernel cuts its span to the rows that exist, and a launch without rows returns at once.
     for (int k = 0; k < K; ++k) {
-        const int rows_k = P.offsets[k + 1] - P.offsets[k];
+        const long long rows_k = rows_of(P, k);
         float* dWk = static_cast<float*>(dW[k]);
-        if (rows_k == 0) {
-            if (!params->accumulate_dW) CUDA_TRY(ctx, cudaMemsetAsync(dWk, 0, sizeof(float) * V * H, st));
-            continue;
+        // nothing accumulates into the dW of a model without rows: it must still read zero
+        if (!params->accumulate_dW) {
+            if (rows_k == 0) CUDA_TRY(ctx, cudaMemsetAsync(dWk, 0, sizeof(float) * V * H, st));
+            else if (P.rows_known[k] < 0) { CUDA_TRY(ctx, launch_zero_if_empty(dWk, static_cast<long long>(V) * H, L.plan, k, st)); nl += 1; }
         }
+        if (rows_k == 0) continue;
         const __nv_bfloat16* Wk = static_cast<const __nv_bfloat16*>(rows->W[k]);
         CUtensorMap tm_W_k, tm_W_mn, tm_W_f;
         if ((rc = make_tmap(ctx, &tm_W_k, Wk, H, V, static_cast<uint64_t>(H) * 2, kTileN / c_grad))) return rc;
         if (stash && (rc = make_tmap(ctx, &tm_W_f, Wk, H, V, static_cast<uint64_t>(H) * 2, kTileN / ctx->ctas[UNITY_PROF_FWD_GEMM]))) return rc;
         if ((rc = make_tmap(ctx, &tm_W_mn, Wk, H, V, static_cast<uint64_t>(H) * 2, kTileK))) return rc;
 
-        for (int c0 = 0; c0 < rows_k; c0 += cr) {
-            const int nc = rows_k - c0 < cr ? rows_k - c0 : cr;          // multiple of kTileM
-            const int slot0 = P.offsets[k] + c0;
+        for (long long c0 = 0; c0 < rows_k; c0 += cr) {
+            const int nc = static_cast<int>(rows_k - c0 < cr ? rows_k - c0 : cr);   // at most this many rows (multiple of kTileM)
+            const RowSpan chunk{L.plan, k, static_cast<int>(c0), nc};
             if (stash) {
                 // forward over this block of rows, keeping its logits; then the per-row loss terms of the block
                 const ZStash z{L.G, cv, static_cast<long long>(cr) * cv, z_base, z_chunks};
-                FwdShape fs;
-                if ((rc = launch_forward(ctx, rows, slot0, nc, L.stats, L.target_p, tm_hp_k, tm_W_f, &z, &fs))) return rc;
+                if ((rc = launch_forward(ctx, rows, P, chunk, false, tm_hp_k, tm_W_f, &z))) return rc;
                 TokenArgs tc = t;
-                tc.slot_begin = slot0; tc.n_slots = slot0 + nc;
-                tc.offsets[k] = slot0; tc.offsets[k + 1] = slot0 + nc;
-                set_token_stats(tc, k, 0, fs, nc, gemm_tile_rows(ctx->ctas[UNITY_PROF_FWD_GEMM]));
+                tc.block = chunk;
                 CUDA_TRY(ctx, launch_finish_rows(tc, true, st, &nl));
                 nl += 1;
             }
@@ -1030,7 +968,7 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                 if (stash) {
                     LogitGradArgs lg;
                     memset(&lg, 0, sizeof(lg));
-                    lg.Z = Gc; lg.ld = cv; lg.rows = nc; lg.cols = vc; lg.row0 = slot0; lg.vocab0 = v0;
+                    lg.Z = Gc; lg.ld = cv; lg.span = chunk; lg.cols = vc; lg.vocab0 = v0;
                     lg.target_p = L.target_p; lg.coef_a = L.coef_a; lg.coef_b = L.coef_b;
                     lg.row_lse = L.row_lse; lg.row_ent = L.row_ent;
                     ProfScope ps(ctx, UNITY_PROF_GRAD_GEMM);
@@ -1047,62 +985,68 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                             if (vc - (q0 + qc) <= tail) qc = vc - q0;
                             GemmArgs g;
                             memset(&g, 0, sizeof(g));
-                            g.m_tiles = nr / gemm_tile_rows(c_grad); g.n_tiles = (qc + kTileN - 1) / kTileN; g.k_iters = H / kTileK;
+                            g.span = RowSpan{L.plan, k, static_cast<int>(c0) + r0, nr}; g.span_mode = kSpanRowsA;
+                            g.m_tiles = 1;                                   // set by the kernel
+                            g.n_tiles = (qc + kTileN - 1) / kTileN; g.k_iters = H / kTileK;
                             g.group_m = ctx->chunk_group[0] / c_grad > 0 ? ctx->chunk_group[0] / c_grad : 1;
-                            g.a_row0 = slot0 + r0; g.b_row0 = v0 + q0; g.m_rows = nr; g.n_cols = qc;
+                            g.a_row0 = 0; g.b_row0 = v0 + q0; g.n_cols = qc;
                             g.target_p = L.target_p; g.vocab0 = v0 + q0; g.scale = rows->inv_temperature;
                             g.coef_a = L.coef_a; g.coef_b = L.coef_b; g.row_lse = L.row_lse; g.row_ent = L.row_ent;
                             g.has_ent = params->ent_coef != 0.f;
                             g.G = Gc + static_cast<long long>(r0) * cv + q0; g.ldg = cv;
                             g.g_wide_store = (reinterpret_cast<uintptr_t>(g.G) % 32 == 0) && (g.ldg * 2 % 32 == 0);
-                            gemm_common(ctx, g, UNITY_PROF_GRAD_GEMM, kEpiLogitGrad, (ctx->chunk_sync & 1) != 0);
+                            gemm_common(ctx, g, UNITY_PROF_GRAD_GEMM, &P.counters, (ctx->chunk_sync & 1) != 0);
                             ProfScope ps(ctx, UNITY_PROF_GRAD_GEMM);
                             CUDA_TRY(ctx, launch_gemm(kEpiLogitGrad, false, c_grad, tm_hp_k, tm_W_k, g, ctx->sm_count, st));
                             nl += 1;
                         }
                     }
                 }
-                // G viewed as [nc rows, vc]: K-major A for dHidden (contract over vc), MN-major A for dW (rows = K)
+                // G viewed as [rows, vc]: K-major A for dHidden (contract over vc), MN-major A for dW (rows = K)
                 CUtensorMap tm_G_k, tm_G_mn;
                 if ((rc = make_tmap(ctx, &tm_G_k, Gc, vc, nc, static_cast<uint64_t>(cv) * 2, kBoxRows))) return rc;
                 if ((rc = make_tmap(ctx, &tm_G_mn, Gc, vc, nc, static_cast<uint64_t>(cv) * 2, kTileK))) return rc;
-                // (2) dH_chunk[nc, H] (+)= G[nc, vc] * W[v0:v0+vc, :]      (B = W, MN-major: rows v are K)
+                // (2) dH_chunk[rows, H] (+)= G[rows, vc] * W[v0:v0+vc, :]      (B = W, MN-major: rows v are K)
                 GemmArgs h;
                 memset(&h, 0, sizeof(h));
                 const bool wide_dh = pick_wide(UNITY_PROF_DH_GEMM, nc / gemm_tile_rows(c_dh));
                 const int mma_n = gemm_mma_n(H);                       // dHidden and dW both have H output columns
                 const int cols_dh = (wide_dh ? 2 : 1) * mma_n;
                 h.mma_n = mma_n;
-                h.m_tiles = nc / gemm_tile_rows(c_dh); h.n_tiles = (H + cols_dh - 1) / cols_dh;
+                h.span = chunk; h.span_mode = kSpanRowsM;
+                h.m_tiles = 1;                                         // set by the kernel
+                h.n_tiles = (H + cols_dh - 1) / cols_dh;
                 h.k_iters = (vc + kTileK - 1) / kTileK;
                 h.group_m = ctx->chunk_group[1] / c_dh > 0 ? ctx->chunk_group[1] / c_dh : 1;
-                h.a_row0 = 0; h.a_k0 = 0; h.b_row0 = 0; h.b_k0 = v0; h.m_rows = nc; h.n_cols = H;
+                h.a_row0 = 0; h.a_k0 = 0; h.b_row0 = 0; h.b_k0 = v0; h.n_cols = H;
                 h.C = L.dHc; h.ldc = H; h.beta = v0 > 0;
-                gemm_common(ctx, h, UNITY_PROF_DH_GEMM, kEpiAccumF32, (ctx->chunk_sync & 2) != 0);
+                gemm_common(ctx, h, UNITY_PROF_DH_GEMM, &P.counters, (ctx->chunk_sync & 2) != 0);
                 {
                     ProfScope ps(ctx, UNITY_PROF_DH_GEMM);
                     CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, false, c_dh, tm_G_k, tm_W_mn, h, ctx->sm_count, st, wide_dh));
                 }
-                // (3) dW[v0:v0+vc, :] (+)= G^T[vc, nc] * hidden[slot0:slot0+nc, :]   (both operands MN-major)
+                // (3) dW[v0:v0+vc, :] (+)= G^T[vc, rows] * hidden[first slot of the chunk ..., :]   (both operands MN-major)
                 GemmArgs w;
                 memset(&w, 0, sizeof(w));
                 w.m_tiles = (vc + gemm_tile_rows(c_dw) - 1) / gemm_tile_rows(c_dw);
                 const bool wide_dw = pick_wide(UNITY_PROF_DW_GEMM, w.m_tiles);
                 const int cols_dw = (wide_dw ? 2 : 1) * mma_n;
                 w.mma_n = mma_n;
-                w.n_tiles = (H + cols_dw - 1) / cols_dw; w.k_iters = nc / kTileK;
+                w.span = chunk; w.span_mode = kSpanRowsK;
+                w.n_tiles = (H + cols_dw - 1) / cols_dw;
+                w.k_iters = 1;                                         // set by the kernel
                 w.group_m = ctx->chunk_group[2] / c_dw > 0 ? ctx->chunk_group[2] / c_dw : 1;
-                w.a_row0 = 0; w.a_k0 = 0; w.b_row0 = 0; w.b_k0 = slot0; w.m_rows = vc; w.n_cols = H;
+                w.a_row0 = 0; w.a_k0 = 0; w.b_row0 = 0; w.b_k0 = 0; w.m_rows = vc; w.n_cols = H;
                 w.C = dWk + static_cast<long long>(v0) * H; w.ldc = H;
                 w.beta = (params->accumulate_dW || c0 > 0) ? 1 : 0;
-                gemm_common(ctx, w, UNITY_PROF_DW_GEMM, kEpiAccumF32, (ctx->chunk_sync & 4) != 0);
+                gemm_common(ctx, w, UNITY_PROF_DW_GEMM, &P.counters, (ctx->chunk_sync & 4) != 0);
                 {
                     ProfScope ps(ctx, UNITY_PROF_DW_GEMM);
                     CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, true, c_dw, tm_G_mn, tm_hp_mn, w, ctx->sm_count, st, wide_dw));
                 }
                 nl += 2;
             }
-            CUDA_TRY(ctx, launch_store_dhidden(L.dHc, L.slot_tok, slot0, nc, H, dH, st));
+            CUDA_TRY(ctx, launch_store_dhidden(L.dHc, L.slot_tok, chunk, H, dH, st));
             nl += 1;
         }
     }

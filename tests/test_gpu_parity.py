@@ -384,6 +384,56 @@ def test_small_shapes_and_ragged_tails(H, V, rows):
     run_all_stages(small_workload(H, V, rows))
 
 
+@pytest.mark.parametrize("name", ["tiny", "search", "stress"])
+def test_fully_asynchronous_calls_match_the_oracle(name):
+    # UNITY_OPT_HOST_COUNTS = 0: the host never learns the row counts, walks every chunk a model could have and the
+    # kernels cut their spans on the device (most launches of a model with few rows return at once)
+    w = wl.make(name, device="cuda", **({} if name == "tiny" else dict(cut_rows=1200, cut_max_len=64)))
+    run_all_stages(w, options=[(ub.OPT_HOST_COUNTS, 0)])
+    if name == "stress":
+        run_all_stages(w, options=[(ub.OPT_HOST_COUNTS, 0), (ub.OPT_LOGIT_STASH, 1)])
+
+
+def test_asynchronous_calls_return_while_the_stream_is_busy():
+    """With UNITY_OPT_HOST_COUNTS = 0 neither call waits for the device: behind a kernel that keeps the stream busy for
+    about a quarter of a second, both calls return long before it ends; with the default the forward call returns
+    only after it (the one synchronisation that reads the row counts)."""
+    import time
+    w = small_workload(128, 2048, 600)
+    d = pu.DeviceInputs(w)
+    ctx = pu.make_ctx(w)
+    n = w.n_tok
+    logp = torch.empty(n, device="cuda")
+    old = torch.full((n,), -7.0, device="cuda")
+    adv = torch.ones(n, device="cuda")
+    loss = torch.empty(w.K, device="cuda")
+    dH = torch.empty(n, w.H, device="cuda", dtype=torch.bfloat16)
+    dW = [torch.empty(w.V, w.H, device="cuda") for _ in range(w.K)]
+
+    def calls():
+        ctx.logprob_fwd(d.hidden, d.W, d.cu_seqlens, d.inv_role, w.role_model.tolist(), d.target, d.tok_mask, 1.0, logp)
+        ctx.ppo_loss_fwd_bwd(d.hidden, d.W, d.cu_seqlens, d.inv_role, w.role_model.tolist(), d.target, d.tok_mask, 1.0, 0.2,
+                             0.2, 0.01, 3, 0.0, None, False, old, old, adv, loss, None, None, None, None, dH, dW)
+
+    calls()                                        # warm-up
+    torch.cuda.synchronize()
+    spin = 500_000_000                             # SM clocks: about 0.25 s at 1.9 GHz
+    seen = {}
+    for mode in (0, 1):
+        ctx.set_option(ub.OPT_HOST_COUNTS, mode)
+        torch.cuda._sleep(spin)
+        t0 = time.perf_counter()
+        calls()
+        seen[mode] = time.perf_counter() - t0
+        busy_after = not torch.cuda.current_stream().query()
+        torch.cuda.synchronize()
+        if mode == 0:
+            assert busy_after
+    ctx.check_status()
+    assert seen[0] < 0.1 and seen[1] > 0.15, seen
+    ctx.close()
+
+
 @pytest.mark.parametrize("rows,valid,ctas", [(7700, 6289, 2), (7700, 6289, 1), (15400, 12326, 2)])
 def test_forward_rounds_with_a_short_last_round(rows, valid, ctas):
     # 6289 valid rows = 25 row tiles of 256 (or 50 of 128): one full round of 24 (48) row tiles x 3 splits and a last
