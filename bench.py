@@ -249,9 +249,8 @@ def measure_streaming():
     t_gat = timed(lambda: ctx.ready_batch_gather(order, cu, out_cu, totals, rewards, r_out, 0.0))
     kept_tok = int(totals[1].item())
     ctx.check_status()
-    # Host-side cost of the one synchronisation inside unity_logprob_fwd / unity_ppo_loss_fwd_bwd (the K row counts are
-    # read back to size the grouped launches): on the smallest configuration, how long the call keeps the host (it
-    # returns once everything is enqueued) and how long until the result is complete.
+    # Host side of unity_logprob_fwd on the smallest configuration: how long the call keeps the host (it returns once
+    # everything is enqueued; nothing in it synchronises) and how long until the result is complete.
     wt = wl.make("tiny", device=dev)
     cxt = ub.Context(0, ub.unity_workspace_bytes(wt.n_tok, wt.H, wt.V, wt.K, wt.n_inv))
     t_cu, t_role, t_tgt, t_mask = wt.cu_seqlens.to(dev), wt.inv_role.to(dev), wt.target.to(dev), wt.tok_mask.to(dev)
@@ -283,8 +282,8 @@ def measure_streaming():
            "ready_batch_gather_f32": {"ms": t_gat, "algorithmic_bytes": 8 * kept_tok, "gbs": 8 * kept_tok / t_gat / 1e6},
            "ready_batch_plan": {"ms": t_plan, "note": "latency-bound: four small launches over the invocations"},
            "logprob_fwd_tiny_host": {"call_returns_after_us": ret_us[len(ret_us) // 2], "complete_after_us": done_us[len(done_us) // 2],
-                                     "note": "median of 20 calls on the tiny configuration; by default the call synchronises the stream "
-                                             "once, after the routing kernels, to read K row counts (UNITY_OPT_HOST_COUNTS)"}}
+                                     "note": "median of 20 calls on the tiny configuration; the call is asynchronous (no stream "
+                                             "synchronisation; UNITY_OPT_HOST_COUNTS = 0)"}}
     for k in ("role_advantage", "device_fill_f32", "gae", "value_loss", "align_rewards", "ready_batch_gather_f32"):
         out[k]["frac"] = out[k]["gbs"] / peaks["hbm_gbs"]
     ctx.close()

@@ -9,11 +9,12 @@
  *   throws, aborts or traps.  unity_last_error() gives a text for the last failure of a context.
  * - Unless marked (host), data pointers are DEVICE pointers owned by the caller; the library never
  *   frees or keeps them beyond the call.  Arrays marked (host) are read during the call.
- * - Work is enqueued on the stream given to unity_create.  By default unity_logprob_fwd and
- *   unity_ppo_loss_fwd_bwd synchronise that stream once, early, to read the K per-model row counts
- *   (a few bytes) and skip launches that would be empty; with UNITY_OPT_HOST_COUNTS = 0 they never
- *   synchronise.  Everything else is asynchronous.  Device-side errors (bad indices in the data, a
- *   bounded wait that expired) are sticky in a status word read by unity_check_status.
+ * - Work is enqueued on the stream given to unity_create and every call is asynchronous: the only
+ *   calls that synchronise are unity_check_status, unity_get_profile and unity_destroy (and, when
+ *   UNITY_OPT_HOST_COUNTS is set to 1, unity_logprob_fwd and unity_ppo_loss_fwd_bwd, once each, to
+ *   read the K per-model row counts and skip launches that would be empty).  Device-side errors
+ *   (bad indices in the data, a bounded wait that expired) are sticky in a status word read by
+ *   unity_check_status.
  * - The library allocates no device memory per call: all scratch lives in the caller's workspace.
  * - Rows with tok_mask == 0 receive 0 in every per-token output and cost no tensor work.
  * - Limits: 1 <= K <= UNITY_MAX_MODELS, 1 <= n_roles <= UNITY_MAX_ROLES, H % 64 == 0, V % 8 == 0,
@@ -116,10 +117,10 @@ int unity_set_profiling(unity_ctx* ctx, int enable);
 #define UNITY_OPT_SYNC_PERIOD_DH 23   /* UNITY_OPT_CHUNK_SYNC); 1 = every tile                                                  */
 #define UNITY_OPT_SYNC_PERIOD_DW 24
 #define UNITY_OPT_HOST_COUNTS 25    /* The kernels of unity_logprob_fwd and unity_ppo_loss_fwd_bwd read the per-model row counts on the
-                                     device.  1 (default): the host reads the K counts back as well (one stream synchronisation
-                                     after the routing kernels) and skips the launches that would be empty.  0: the calls never
-                                     synchronise; the host walks every chunk a model could have and a launch without rows returns
-                                     at once (0.3-0.6 % slower on the measured workloads).  Same results either way. */
+                                     device.  0 (default): the calls never synchronise; the host walks every chunk a model could
+                                     have and a launch without rows returns at once.  1: the host reads the K counts back as well
+                                     (one stream synchronisation after the routing kernels) and skips the launches that would be
+                                     empty (0.1-0.9 % faster on the measured workloads).  Same results either way. */
 #define UNITY_OPT_WAIT_KCYCLES 20  /* bound of every in-kernel wait in thousands of SM clocks (default 4 000 000, about 2 s); when
                                      it runs out the kernel records UNITY_ERR_TIMEOUT, frees its tensor memory and returns */
 #define UNITY_OPT_TEST_DROP_SLAB 21 /* TEST HOOK for the timeout path; accepted only while UNITY_OPT_WAIT_KCYCLES <= 1000.

@@ -128,6 +128,10 @@ __device__ __noinline__ GemmArgs resolve_span(const GemmArgs& in) {
         g.last_stats_off = static_cast<long long>(fs.splits) * n_rows;
         g.last_pitch = n_rows - static_cast<long long>(fs.last_m0) * TILE_ROWS;
         g.stats_pitch = n_rows;
+        {   // the most units any round holds: a full round, or the short last one with its own split count
+            const int full = min(g.m_tiles, fs.gm) * fs.splits, last = (g.m_tiles - fs.last_m0) * fs.last_splits;
+            g.n_active = max(full, last);
+        }
         if (in.stats_from_plan) g.stats = in.stats + in.span.plan->stats_base[in.span.model];
     } else if (in.span_mode == kSpanRowsA) {
         g.a_row0 = in.a_row0 + slot0;
@@ -151,6 +155,7 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
     // thread of both CTAs reads the same plan, so a launch whose span is empty is left by all of them, here.
     const GemmArgs g = resolve_span<C::kTileRows>(g_in);
     if (g.m_tiles <= 0 || g.n_tiles <= 0 || g.k_iters <= 0) return;
+    if (g.n_active > 0 && (CTAS == 2 ? blockIdx.x >> 1 : blockIdx.x) >= g.n_active) return;   // never holds a unit
     constexpr int kStages = C::kStages, kStageBytes = C::kStageBytes, kABytes = C::kABytes, kBBytes = C::kBBytes;
     constexpr int kAccStages = C::kAccStages, kTileCols = C::kTileCols;
     static_assert(NB == 1 || (EPI == kEpiAccumF32 && CTAS == 2), "two-block tiles: fp32-accumulate epilogue, CTA pairs");
@@ -168,7 +173,8 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cta_rank = CTAS == 2 ? ptx::cluster_ctarank() : 0u;     // 0: issues the MMAs, 1: its peer
     const int pair = CTAS == 2 ? blockIdx.x >> 1 : blockIdx.x;              // index of this worker (CTA or CTA pair)
-    const int n_pairs = CTAS == 2 ? gridDim.x >> 1 : gridDim.x;
+    const int n_launched = CTAS == 2 ? gridDim.x >> 1 : gridDim.x;
+    const int n_pairs = g.n_active > 0 && g.n_active < n_launched ? g.n_active : n_launched;   // workers at work
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
@@ -612,11 +618,11 @@ int gemm_mma_n(int n_cols) {
 }
 
 cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, int ctas, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                        const GemmArgs& args, int sm_count, cudaStream_t stream, bool wide) {
+                        const GemmArgs& args, int sm_count, cudaStream_t stream, bool wide, int workers_known) {
     // softmax: one round handles group_m row tiles x n_splits; other epilogues: plain striding over all tiles.  With the
     // row extent known on the device only, the launch takes the whole machine; workers without a unit leave at once.
     const int max_workers = sm_count / ctas;                                   // one CTA per SM
-    int workers = max_workers;
+    int workers = workers_known > 0 && workers_known < max_workers ? workers_known : max_workers;
     if (args.span.plan == nullptr) {
         const long long units = epi == kEpiSoftmaxStats
                                     ? static_cast<long long>(args.group_m < args.m_tiles ? args.group_m : args.m_tiles) * args.n_splits

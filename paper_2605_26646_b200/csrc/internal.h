@@ -122,6 +122,8 @@ struct GemmArgs {
     int m_rows, n_cols;       // valid extent of C from (a_row0, b_row0): epilogue writes nothing beyond it
     // kEpiSoftmaxStats: a unit is (row tile, vocabulary split); a CTA keeps a unit's running statistics
     int n_splits, tiles_per_split;
+    int n_active;             // workers that ever hold a unit (0 = all launched): the others leave at once and the round
+                              // rendezvous counts only these
     // ... and the last round, when it holds fewer row tiles than the others, may cut the vocabulary into more splits so
     // that it still occupies the machine: row tiles >= last_m0 use last_splits / last_tiles_per_split and write their
     // statistics to stats[last_stats_off + split * last_pitch + (row - first row of tile last_m0)]
@@ -176,8 +178,10 @@ struct GemmArgs {
 // gemm_tile_rows(ctas) rows.
 // wide: output tiles two MMA blocks wide (kEpiAccumF32 with ctas = 2 only); args.n_tiles then counts tiles of
 // 2 * args.mma_n columns instead of args.mma_n.
+// workers: CTAs (or CTA pairs) to launch when the caller knows how many units a round holds; 0 = the whole machine
+// (a worker without a unit leaves at once).
 cudaError_t launch_gemm(GemmEpilogue epi, bool a_mn, int ctas, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                        const GemmArgs& args, int sm_count, cudaStream_t stream, bool wide = false);
+                        const GemmArgs& args, int sm_count, cudaStream_t stream, bool wide = false, int workers = 0);
 int gemm_tile_rows(int ctas);
 int gemm_mma_n(int n_cols);   // block width for an fp32-accumulate GEMM with n_cols output columns
 cudaError_t gemm_set_attributes();
