@@ -32,8 +32,8 @@ UNIT = "tokens/s"
 # (valid rows x vocabulary columns).  Traffic grows in proportion to the logits covered (same chunk and group sizes),
 # so a full-size launch is estimated as bytes_per_logit x its logits.  Valid only for the kernel source it was taken
 # from: when the hash of gemm_tcgen05.cu differs, the benchmark reports null.
-NCU_TRAFFIC = {"source_sha256_16": "15538ac9efb39bde",
-               "bytes_per_logit": {"fwd_gemm": 1.959, "grad_gemm": 3.942, "dh_gemm": 6.354, "dw_gemm": 6.352}}
+NCU_TRAFFIC = {"source_sha256_16": "b76133cc36e845e0",
+               "bytes_per_logit": {"fwd_gemm": 1.977, "grad_gemm": 3.985, "dh_gemm": 6.410, "dw_gemm": 6.395}}
 
 
 def ncu_traffic_per_launch(cls: str, logits_per_launch: float):
@@ -676,7 +676,9 @@ def main():
                 "traffic": ncu_traffic_per_launch(dom, float(V) * n_valid_local * args.steps / dp["launches"]),
                 "peak_source": f"{peaks['source']} bf16 GEMM, sustained",
                 "flops_per_launch": flops_per_tok * n_valid_local * args.steps / dp["launches"],
-                "avg_launch_ms": dp["ms_total"] / dp["launches"]}
+                "avg_launch_ms": dp["ms_total"] / dp["launches"],
+                "launches_note": "per-launch figures average over every launch of the class, including those whose span "
+                                 "of rows was empty and returned at once (the host does not know the row counts)"}
     step_tflops_alg = 6.0 * H * V * n_valid_local / (ms_step * 1e-3) / 1e12
     step_tflops_exe = 8.0 * H * V * n_valid_local / (ms_step * 1e-3) / 1e12
 
