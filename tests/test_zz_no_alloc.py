@@ -29,7 +29,7 @@ def both_ways(ctx, w):
     oracle = pu.oracle_advantage(w)
     for k in ref:
         assert (out[k] - ref[k]).abs().max().item() <= pu.TOL_ADV, k
-        assert np.abs(out[k].cpu().numpy() - oracle[k]).max() <= pu.TOL_ADV, k       # the oracle is the judge
+        assert np.abs(out[k].cpu().numpy() - oracle[k]).max() <= pu.TOL_ADV, k       # parity is defined against the oracle
     return int(flag.item())
 
 
