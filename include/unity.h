@@ -97,7 +97,8 @@ int unity_set_profiling(unity_ctx* ctx, int enable);
 #define UNITY_OPT_CHUNK_GROUP 5   /* raster group of all three gradient-chunk GEMMs in 128-row tiles (defaults 40, 32, 32)       */
 #define UNITY_OPT_CHUNK_ROWS 6    /* gradient chunk rows = value x 18944 (default 2; larger needs a larger workspace)   */
 #define UNITY_OPT_CHUNK_VOCAB 7   /* gradient chunk vocabulary entries = value x 18944 (default 2)                      */
-#define UNITY_OPT_FWD_GROUP 8     /* 128-row tiles per round of the forward kernel (default 48; 0 = a quarter of the SMs) */
+#define UNITY_OPT_FWD_GROUP 8     /* 128-row tiles per round of the forward kernel; 0 = a quarter of the SMs; -1 (default): half
+                                     the SMs where that many hidden rows fit a 45 MB share of L2 (H <= 2368), else 48 */
 #define UNITY_OPT_FWD_SYNC 9      /* 1 (default): workers of the forward kernel meet at each round start (bounded wait) */
 #define UNITY_OPT_CHUNK_SYNC 10   /* same for the gradient-chunk GEMMs: bit 0 recompute, bit 1 dHidden, bit 2 dW (default 7) */
 #define UNITY_OPT_WIDE_ACC 11     /* 1 (default): the dHidden / dW chunk GEMMs of CTA pairs use 256 x 512 output tiles    */
@@ -121,6 +122,17 @@ int unity_set_profiling(unity_ctx* ctx, int enable);
                                      have and a launch without rows returns at once.  1: the host reads the K counts back as well
                                      (one stream synchronisation after the routing kernels) and skips the launches that would be
                                      empty (0.1-0.9 % faster on the measured workloads).  Same results either way. */
+#define UNITY_OPT_GRAD_ROUNDS 26    /* Schedule of the recompute GEMM.  0: one output tile per unit, workers stride over the tiles
+                                     in raster groups and meet at every tile.  n > 0: the forward kernel's schedule: a round =
+                                     at most n 128-row tiles x vocabulary splits of the launch's columns, a worker sweeps the
+                                     tiles of its split with one row tile and the workers meet once per round.  -1 (default):
+                                     rounds of half the SMs where UNITY_OPT_FWD_GROUP's rule allows them (H <= 2368), else 0. */
+#define UNITY_OPT_GRAD_RUNS 28      /* The recompute GEMM outside rounds.  0: a unit is one output tile.  n > 0: a unit is a run of column
+                                     tiles of one row tile; the kernel cuts the launch's columns into the number of runs that fills
+                                     its workers best while about n 128-row tiles are in flight.  -1 (default): n = the tiles whose
+                                     hidden rows fit a 45 MB share of L2. */
+#define UNITY_OPT_GRAD_BLOCK 27     /* one recompute launch covers value x 18944 rows and vocabulary entries of the gradient
+                                     chunk per side; 0 (default): the whole chunk when it runs in rounds or runs of tiles, else 1 */
 #define UNITY_OPT_WAIT_KCYCLES 20  /* bound of every in-kernel wait in thousands of SM clocks (default 4 000 000, about 2 s); when
                                      it runs out the kernel records UNITY_ERR_TIMEOUT, frees its tensor memory and returns */
 #define UNITY_OPT_TEST_DROP_SLAB 21 /* TEST HOOK for the timeout path; accepted only while UNITY_OPT_WAIT_KCYCLES <= 1000.

@@ -179,6 +179,9 @@ OPT_LOGIT_STASH = 15
 OPT_WAIT_KCYCLES = 20
 OPT_HOST_COUNTS = 25
 OPT_TEST_DROP_SLAB = 21
+OPT_GRAD_ROUNDS = 26
+OPT_GRAD_BLOCK = 27
+OPT_GRAD_RUNS = 28
 
 
 def unity_create(device: int, stream_ptr: int, workspace: torch.Tensor) -> C.c_void_p:

@@ -62,7 +62,19 @@ struct Cfg {
 
 struct Unit {
     int m_tile, n_begin, n_end, split;
+    bool rev;     // walk the unit's column tiles from n_end - 1 down to n_begin
 };
+
+// The logit-gradient epilogue can run on the softmax epilogue's schedule (rounds of row tiles x vocabulary splits): the
+// launch says so by carrying a split count.
+template <int EPI>
+__device__ __forceinline__ int stride_unit_tiles(const GemmArgs& g) {
+    return EPI == kEpiLogitGrad && g.unit_tiles > 1 ? g.unit_tiles : 1;
+}
+template <int EPI>
+__device__ __forceinline__ bool in_rounds(const GemmArgs& g) {
+    return EPI == kEpiSoftmaxStats || (EPI == kEpiLogitGrad && g.n_splits > 0);
+}
 
 // Work decomposition over CTA pairs; `it` counts the rounds of a pair's persistent loop.
 // Softmax: a unit is (256-row tile, vocabulary split).  Round `it` works on row-tile group `it` (gm row tiles): pair
@@ -74,7 +86,8 @@ struct Unit {
 // Returns false when the pair has no more work; `valid` is false for a round the pair sits out.
 template <int EPI>
 __device__ __forceinline__ bool next_unit(const GemmArgs& g, int it, int pair, int n_pairs, int gm, Unit& t, bool& valid) {
-    if (EPI == kEpiSoftmaxStats) {
+    t.rev = false;
+    if (in_rounds<EPI>(g)) {
         const int m0 = it * gm;
         if (m0 >= g.m_tiles) return false;
         const int gm_here = min(gm, g.m_tiles - m0);
@@ -86,21 +99,34 @@ __device__ __forceinline__ bool next_unit(const GemmArgs& g, int it, int pair, i
         t.m_tile = m0 + (pair - t.split * gm_here);
         t.n_begin = t.split * tps;
         t.n_end = min(t.n_begin + tps, g.n_tiles);
+        // logit gradient: odd rounds sweep their split backwards, so a round starts on the W tiles the round before it
+        // ended with (the statistics of the softmax epilogue depend on the order of the sweep and keep it)
+        t.rev = EPI == kEpiLogitGrad && (it & 1);
         return true;
     } else {
+        // a unit is one output tile, or (logit gradient, GemmArgs::unit_tiles > 1) a run of that many column tiles of one
+        // row tile: all units of a launch are then nearly equally long, every worker holds one at any time, and the
+        // workers that hold the same run of columns sweep its W tiles in step
+        const int tpu = stride_unit_tiles<EPI>(g);
+        const int ncu = (g.n_tiles + tpu - 1) / tpu;
         const int u = pair + it * n_pairs;
-        if (u >= g.m_tiles * g.n_tiles) return false;
-        const int per_group = gm * g.n_tiles;
+        if (u >= g.m_tiles * ncu) return false;
+        const int per_group = gm * ncu;
         const int grp = u / per_group, r = u - grp * per_group;
         const int m0 = grp * gm;
         const int gm_here = min(gm, g.m_tiles - m0);
         const int q = r / gm_here;
         t.m_tile = m0 + (r - q * gm_here);
         t.split = 0;
-        // odd groups walk the columns backwards: the B tiles a group ends with are the ones the next group starts
-        // with, while they are still in L2
-        t.n_begin = (grp & 1) ? g.n_tiles - 1 - q : q;
-        t.n_end = t.n_begin + 1;
+        if (tpu == 1) {
+            // odd groups walk the columns backwards: the B tiles a group ends with are the ones the next group starts
+            // with, while they are still in L2
+            t.n_begin = (grp & 1) ? g.n_tiles - 1 - q : q;
+            t.n_end = t.n_begin + 1;
+        } else {
+            t.n_begin = q * tpu;
+            t.n_end = min(t.n_begin + tpu, g.n_tiles);
+        }
         valid = true;
         return true;
     }
@@ -137,6 +163,30 @@ __device__ __noinline__ GemmArgs resolve_span(const GemmArgs& in) {
         g.a_row0 = in.a_row0 + slot0;
         g.m_rows = n_rows;
         g.m_tiles = n_rows / TILE_ROWS;
+        if (in.fwd.n_pairs > 0 && in.plan_runs) {
+            // Units = runs of column tiles.  More runs than the L2 budget asks for (fwd.gmax row tiles in flight) are
+            // fine; among a few counts take the one whose units fill the workers' iterations best.
+            const int np = in.fwd.n_pairs, nt = in.n_tiles;
+            const int ncu_min = max(1, (np + in.fwd.gmax - 1) / in.fwd.gmax);
+            int best_tpu = nt, best_ncu = 1;
+            long long best_cost = -1;
+            for (int want = ncu_min; want <= min(nt, ncu_min + 12); ++want) {
+                const int tpu = (nt + want - 1) / want, ncu = (nt + tpu - 1) / tpu;
+                const long long cost = (static_cast<long long>(g.m_tiles) * ncu + np - 1) / np * tpu;
+                if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_tpu = tpu; best_ncu = ncu; }
+            }
+            g.unit_tiles = best_tpu;
+            g.group_m = max(1, min(g.m_tiles, (np + best_ncu - 1) / best_ncu));
+            const long long units = static_cast<long long>(g.m_tiles) * best_ncu;
+            g.n_active = static_cast<int>(min(static_cast<long long>(np), units));
+        } else if (in.fwd.n_pairs > 0) {
+            // the recompute GEMM on the forward's schedule: rounds of row tiles x vocabulary splits of this launch's columns
+            const FwdShape fs = forward_shape(in.fwd, n_rows);
+            g.group_m = fs.gm; g.n_splits = fs.splits; g.tiles_per_split = fs.tps;
+            g.last_m0 = fs.last_m0; g.last_splits = fs.last_splits; g.last_tiles_per_split = fs.last_tps;
+            const int full = min(g.m_tiles, fs.gm) * fs.splits, last = (g.m_tiles - fs.last_m0) * fs.last_splits;
+            g.n_active = max(full, last);
+        }
     } else if (in.span_mode == kSpanRowsM) {
         g.m_rows = n_rows;
         g.m_tiles = n_rows / TILE_ROWS;
@@ -207,7 +257,7 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                 Unit t;
                 bool valid;
                 if (!next_unit<EPI>(g, it, pair, n_pairs, gm, t, valid)) break;
-                if (g.round_counter != nullptr && cta_rank == 0 && (EPI == kEpiSoftmaxStats || it % g.sync_period == 0)) {
+                if (g.round_counter != nullptr && cta_rank == 0 && (in_rounds<EPI>(g) || it % g.sync_period == 0)) {
                     // Soft rendezvous at the start of a round (softmax: every round; other epilogues, whose round is one
                     // tile: every sync_period-th): the workers that share a stream of W tiles stay in step only while
                     // they start together, and once they drift apart by more than L2 can bridge each of them fetches the
@@ -218,11 +268,12 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                     // arrivals expected by the end of this rendezvous: every worker (softmax), or every worker that
                     // still has a tile (the last ones of the other epilogues may be partial)
                     unsigned expect;
-                    if (EPI == kEpiSoftmaxStats) {
+                    if (in_rounds<EPI>(g)) {
                         expect = static_cast<unsigned>(it + 1) * static_cast<unsigned>(n_pairs);
                     } else {
                         const long long before = static_cast<long long>(it) * n_pairs;      // units of earlier rounds
-                        const long long left = static_cast<long long>(g.m_tiles) * g.n_tiles - before;
+                        const int tpu = stride_unit_tiles<EPI>(g);
+                        const long long left = static_cast<long long>(g.m_tiles) * ((g.n_tiles + tpu - 1) / tpu) - before;
                         expect = static_cast<unsigned>(it / g.sync_period) * static_cast<unsigned>(n_pairs) +
                                  static_cast<unsigned>(left < n_pairs ? left : n_pairs);
                     }
@@ -233,14 +284,15 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                 }
                 if (!valid) continue;
                 const int a_row = g.a_row0 + t.m_tile * C::kTileRows + static_cast<int>(cta_rank) * kCtaM;
-                for (int nt = t.n_begin; nt < t.n_end && ok; ++nt) {
+                for (int ni = t.n_begin; ni < t.n_end && ok; ++ni) {
+                    const int nt = t.rev ? t.n_begin + t.n_end - 1 - ni : ni;
                     // fp32-accumulate tiles may be narrower than 256 columns per MMA (mma_n); the B boxes keep their size, the
                     // MMA simply leaves their last columns unread
                     const int mma_n = EPI == kEpiAccumF32 ? g.mma_n : kTileN;
                     const int b_row = g.b_row0 + nt * (NB * mma_n) + static_cast<int>(cta_rank) * (mma_n / CTAS);
                     for (int k = 0; k < g.k_iters; ++k) {
                         if (!ptx::mbar_wait(&empty[stage], phase ^ 1, g.wait_budget) || *abort_flag) { ok = false; break; }
-                        if (g.test_drop_slab && it == 0 && nt == t.n_begin && k == (g.k_iters > 1 ? 1 : 0)) {
+                        if (g.test_drop_slab && it == 0 && ni == t.n_begin && k == (g.k_iters > 1 ? 1 : 0)) {
                             // test hook: this slab never arrives; the MMA issuer's wait for it must run out
                             if (++stage == kStages) { stage = 0; phase ^= 1; }
                             continue;
@@ -374,7 +426,8 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
                 }
             }
 
-            for (int nt = t.n_begin; nt < t.n_end && ok; ++nt) {
+            for (int ni = t.n_begin; ni < t.n_end && ok; ++ni) {
+                const int nt = t.rev ? t.n_begin + t.n_end - 1 - ni : ni;
                 if (!ptx::mbar_wait(&acc_full[acc], acc_phase, g.wait_budget) || *abort_flag) { ok = false; break; }
                 ptx::tc_fence_after();
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kTileCols;

@@ -78,6 +78,9 @@ __host__ __device__ inline FwdShape forward_shape(const FwdPlanParams& p, int ro
         sp = sp > 32 ? 32 : sp;
         sp = sp > p.n_tiles ? p.n_tiles : sp;
         sp = sp < 1 ? 1 : sp;
+        // several rounds: at most 4 splits, which bounds the statistics a launch writes by 4 per row (plus the short last
+        // round's, at most one per worker and tile row); only a round size far below the default runs into this
+        if (c < m_tiles && sp > 4) sp = 4;
         const int full_rounds = m_tiles / c, rest = m_tiles - full_rounds * c;
         int sp_last = sp;
         if (rest > 0) {
@@ -130,6 +133,9 @@ struct GemmArgs {
     int last_m0, last_splits, last_tiles_per_split;
     long long last_stats_off, last_pitch;
     unsigned* round_counter;  // this launch's arrival counter, zero before the launch (null = no rendezvous between rounds)
+    int unit_tiles;           // logit gradient outside rounds: column tiles per unit (0 or 1: one output tile per unit)
+    int plan_runs;            // logit gradient, rows known on the device only: the kernel picks unit_tiles and group_m itself
+                              // from fwd.n_pairs (workers) and fwd.gmax (row tiles in flight that fit L2)
     int sync_period;          // epilogues other than softmax: rendezvous at every sync_period-th tile of a worker (>= 1)
     float4* stats;            // [n_splits][stats_pitch], row relative to a_row0: (max acc, sum e, sum e*acc, target acc)
     long long stats_pitch;

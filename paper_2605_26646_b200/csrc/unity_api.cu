@@ -34,7 +34,7 @@ struct unity_ctx {
     int l2_promotion;               // tensor-map L2 promotion: 0 none, 1 64 B, 2 128 B, 3 256 B
     int chunk_group[3];             // raster group of the recompute / dHidden / dW chunk GEMMs, in 128-row tiles
     int chunk_rows_mult, chunk_vocab_mult;   // gradient chunk = mult x 18944 rows / vocabulary entries
-    int fwd_group;                  // row tiles (128 rows) per round of the forward kernel; 0 = a quarter of the SMs
+    int fwd_group;                  // row tiles (128 rows) per round of the forward kernel; 0 = a quarter of the SMs; -1: by H
     int fwd_sync;                   // 1: workers of the forward kernel meet (softly) at every round start
     int chunk_sync;                 // bit 0: same for the recompute GEMM, bit 1: dHidden GEMM, bit 2: dW GEMM
     int logit_stash;                // 1: the loss call keeps the logits of one row block instead of recomputing them
@@ -45,6 +45,12 @@ struct unity_ctx {
     int chunk_sync_period[3];       // recompute / dHidden / dW GEMM: rendezvous at every n-th tile of a worker
     long long wait_budget;          // SM clocks after which an in-kernel wait gives up
     int test_drop;                  // test hook: 1 + GEMM class whose producer leaves out one K slab; 0 = off
+    int grad_rounds;                // > 0: the recompute GEMM runs on the forward's schedule (rounds of at most this many
+                                    // 128-row tiles x vocabulary splits); 0: one tile per unit in raster groups; -1: by H
+    int grad_runs;                  // recompute GEMM outside rounds: 0: one output tile per unit; n > 0: units are runs of column
+                                    // tiles, planned by the kernel so that about n 128-row tiles are in flight; -1: n from H
+    int grad_block;                 // blocks of 18944 rows / vocabulary entries one recompute launch covers per side;
+                                    // 0: the whole chunk when the launch runs in rounds, else 1
 };
 
 namespace {
@@ -263,14 +269,24 @@ struct RowPlan {
     long long rows_bound;                 // padded rows a model can have at most: every row of the batch
 };
 
+// A round of the forward schedule keeps its hidden rows in L2 while the W tiles stream past.  Where half the machine's
+// worth of 256-row tiles (37 on 148 SMs) fits a 45 MB budget (H <= 2368) the rounds are that large: every worker of a
+// two-split round then shares its W stream with 36 others.  Measured at H = 896 / 1536: forward +2 %, recompute GEMM
+// +19 % / +11 % over rounds of 24 / one tile per unit; at H = 3584 / 5120 such rounds overflow L2 (SM clock -3 %).
+bool large_rounds_fit(const unity_ctx* ctx, int H) {
+    const long long tiles = ctx->sm_count / 4;
+    return tiles * kTileM * H * 2 <= 45ll << 20;
+}
+
 // Inputs of the forward planner that the host knows.
-FwdPlanParams fwd_params(const unity_ctx* ctx, int V) {
+FwdPlanParams fwd_params(const unity_ctx* ctx, int V, int H) {
     const int ctas = ctx->ctas[UNITY_PROF_FWD_GEMM];
     FwdPlanParams p;
     p.n_pairs = ctx->sm_count / ctas;
     p.tile_rows = gemm_tile_rows(ctas);
     p.n_tiles = (V + kTileN - 1) / kTileN;
-    int gmax = ctx->fwd_group > 0 ? ctx->fwd_group / ctas : p.n_pairs / 4;
+    const int group = ctx->fwd_group >= 0 ? ctx->fwd_group : (large_rounds_fit(ctx, H) ? ctx->sm_count / 2 : 48);
+    int gmax = group > 0 ? group / ctas : p.n_pairs / 4;
     if (gmax < 1) gmax = 1;
     if (gmax > p.n_pairs) gmax = p.n_pairs;
     p.gmax = gmax;
@@ -329,7 +345,7 @@ int forward_sweep(unity_ctx* ctx, const unity_rows* r, RowPlan& P, bool run_gemm
     const Layout& L = P.L;
     cudaStream_t st = ctx->stream;
     int nl = 0;
-    P.fwd = fwd_params(ctx, r->V);
+    P.fwd = fwd_params(ctx, r->V, r->H);
     P.counters = SyncCounters{L.sync_counters, 0, kSyncCounters};
     P.rows_bound = static_cast<long long>(up(r->n_tok, kTileM));
     for (int k = 0; k < UNITY_MAX_MODELS; ++k) P.rows_known[k] = -1;
@@ -421,7 +437,7 @@ int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace
     c->l2_promotion = 3;
     c->chunk_group[0] = 40;          // recompute: least DRAM traffic of 32 / 40 / 48 / 64 (3.9 bytes per logit), same time
     c->chunk_group[1] = c->chunk_group[2] = 32;
-    c->fwd_group = 48;
+    c->fwd_group = -1;
     c->fwd_sync = 1;
     c->chunk_sync = 7;
     c->chunk_rows_mult = kDefaultChunkMult;
@@ -438,6 +454,9 @@ int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace
     c->host_counts = 0;
     c->wait_budget = kWaitBudgetCycles;
     c->test_drop = 0;
+    c->grad_rounds = -1;
+    c->grad_runs = -1;
+    c->grad_block = 0;
     c->ev_pool = new (std::nothrow) std::vector<cudaEvent_t>();
     c->ev_class = new (std::nothrow) std::vector<int>();
     if (cudaMalloc(&c->d_status, 256) != cudaSuccess || cudaMallocHost(&c->h_pinned, 4096) != cudaSuccess ||
@@ -539,7 +558,7 @@ int unity_set_option(unity_ctx* ctx, int option, int value) {
     }
     if (option == UNITY_OPT_FWD_SYNC && (value == 0 || value == 1)) { ctx->fwd_sync = value; return UNITY_OK; }
     if (option == UNITY_OPT_CHUNK_SYNC && value >= 0 && value <= 7) { ctx->chunk_sync = value; return UNITY_OK; }
-    if (option == UNITY_OPT_FWD_GROUP && value >= 0 && value <= 148) { ctx->fwd_group = value; return UNITY_OK; }
+    if (option == UNITY_OPT_FWD_GROUP && value >= -1 && value <= 148) { ctx->fwd_group = value; return UNITY_OK; }
     if (option == UNITY_OPT_CHUNK_ROWS && value >= 1 && value <= 8) { ctx->chunk_rows_mult = value; return UNITY_OK; }
     if (option == UNITY_OPT_CHUNK_VOCAB && value >= 1 && value <= 8) { ctx->chunk_vocab_mult = value; return UNITY_OK; }
     if (option == UNITY_OPT_LOGIT_STASH && (value == 0 || value == 1)) { ctx->logit_stash = value; return UNITY_OK; }
@@ -553,6 +572,9 @@ int unity_set_option(unity_ctx* ctx, int option, int value) {
         return UNITY_OK;
     }
     if (option == UNITY_OPT_HOST_COUNTS && (value == 0 || value == 1)) { ctx->host_counts = value; return UNITY_OK; }
+    if (option == UNITY_OPT_GRAD_ROUNDS && value >= -1 && value <= 148) { ctx->grad_rounds = value; return UNITY_OK; }
+    if (option == UNITY_OPT_GRAD_RUNS && value >= -1 && value <= 148) { ctx->grad_runs = value; return UNITY_OK; }
+    if (option == UNITY_OPT_GRAD_BLOCK && value >= 0 && value <= 8) { ctx->grad_block = value; return UNITY_OK; }
     if (option == UNITY_OPT_WAIT_KCYCLES && value >= 1) {
         ctx->wait_budget = static_cast<long long>(value) * 1000;
         if (ctx->wait_budget > 1000000) ctx->test_drop = 0;      // the test hook lives only under a short bound
@@ -989,10 +1011,19 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                     // recompute the logits.  Whatever the chunk size, one launch covers at most kChunkRows x
                     // (kChunkVocab + tail) of it: the kernel re-reads its W block once per group of row tiles, and
                     // that block has to stay small enough for the group's hidden rows to survive in L2 meanwhile.
-                    for (int r0 = 0; r0 < nc; r0 += kChunkRows) {
-                        const int nr = nc - r0 < kChunkRows ? nc - r0 : kChunkRows;
+                    // (On the forward's schedule a round bounds the rows in flight by itself and a launch may cover more.)
+                    const int rounds = ctx->grad_rounds >= 0 ? ctx->grad_rounds : (large_rounds_fit(ctx, H) ? ctx->sm_count / 2 : 0);
+                    int runs = rounds > 0 ? 0 : ctx->grad_runs;
+                    if (runs < 0) {   // 128-row tiles whose hidden rows fit the 45 MB share of L2
+                        runs = static_cast<int>((45ll << 20) / (128ll * H * 2));
+                        runs = runs < 8 ? 8 : (runs > ctx->sm_count / 2 ? ctx->sm_count / 2 : runs);
+                    }
+                    const int per_side = ctx->grad_block > 0 ? ctx->grad_block : (rounds > 0 || runs > 0 ? 8 : 1);
+                    const int blk_rows = kChunkRows * per_side, blk_cols = kChunkVocab * per_side;
+                    for (int r0 = 0; r0 < nc; r0 += blk_rows) {
+                        const int nr = nc - r0 < blk_rows ? nc - r0 : blk_rows;
                         for (int q0 = 0, qc = 0; q0 < vc; q0 += qc) {
-                            qc = vc - q0 < kChunkVocab ? vc - q0 : kChunkVocab;
+                            qc = vc - q0 < blk_cols ? vc - q0 : blk_cols;
                             if (vc - (q0 + qc) <= tail) qc = vc - q0;
                             GemmArgs g;
                             memset(&g, 0, sizeof(g));
@@ -1000,6 +1031,20 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                             g.m_tiles = 1;                                   // set by the kernel
                             g.n_tiles = (qc + kTileN - 1) / kTileN; g.k_iters = H / kTileK;
                             g.group_m = ctx->chunk_group[0] / c_grad > 0 ? ctx->chunk_group[0] / c_grad : 1;
+                            if (runs > 0) {
+                                g.plan_runs = 1;
+                                g.fwd.n_pairs = ctx->sm_count / c_grad;
+                                g.fwd.tile_rows = gemm_tile_rows(c_grad);
+                                g.fwd.n_tiles = g.n_tiles;
+                                g.fwd.gmax = runs / c_grad > 0 ? runs / c_grad : 1;
+                            }
+                            if (rounds > 0) {
+                                g.fwd.n_pairs = ctx->sm_count / c_grad;
+                                g.fwd.tile_rows = gemm_tile_rows(c_grad);
+                                g.fwd.n_tiles = g.n_tiles;
+                                g.fwd.gmax = rounds / c_grad > 0 ? rounds / c_grad : 1;
+                                if (g.fwd.gmax > g.fwd.n_pairs) g.fwd.gmax = g.fwd.n_pairs;
+                            }
                             g.a_row0 = 0; g.b_row0 = v0 + q0; g.n_cols = qc;
                             g.target_p = L.target_p; g.vocab0 = v0 + q0; g.scale = rows->inv_temperature;
                             g.coef_a = L.coef_a; g.coef_b = L.coef_b; g.row_lse = L.row_lse; g.row_ent = L.row_ent;

@@ -442,7 +442,27 @@ def test_forward_rounds_with_a_short_last_round(rows, valid, ctas):
     # two full rounds and a last one of one tile
     w = small_workload(128, 8192 + 264, rows, max_len=200, role_model=[0, 0, 0], K=1)
     assert (w.tok_mask != 0).sum().item() == valid
-    run_all_stages(w, ctas=(ctas,) * 4)
+    run_all_stages(w, ctas=(ctas,) * 4, options=[(8, 48)])      # rounds of 48 tiles of 128 rows whatever the hidden size
+
+
+@pytest.mark.parametrize("ctas,gmax,block", [(2, 16, 1), (1, 16, 1), (2, 48, 2), (2, 148, 1)])
+def test_recompute_gemm_on_the_forward_schedule(ctas, gmax, block):
+    # the recompute GEMM in rounds of row tiles x vocabulary splits (a worker sweeps its split with one row tile, odd
+    # rounds backwards): 25 row tiles of 256 give full rounds and a short last one that is cut into more splits
+    w = small_workload(128, 8192 + 264, 7700, max_len=200, role_model=[0, 0, 0], K=1)
+    run_all_stages(w, ctas=(ctas,) * 4, options=[(ub.OPT_GRAD_ROUNDS, gmax), (ub.OPT_GRAD_BLOCK, block)], ent_coef=0.01)
+    if gmax == 48:       # and once at a full-size hidden width and vocabulary (four models, H = 5120)
+        run_all_stages(wl.make("stress", device="cuda", cut_rows=300, cut_max_len=64),
+                       options=[(ub.OPT_GRAD_ROUNDS, gmax), (ub.OPT_GRAD_BLOCK, block)])
+
+
+@pytest.mark.parametrize("ctas,in_flight", [(2, 0), (2, 12), (1, 12), (2, 148)])
+def test_recompute_gemm_in_runs_of_column_tiles(ctas, in_flight):
+    # outside rounds a unit of the recompute GEMM is one output tile (0) or a run of column tiles that the kernel sizes
+    # from the rows it finds (25 row tiles of 256, 34 column tiles, the last one ragged)
+    w = small_workload(128, 8192 + 264, 7700, max_len=200, role_model=[0, 0, 0], K=1)
+    options = [(ub.OPT_GRAD_ROUNDS, 0), (ub.OPT_GRAD_RUNS, in_flight)]
+    run_all_stages(w, ctas=(ctas,) * 4, options=options, ent_coef=0.01)
 
 
 @pytest.mark.parametrize("ctas", [(1, 1, 1, 1), (2, 2, 2, 2), (2, 1, 1, 2)])
@@ -453,8 +473,8 @@ def test_single_cta_and_cta_pair_kernels(ctas):
 
 
 def test_scheduling_options_do_not_change_results():
-    """Raster groups, rendezvous switches and periods, L2 hints and tensor-map promotion only move work in time or
-    space: every output must be bitwise what the defaults give.  The forward round size changes the number of
+    """Raster groups, rendezvous switches and periods, L2 hints, tensor-map promotion and the schedule of the recompute
+    GEMM (tile by tile or in rounds, per block or per chunk) only move work in time or space: every output must be bitwise what the defaults give.  The forward round size changes the number of
     vocabulary splits and with it the order of a four-term merge: equal within rounding."""
     w = small_workload(320, 4096 + 264, 900)
     d = pu.DeviceInputs(w)
@@ -473,7 +493,8 @@ def test_scheduling_options_do_not_change_results():
 
     base = run([])
     same = [[(4, 0)], [(5, 8)], [(9, 0)], [(10, 0)], [(10, 5)], [(12, 4), (13, 6), (14, 2)], [(16, 0), (17, 0)],
-            [(17, 41), (18, 9), (19, 38)], [(22, 3), (23, 2), (24, 5)]]
+            [(17, 41), (18, 9), (19, 38)], [(22, 3), (23, 2), (24, 5)], [(26, 4)], [(26, 48), (27, 2)], [(26, 2), (10, 0)], [(26, 0), (28, 0)], [(26, 0), (28, 8)],
+            [(26, 0), (28, 40), (27, 1)]]
     for options in same:
         out = run(options)
         for key in ("loss", "logp", "entropy", "tok_loss", "dHidden", "metrics"):
