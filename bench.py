@@ -32,8 +32,8 @@ UNIT = "tokens/s"
 # (valid rows x vocabulary columns).  Traffic grows in proportion to the logits covered (same chunk and group sizes),
 # so a full-size launch is estimated as bytes_per_logit x its logits.  Valid only for the kernel source it was taken
 # from: when the hash of gemm_tcgen05.cu differs, the benchmark reports null.
-NCU_TRAFFIC = {"source_sha256_16": "b76133cc36e845e0",
-               "bytes_per_logit": {"fwd_gemm": 1.977, "grad_gemm": 3.985, "dh_gemm": 6.410, "dw_gemm": 6.395}}
+NCU_TRAFFIC = {"source_sha256_16": "29857bc22ec90b32",
+               "bytes_per_logit": {"fwd_gemm": 1.754, "grad_gemm": 4.006, "dh_gemm": 6.530, "dw_gemm": 6.344}}
 
 
 def ncu_traffic_per_launch(cls: str, logits_per_launch: float):

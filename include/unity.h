@@ -131,6 +131,9 @@ int unity_set_profiling(unity_ctx* ctx, int enable);
                                      tiles of one row tile; the kernel cuts the launch's columns into the number of runs that fills
                                      its workers best while about n 128-row tiles are in flight.  -1 (default): n = the tiles whose
                                      hidden rows fit a 45 MB share of L2. */
+#define UNITY_OPT_DW_TAIL 29        /* 1 (default): when the vocabulary tiles of a gradient chunk leave a remainder that would fill
+                                     less than half of one more wave of CTA pairs, the dW GEMM runs those tiles as a second
+                                     launch with narrow column tiles spread over the machine.  0: one launch per chunk. */
 #define UNITY_OPT_GRAD_BLOCK 27     /* one recompute launch covers value x 18944 rows and vocabulary entries of the gradient
                                      chunk per side; 0 (default): the whole chunk when it runs in rounds or runs of tiles, else 1 */
 #define UNITY_OPT_WAIT_KCYCLES 20  /* bound of every in-kernel wait in thousands of SM clocks (default 4 000 000, about 2 s); when

@@ -65,25 +65,26 @@ struct Unit {
     bool rev;     // walk the unit's column tiles from n_end - 1 down to n_begin
 };
 
-// The logit-gradient epilogue can run on the softmax epilogue's schedule (rounds of row tiles x vocabulary splits): the
-// launch says so by carrying a split count.
+// Column tiles per unit of the striding schedule (below): one, or a run of GemmArgs::unit_tiles (logit gradient only).
 template <int EPI>
 __device__ __forceinline__ int stride_unit_tiles(const GemmArgs& g) {
     return EPI == kEpiLogitGrad && g.unit_tiles > 1 ? g.unit_tiles : 1;
 }
+// The logit-gradient epilogue can run on the softmax epilogue's schedule of rounds: the launch says so by carrying a
+// split count.
 template <int EPI>
 __device__ __forceinline__ bool in_rounds(const GemmArgs& g) {
     return EPI == kEpiSoftmaxStats || (EPI == kEpiLogitGrad && g.n_splits > 0);
 }
 
-// Work decomposition over CTA pairs; `it` counts the rounds of a pair's persistent loop.
-// Softmax: a unit is (256-row tile, vocabulary split).  Round `it` works on row-tile group `it` (gm row tiles): pair
-// p takes split p / gm_here of row tile p % gm_here and pairs beyond gm_here * n_splits sit the round out.  All pairs
-// of a round therefore share gm A tiles (L2 resident) and each split's stream of B tiles is fetched from HBM once, by
-// pairs that sweep it in step.  Other epilogues: one 256 x 256 output tile per unit, unit = pair + it * n_pairs, m
-// fastest inside groups of gm row tiles.
-// Other epilogues, continued: the column order alternates from one group of row tiles to the next.
-// Returns false when the pair has no more work; `valid` is false for a round the pair sits out.
+// Work decomposition over workers (CTAs or CTA pairs); `it` counts the iterations of a worker's persistent loop.
+// Rounds (softmax statistics always; logit gradient when the launch carries a split count): a unit is (row tile,
+// vocabulary split).  Round `it` works on row-tile group `it` (gm row tiles): worker p takes split p / gm_here of row
+// tile p % gm_here and workers beyond gm_here * n_splits sit the round out.  All workers of a round therefore share gm
+// A tiles (L2 resident) and each split's stream of B tiles is fetched from HBM once, by workers that sweep it in step.
+// Striding (the other launches): unit = worker + it * workers, m fastest inside groups of gm row tiles; a unit is one
+// output tile, with the column order alternating from one group of row tiles to the next, or a run of column tiles.
+// Returns false when the worker has no more work; `valid` is false for a round the worker sits out.
 template <int EPI>
 __device__ __forceinline__ bool next_unit(const GemmArgs& g, int it, int pair, int n_pairs, int gm, Unit& t, bool& valid) {
     t.rev = false;

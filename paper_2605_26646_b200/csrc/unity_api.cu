@@ -47,6 +47,7 @@ struct unity_ctx {
     int test_drop;                  // test hook: 1 + GEMM class whose producer leaves out one K slab; 0 = off
     int grad_rounds;                // > 0: the recompute GEMM runs on the forward's schedule (rounds of at most this many
                                     // 128-row tiles x vocabulary splits); 0: one tile per unit in raster groups; -1: by H
+    int dw_tail;                    // 1: the dW GEMM's last few vocabulary tiles of a chunk run as a launch of narrow tiles
     int grad_runs;                  // recompute GEMM outside rounds: 0: one output tile per unit; n > 0: units are runs of column
                                     // tiles, planned by the kernel so that about n 128-row tiles are in flight; -1: n from H
     int grad_block;                 // blocks of 18944 rows / vocabulary entries one recompute launch covers per side;
@@ -456,6 +457,7 @@ int unity_create(unity_ctx** out, int device, void* cuda_stream, void* workspace
     c->test_drop = 0;
     c->grad_rounds = -1;
     c->grad_runs = -1;
+    c->dw_tail = 1;
     c->grad_block = 0;
     c->ev_pool = new (std::nothrow) std::vector<cudaEvent_t>();
     c->ev_class = new (std::nothrow) std::vector<int>();
@@ -574,6 +576,7 @@ int unity_set_option(unity_ctx* ctx, int option, int value) {
     if (option == UNITY_OPT_HOST_COUNTS && (value == 0 || value == 1)) { ctx->host_counts = value; return UNITY_OK; }
     if (option == UNITY_OPT_GRAD_ROUNDS && value >= -1 && value <= 148) { ctx->grad_rounds = value; return UNITY_OK; }
     if (option == UNITY_OPT_GRAD_RUNS && value >= -1 && value <= 148) { ctx->grad_runs = value; return UNITY_OK; }
+    if (option == UNITY_OPT_DW_TAIL && (value == 0 || value == 1)) { ctx->dw_tail = value; return UNITY_OK; }
     if (option == UNITY_OPT_GRAD_BLOCK && value >= 0 && value <= 8) { ctx->grad_block = value; return UNITY_OK; }
     if (option == UNITY_OPT_WAIT_KCYCLES && value >= 1) {
         ctx->wait_budget = static_cast<long long>(value) * 1000;
@@ -1082,25 +1085,44 @@ int unity_ppo_loss_fwd_bwd(unity_ctx* ctx, const unity_rows* rows, const unity_p
                     CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, false, c_dh, tm_G_k, tm_W_mn, h, ctx->sm_count, st, wide_dh));
                 }
                 // (3) dW[v0:v0+vc, :] (+)= G^T[vc, rows] * hidden[first slot of the chunk ..., :]   (both operands MN-major)
-                GemmArgs w;
-                memset(&w, 0, sizeof(w));
-                w.m_tiles = (vc + gemm_tile_rows(c_dw) - 1) / gemm_tile_rows(c_dw);
-                const bool wide_dw = pick_wide(UNITY_PROF_DW_GEMM, w.m_tiles);
-                const int cols_dw = (wide_dw ? 2 : 1) * mma_n;
-                w.mma_n = mma_n;
-                w.span = chunk; w.span_mode = kSpanRowsK;
-                w.n_tiles = (H + cols_dw - 1) / cols_dw;
-                w.k_iters = 1;                                         // set by the kernel
-                w.group_m = ctx->chunk_group[2] / c_dw > 0 ? ctx->chunk_group[2] / c_dw : 1;
-                w.a_row0 = 0; w.a_k0 = 0; w.b_row0 = 0; w.b_k0 = 0; w.m_rows = vc; w.n_cols = H;
-                w.C = dWk + static_cast<long long>(v0) * H; w.ldc = H;
-                w.beta = (params->accumulate_dW || c0 > 0) ? 1 : 0;
-                gemm_common(ctx, w, UNITY_PROF_DW_GEMM, &P.counters, (ctx->chunk_sync & 4) != 0);
-                {
+                // The vocabulary tiles of a chunk are known here.  When the last few of them would open one more wave of
+                // workers and fill less than half of it (V = 152064: a last chunk of 150 tiles after three of 148), they run
+                // as a launch of their own with narrow tiles, so that they spread over the machine instead of occupying a
+                // seventh of it for a whole tile time.
+                const int tile_v = gemm_tile_rows(c_dw), vt = (vc + tile_v - 1) / tile_v;
+                const bool wide_all = pick_wide(UNITY_PROF_DW_GEMM, vt);
+                int vt_main = vt, narrow_n = 0;
+                if (ctx->dw_tail && c_dw == 2 && vt > n_workers) {
+                    const int nt_main = (H + (wide_all ? 2 : 1) * mma_n - 1) / ((wide_all ? 2 : 1) * mma_n);
+                    const int rem = vt % n_workers;
+                    if (rem > 0 && 2 * rem * nt_main < n_workers) {
+                        for (int cand = 64; cand <= kTileN && narrow_n == 0; cand += 32)
+                            if (static_cast<long long>(rem) * ((H + cand - 1) / cand) <= n_workers) narrow_n = cand;
+                        if (narrow_n > 0) vt_main = vt - rem;
+                    }
+                }
+                for (int part = 0; part < (narrow_n > 0 ? 2 : 1); ++part) {
+                    const int t0 = part == 0 ? 0 : vt_main, t1 = part == 0 ? vt_main : vt;
+                    const int row0 = t0 * tile_v, rows_here = (t1 * tile_v < vc ? t1 * tile_v : vc) - row0;
+                    GemmArgs w;
+                    memset(&w, 0, sizeof(w));
+                    w.m_tiles = t1 - t0;
+                    const bool wide_dw = part == 0 && pick_wide(UNITY_PROF_DW_GEMM, w.m_tiles);
+                    w.mma_n = part == 0 ? mma_n : narrow_n;
+                    const int cols_dw = (wide_dw ? 2 : 1) * w.mma_n;
+                    w.span = chunk; w.span_mode = kSpanRowsK;
+                    w.n_tiles = (H + cols_dw - 1) / cols_dw;
+                    w.k_iters = 1;                                         // set by the kernel
+                    w.group_m = ctx->chunk_group[2] / c_dw > 0 ? ctx->chunk_group[2] / c_dw : 1;
+                    w.a_row0 = row0; w.a_k0 = 0; w.b_row0 = 0; w.b_k0 = 0; w.m_rows = rows_here; w.n_cols = H;
+                    w.C = dWk + static_cast<long long>(v0 + row0) * H; w.ldc = H;
+                    w.beta = (params->accumulate_dW || c0 > 0) ? 1 : 0;
+                    gemm_common(ctx, w, UNITY_PROF_DW_GEMM, &P.counters, (ctx->chunk_sync & 4) != 0);
                     ProfScope ps(ctx, UNITY_PROF_DW_GEMM);
                     CUDA_TRY(ctx, launch_gemm(kEpiAccumF32, true, c_dw, tm_G_mn, tm_hp_mn, w, ctx->sm_count, st, wide_dw));
+                    nl += 1;
                 }
-                nl += 2;
+                nl += 1;
             }
             CUDA_TRY(ctx, launch_store_dhidden(L.dHc, L.slot_tok, chunk, H, dH, st));
             nl += 1;
