@@ -652,6 +652,44 @@ def test_small_workspace_uses_smaller_chunks_and_too_small_is_an_error():
     ctx.close()
 
 
+@pytest.mark.parametrize("case", range(10))
+def test_seeded_random_shapes_schedules_and_workspaces(case):
+    """Shapes, model mappings, scheduling options and workspace sizes drawn from a seeded generator: every combination
+    must match the oracle within the stated tolerances (the planners that cut launches into rounds, runs, chunks and
+    tail launches see extents here that no hand-picked case covers)."""
+    rng = np.random.default_rng(20260528 + case)
+    H = int(rng.choice([64, 128, 192, 320, 448, 512]))
+    V = 8 * int(rng.integers(16, 450))
+    rows = int(rng.integers(40, 1400))
+    K = int(rng.integers(1, 4))
+    role_model = [int(x) for x in rng.integers(0, K, 3)]
+    role_model[int(rng.integers(0, 3))] = K - 1                    # the last model is used; others may stay empty
+    w = small_workload(H, V, rows, role_model=role_model, K=K, max_len=int(rng.choice([16, 48, 200])), seed_offset=case)
+    options = [(ub.OPT_GRAD_ROUNDS, int(rng.choice([-1, 0, 4, 16, 148]))), (ub.OPT_GRAD_RUNS, int(rng.choice([-1, 0, 8, 40]))),
+               (ub.OPT_GRAD_BLOCK, int(rng.choice([0, 1, 2]))), (8, int(rng.choice([-1, 0, 16, 48]))),
+               (11, int(rng.integers(0, 2))), (29, int(rng.integers(0, 2))), (ub.OPT_HOST_COUNTS, int(rng.integers(0, 2)))]
+    ctas = [int(x) for x in rng.integers(1, 3, 4)]
+    ent_coef = float(rng.choice([0.0, 0.01]))
+    need = ub.unity_workspace_bytes(w.n_tok, w.H, w.V, w.K, w.n_inv)
+    least = ub.unity_workspace_min_bytes(w.n_tok, w.H, w.V, w.K, w.n_inv)
+    size = [need, least, (need + least) // 2][int(rng.integers(0, 3))]
+    d = pu.DeviceInputs(w)
+    ctx = ub.Context(0, size)
+    try:
+        for option, value in list(enumerate(ctas)) + options:
+            ctx.set_option(option, value)
+        gl, ol = pu.gpu_logprob(ctx, w, d), pu.oracle_logprob(w)
+        check_forward(gl, ol, w.tok_mask.numpy() != 0)
+        cur = torch.from_numpy(ol["logp"].astype(np.float32))
+        old, ref = cur + w.noise_old, cur + w.noise_ref
+        adv = wl.normal(5, 99 + case, w.n_tok)
+        gp = pu.gpu_ppo(ctx, w, d, old.cuda(), ref.cuda(), adv.cuda(), ent_coef=ent_coef)
+        op = pu.oracle_ppo(w, old.numpy(), ref.numpy(), adv.numpy(), ent_coef=ent_coef)
+        check_ppo(gp, op, w)
+    finally:
+        ctx.close()
+
+
 def test_argument_errors_return_codes():
     w = small_workload(128, 1024, 100)
     d = pu.DeviceInputs(w)
