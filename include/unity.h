@@ -238,7 +238,8 @@ int unity_gae(unity_ctx* ctx, int32_t n_inv, int64_t n_tok, const int64_t* cu_se
  *   loss : out f32 [K];  clip_frac : out f32 [K] or NULL (share of valid tokens on the clipped branch)
  *   tok_loss : out f32 [n_tok] or NULL;  dvalues : out f32 [n_tok]; masked tokens receive 0 in both
  * An out-of-range role or model id flags UNITY_ERR_BAD_INDEX and the invocation's tokens count as masked.
- * Needs 12 bytes of workspace per invocation.  Deterministic (fixed-order sums, no floating-point atomics). */
+ * Needs 12 bytes of workspace per invocation plus 5 KiB.  Deterministic (fixed-order sums of floating-point values, integer
+ * atomics for the token counts). */
 int unity_value_loss_fwd_bwd(unity_ctx* ctx, int32_t n_inv, int32_t n_roles, int32_t K, int64_t n_tok,
                              const int64_t* cu_seqlens, const int32_t* inv_role, const int32_t* role_model,
                              const uint8_t* tok_mask, const float* values, const float* old_values,

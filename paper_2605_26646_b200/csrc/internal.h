@@ -325,10 +325,14 @@ struct ValueArgs {
     int vec_ok;         // token arrays 16-byte aligned and the mask 4-byte aligned: 128-bit accesses allowed
     float norm[UNITY_MAX_MODELS];
     float* inv_sums;    // [n_inv * 3] count, sum of token losses, clipped tokens
-    float* Mk;          // [2 * UNITY_MAX_MODELS] denominators M_k, then max(valid tokens, 1) per model
+    unsigned long long* model_cnt;   // [UNITY_MAX_MODELS] valid tokens per model, directly followed by ...
+    int* tickets;       // [UNITY_MAX_MODELS] ... the arrival counters of k_value_class (value_counters_bytes() in all)
+    float* partial;     // [UNITY_MAX_MODELS * kValueSlices * 2] per-slice sums of k_value_class
     float *loss, *clip_frac, *tok_loss, *dvalues;
     int* status;
 };
+constexpr int kValueSlices = 32;      // slices of the invocations in the last pass of the value loss
+size_t value_counters_bytes();
 cudaError_t launch_value_loss(const ValueArgs& a, cudaStream_t stream, int* n_launches);
 
 // ----------------------------------------------------------------------------------------------

@@ -801,38 +801,52 @@ __device__ __forceinline__ ValueTerm value_term(float v, float ov, float ret, fl
     return t;
 }
 
-// (1) valid tokens per invocation (mask bytes only).
+// Denominator of model k: the caller's norm, else the valid tokens counted by k_value_count (at least 1).
+__device__ __forceinline__ float value_Mk(const ValueArgs& a, int k) {
+    return a.has_norm ? a.norm[k] : fmaxf(static_cast<float>(a.model_cnt[k]), 1.f);
+}
+
+// (1) valid tokens per invocation (mask bytes only) and per model.  The per-model totals are integers added with atomics
+// (one per block and model): exact and independent of the order in which the blocks arrive.
 __global__ void k_value_count(ValueArgs a) {
+    __shared__ int block_cnt[UNITY_MAX_MODELS];
+    if (threadIdx.x < UNITY_MAX_MODELS) block_cnt[threadIdx.x] = 0;
+    __syncthreads();
     const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
-    if (s >= a.n_inv) return;
-    const int role = a.inv_role[s];
-    const bool role_ok = role >= 0 && role < a.n_roles && a.role_model[role] >= 0 && a.role_model[role] < a.K;
-    const long long lo = a.cu_seqlens[s], hi = a.cu_seqlens[s + 1];
-    int cnt = 0;
-    if (role_ok) {
-        if (a.tok_mask == nullptr) {
-            cnt = lane == 0 ? static_cast<int>(hi - lo) : 0;
-        } else {
-            // bytes up to the next 16-byte boundary one by one, then 16 mask bytes per lane and load, then the rest
-            const uintptr_t addr = reinterpret_cast<uintptr_t>(a.tok_mask) + static_cast<uintptr_t>(lo);
-            const long long head_end = min(hi, lo + static_cast<long long>((16 - (addr & 15)) & 15));
-            for (long long i = lo + lane; i < head_end; i += 32) cnt += a.tok_mask[i] != 0;
-            const long long n_vec = (hi - head_end) >> 4;
-            const uint4* mv = reinterpret_cast<const uint4*>(a.tok_mask + head_end);
-            for (long long q = lane; q < n_vec; q += 32) {
-                const uint4 m = mv[q];
-                cnt += (__popc(__vcmpne4(m.x, 0u)) + __popc(__vcmpne4(m.y, 0u)) + __popc(__vcmpne4(m.z, 0u)) +
-                        __popc(__vcmpne4(m.w, 0u))) >> 3;
+    if (s < a.n_inv) {
+        const int role = a.inv_role[s];
+        const bool role_ok = role >= 0 && role < a.n_roles && a.role_model[role] >= 0 && a.role_model[role] < a.K;
+        const long long lo = a.cu_seqlens[s], hi = a.cu_seqlens[s + 1];
+        int cnt = 0;
+        if (role_ok) {
+            if (a.tok_mask == nullptr) {
+                cnt = lane == 0 ? static_cast<int>(hi - lo) : 0;
+            } else {
+                // bytes up to the next 16-byte boundary one by one, then 16 mask bytes per lane and load, then the rest
+                const uintptr_t addr = reinterpret_cast<uintptr_t>(a.tok_mask) + static_cast<uintptr_t>(lo);
+                const long long head_end = min(hi, lo + static_cast<long long>((16 - (addr & 15)) & 15));
+                for (long long i = lo + lane; i < head_end; i += 32) cnt += a.tok_mask[i] != 0;
+                const long long n_vec = (hi - head_end) >> 4;
+                const uint4* mv = reinterpret_cast<const uint4*>(a.tok_mask + head_end);
+                for (long long q = lane; q < n_vec; q += 32) {
+                    const uint4 m = mv[q];
+                    cnt += (__popc(__vcmpne4(m.x, 0u)) + __popc(__vcmpne4(m.y, 0u)) + __popc(__vcmpne4(m.z, 0u)) +
+                            __popc(__vcmpne4(m.w, 0u))) >> 3;
+                }
+                for (long long i = head_end + (n_vec << 4) + lane; i < hi; i += 32) cnt += a.tok_mask[i] != 0;
             }
-            for (long long i = head_end + (n_vec << 4) + lane; i < hi; i += 32) cnt += a.tok_mask[i] != 0;
+        }
+        cnt = warp_sum_int(cnt);
+        if (lane == 0) {
+            if (!role_ok && hi > lo) atomicOr(a.status, kStatusBadIndex);
+            a.inv_sums[s * 3 + 0] = static_cast<float>(cnt);
+            if (role_ok && cnt > 0) atomicAdd(&block_cnt[a.role_model[role]], cnt);
         }
     }
-    cnt = warp_sum_int(cnt);
-    if (lane == 0) {
-        if (!role_ok && hi > lo) atomicOr(a.status, kStatusBadIndex);
-        a.inv_sums[s * 3 + 0] = static_cast<float>(cnt);
-    }
+    __syncthreads();
+    if (threadIdx.x < a.K && block_cnt[threadIdx.x] > 0)
+        atomicAdd(&a.model_cnt[threadIdx.x], static_cast<unsigned long long>(block_cnt[threadIdx.x]));
 }
 
 // Fixed-order sum over the 1024 threads of a block: lanes, then the 32 warp totals.
@@ -846,27 +860,6 @@ __device__ __forceinline__ float block_sum_1024(float v, float* sh) {
     return t;                                          // valid in warp 0
 }
 
-// (2) denominators M_k (one block of 1024 threads per model, fixed order).
-__global__ void k_value_norm(ValueArgs a) {
-    __shared__ float sh[32];
-    const int k = blockIdx.x;
-    float cnt = 0.f;
-    // branch-free body, eight invocations per step: the loads of a step are independent and issue together (a thread
-    // still adds its values in index order)
-#pragma unroll 8
-    for (int s = threadIdx.x; s < a.n_inv; s += 1024) {
-        const int role = a.inv_role[s];
-        const float c = a.inv_sums[s * 3 + 0];
-        const bool mine = role >= 0 && role < a.n_roles && a.role_model[role] == k;
-        cnt += mine ? c : 0.f;
-    }
-    cnt = block_sum_1024(cnt, sh);
-    if (threadIdx.x == 0) {
-        a.Mk[k] = a.has_norm ? a.norm[k] : fmaxf(cnt, 1.f);
-        a.Mk[UNITY_MAX_MODELS + k] = fmaxf(cnt, 1.f);
-    }
-}
-
 // (3) the one pass over the token data: loss terms, gradient (already divided by M_k), per-invocation sums.
 __global__ void k_value_main(ValueArgs a) {
     const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -874,7 +867,7 @@ __global__ void k_value_main(ValueArgs a) {
     if (s >= a.n_inv) return;
     const int role = a.inv_role[s];
     const bool role_ok = role >= 0 && role < a.n_roles && a.role_model[role] >= 0 && a.role_model[role] < a.K;
-    const float inv_M = 1.f / (role_ok ? a.Mk[a.role_model[role]] : 1.f);
+    const float inv_M = 1.f / (role_ok ? value_Mk(a, a.role_model[role]) : 1.f);
     const long long lo = a.cu_seqlens[s], hi = a.cu_seqlens[s + 1];
     float sum = 0.f, clp = 0.f;
     auto one = [&](long long i) {
@@ -919,13 +912,18 @@ __global__ void k_value_main(ValueArgs a) {
     if (lane == 0) { a.inv_sums[s * 3 + 1] = sum; a.inv_sums[s * 3 + 2] = clp; }
 }
 
-// (4) loss and clip fraction per model (one block per model).
+// (4) loss and clip fraction per model.  Block (j, k) sums slice j of the invocations for model k in a fixed order; the
+// block that finishes last for a model (a ticket counter, which it leaves at zero) adds the slices' partial sums in index
+// order.  The result depends on neither the order nor the timing of the blocks.
 __global__ void k_value_class(ValueArgs a) {
     __shared__ float sh[32];
-    const int k = blockIdx.x;
+    __shared__ int last;
+    const int k = blockIdx.y, j = blockIdx.x, n_slices = gridDim.x;
+    const int per = (a.n_inv + n_slices - 1) / n_slices;
+    const int s_end = min(a.n_inv, (j + 1) * per);
     float sum = 0.f, clp = 0.f;
-#pragma unroll 8
-    for (int s = threadIdx.x; s < a.n_inv; s += 1024) {
+#pragma unroll 4
+    for (int s = j * per + threadIdx.x; s < s_end; s += 1024) {
         const int role = a.inv_role[s];
         const float l = a.inv_sums[s * 3 + 1], c = a.inv_sums[s * 3 + 2];
         const bool mine = role >= 0 && role < a.n_roles && a.role_model[role] == k;
@@ -934,9 +932,23 @@ __global__ void k_value_class(ValueArgs a) {
     }
     sum = block_sum_1024(sum, sh);
     clp = block_sum_1024(clp, sh);
-    if (threadIdx.x != 0) return;
-    a.loss[k] = sum / a.Mk[k];
-    if (a.clip_frac) a.clip_frac[k] = clp / a.Mk[UNITY_MAX_MODELS + k];
+    if (threadIdx.x == 0) {
+        a.partial[(k * kValueSlices + j) * 2 + 0] = sum;
+        a.partial[(k * kValueSlices + j) * 2 + 1] = clp;
+        __threadfence();
+        last = atomicAdd(&a.tickets[k], 1) == n_slices - 1;
+    }
+    __syncthreads();
+    if (!last || threadIdx.x != 0) return;
+    __threadfence();
+    float tot = 0.f, tot_c = 0.f;
+    for (int q = 0; q < n_slices; ++q) {
+        tot += __ldcg(&a.partial[(k * kValueSlices + q) * 2 + 0]);
+        tot_c += __ldcg(&a.partial[(k * kValueSlices + q) * 2 + 1]);
+    }
+    a.tickets[k] = 0;
+    a.loss[k] = tot / value_Mk(a, k);
+    if (a.clip_frac) a.clip_frac[k] = tot_c / fmaxf(static_cast<float>(a.model_cnt[k]), 1.f);
 }
 
 }  // namespace
@@ -944,6 +956,8 @@ __global__ void k_value_class(ValueArgs a) {
 // ------------------------------------------------------------------------------------------------
 // launchers
 // ------------------------------------------------------------------------------------------------
+size_t value_counters_bytes() { return sizeof(unsigned long long) * UNITY_MAX_MODELS + sizeof(int) * UNITY_MAX_MODELS; }
+
 size_t advantage_table_bytes(long long n_seg) { return kSegHeaderBytes + static_cast<size_t>(n_seg) * 32; }
 
 cudaError_t launch_advantage(const AdvArgs& a, cudaStream_t stream, int* n_launches) {
@@ -1094,11 +1108,15 @@ cudaError_t launch_reward_assembly(const RewardArgs& a, cudaStream_t stream) {
 
 cudaError_t launch_value_loss(const ValueArgs& a, cudaStream_t stream, int* n_launches) {
     const int gi = (a.n_inv + 7) / 8;
+    // per-model token counts and the tickets of the last pass start at zero (one small clear)
+    cudaError_t e = cudaMemsetAsync(a.model_cnt, 0, value_counters_bytes(), stream);
+    if (e != cudaSuccess) return e;
     if (a.n_inv > 0) { k_value_count<<<gi, 256, 0, stream>>>(a); *n_launches += 1; }
-    k_value_norm<<<a.K, 1024, 0, stream>>>(a);
     if (a.n_inv > 0) { k_value_main<<<gi, 256, 0, stream>>>(a); *n_launches += 1; }
-    k_value_class<<<a.K, 1024, 0, stream>>>(a);
-    *n_launches += 2;
+    int slices = (a.n_inv + 2047) / 2048;
+    slices = slices < 1 ? 1 : (slices > kValueSlices ? kValueSlices : slices);
+    k_value_class<<<dim3(slices, a.K), 1024, 0, stream>>>(a);
+    *n_launches += 1;
     return cudaGetLastError();
 }
 

@@ -726,7 +726,9 @@ int unity_value_loss_fwd_bwd(unity_ctx* ctx, int32_t n_inv, int32_t n_roles, int
     for (int v = 0; v < n_roles; ++v) a.role_model[v] = role_model[v];
     CUDA_TRY(ctx, cudaSetDevice(ctx->device));
     Bump b{ctx->ws, 0, ctx->ws_bytes, true};
-    a.Mk = b.take<float>(2 * UNITY_MAX_MODELS);
+    a.model_cnt = reinterpret_cast<unsigned long long*>(b.take<char>(value_counters_bytes()));
+    a.tickets = reinterpret_cast<int*>(a.model_cnt + UNITY_MAX_MODELS);
+    a.partial = b.take<float>(static_cast<size_t>(UNITY_MAX_MODELS) * kValueSlices * 2);
     a.inv_sums = b.take<float>(static_cast<size_t>(n_inv) * 3 + 4);
     if (!b.ok) return fail(ctx, UNITY_ERR_WORKSPACE, "workspace too small: need %zu bytes", b.off);
     a.n_inv = n_inv; a.n_roles = n_roles; a.K = K;
