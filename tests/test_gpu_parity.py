@@ -384,12 +384,15 @@ def test_small_shapes_and_ragged_tails(H, V, rows):
     run_all_stages(small_workload(H, V, rows))
 
 
-@pytest.mark.parametrize("name", ["tiny", "search", "stress"])
+@pytest.mark.parametrize("name", ["tiny", "search", "four_models"])
 def test_calls_with_host_side_row_counts_match_the_oracle(name):
     # By default the host never learns the row counts: it walks every chunk a model could have and the kernels cut their
     # spans on the device (most launches of a model with few rows return at once) - that is what every other test runs.
     # UNITY_OPT_HOST_COUNTS = 1: the counts are read back once and launches that would be empty are skipped.
-    w = wl.make(name, device="cuda", **({} if name == "tiny" else dict(cut_rows=1200, cut_max_len=64)))
+    if name == "four_models":      # four models, one of them without rows (the stress configuration's mapping, small sizes)
+        w = small_workload(320, 2048 + 264, 1200, role_model=[0, 3, 1], K=4)
+    else:
+        w = wl.make(name, device="cuda", **({} if name == "tiny" else dict(cut_rows=1200, cut_max_len=64)))
     run_all_stages(w, options=[(ub.OPT_HOST_COUNTS, 1)])
     if name == "tiny":
         run_all_stages(w, options=[(ub.OPT_HOST_COUNTS, 1), (ub.OPT_LOGIT_STASH, 1)])
@@ -451,8 +454,8 @@ def test_recompute_gemm_on_the_forward_schedule(ctas, gmax, block):
     # rounds backwards): 25 row tiles of 256 give full rounds and a short last one that is cut into more splits
     w = small_workload(128, 8192 + 264, 7700, max_len=200, role_model=[0, 0, 0], K=1)
     run_all_stages(w, ctas=(ctas,) * 4, options=[(ub.OPT_GRAD_ROUNDS, gmax), (ub.OPT_GRAD_BLOCK, block)], ent_coef=0.01)
-    if gmax == 48:       # and once at a full-size hidden width and vocabulary (four models, H = 5120)
-        run_all_stages(wl.make("stress", device="cuda", cut_rows=300, cut_max_len=64),
+    if gmax == 48:       # and once at a full-size hidden width and vocabulary (two models, H = 1536, V = 151936)
+        run_all_stages(wl.make("search", device="cuda", cut_rows=300, cut_max_len=64),
                        options=[(ub.OPT_GRAD_ROUNDS, gmax), (ub.OPT_GRAD_BLOCK, block)])
 
 
@@ -515,10 +518,11 @@ def test_accumulate_gemms_with_256_and_512_column_tiles(wide):
         run_all_stages(small_workload(H, V, rows), ctas=(2, 2, 2, 2), options=[(11, wide)])
 
 
-@pytest.mark.parametrize("name", ["tiny", "rag_qa", "code", "stress"])
+@pytest.mark.parametrize("name", ["tiny", "rag_qa", "code"])
 def test_logit_stash_instead_of_recompute(name):
     # the loss call keeps the scaled logits of a row block in bf16 and turns them into dL/dz in place; same outputs
-    # within the same tolerances (V = 151936 ends in a half tile; the cuts span all eight vocabulary chunks)
+    # within the same tolerances (V = 151936 ends in a half tile; the cuts span all eight vocabulary chunks); the stress
+    # configuration runs with the stash at full size in test_gpu_fullsize.py
     w = wl.make(name, device="cuda") if name == "tiny" else wl.make(name, device="cuda", cut_rows=300, cut_max_len=64)
     run_all_stages(w, options=[(ub.OPT_LOGIT_STASH, 1)])
 
