@@ -127,6 +127,8 @@ int unity_set_profiling(unity_ctx* ctx, int enable);
                                      at most n 128-row tiles x vocabulary splits of the launch's columns, a worker sweeps the
                                      tiles of its split with one row tile and the workers meet once per round.  -1 (default):
                                      rounds of half the SMs where UNITY_OPT_FWD_GROUP's rule allows them (H <= 2368), else 0. */
+#define UNITY_OPT_GRAD_BLOCK 27     /* one recompute launch covers value x 18944 rows and vocabulary entries of the gradient
+                                     chunk per side; 0 (default): the whole chunk when it runs in rounds or runs of tiles, else 1 */
 #define UNITY_OPT_GRAD_RUNS 28      /* The recompute GEMM outside rounds.  0: a unit is one output tile.  n > 0: a unit is a run of column
                                      tiles of one row tile; the kernel cuts the launch's columns into the number of runs that fills
                                      its workers best while about n 128-row tiles are in flight.  -1 (default): n = the tiles whose
@@ -134,8 +136,6 @@ int unity_set_profiling(unity_ctx* ctx, int enable);
 #define UNITY_OPT_DW_TAIL 29        /* 1 (default): when the vocabulary tiles of a gradient chunk leave a remainder that would fill
                                      less than half of one more wave of CTA pairs, the dW GEMM runs those tiles as a second
                                      launch with narrow column tiles spread over the machine.  0: one launch per chunk. */
-#define UNITY_OPT_GRAD_BLOCK 27     /* one recompute launch covers value x 18944 rows and vocabulary entries of the gradient
-                                     chunk per side; 0 (default): the whole chunk when it runs in rounds or runs of tiles, else 1 */
 #define UNITY_OPT_WAIT_KCYCLES 20  /* bound of every in-kernel wait in thousands of SM clocks (default 4 000 000, about 2 s); when
                                      it runs out the kernel records UNITY_ERR_TIMEOUT, frees its tensor memory and returns */
 #define UNITY_OPT_TEST_DROP_SLAB 21 /* TEST HOOK for the timeout path; accepted only while UNITY_OPT_WAIT_KCYCLES <= 1000.
