@@ -468,6 +468,27 @@ def test_recompute_gemm_in_runs_of_column_tiles(ctas, in_flight):
     run_all_stages(w, ctas=(ctas,) * 4, options=options, ent_coef=0.01)
 
 
+def test_dw_gemm_runs_its_last_vocabulary_tiles_as_a_narrow_launch():
+    # 77 vocabulary tiles (the last one ragged) on 74 CTA pairs: the dW GEMM runs tiles 74..76 as a second launch with
+    # 64-column tiles; same bits as the single launch (a tile's sum over the rows does not depend on its width), and
+    # both match the oracle
+    w = small_workload(320, 76 * 256 + 8, 300)
+    run_all_stages(w)
+    d = pu.DeviceInputs(w)
+    ol = pu.oracle_logprob(w)
+    cur = torch.from_numpy(ol["logp"].astype(np.float32))
+    old, ref = (cur + w.noise_old).cuda(), (cur + w.noise_ref).cuda()
+    adv = wl.normal(6, 96, w.n_tok).cuda()
+    outs = []
+    for tail in (0, 1):
+        ctx = pu.make_ctx(w)
+        ctx.set_option(29, tail)
+        outs.append(pu.gpu_ppo(ctx, w, d, old, ref, adv))
+        ctx.close()
+    assert all(torch.equal(a, b) for a, b in zip(outs[0]["dW"], outs[1]["dW"]))
+    assert torch.equal(outs[0]["dHidden"], outs[1]["dHidden"])
+
+
 @pytest.mark.parametrize("ctas", [(1, 1, 1, 1), (2, 2, 2, 2), (2, 1, 1, 2)])
 def test_single_cta_and_cta_pair_kernels(ctas):
     # every GEMM class exists as a one-CTA kernel (128-row tiles) and as a CTA-pair kernel (256-row tiles)
