@@ -687,7 +687,8 @@ def main():
         old_h, ref_h, adv_h = old.cpu().numpy(), ref.cpu().numpy(), adv_tok.cpu().numpy()
         w.hidden = w.hidden.cpu()
         w.W = [x.cpu() for x in w.W]
-        dt, rows = oracle_sample_run(w, args.ref_rows, old_h, ref_h, adv_h)
+        # twice the reference arm's per-step sample: one pass of about 12 s on 16 host cores
+        dt, rows = oracle_sample_run(w, 2 * args.ref_rows, old_h, ref_h, adv_h)
         cpu_baseline = {"value": rows / dt, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
                         "sample": f"{rows} valid rows of the {args.workload} workload (one oracle pass, {dt:.1f} s), fp64 numpy"}
         # and the smallest configuration at full size: advantage, log-prob and loss forward + backward on every row
